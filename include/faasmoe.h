@@ -1,0 +1,214 @@
+/*
+ * faasmoe.h -- C ABI of the B200 (sm_100a) multi-tenant Mixture-of-Experts layer.
+ *
+ * The layer is the one FaaSMoE serves as a shared pool of stateless expert
+ * functions for many tenants: gating and top-k selection (paper Sec. 2.1), the
+ * construction of micro-batched routing requests per expert block (Sec. 3,
+ * Sec. 4.1), expert execution on the assigned tokens (Sec. 3), and the
+ * aggregation of expert outputs per token (Sec. 3, Sec. 4.2).  The paper's
+ * expert-block granularity (G experts per function, Sec. 3 / Sec. 5) is a
+ * partition parameter of the expert work; it never changes a result.
+ *
+ * Conventions
+ *  - Every pointer is a DEVICE pointer unless its comment says "host".
+ *  - bf16 tensors are passed as `const void*` (16-bit elements, row-major).
+ *  - The caller owns every buffer it passes.  Weight buffers are used in
+ *    place (no copy is made): they must stay valid and unchanged while any
+ *    call that uses them may still run.
+ *  - The context owns only its workspace, its tables and its TMA descriptors.
+ *  - `stream` is a cudaStream_t passed as `void*` (NULL = default stream).
+ *    No call synchronises the stream unless stated.
+ *  - Every call returns an int status: MOE_OK (0) or a negative MOE_ERR_*.
+ *    Errors the host can detect return before anything is launched.
+ *    Data-dependent errors (an id out of range inside a device buffer, a
+ *    bounded device-side wait that ran out) set bits in a sticky device
+ *    status word, never fault, and are read with moe_last_status().
+ *  - Shapes: hidden, inter and shared_inter must be multiples of 128;
+ *    1 <= top_k <= min(n_experts, 8); n_experts <= 256.
+ *  - One context serves one device (the device current at moe_create) and
+ *    one stream at a time: calls on one context must not overlap on the GPU,
+ *    because they share its workspace.
+ */
+#ifndef FAASMOE_H
+#define FAASMOE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct moe_ctx moe_ctx;
+
+enum {
+    MOE_OK = 0,
+    MOE_ERR_NULL = -1,        /* a required pointer is NULL */
+    MOE_ERR_SHAPE = -2,       /* a size or id is out of range (T > max_tokens, bad layer/model, ...) */
+    MOE_ERR_G = -3,           /* G < 1 or G > n_experts */
+    MOE_ERR_STATE = -4,       /* weights for the requested layer/model were not set */
+    MOE_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed (see moe_strerror) */
+    MOE_ERR_ALLOC = -6,       /* workspace allocation failed */
+    MOE_ERR_UNSUPPORTED = -7  /* the shape is outside what the kernels support */
+};
+
+/* bits of the device status word */
+enum {
+    MOE_DEV_BAD_TENANT = 1,   /* tenant id outside [0, n_tenants): the token's output is zero */
+    MOE_DEV_BAD_EXPERT = 2,   /* expert id outside [0, n_experts) in a caller-supplied topk_idx */
+    MOE_DEV_TIMEOUT = 8       /* a bounded wait inside a kernel ran out; outputs are invalid */
+};
+
+/* values of MOE_OPT_EXPERT_PATH */
+enum { MOE_PATH_AUTO = 0, MOE_PATH_FMA = 1, MOE_PATH_TCGEN05 = 2 };
+enum { MOE_OPT_EXPERT_PATH = 1 };
+
+typedef struct {
+    int32_t hidden;        /* H */
+    int32_t n_experts;     /* E: routed experts per tenant model */
+    int32_t inter;         /* I: intermediate size of one routed expert */
+    int32_t top_k;         /* k */
+    int32_t shared_inter;  /* I_s: intermediate size of the shared expert, 0 = none */
+    int32_t n_models;      /* M: tenant models whose experts live in the pool */
+    int32_t n_tenants;     /* tenant ids are 0 .. n_tenants-1 */
+    int32_t n_slots;       /* S: routed-expert slots in the pool of each layer (>= 1) */
+    int32_t max_tokens;    /* largest T any call will pass */
+    int32_t n_layers;      /* L: 1 for a single layer */
+    float   rms_eps;       /* epsilon of the RMSNorm in moe_stack_forward */
+} moe_config;
+
+/* Creates a context on the current device and allocates its workspace
+ * (O(max_tokens * top_k * (2*H + I)) bytes).  cfg is a host pointer. */
+int moe_create(const moe_config* cfg, moe_ctx** out);
+int moe_destroy(moe_ctx* ctx);
+
+/*
+ * Registers the routed-expert pool of one layer (Sec. 4.1: experts are
+ * extracted from each MoE layer and packaged by layer and expert id).
+ *   w_gate, w_up : bf16 [S, I, H]    w_down : bf16 [S, H, I]
+ * Slot s holds one SwiGLU expert: y = W_down . (silu(W_gate . x) * (W_up . x)).
+ * The buffers are used in place.  16-byte aligned.
+ */
+int moe_set_expert_pool(moe_ctx* ctx, int layer, const void* w_gate, const void* w_up, const void* w_down);
+
+/*
+ * Registers the non-pooled weights of tenant model `model` in layer `layer`:
+ *   router_w      bf16 [E, H]          gating network (Sec. 2.1)
+ *   router_bias   f32  [E] or NULL     added to the router logits
+ *   shared_gate_w bf16 [H] or NULL     sigmoid scalar gate of the shared expert
+ *   ws_gate/ws_up bf16 [I_s, H], ws_down bf16 [H, I_s], or all NULL if I_s = 0
+ *                                      (Sec. 5: the always-active shared experts)
+ *   rms_w         bf16 [H] or NULL     RMSNorm scale, needed by moe_stack_forward only
+ * Used in place.
+ */
+int moe_set_model_weights(moe_ctx* ctx, int layer, int model, const void* router_w, const float* router_bias,
+                          const void* shared_gate_w, const void* ws_gate, const void* ws_up, const void* ws_down,
+                          const void* rms_w);
+
+/* Expert (m, e) lives in pool slot slot[m*E + e] (host pointer, M*E entries, each in
+ * [0, S)).  The default is the identity m*E + e.  Copied; synchronises the device. */
+int moe_set_slot_table(moe_ctx* ctx, const int32_t* slot);
+
+/* Tenant u runs model model_of_tenant[u] (host pointer, n_tenants entries in [0, M)).
+ * Default: u % M.  Copied; synchronises the device. */
+int moe_set_tenant_models(moe_ctx* ctx, const int32_t* model_of_tenant);
+
+int moe_set_option(moe_ctx* ctx, int option, int value);
+
+/*
+ * Gating (Sec. 2.1; Sec. 3: gating modules of the orchestrator).
+ * For token t of tenant u = tenant_id[t], model m = model_of_tenant[u]:
+ *   z[e] = x[t] . router_w[m][e] + bias[m][e]   (bf16 inputs, fp32 accumulation)
+ *   p = softmax(z) in fp32; the k experts of largest p, ordered by (p descending,
+ *   expert id ascending); weights are the raw probabilities (no renormalisation).
+ *   shared_gate[t] = sigmoid(x[t] . shared_gate_w[m])
+ *   tie_flag[t] = 1 if two neighbouring ranks among ranks 1..k+1 differ by less
+ *   than 1e-5 relative (the order is then not decidable in fp32).
+ * x bf16 [T,H]; tenant_id int32 [T]; topk_idx int32 [T,k]; topk_w f32 [T,k];
+ * shared_gate f32 [T] or NULL; tie_flag u8 [T] or NULL.
+ */
+int moe_route(moe_ctx* ctx, int layer, const void* x, const int32_t* tenant_id, int T,
+              int32_t* topk_idx, float* topk_w, float* shared_gate, uint8_t* tie_flag, void* stream);
+
+/*
+ * Micro-batched routing requests (Sec. 3; Sec. 4.1: all tokens routed to the same
+ * expert block are consolidated into one batched invocation).
+ * Row (t, j) has flat id t*k + j.  Rows are sorted by (model, expert, tenant, token):
+ *   perm[r'] = flat id placed at position r';  inv_perm = its inverse      int32 [T*k]
+ *   tenant_expert_count[u*E + e] = rows of tenant u routed to expert e    int32 [n_tenants*E]
+ *   expert_off[m*E + e] = first position of expert (m,e); last entry T*k  int32 [M*E+1]
+ *   group_off[m*B + b] = first position of block b = experts [b*G, min((b+1)*G, E))
+ *                        of model m, B = ceil(E/G); last entry T*k        int32 [M*B+1]
+ *   x_perm[r'] = x[perm[r'] / k]                                          bf16 [T*k, H] or NULL
+ * perm does not depend on G (Sec. 3: block size does not affect routing correctness).
+ * Any output pointer except perm/inv_perm/expert_off may be NULL.
+ */
+int moe_dispatch(moe_ctx* ctx, const void* x, const int32_t* topk_idx, const int32_t* tenant_id, int T, int G,
+                 int32_t* perm, int32_t* inv_perm, int32_t* tenant_expert_count, int32_t* expert_off,
+                 int32_t* group_off, void* x_perm, void* stream);
+
+/*
+ * Expert execution (Sec. 3: each expert block performs stateless computation on its
+ * assigned tokens).  Only experts that received rows are touched.
+ *   y_perm[r'] = FFN_{slot(m,e)}(x_perm[r'])    for r' in expert (m,e)'s segment   bf16 [T*k, H]
+ *   y_shared[t] = FFN_shared,m(x[t])  (ungated)                                    bf16 [T, H] or NULL
+ * G orders the work by expert block; results are bit-identical for every G.
+ * x bf16 [T,H] and tenant_id are needed only when y_shared is requested.
+ * x_perm must be readable for 128 rows past T*k (the tensor-core path loads whole
+ * row tiles; what lies there is never used).
+ */
+int moe_experts(moe_ctx* ctx, int layer, const void* x, const void* x_perm, const int32_t* expert_off,
+                const int32_t* tenant_id, int T, int G, void* y_perm, void* y_shared, void* stream);
+
+/*
+ * Aggregation (Sec. 3, Sec. 4.2):
+ *   out[t] = sum_{j=0..k-1} topk_w[t,j] * y_perm[inv_perm[t*k+j]] + shared_gate[t] * y_shared[t]
+ * accumulated in fp32 in that fixed order, rounded once to bf16.  out bf16 [T,H].
+ * y_shared / shared_gate may both be NULL.
+ */
+int moe_combine(moe_ctx* ctx, const void* y_perm, const int32_t* inv_perm, const float* topk_w,
+                const void* y_shared, const float* shared_gate, int T, void* out, void* stream);
+
+/* route -> dispatch -> experts -> combine on the context's workspace; bit-identical to
+ * the four calls above.  out bf16 [T,H]. */
+int moe_layer_forward(moe_ctx* ctx, int layer, const void* x, const int32_t* tenant_id, int T, int G,
+                      void* out, void* stream);
+
+/* Same, with HOST buffers: copies x and tenant_id to the device, runs the layer,
+ * copies out back and synchronises the stream.  For best speed pass pinned memory. */
+int moe_layer_forward_host(moe_ctx* ctx, int layer, const void* x_host, const int32_t* tenant_id_host, int T, int G,
+                           void* out_host, void* stream);
+
+/* moe_layer_forward with a CUDA event recorded on `stream` after every stage; synchronises the
+ * stream and writes the stage durations in milliseconds to stage_ms_host (host, 6 floats):
+ * route, dispatch, plan, experts gate/up, experts down, combine. */
+int moe_layer_forward_timed(moe_ctx* ctx, int layer, const void* x, const int32_t* tenant_id, int T, int G,
+                            void* out, float* stage_ms_host, void* stream);
+
+/*
+ * n_layers blocks of: xn = bf16(RMSNorm(x) * rms_w);  o = layer(xn);  x = bf16(x + o).
+ * x_inout bf16 [T,H] is updated in place.  dbg_layer_inputs, if not NULL, receives the
+ * xn of every block, and dbg_layer_outputs, if not NULL, the residual stream x after every
+ * block: bf16 [L, T, H] each.
+ */
+int moe_stack_forward(moe_ctx* ctx, void* x_inout, const int32_t* tenant_id, int T, int G,
+                      void* dbg_layer_inputs, void* dbg_layer_outputs, void* stream);
+
+/* Device pointers into the workspace holding the routing results of the last
+ * moe_layer_forward (valid until the next call on this context). */
+int moe_get_workspace(moe_ctx* ctx, int32_t** topk_idx, float** topk_w, float** shared_gate, uint8_t** tie_flag,
+                      int32_t** perm, int32_t** inv_perm, int32_t** expert_off, int32_t** group_off);
+
+/* Synchronises the device, returns the device status word in *status_host and clears it.
+ * Also reports, if not NULL, stats_host[0] = non-empty expert blocks (invocations) and
+ * stats_host[1] = active routed experts of the last dispatch. */
+int moe_last_status(moe_ctx* ctx, int32_t* status_host, int32_t* stats_host);
+
+/* Number of kernels this library has launched on this context since creation. */
+int64_t moe_launch_count(moe_ctx* ctx);
+
+const char* moe_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FAASMOE_H */
