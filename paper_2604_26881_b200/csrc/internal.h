@@ -1,0 +1,170 @@
+// Internal declarations shared by the translation units of libfaasmoe.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda.h>
+#include <stdint.h>
+#include <vector>
+
+#include "faasmoe.h"
+
+namespace faasmoe {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kMaxTopK = 8;
+constexpr int kMaxExperts = 256;
+constexpr int kMaxBins = 8192;       // E * n_tenants
+constexpr int kTileRows = 128;       // rows (tokens) of one expert handled by one work unit
+constexpr int kDispatchChunk = 256;  // routed rows ranked by one block of the dispatch kernels
+
+// Per (layer, model) weight pointers, as the kernels see them.
+struct ModelWeights {
+    const bf16* router_w;       // [E,H]
+    const float* router_bias;   // [E] or null
+    const bf16* shared_gate_w;  // [H] or null
+    const bf16* ws_gate;        // [Is,H]
+    const bf16* ws_up;          // [Is,H]
+    const bf16* ws_down;        // [H,Is]
+    const bf16* rms_w;          // [H]
+};
+
+struct PoolWeights {
+    const bf16* w_gate;  // [S,I,H]
+    const bf16* w_up;    // [S,I,H]
+    const bf16* w_down;  // [S,H,I]
+};
+
+// One tile of rows that share an expert: rows [row0, row0+nrows) of the activation
+// matrix, weights of `slot` (routed: pool slot; shared: model index).
+struct Tile {
+    int32_t row0;
+    int32_t nrows;
+    int32_t slot;
+    int32_t group;   // expert block (m*B + b) for routed tiles, model for shared tiles
+};
+
+// Work unit of the tensor-core grouped GEMM: a tile (>= 0 routed, < 0: shared tile ~tile)
+// and a block of weight rows.
+struct Unit {
+    int32_t tile;
+    int32_t colblock;
+};
+
+struct TensorMaps;   // defined in experts_tc.cu
+
+struct Workspace {
+    // routing results
+    int32_t* topk_idx = nullptr;   // [T,k]
+    float* topk_w = nullptr;       // [T,k]
+    float* shared_gate = nullptr;  // [T]
+    uint8_t* tie_flag = nullptr;   // [T]
+    // dispatch results
+    int32_t* perm = nullptr;       // [R]
+    int32_t* inv_perm = nullptr;   // [R]
+    int32_t* tenant_expert_count = nullptr;  // [Nt*E]
+    int32_t* expert_off = nullptr; // [M*E+1]
+    int32_t* group_off = nullptr;  // [M*E+1] (largest B is E)
+    // dispatch scratch
+    int32_t* block_cnt = nullptr;  // [nblk, nbins]
+    int32_t* bin_off = nullptr;    // [nbins+1]
+    int32_t* tok_block_cnt = nullptr;  // [nblk_tok, M]
+    int32_t* model_tok_off = nullptr;  // [M+1]
+    int32_t* tok_perm = nullptr;   // [T] tokens sorted by (model, token)
+    int32_t* tok_inv = nullptr;    // [T]
+    // plan
+    Tile* tiles = nullptr;         // routed tiles
+    Tile* stiles = nullptr;        // shared-expert tiles
+    int32_t* plan_counts = nullptr;  // [8]: n_tiles, n_stiles, n_units1, n_units2
+    Unit* units1 = nullptr;        // gate/up GEMM units (shared, then routed)
+    Unit* units2 = nullptr;        // down GEMM units
+    // activations
+    bf16* x_perm = nullptr;        // [R,H]
+    bf16* xs_perm = nullptr;       // [T,H] tokens grouped by model (M > 1 only)
+    bf16* h = nullptr;             // [R,I]
+    bf16* hs = nullptr;            // [T,Is]
+    bf16* y_perm = nullptr;        // [R,H]
+    bf16* y_shared = nullptr;      // [T,H]
+    bf16* xn = nullptr;            // [T,H] normalised input of a block (stack)
+    // staging of the host-buffer entry point
+    bf16* x_stage = nullptr;       // [T,H]
+    int32_t* tenant_stage = nullptr;  // [T]
+    bf16* out_stage = nullptr;     // [T,H]
+    // status
+    int32_t* status = nullptr;     // [1] sticky status bits
+    int32_t* stats = nullptr;      // [4]
+};
+
+}  // namespace faasmoe
+
+struct moe_ctx {
+    moe_config cfg;
+    int device;
+    int sm_count;
+    int expert_path;
+    int64_t launches;
+    int max_tiles, max_stiles, max_units1, max_units2;
+    int nblk_rows, nblk_tok, nbins;
+    std::vector<faasmoe::PoolWeights> pools;     // [L]
+    std::vector<uint8_t> pool_set;               // [L]
+    std::vector<faasmoe::ModelWeights> models;   // [L*M]
+    std::vector<uint8_t> model_set;              // [L*M]
+    faasmoe::ModelWeights* d_models;             // [L*M] device copy
+    std::vector<int32_t> h_slot, h_model_of_tenant;
+    int32_t* d_slot;              // [M*E]
+    int32_t* d_model_of_tenant;   // [Nt]
+    int32_t* d_tenant_local;      // [Nt] index of the tenant among the tenants of its model
+    int32_t* d_bin_base;          // [M+1] first bin of each model (bins = (model, expert, tenant of model))
+    int32_t* d_tenants_in_model;  // [M]
+    faasmoe::Workspace ws;
+    faasmoe::TensorMaps* tmaps;   // TMA descriptors of the tensor-core path (host)
+    bool timing;                  // record an event after every stage (moe_layer_forward_timed)
+    cudaEvent_t ev[8];
+    char errbuf[256];
+};
+
+// stage boundaries of one layer pass
+enum { kEvBegin = 0, kEvRoute, kEvDispatch, kEvPlan, kEvGateUp, kEvDown, kEvCombine, kEvCount };
+
+static inline void stage_mark(moe_ctx* c, cudaStream_t st, int i)
+{
+    if (c->timing) cudaEventRecord(c->ev[i], st);
+}
+
+namespace faasmoe {
+
+// --- launchers (each returns a cudaError_t from the launch) -------------------------------
+
+cudaError_t launch_route(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,
+                         float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st);
+
+cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, const int32_t* tenant_id, int T, int G,
+                            int32_t* perm, int32_t* inv_perm, int32_t* tenant_expert_count, int32_t* expert_off,
+                            int32_t* group_off, bf16* x_perm, cudaStream_t st);
+
+// Sorts tokens by (model, token) into ws.tok_perm / tok_inv / model_tok_off and gathers ws.xs_perm (M > 1).
+cudaError_t launch_token_sort(moe_ctx* c, const bf16* x, const int32_t* tenant_id, int T, cudaStream_t st);
+
+// Builds the tile lists (and the unit lists of the tensor-core path) from expert_off.
+cudaError_t launch_plan(moe_ctx* c, const int32_t* expert_off, int T, int G, bool with_shared, cudaStream_t st);
+
+cudaError_t launch_experts_fma(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, bf16* y_perm,
+                               bf16* y_shared, const int32_t* shared_dst_rows, cudaStream_t st);
+
+cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, bf16* y_perm,
+                              bf16* y_shared, const int32_t* shared_dst_rows, cudaStream_t st);
+
+cudaError_t launch_combine(moe_ctx* c, const bf16* y_perm, const int32_t* inv_perm, const float* topk_w,
+                           const bf16* y_shared, const float* shared_gate, const bf16* residual, int T, bf16* out,
+                           cudaStream_t st);
+
+cudaError_t launch_rmsnorm(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, bf16* xn,
+                           cudaStream_t st);
+
+// tensor-core path set-up / tear-down (TMA descriptors); returns MOE_* status
+int tc_setup_layer(moe_ctx* c, int layer);
+void tc_destroy(moe_ctx* c);
+bool tc_supported(const moe_ctx* c);
+
+}  // namespace faasmoe
