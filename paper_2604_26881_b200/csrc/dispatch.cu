@@ -1,0 +1,299 @@
+// Micro-batched routing requests: per-(tenant, expert) histogram, prefix scan, stable ranks,
+// token permute into expert segments (paper Sec. 3: the orchestrator "constructs micro-batched
+// routing requests"; Sec. 4.1: all tokens routed to the same expert block become one batched
+// invocation).  Rows are ordered by (model, expert, tenant, token); the order is produced
+// without order-dependent atomics so that the permutation is reproducible bit for bit.
+#include "internal.h"
+
+namespace faasmoe {
+
+namespace {
+
+// bin of a routed row: bins are laid out (model, expert, tenant-of-that-model)
+struct BinMap {
+    const int32_t* model_of_tenant;
+    const int32_t* tenant_local;
+    const int32_t* bin_base;          // [M+1]
+    const int32_t* tenants_in_model;  // [M]
+    int n_tenants, E;
+};
+
+__device__ __forceinline__ int row_bin(const BinMap& bm, int tenant, int expert, int32_t* status)
+{
+    if (tenant < 0 || tenant >= bm.n_tenants) { atomicOr(status, MOE_DEV_BAD_TENANT); tenant = 0; }
+    if (expert < 0 || expert >= bm.E) { atomicOr(status, MOE_DEV_BAD_EXPERT); expert = 0; }
+    const int m = bm.model_of_tenant[tenant];
+    return bm.bin_base[m] + expert * bm.tenants_in_model[m] + bm.tenant_local[tenant];
+}
+
+// D1: each block counts the rows of its chunk per bin.  One warp per block.
+__global__ void __launch_bounds__(32)
+dispatch_hist_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ tenant_id, int R, int k,
+                     BinMap bm, int nbins, int32_t* __restrict__ block_cnt, int32_t* __restrict__ status)
+{
+    extern __shared__ int32_t s_cnt[];
+    for (int b = threadIdx.x; b < nbins; b += 32) s_cnt[b] = 0;
+    __syncwarp();
+    const int r0 = blockIdx.x * kDispatchChunk;
+    const int r1 = min(R, r0 + kDispatchChunk);
+    for (int r = r0 + threadIdx.x; r < r1; r += 32) {
+        const int bin = row_bin(bm, tenant_id[r / k], topk_idx[r], status);
+        atomicAdd(&s_cnt[bin], 1);      // counts only: the result does not depend on the order
+    }
+    __syncwarp();
+    int32_t* dst = block_cnt + (size_t)blockIdx.x * nbins;
+    for (int b = threadIdx.x; b < nbins; b += 32) dst[b] = s_cnt[b];
+}
+
+// D2: one block.  Totals per bin, exclusive scan in key order, per-block bases, and the
+// offset tables the caller sees.
+__global__ void __launch_bounds__(1024)
+dispatch_scan_kernel(int nblk, int nbins, int R, int E, int M, int G, int n_tenants, BinMap bm,
+                     int32_t* __restrict__ block_cnt, int32_t* __restrict__ bin_off,
+                     int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
+                     int32_t* __restrict__ group_off, int32_t* __restrict__ stats)
+{
+    extern __shared__ int32_t s_tot[];       // [nbins] totals, then exclusive offsets
+    __shared__ int32_t s_part[1024];
+    __shared__ int32_t s_count[2];
+    const int tid = threadIdx.x, nth = blockDim.x;
+    // totals per bin; block_cnt becomes the exclusive prefix over blocks
+    for (int b = tid; b < nbins; b += nth) {
+        int run = 0;
+        for (int blk = 0; blk < nblk; ++blk) {
+            const int c = block_cnt[(size_t)blk * nbins + b];
+            block_cnt[(size_t)blk * nbins + b] = run;
+            run += c;
+        }
+        s_tot[b] = run;
+    }
+    if (tid < 2) s_count[tid] = 0;
+    __syncthreads();
+    if (tenant_expert_count) {
+        for (int i = tid; i < n_tenants * E; i += nth) {
+            const int u = i / E, e = i - u * E;
+            const int m = bm.model_of_tenant[u];
+            tenant_expert_count[i] = s_tot[bm.bin_base[m] + e * bm.tenants_in_model[m] + bm.tenant_local[u]];
+        }
+    }
+    __syncthreads();
+    // exclusive scan over bins: each thread owns a contiguous run of bins
+    const int per = (nbins + nth - 1) / nth;
+    const int b0 = min(nbins, tid * per), b1 = min(nbins, b0 + per);
+    int sum = 0;
+    for (int b = b0; b < b1; ++b) sum += s_tot[b];
+    s_part[tid] = sum;
+    __syncthreads();
+    for (int off = 1; off < nth; off <<= 1) {          // Hillis-Steele inclusive scan of the partials
+        int v = (tid >= off) ? s_part[tid - off] : 0;
+        __syncthreads();
+        s_part[tid] += v;
+        __syncthreads();
+    }
+    int run = s_part[tid] - sum;
+    for (int b = b0; b < b1; ++b) { const int c = s_tot[b]; s_tot[b] = run; run += c; }
+    __syncthreads();
+    for (int b = tid; b < nbins; b += nth) bin_off[b] = s_tot[b];
+    if (tid == 0) bin_off[nbins] = R;
+    // expert_off[m*E + e] = offset of the first bin of (m, e); a model without tenants owns
+    // no bins, so its experts start where the next model's bins start
+    for (int i = tid; i <= M * E; i += nth) {
+        int v = R;
+        if (i < M * E) {
+            const int m = i / E, e = i - m * E;
+            const int first = bm.bin_base[m] + e * bm.tenants_in_model[m];
+            v = (first < nbins) ? s_tot[first] : R;
+        }
+        expert_off[i] = v;
+    }
+    __syncthreads();
+    // expert blocks of G experts; invocation statistics
+    const int B = (E + G - 1) / G;
+    for (int i = tid; i <= M * B; i += nth) {
+        int v = R;
+        if (i < M * B) {
+            const int m = i / B, b = i - m * B;
+            const int e0 = b * G, e1 = min(E, e0 + G);
+            v = expert_off[m * E + e0];
+            if (expert_off[m * E + e1] > v) atomicAdd(&s_count[0], 1);
+        }
+        if (group_off) group_off[i] = v;
+    }
+    for (int i = tid; i < M * E; i += nth)
+        if (expert_off[i + 1] > expert_off[i]) atomicAdd(&s_count[1], 1);
+    __syncthreads();
+    if (tid < 2) stats[tid] = s_count[tid];
+}
+
+// D3: stable rank of every row inside its bin.  One warp per block walks its chunk in row
+// order; rows that share a bin inside one step are ranked by lane order (= row order).
+__global__ void __launch_bounds__(32)
+dispatch_rank_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ tenant_id, int R, int k,
+                     BinMap bm, int nbins, const int32_t* __restrict__ block_cnt, const int32_t* __restrict__ bin_off,
+                     int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, int32_t* __restrict__ status)
+{
+    extern __shared__ int32_t s_next[];      // next free position of each bin for this block
+    const int lane = threadIdx.x;
+    const int32_t* base = block_cnt + (size_t)blockIdx.x * nbins;
+    for (int b = lane; b < nbins; b += 32) s_next[b] = bin_off[b] + base[b];
+    __syncwarp();
+    const int r0 = blockIdx.x * kDispatchChunk;
+    const int r1 = min(R, r0 + kDispatchChunk);
+    for (int rr = r0; rr < r1; rr += 32) {
+        const int r = rr + lane;
+        const bool live = r < r1;
+        int bin = -1 - lane;                 // distinct dummy keys for idle lanes
+        if (live) bin = row_bin(bm, tenant_id[r / k], topk_idx[r], status);
+        const unsigned peers = __match_any_sync(0xffffffffu, bin);
+        const int leader = __ffs(peers) - 1;
+        const int rank = __popc(peers & ((1u << lane) - 1u));
+        int start = 0;
+        if (live && lane == leader) { start = s_next[bin]; s_next[bin] = start + __popc(peers); }
+        start = __shfl_sync(0xffffffffu, start, leader);
+        if (live) {
+            const int pos = start + rank;
+            perm[pos] = r;
+            inv_perm[r] = pos;
+        }
+        __syncwarp();
+    }
+}
+
+// D4: x_perm[pos] = x[perm[pos] / k].  One warp per row, 16-byte vectors.
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ perm, int R, int k, int H,
+                   bf16* __restrict__ x_perm)
+{
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= R) return;
+    const int t = perm[warp] / k;
+    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * H);
+    uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)warp * H);
+    for (int v = lane; v < (H >> 3); v += 32) dst[v] = src[v];
+}
+
+// Token sort by (model, token) for the shared experts of a multi-model pool.
+__global__ void __launch_bounds__(32)
+token_hist_kernel(const int32_t* __restrict__ tenant_id, int T, int n_tenants, int M,
+                  const int32_t* __restrict__ model_of_tenant, int32_t* __restrict__ tok_block_cnt)
+{
+    __shared__ int32_t s_cnt[kMaxExperts];
+    for (int m = threadIdx.x; m < M; m += 32) s_cnt[m] = 0;
+    __syncwarp();
+    const int t0 = blockIdx.x * kDispatchChunk, t1 = min(T, t0 + kDispatchChunk);
+    for (int t = t0 + threadIdx.x; t < t1; t += 32) {
+        int u = tenant_id[t];
+        if (u < 0 || u >= n_tenants) u = 0;
+        atomicAdd(&s_cnt[model_of_tenant[u]], 1);
+    }
+    __syncwarp();
+    for (int m = threadIdx.x; m < M; m += 32) tok_block_cnt[(size_t)blockIdx.x * M + m] = s_cnt[m];
+}
+
+__global__ void __launch_bounds__(256)
+token_scan_kernel(int nblk, int M, int T, int32_t* __restrict__ tok_block_cnt, int32_t* __restrict__ model_tok_off)
+{
+    __shared__ int32_t s_tot[kMaxExperts];
+    for (int m = threadIdx.x; m < M; m += blockDim.x) {
+        int run = 0;
+        for (int blk = 0; blk < nblk; ++blk) {
+            const int c = tok_block_cnt[(size_t)blk * M + m];
+            tok_block_cnt[(size_t)blk * M + m] = run;
+            run += c;
+        }
+        s_tot[m] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int m = 0; m < M; ++m) { model_tok_off[m] = run; run += s_tot[m]; }
+        model_tok_off[M] = run;
+    }
+}
+
+__global__ void __launch_bounds__(32)
+token_rank_kernel(const int32_t* __restrict__ tenant_id, int T, int n_tenants, int M,
+                  const int32_t* __restrict__ model_of_tenant, const int32_t* __restrict__ tok_block_cnt,
+                  const int32_t* __restrict__ model_tok_off, int32_t* __restrict__ tok_perm,
+                  int32_t* __restrict__ tok_inv)
+{
+    __shared__ int32_t s_next[kMaxExperts];
+    const int lane = threadIdx.x;
+    for (int m = lane; m < M; m += 32) s_next[m] = model_tok_off[m] + tok_block_cnt[(size_t)blockIdx.x * M + m];
+    __syncwarp();
+    const int t0 = blockIdx.x * kDispatchChunk, t1 = min(T, t0 + kDispatchChunk);
+    for (int tt = t0; tt < t1; tt += 32) {
+        const int t = tt + lane;
+        const bool live = t < t1;
+        int key = -1 - lane;
+        if (live) {
+            int u = tenant_id[t];
+            if (u < 0 || u >= n_tenants) u = 0;
+            key = model_of_tenant[u];
+        }
+        const unsigned peers = __match_any_sync(0xffffffffu, key);
+        const int leader = __ffs(peers) - 1;
+        const int rank = __popc(peers & ((1u << lane) - 1u));
+        int start = 0;
+        if (live && lane == leader) { start = s_next[key]; s_next[key] = start + __popc(peers); }
+        start = __shfl_sync(0xffffffffu, start, leader);
+        if (live) { tok_perm[start + rank] = t; tok_inv[t] = start + rank; }
+        __syncwarp();
+    }
+}
+
+BinMap make_binmap(const moe_ctx* c)
+{
+    BinMap bm;
+    bm.model_of_tenant = c->d_model_of_tenant;
+    bm.tenant_local = c->d_tenant_local;
+    bm.bin_base = c->d_bin_base;
+    bm.tenants_in_model = c->d_tenants_in_model;
+    bm.n_tenants = c->cfg.n_tenants;
+    bm.E = c->cfg.n_experts;
+    return bm;
+}
+
+}  // namespace
+
+cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, const int32_t* tenant_id, int T, int G,
+                            int32_t* perm, int32_t* inv_perm, int32_t* tenant_expert_count, int32_t* expert_off,
+                            int32_t* group_off, bf16* x_perm, cudaStream_t st)
+{
+    const moe_config& g = c->cfg;
+    const int k = g.top_k, R = T * k;
+    const int nblk = (R + kDispatchChunk - 1) / kDispatchChunk;
+    const int nbins = c->nbins;
+    const BinMap bm = make_binmap(c);
+    const size_t smem = (size_t)nbins * sizeof(int32_t);
+    dispatch_hist_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, c->ws.block_cnt, c->ws.status);
+    dispatch_scan_kernel<<<1, 1024, smem, st>>>(nblk, nbins, R, g.n_experts, g.n_models, G, g.n_tenants, bm,
+                                                c->ws.block_cnt, c->ws.bin_off, tenant_expert_count, expert_off,
+                                                group_off, c->ws.stats);
+    dispatch_rank_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, c->ws.block_cnt, c->ws.bin_off,
+                                                 perm, inv_perm, c->ws.status);
+    c->launches += 3;
+    if (x_perm) {
+        const int blocks = (R * 32 + 255) / 256;
+        gather_rows_kernel<<<blocks, 256, 0, st>>>(x, perm, R, k, g.hidden, x_perm);
+        c->launches += 1;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_token_sort(moe_ctx* c, const bf16* x, const int32_t* tenant_id, int T, cudaStream_t st)
+{
+    const moe_config& g = c->cfg;
+    const int nblk = (T + kDispatchChunk - 1) / kDispatchChunk;
+    token_hist_kernel<<<nblk, 32, 0, st>>>(tenant_id, T, g.n_tenants, g.n_models, c->d_model_of_tenant,
+                                           c->ws.tok_block_cnt);
+    token_scan_kernel<<<1, 256, 0, st>>>(nblk, g.n_models, T, c->ws.tok_block_cnt, c->ws.model_tok_off);
+    token_rank_kernel<<<nblk, 32, 0, st>>>(tenant_id, T, g.n_tenants, g.n_models, c->d_model_of_tenant,
+                                           c->ws.tok_block_cnt, c->ws.model_tok_off, c->ws.tok_perm, c->ws.tok_inv);
+    const int blocks = (T * 32 + 255) / 256;
+    gather_rows_kernel<<<blocks, 256, 0, st>>>(x, c->ws.tok_perm, T, 1, g.hidden, c->ws.xs_perm);
+    c->launches += 4;
+    return cudaGetLastError();
+}
+
+}  // namespace faasmoe
