@@ -1,0 +1,257 @@
+"""GPU parity: the C-ABI CUDA path against the fp64 CPU oracle, element by element on
+seeded inputs (small and reduced cases), and on sampled tokens at the full sizes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from harness import GpuLayer, assert_close, bf16_to_f64, check_routing, compare_four_calls, oracle_layer
+from paper_2604_26881_b200 import binding as B
+from paper_2604_26881_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+PATHS = [B.MOE_PATH_FMA, B.MOE_PATH_AUTO]
+
+
+@pytest.fixture(scope="module")
+def qwen_weights():
+    return W.make_weights(W.WORKLOADS["prefill"], seed=0)
+
+
+def run_and_compare(wl, wts, x, tenant, mot, G, path, max_tokens=None):
+    g = GpuLayer(wl, [wts], max_tokens or x.shape[0], model_of_tenant=mot)
+    try:
+        B.moe_set_option(g.ctx, B.MOE_OPT_EXPERT_PATH, path)
+        o = g.four_calls(x, tenant, G)
+        ref = oracle_layer(wl, wts, x, tenant, mot, G, o["topk_idx"].cpu().numpy(), o["topk_w"].cpu().numpy())
+        compare_four_calls(o, ref, wl, x)
+        # the fused entry point equals the four calls bit for bit, and is reproducible
+        out1 = g.forward(x, tenant, G)
+        out2 = g.forward(x, tenant, G)
+        assert torch.equal(out1, o["out"]) and torch.equal(out1, out2)
+        return o, ref
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_tiny_config(path):
+    wl = W.WORKLOADS["tiny"]
+    wts = W.make_weights(wl, seed=0)
+    x, tenant, mot = W.make_tokens(wl, seed=0)
+    run_and_compare(wl, wts, x, tenant, mot, wl.G, path)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("G", [1, 5, 12])
+def test_small_multi_model_pool(path, G):
+    # 3 tenant models, 5 tenants, shuffled slot table, router bias, shared expert, G not dividing E,
+    # a row count that spans several dispatch chunks and row tiles with ragged tails
+    wl = W.MoEWorkload("small-pool", T=333, H=256, E=12, I=128, k=3, Is=256, M=3, n_tenants=5, G=G,
+                       zipf_bias=True, tenant_layout="uniform")
+    wts = W.make_weights(wl, seed=3, shuffle_slots=True)
+    x, tenant, mot = W.make_tokens(wl, seed=3)
+    o, ref = run_and_compare(wl, wts, x, tenant, mot, G, path, max_tokens=400)
+    assert ref.dispatch.n_invocations <= 3 * -(-12 // G)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_decode_config(qwen_weights, path):
+    wl = W.WORKLOADS["decode"]
+    wts = dict(qwen_weights, router_bias=None)
+    x, tenant, mot = W.make_tokens(wl, seed=0)
+    o, ref = run_and_compare(wl, wts, x, tenant, mot, wl.G, path)
+    assert 30 <= o["active_experts"] <= 60
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_prefill_reduced(qwen_weights, path):
+    # the prefill layer (Zipf-skewed router) on 300 tokens: every element against the oracle
+    wl = W.scaled(W.WORKLOADS["prefill"], T=300)
+    x, tenant, mot = W.make_tokens(wl, seed=1)
+    run_and_compare(wl, qwen_weights, x, tenant, mot, wl.G, path)
+
+
+def test_prefill_full_size_sampled(qwen_weights):
+    # full 4096-token prefill in the launch configuration the benchmark times: routing and
+    # dispatch compared in full, layer outputs on sampled tokens (tokens are independent, so the
+    # oracle evaluates the sample alone)
+    wl = W.WORKLOADS["prefill"]
+    x, tenant, mot = W.make_tokens(wl, seed=0)
+    g = GpuLayer(wl, [qwen_weights], wl.T, model_of_tenant=mot)
+    try:
+        out = g.forward(x, tenant, wl.G)
+        ws = B.moe_get_workspace(g.ctx)
+        status = B.moe_last_status(g.ctx)
+        assert status[0] == 0
+        T, k, E = wl.T, wl.k, wl.E
+        idx = B.wrap_device_pointer(ws["topk_idx"], (T, k), torch.int32, g.dev).cpu().numpy()
+        wgt = B.wrap_device_pointer(ws["topk_w"], (T, k), torch.float32, g.dev).cpu().numpy()
+        perm = B.wrap_device_pointer(ws["perm"], (T * k,), torch.int32, g.dev).cpu().numpy()
+        inv = B.wrap_device_pointer(ws["inv_perm"], (T * k,), torch.int32, g.dev).cpu().numpy()
+        eoff = B.wrap_device_pointer(ws["expert_off"], (E + 1,), torch.int32, g.dev).cpu().numpy()
+        goff = B.wrap_device_pointer(ws["group_off"], (E // wl.G + 1,), torch.int32, g.dev).cpu().numpy()
+        wn = W.weights_as_numpy(qwen_weights)
+        r = oracle.route(W.as_u16(x), tenant.numpy(), mot.numpy(), wn["router_w"], wn["router_bias"],
+                         wn["shared_gate_w"], k=k)
+        idx_o, mask = check_routing(idx, wgt, r, k)
+        ref_idx = np.where(mask[:, None], idx_o, r.topk_idx)
+        assert np.array_equal(idx, ref_idx)
+        d = oracle.dispatch(ref_idx, tenant.numpy(), mot.numpy(), n_models=1, E=E, G=wl.G)
+        assert np.array_equal(perm, d.perm) and np.array_equal(inv, d.inv_perm)
+        assert np.array_equal(eoff, d.expert_off) and np.array_equal(goff, d.group_off)
+        assert status[1] == d.n_invocations
+        # expert load is skewed as the workload asks
+        load = np.diff(d.expert_off)
+        assert load.max() > 8 * max(1, np.median(load))
+        sample = np.random.default_rng(0).choice(T, 40, replace=False)
+        sample.sort()
+        xs, ts = x[sample].contiguous(), tenant[sample].contiguous()
+        ref = oracle.layer_forward(W.as_u16(xs), ts.numpy(), mot.numpy(), wn, k=k, G=wl.G,
+                                   topk_override=(idx[sample], np.ones(len(sample), bool)))
+        assert_close("out[sample]", bf16_to_f64(out[sample]), ref.out)
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_pool_config_reduced_and_G_sweep(path):
+    # 4 tenant models in one pool, top-4 inside each tenant's own experts, uniform tenant ids
+    wl = W.scaled(W.WORKLOADS["pool"], T=192, H=512, I=256, Is=512, E=60)
+    wts = W.make_weights(wl, seed=5, shuffle_slots=True)
+    x, tenant, mot = W.make_tokens(wl, seed=5)
+    o, ref = run_and_compare(wl, wts, x, tenant, mot, 1, path)
+    g = GpuLayer(wl, [wts], wl.T, model_of_tenant=mot)
+    try:
+        B.moe_set_option(g.ctx, B.MOE_OPT_EXPERT_PATH, path)
+        base = g.forward(x, tenant, 1)
+        assert torch.equal(base, o["out"])
+        invocations = []
+        for G in (1, 2, 4, 6, 12, 60):
+            out = g.forward(x, tenant, G)
+            assert torch.equal(out, base), f"output changed with G={G}"      # bit-identical for every G
+            invocations.append(B.moe_last_status(g.ctx)[1])
+        assert invocations == sorted(invocations, reverse=True) and invocations[-1] == 4
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_stack_teacher_forced(path):
+    # 3 blocks of RMSNorm -> MoE (+shared) -> residual; ragged multi-tenant batch
+    wl = W.scaled(W.WORKLOADS["stack"], H=512, I=256, Is=512, E=24, n_layers=3, n_tenants=6)
+    layers = [W.make_weights(wl, seed=7, layer=l) for l in range(wl.n_layers)]
+    x, tenant, mot = W.make_tokens(wl, seed=7)
+    x, tenant = x[:700].contiguous(), tenant[:700].contiguous()
+    T = x.shape[0]
+    g = GpuLayer(wl, layers, T, model_of_tenant=mot)
+    try:
+        B.moe_set_option(g.ctx, B.MOE_OPT_EXPERT_PATH, path)
+        xd, td = x.to(g.dev).clone(), tenant.to(g.dev)
+        dbg_in = torch.zeros((wl.n_layers, T, wl.H), dtype=torch.bfloat16, device=g.dev)
+        dbg_out = torch.zeros_like(dbg_in)
+        B.moe_stack_forward(g.ctx, xd, td, T, wl.G, dbg_in, dbg_out)
+        torch.cuda.synchronize()
+        assert B.moe_last_status(g.ctx)[0] == 0
+        assert torch.equal(dbg_out[-1], xd)
+        # teacher forcing: block l of the oracle starts from the GPU's residual stream and the GPU's
+        # normalised input, so every block is compared on identical inputs
+        x_in = x
+        for l in range(wl.n_layers):
+            wn = W.weights_as_numpy(layers[l])
+            xn_ref = oracle.rmsnorm(W.as_u16(x_in), wn["rms_w"], wl.rms_eps)
+            xn_gpu = dbg_in[l].cpu()
+            ulp = 2.0 ** (np.floor(np.log2(np.abs(xn_ref) + 1e-300)) - 7)      # spacing of bf16 at each value
+            err = np.abs(bf16_to_f64(xn_gpu) - xn_ref) / ulp
+            assert err.max() <= 1.0, f"block {l}: RMSNorm differs by {err.max()} bf16 ulp"
+            # the gate alone on the GPU's xn, to apply the near-tie protocol to this block
+            tk_i = torch.zeros((T, wl.k), dtype=torch.int32, device=g.dev)
+            tk_w = torch.zeros((T, wl.k), dtype=torch.float32, device=g.dev)
+            B.moe_route(g.ctx, l, dbg_in[l], td, T, tk_i, tk_w)
+            torch.cuda.synchronize()
+            r = oracle.route(W.as_u16(xn_gpu), tenant.numpy(), mot.numpy(), wn["router_w"], wn["router_bias"],
+                             wn["shared_gate_w"], k=wl.k)
+            ov = check_routing(tk_i.cpu().numpy(), tk_w.cpu().numpy(), r, wl.k)
+            _, _, res = oracle.block_forward(W.as_u16(x_in), tenant.numpy(), mot.numpy(), wn, k=wl.k, G=wl.G,
+                                             eps=wl.rms_eps, xn_override=W.as_u16(xn_gpu), topk_override=ov)
+            assert_close(f"block {l} residual stream", bf16_to_f64(dbg_out[l]), bf16_to_f64(x_in) + res.out)
+            x_in = dbg_out[l].cpu()
+        # the stack without debug buffers gives the same bits
+        xd2 = x.to(g.dev).clone()
+        B.moe_stack_forward(g.ctx, xd2, td, T, wl.G)
+        torch.cuda.synchronize()
+        assert torch.equal(xd2, xd)
+    finally:
+        g.close()
+
+
+def test_host_entry_point_matches_device_entry_point():
+    wl = W.WORKLOADS["tiny"]
+    wts = W.make_weights(wl, seed=0)
+    x, tenant, mot = W.make_tokens(wl, seed=0)
+    g = GpuLayer(wl, [wts], wl.T, model_of_tenant=mot)
+    try:
+        assert torch.equal(g.forward_host(x, tenant, 1), g.forward(x, tenant, 1).cpu())
+    finally:
+        g.close()
+
+
+def test_edge_cases_and_errors():
+    wl = W.MoEWorkload("edge", T=5, H=256, E=8, I=128, k=2, Is=128, M=1, n_tenants=3)
+    wts = W.make_weights(wl, seed=9)
+    x, tenant, mot = W.make_tokens(wl, seed=9)
+    g = GpuLayer(wl, [wts], 64, model_of_tenant=mot)
+    try:
+        dev = g.dev
+        out = torch.zeros((5, wl.H), dtype=torch.bfloat16, device=dev)
+        xd, td = x.to(dev), tenant.to(dev)
+        # T = 0 is a no-op
+        B.moe_layer_forward(g.ctx, 0, xd, td, 0, 1, out)
+        # a single token
+        one = g.forward(x[:1].contiguous(), tenant[:1].contiguous(), 1)
+        full = g.forward(x, tenant, 1)
+        assert torch.equal(one[0], full[0])
+        ref = oracle_layer(wl, wts, x, tenant, mot, 1)
+        assert_close("edge out", bf16_to_f64(full), ref.out)
+        # host-detectable errors launch nothing
+        n0 = B.moe_launch_count(g.ctx)
+        for G in (0, wl.E + 1):
+            with pytest.raises(B.MoeError) as e:
+                B.moe_layer_forward(g.ctx, 0, xd, td, 5, G, out)
+            assert e.value.status == B.MOE_ERR_G
+        with pytest.raises(B.MoeError) as e:
+            B.moe_layer_forward(g.ctx, 0, xd, td, 65, 1, out)
+        assert e.value.status == B.MOE_ERR_SHAPE
+        with pytest.raises(B.MoeError) as e:
+            B.moe_layer_forward(g.ctx, 1, xd, td, 5, 1, out)
+        assert e.value.status == B.MOE_ERR_SHAPE
+        with pytest.raises(B.MoeError) as e:
+            B.moe_layer_forward(g.ctx, 0, None, td, 5, 1, out)
+        assert e.value.status == B.MOE_ERR_NULL
+        assert B.moe_launch_count(g.ctx) == n0
+        # an out-of-range tenant id is reported through the status word; that token's output is zero
+        bad = tenant.clone(); bad[2] = 7
+        outb = g.forward(x, bad, 1)
+        st = B.moe_last_status(g.ctx)[0]
+        assert st & B.MOE_DEV_BAD_TENANT
+        assert torch.count_nonzero(outb[2]) == 0
+        keep = [0, 1, 3, 4]
+        assert torch.equal(outb[keep], full[keep])
+        assert B.moe_last_status(g.ctx)[0] == 0          # cleared by the read
+    finally:
+        g.close()
+    # weights not set -> MOE_ERR_STATE
+    ctx = B.moe_create(hidden=256, n_experts=8, inter=128, top_k=2, max_tokens=8)
+    try:
+        t = torch.zeros((8, 256), dtype=torch.bfloat16, device="cuda")
+        with pytest.raises(B.MoeError) as e:
+            B.moe_layer_forward(ctx, 0, t, torch.zeros(8, dtype=torch.int32, device="cuda"), 8, 1, t)
+        assert e.value.status == B.MOE_ERR_STATE
+    finally:
+        B.moe_destroy(ctx)
+    for kw in (dict(hidden=250), dict(top_k=9), dict(n_experts=0), dict(inter=100)):
+        args = dict(hidden=256, n_experts=8, inter=128, top_k=2, max_tokens=8)
+        args.update(kw)
+        with pytest.raises(B.MoeError):
+            B.moe_create(**args)
