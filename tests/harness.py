@@ -19,6 +19,12 @@ from paper_2604_26881_b200 import workloads as W
 
 RTOL, ATOL = 2e-2, 2e-3
 W_RTOL = 1e-4          # router weights: fp32 softmax against fp64
+# Un-gated, un-weighted expert outputs (y_perm, y_shared) are intermediates of magnitude ~0.4-0.7
+# that the layer output scales by p ~ 0.1 or the gate ~ 0.5.  Their error is dominated by the bf16
+# rounding of the SwiGLU activations h: each of the I (or I_s) terms of a down-projection carries a
+# relative error of std 2^-9/sqrt(3), which sums to an absolute std of about 4e-4 (I = 1408) or
+# 8e-4 (I_s = 5632) whatever the size of the result.  6e-3 is seven of the larger sigmas.
+INTERMEDIATE_ATOL = 6e-3
 
 
 def bf16_to_f64(t: torch.Tensor) -> np.ndarray:
@@ -169,7 +175,7 @@ def compare_four_calls(o: dict, ref, wl, x: torch.Tensor):
     xp = o["x_perm"].cpu().view(torch.int16).numpy()
     xs = x.view(torch.int16).numpy()
     assert np.array_equal(xp, xs[d.perm // k])
-    assert_close("y_perm", bf16_to_f64(o["y_perm"]), ref.y_perm)
+    assert_close("y_perm", bf16_to_f64(o["y_perm"]), ref.y_perm, atol=INTERMEDIATE_ATOL)
     if wl.Is:
-        assert_close("y_shared", bf16_to_f64(o["y_shared"]), ref.y_shared)
+        assert_close("y_shared", bf16_to_f64(o["y_shared"]), ref.y_shared, atol=INTERMEDIATE_ATOL)
     assert_close("out", bf16_to_f64(o["out"]), ref.out)
