@@ -59,7 +59,12 @@ int alloc_workspace(moe_ctx* c)
     // activations: one extra tile of rows so that a whole-tile load never leaves the buffer
     A(&w.x_perm, (R + kTileRows) * H); A(&w.h, (R + kTileRows) * I); A(&w.y_perm, R * H);
     if (g.n_models > 1) A(&w.xs_perm, (T + kTileRows) * H);
-    if (Is > 0) { A(&w.hs, (T + kTileRows) * Is); A(&w.y_shared, T * H); }
+    if (Is > 0) {
+        bf16* hs16 = nullptr;                       // same element size as fp16
+        A(&hs16, (T + kTileRows) * Is);
+        w.hs = hs16;
+        A(&w.y_shared, T * H);
+    }
     A(&w.xn, (T + kTileRows) * H);
     A(&w.x_stage, (T + kTileRows) * H); A(&w.tenant_stage, T); A(&w.out_stage, T * H);
     A(&w.status, 1); A(&w.stats, 4);

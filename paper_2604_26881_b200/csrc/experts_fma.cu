@@ -1,6 +1,8 @@
 // CUDA-core expert execution: the plain, tile-wise SwiGLU FFN used for shapes the tensor-core
 // path does not cover and as the A/B reference of that path.  (Paper Sec. 3: an expert block
 // performs stateless computation on its assigned tokens; only activated experts are touched.)
+#include <cuda_fp16.h>
+
 #include "internal.h"
 
 namespace faasmoe {
@@ -15,6 +17,20 @@ __device__ __forceinline__ float warp_sum_f(float v)
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
+}
+
+// weights bf16, activations fp16 (the shared expert's SwiGLU activations, see launch_experts_fma)
+__device__ __forceinline__ void fma8_half(const uint4& w, const uint4& a, float& acc)
+{
+    const __nv_bfloat162* pw = reinterpret_cast<const __nv_bfloat162*>(&w);
+    const __half2* pa = reinterpret_cast<const __half2*>(&a);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 fw = __bfloat1622float2(pw[i]);
+        const float2 fa = __half22float2(pa[i]);
+        acc = fmaf(fw.x, fa.x, acc);
+        acc = fmaf(fw.y, fa.y, acc);
+    }
 }
 
 __device__ __forceinline__ void fma8(const uint4& w, const uint4& a, float& acc)
@@ -32,10 +48,11 @@ __device__ __forceinline__ void fma8(const uint4& w, const uint4& a, float& acc)
 
 // out[dst(r), c] = epi( W0[c,:] . act[r,:], W1[c,:] . act[r,:] ) for the rows r of one tile and
 // 64 weight rows c.  SWIGLU: epi = silu(a) * b; otherwise epi = a (W1 unused).
+// The shared expert's intermediate (SWIGLU && SHARED output, !SWIGLU && SHARED input) is fp16.
 template <bool SWIGLU, bool SHARED>
 __global__ void __launch_bounds__(256)
 ffn_fma_kernel(const Tile* __restrict__ tiles, const int32_t* __restrict__ n_tiles_ptr, const bf16* __restrict__ act,
-               int K, int ncols, PoolWeights pool, const ModelWeights* __restrict__ models, bf16* __restrict__ out,
+               int K, int ncols, PoolWeights pool, const ModelWeights* __restrict__ models, void* __restrict__ out_raw,
                int ld_out, const int32_t* __restrict__ dst_rows)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -81,7 +98,8 @@ ffn_fma_kernel(const Tile* __restrict__ tiles, const int32_t* __restrict__ n_til
 #pragma unroll
                 for (int r = 0; r < kRowsPerPass; ++r) {
                     const uint4 xv = reinterpret_cast<const uint4*>(a_s)[r * kv + v];
-                    fma8(a, xv, acc0[r]);
+                    if (!SWIGLU && SHARED) fma8_half(a, xv, acc0[r]);
+                    else fma8(a, xv, acc0[r]);
                     if (SWIGLU) fma8(b, xv, acc1[r]);
                 }
             }
@@ -93,7 +111,8 @@ ffn_fma_kernel(const Tile* __restrict__ tiles, const int32_t* __restrict__ n_til
                     const float val = SWIGLU ? (s0 / (1.f + expf(-s0))) * s1 : s0;
                     const int row = tile.row0 + r0 + r;
                     const int drow = dst_rows ? dst_rows[row] : row;
-                    out[(size_t)drow * ld_out + c] = __float2bfloat16_rn(val);
+                    if (SWIGLU && SHARED) reinterpret_cast<__half*>(out_raw)[(size_t)drow * ld_out + c] = __float2half_rn(val);
+                    else reinterpret_cast<bf16*>(out_raw)[(size_t)drow * ld_out + c] = __float2bfloat16_rn(val);
                 }
             }
         }
@@ -140,7 +159,7 @@ cudaError_t launch_experts_fma(moe_ctx* c, int layer, const bf16* x_or_xs, const
                                                           nullptr);
     if (shared) {
         dim3 gs2(c->max_stiles, (H + kColsPerBlock - 1) / kColsPerBlock);
-        ffn_fma_kernel<false, true><<<gs2, 256, smem_is, st>>>(c->ws.stiles, n_tiles + 1, c->ws.hs, Is, H, pool, models,
+        ffn_fma_kernel<false, true><<<gs2, 256, smem_is, st>>>(c->ws.stiles, n_tiles + 1, (const bf16*)c->ws.hs, Is, H, pool, models,
                                                                y_shared, H, shared_dst_rows);
     }
     stage_mark(c, st, kEvDown);

@@ -83,7 +83,9 @@ struct Workspace {
     bf16* x_perm = nullptr;        // [R,H]
     bf16* xs_perm = nullptr;       // [T,H] tokens grouped by model (M > 1 only)
     bf16* h = nullptr;             // [R,I]
-    bf16* hs = nullptr;            // [T,Is]
+    void* hs = nullptr;            // [T,Is] fp16: SwiGLU activations of the shared expert.  fp16 rather than
+                                   // bf16 because the 4x wider down-projection sums 4x more rounding errors and
+                                   // the gated result enters the output with a weight of ~0.5 instead of ~0.1
     bf16* y_perm = nullptr;        // [R,H]
     bf16* y_shared = nullptr;      // [T,H]
     bf16* xn = nullptr;            // [T,H] normalised input of a block (stack)
