@@ -149,24 +149,28 @@ int moe_dispatch(moe_ctx* ctx, const void* x, const int32_t* topk_idx, const int
 /*
  * Expert execution (Sec. 3: each expert block performs stateless computation on its
  * assigned tokens).  Only experts that received rows are touched.
- *   y_perm[r'] = FFN_{slot(m,e)}(x_perm[r'])    for r' in expert (m,e)'s segment   bf16 [T*k, H]
- *   y_shared[t] = FFN_shared,m(x[t])  (ungated)                                    bf16 [T, H] or NULL
+ *   y_perm[r'] = FFN_{slot(m,e)}(x_perm[r'])    for r' in expert (m,e)'s segment   f32 [T*k, H]
+ *   y_shared[t] = FFN_shared,m(x[t])  (ungated)                                    f32 [T, H] or NULL
+ * (bf16 operands, fp32 accumulation; the SwiGLU activations are rounded to bf16 for the
+ * routed experts and to fp16 for the shared expert before the down projection; the
+ * results stay in fp32 so that the aggregation rounds only once)
  * G orders the work by expert block; results are bit-identical for every G.
  * x bf16 [T,H] and tenant_id are needed only when y_shared is requested.
  * x_perm must be readable for 128 rows past T*k (the tensor-core path loads whole
  * row tiles; what lies there is never used).
  */
 int moe_experts(moe_ctx* ctx, int layer, const void* x, const void* x_perm, const int32_t* expert_off,
-                const int32_t* tenant_id, int T, int G, void* y_perm, void* y_shared, void* stream);
+                const int32_t* tenant_id, int T, int G, float* y_perm, float* y_shared, void* stream);
 
 /*
  * Aggregation (Sec. 3, Sec. 4.2):
  *   out[t] = sum_{j=0..k-1} topk_w[t,j] * y_perm[inv_perm[t*k+j]] + shared_gate[t] * y_shared[t]
- * accumulated in fp32 in that fixed order, rounded once to bf16.  out bf16 [T,H].
+ * accumulated in fp32 in that fixed order, rounded once to bf16.  y_perm f32 [T*k,H],
+ * y_shared f32 [T,H], out bf16 [T,H].
  * y_shared / shared_gate may both be NULL.
  */
-int moe_combine(moe_ctx* ctx, const void* y_perm, const int32_t* inv_perm, const float* topk_w,
-                const void* y_shared, const float* shared_gate, int T, void* out, void* stream);
+int moe_combine(moe_ctx* ctx, const float* y_perm, const int32_t* inv_perm, const float* topk_w,
+                const float* y_shared, const float* shared_gate, int T, void* out, void* stream);
 
 /* route -> dispatch -> experts -> combine on the context's workspace; bit-identical to
  * the four calls above.  out bf16 [T,H]. */

@@ -124,7 +124,7 @@ bool use_tc(const moe_ctx* c)
 }
 
 int experts_impl(moe_ctx* c, int layer, const bf16* x, const bf16* x_perm, const int32_t* expert_off,
-                 const int32_t* tenant_id, int T, int G, bf16* y_perm, bf16* y_shared, cudaStream_t st)
+                 const int32_t* tenant_id, int T, int G, float* y_perm, float* y_shared, cudaStream_t st)
 {
     const moe_config& g = c->cfg;
     const bool with_shared = y_shared != nullptr && g.shared_inter > 0;
@@ -345,7 +345,7 @@ int moe_dispatch(moe_ctx* c, const void* x, const int32_t* topk_idx, const int32
 }
 
 int moe_experts(moe_ctx* c, int layer, const void* x, const void* x_perm, const int32_t* expert_off,
-                const int32_t* tenant_id, int T, int G, void* y_perm, void* y_shared, void* stream)
+                const int32_t* tenant_id, int T, int G, float* y_perm, float* y_shared, void* stream)
 {
     if (!c || !x_perm || !expert_off || !y_perm) return MOE_ERR_NULL;
     if (y_shared && (!x || !tenant_id)) return MOE_ERR_NULL;
@@ -354,18 +354,18 @@ int moe_experts(moe_ctx* c, int layer, const void* x, const void* x_perm, const 
     const int rc = check_layer_ready(c, layer, true, y_shared != nullptr);
     if (rc != MOE_OK) return rc;
     if (T == 0) return MOE_OK;
-    return experts_impl(c, layer, (const bf16*)x, (const bf16*)x_perm, expert_off, tenant_id, T, G, (bf16*)y_perm,
-                        (bf16*)y_shared, (cudaStream_t)stream);
+    return experts_impl(c, layer, (const bf16*)x, (const bf16*)x_perm, expert_off, tenant_id, T, G, (float*)y_perm,
+                        (float*)y_shared, (cudaStream_t)stream);
 }
 
-int moe_combine(moe_ctx* c, const void* y_perm, const int32_t* inv_perm, const float* topk_w, const void* y_shared,
+int moe_combine(moe_ctx* c, const float* y_perm, const int32_t* inv_perm, const float* topk_w, const float* y_shared,
                 const float* shared_gate, int T, void* out, void* stream)
 {
     if (!c || !y_perm || !inv_perm || !topk_w || !out) return MOE_ERR_NULL;
     if ((y_shared == nullptr) != (shared_gate == nullptr)) return MOE_ERR_NULL;
     if (T < 0 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
     if (T == 0) return MOE_OK;
-    MOE_CUDA(c, launch_combine(c, (const bf16*)y_perm, inv_perm, topk_w, (const bf16*)y_shared, shared_gate, nullptr,
+    MOE_CUDA(c, launch_combine(c, (const float*)y_perm, inv_perm, topk_w, (const float*)y_shared, shared_gate, nullptr,
                                T, (bf16*)out, (cudaStream_t)stream));
     return MOE_OK;
 }

@@ -18,6 +18,13 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f)
     }
 }
 
+__device__ __forceinline__ void load8(const float* p, float* f)
+{
+    const float4 a = reinterpret_cast<const float4*>(p)[0], b = reinterpret_cast<const float4*>(p)[1];
+    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w;
+    f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+}
+
 __device__ __forceinline__ uint4 pack8(const float* f)
 {
     uint4 v;
@@ -31,8 +38,8 @@ __device__ __forceinline__ uint4 pack8(const float* f)
 // (fp32, fixed order: residual, j = 0..k-1, shared), one rounding to bf16.
 // One thread per 8 consecutive features.
 __global__ void __launch_bounds__(256)
-combine_kernel(const bf16* __restrict__ y_perm, const int32_t* __restrict__ inv_perm, const float* __restrict__ topk_w,
-               const bf16* __restrict__ y_shared, const float* __restrict__ shared_gate,
+combine_kernel(const float* __restrict__ y_perm, const int32_t* __restrict__ inv_perm, const float* __restrict__ topk_w,
+               const float* __restrict__ y_shared, const float* __restrict__ shared_gate,
                const bf16* residual, int T, int H, int k, bf16* out)
 {
     const int hv = H >> 3;
@@ -46,13 +53,13 @@ combine_kernel(const bf16* __restrict__ y_perm, const int32_t* __restrict__ inv_
     for (int j = 0; j < k; ++j) {
         const int r = inv_perm[(size_t)t * k + j];
         const float w = topk_w[(size_t)t * k + j];
-        unpack8(reinterpret_cast<const uint4*>(y_perm + (size_t)r * H)[v], tmp);
+        load8(y_perm + (size_t)r * H + 8 * v, tmp);
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, tmp[i], acc[i]);
     }
     if (y_shared) {
         const float s = shared_gate[t];
-        unpack8(reinterpret_cast<const uint4*>(y_shared + (size_t)t * H)[v], tmp);
+        load8(y_shared + (size_t)t * H + 8 * v, tmp);
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = fmaf(s, tmp[i], acc[i]);
     }
@@ -93,8 +100,8 @@ rmsnorm_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ tenant_id
 
 }  // namespace
 
-cudaError_t launch_combine(moe_ctx* c, const bf16* y_perm, const int32_t* inv_perm, const float* topk_w,
-                           const bf16* y_shared, const float* shared_gate, const bf16* residual, int T, bf16* out,
+cudaError_t launch_combine(moe_ctx* c, const float* y_perm, const int32_t* inv_perm, const float* topk_w,
+                           const float* y_shared, const float* shared_gate, const bf16* residual, int T, bf16* out,
                            cudaStream_t st)
 {
     const moe_config& g = c->cfg;

@@ -111,8 +111,10 @@ ffn_fma_kernel(const Tile* __restrict__ tiles, const int32_t* __restrict__ n_til
                     const float val = SWIGLU ? (s0 / (1.f + expf(-s0))) * s1 : s0;
                     const int row = tile.row0 + r0 + r;
                     const int drow = dst_rows ? dst_rows[row] : row;
-                    if (SWIGLU && SHARED) reinterpret_cast<__half*>(out_raw)[(size_t)drow * ld_out + c] = __float2half_rn(val);
-                    else reinterpret_cast<bf16*>(out_raw)[(size_t)drow * ld_out + c] = __float2bfloat16_rn(val);
+                    const size_t o = (size_t)drow * ld_out + c;
+                    if (!SWIGLU) reinterpret_cast<float*>(out_raw)[o] = val;                       // y: fp32
+                    else if (SHARED) reinterpret_cast<__half*>(out_raw)[o] = __float2half_rn(val);  // hs: fp16
+                    else reinterpret_cast<bf16*>(out_raw)[o] = __float2bfloat16_rn(val);            // h: bf16
                 }
             }
         }
@@ -121,8 +123,8 @@ ffn_fma_kernel(const Tile* __restrict__ tiles, const int32_t* __restrict__ n_til
 
 }  // namespace
 
-cudaError_t launch_experts_fma(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, bf16* y_perm,
-                               bf16* y_shared, const int32_t* shared_dst_rows, cudaStream_t st)
+cudaError_t launch_experts_fma(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, float* y_perm,
+                               float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st)
 {
     const moe_config& g = c->cfg;
     const PoolWeights pool = c->pools[layer];

@@ -9,7 +9,7 @@ bool tc_supported(const moe_ctx*) { return false; }
 int tc_setup_layer(moe_ctx*, int) { return MOE_ERR_UNSUPPORTED; }
 void tc_destroy(moe_ctx*) {}
 
-cudaError_t launch_experts_tc(moe_ctx*, int, const bf16*, const bf16*, int, bf16*, bf16*, const int32_t*, cudaStream_t)
+cudaError_t launch_experts_tc(moe_ctx*, int, const bf16*, const bf16*, int, float*, float*, const int32_t*, cudaStream_t)
 {
     return cudaErrorNotSupported;
 }

@@ -86,8 +86,8 @@ struct Workspace {
     void* hs = nullptr;            // [T,Is] fp16: SwiGLU activations of the shared expert.  fp16 rather than
                                    // bf16 because the 4x wider down-projection sums 4x more rounding errors and
                                    // the gated result enters the output with a weight of ~0.5 instead of ~0.1
-    bf16* y_perm = nullptr;        // [R,H]
-    bf16* y_shared = nullptr;      // [T,H]
+    float* y_perm = nullptr;       // [R,H] fp32: un-weighted expert outputs; kept in fp32 because the combine
+    float* y_shared = nullptr;     // [T,H]       adds terms of opposite sign and bf16 rounding would not cancel
     bf16* xn = nullptr;            // [T,H] normalised input of a block (stack)
     // staging of the host-buffer entry point
     bf16* x_stage = nullptr;       // [T,H]
@@ -151,14 +151,14 @@ cudaError_t launch_token_sort(moe_ctx* c, const bf16* x, const int32_t* tenant_i
 // Builds the tile lists (and the unit lists of the tensor-core path) from expert_off.
 cudaError_t launch_plan(moe_ctx* c, const int32_t* expert_off, int T, int G, bool with_shared, cudaStream_t st);
 
-cudaError_t launch_experts_fma(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, bf16* y_perm,
-                               bf16* y_shared, const int32_t* shared_dst_rows, cudaStream_t st);
+cudaError_t launch_experts_fma(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, float* y_perm,
+                               float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st);
 
-cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, bf16* y_perm,
-                              bf16* y_shared, const int32_t* shared_dst_rows, cudaStream_t st);
+cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, float* y_perm,
+                              float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st);
 
-cudaError_t launch_combine(moe_ctx* c, const bf16* y_perm, const int32_t* inv_perm, const float* topk_w,
-                           const bf16* y_shared, const float* shared_gate, const bf16* residual, int T, bf16* out,
+cudaError_t launch_combine(moe_ctx* c, const float* y_perm, const int32_t* inv_perm, const float* topk_w,
+                           const float* y_shared, const float* shared_gate, const bf16* residual, int T, bf16* out,
                            cudaStream_t st);
 
 cudaError_t launch_rmsnorm(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, bf16* xn,

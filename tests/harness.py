@@ -68,8 +68,8 @@ class GpuLayer:
             "group_off": torch.full((M * Bn + 1,), -7, dtype=torch.int32, device=dev),
             # one spare tile of rows: the tensor-core path reads whole row tiles
             "x_perm": torch.zeros((R + 128, H), dtype=torch.bfloat16, device=dev),
-            "y_perm": torch.zeros((R, H), dtype=torch.bfloat16, device=dev),
-            "y_shared": torch.zeros((T, H), dtype=torch.bfloat16, device=dev) if wl.Is else None,
+            "y_perm": torch.zeros((R, H), dtype=torch.float32, device=dev),
+            "y_shared": torch.zeros((T, H), dtype=torch.float32, device=dev) if wl.Is else None,
             "out": torch.zeros((T, H), dtype=torch.bfloat16, device=dev),
         }
         B.moe_route(self.ctx, layer, xd, td, T, o["topk_idx"], o["topk_w"], o["shared_gate"] if wl.Is else None,
