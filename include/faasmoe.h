@@ -172,6 +172,40 @@ int moe_experts(moe_ctx* ctx, int layer, const void* x, const void* x_perm, cons
 int moe_combine(moe_ctx* ctx, const float* y_perm, const int32_t* inv_perm, const float* topk_w,
                 const float* y_shared, const float* shared_gate, int T, void* out, void* stream);
 
+/*
+ * moe_dispatch for callers that must not allocate device memory (the paper has no
+ * counterpart; this is a convenience of this library).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a host application
+ * whose device memory pool is fixed at start-up, on a latency-critical path that cannot
+ * afford cudaMalloc's implicit synchronisation, or in a process that already spent its
+ * memory budget.  Such a caller cannot use moe_create either (it allocates the workspace),
+ * so this call takes no context: the shapes and the tenant -> model table are arguments, and
+ * the scratch the dispatch kernels need lives in a fixed array of
+ * MOE_DISPATCH_NOALLOC_MAX_WORDS 32-bit words (1 MiB) inside the library, held by every GPU
+ * that loads the library until the process exits.  The call itself and everything it
+ * launches call no cudaMalloc, cudaFree or allocating library routine.
+ *
+ * Inputs and outputs are those of moe_dispatch (device pointers, same layouts and meaning,
+ * without x / x_perm): topk_idx int32 [T,k], tenant_id int32 [T], model_of_tenant int32
+ * [n_tenants] (DEVICE; an entry outside [0, M) counts as model 0), perm / inv_perm int32 [T*k], tenant_expert_count int32
+ * [n_tenants*E] or NULL, expert_off int32 [M*E+1], group_off int32 [M*ceil(E/G)+1] or NULL.
+ * status_out, if not NULL, is a device int32 that receives the MOE_DEV_* bits of this call
+ * (it is cleared first).
+ *
+ * Limit: 10 + 2*n_tenants + 2*M + (ceil(T*k/256) + 1) * E*n_tenants words must fit in the
+ * array; larger problems return MOE_ERR_UNSUPPORTED and launch nothing.
+ * The first call on each device looks up the array's device address; make that first call
+ * before any stream capture.  All calls on a device share the array and it keeps the last
+ * call's contents (what must start at zero is cleared by the call itself): two calls that
+ * overlap on the GPU -- different streams, or different host threads -- race on it.
+ */
+#define MOE_DISPATCH_NOALLOC_MAX_WORDS (1 << 18)
+int moe_dispatch_noalloc(const int32_t* topk_idx, const int32_t* tenant_id, const int32_t* model_of_tenant,
+                         int T, int k, int E, int M, int n_tenants, int G, int32_t* perm, int32_t* inv_perm,
+                         int32_t* tenant_expert_count, int32_t* expert_off, int32_t* group_off,
+                         int32_t* status_out, void* stream);
+
 /* route -> dispatch -> experts -> combine on the context's workspace; bit-identical to
  * the four calls above.  out bf16 [T,H]. */
 int moe_layer_forward(moe_ctx* ctx, int layer, const void* x, const int32_t* tenant_id, int T, int G,

@@ -26,7 +26,8 @@ MOE_PATH_AUTO, MOE_PATH_FMA, MOE_PATH_TCGEN05 = 0, 1, 2
 EXPORTS = ["moe_create", "moe_destroy", "moe_set_expert_pool", "moe_set_model_weights", "moe_set_slot_table",
            "moe_set_tenant_models", "moe_set_option", "moe_route", "moe_dispatch", "moe_experts", "moe_combine",
            "moe_layer_forward", "moe_layer_forward_host", "moe_layer_forward_timed", "moe_stack_forward",
-           "moe_get_workspace", "moe_last_status", "moe_launch_count", "moe_strerror"]
+           "moe_get_workspace", "moe_last_status", "moe_launch_count", "moe_strerror", "moe_dispatch_noalloc"]
+MOE_DISPATCH_NOALLOC_MAX_WORDS = 1 << 18
 
 STAGES = ["route", "dispatch", "plan", "experts_gateup", "experts_down", "combine"]
 
@@ -77,6 +78,7 @@ def load_library(path: str | None = None):
         lib.moe_layer_forward_timed.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int, c_int, c_void_p,
                                                 POINTER(c_float), c_void_p]
         lib.moe_stack_forward.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p]
+        lib.moe_dispatch_noalloc.argtypes = [c_void_p] * 3 + [c_int] * 6 + [c_void_p] * 7
         lib.moe_get_workspace.argtypes = [c_void_p] + [POINTER(c_void_p)] * 8
         lib.moe_last_status.argtypes = [c_void_p, POINTER(c_int32), POINTER(c_int32)]
         _lib = lib
@@ -155,6 +157,15 @@ def moe_dispatch(ctx, x, topk_idx, tenant_id, T, G, perm, inv_perm, tenant_exper
     _check("moe_dispatch", load_library().moe_dispatch(
         ctx, _ptr(x), _ptr(topk_idx), _ptr(tenant_id), T, G, _ptr(perm), _ptr(inv_perm), _ptr(tenant_expert_count),
         _ptr(expert_off), _ptr(group_off), _ptr(x_perm), _stream(stream)))
+
+
+def moe_dispatch_noalloc(topk_idx, tenant_id, model_of_tenant, T, k, E, M, n_tenants, G, perm, inv_perm,
+                         tenant_expert_count=None, expert_off=None, group_off=None, status_out=None, stream=None):
+    """moe_dispatch without a context and without any allocation inside the library: for callers that
+    may not call cudaMalloc.  model_of_tenant is a DEVICE tensor here.  See include/faasmoe.h."""
+    _check("moe_dispatch_noalloc", load_library().moe_dispatch_noalloc(
+        _ptr(topk_idx), _ptr(tenant_id), _ptr(model_of_tenant), T, k, E, M, n_tenants, G, _ptr(perm), _ptr(inv_perm),
+        _ptr(tenant_expert_count), _ptr(expert_off), _ptr(group_off), _ptr(status_out), _stream(stream)))
 
 
 def moe_experts(ctx, layer, x, x_perm, expert_off, tenant_id, T, G, y_perm, y_shared=None, stream=None):

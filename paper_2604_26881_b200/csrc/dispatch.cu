@@ -3,6 +3,8 @@
 // routing requests"; Sec. 4.1: all tokens routed to the same expert block become one batched
 // invocation).  Rows are ordered by (model, expert, tenant, token); the order is produced
 // without order-dependent atomics so that the permutation is reproducible bit for bit.
+#include <mutex>
+
 #include "internal.h"
 
 namespace faasmoe {
@@ -297,3 +299,122 @@ cudaError_t launch_token_sort(moe_ctx* c, const bf16* x, const int32_t* tenant_i
 }
 
 }  // namespace faasmoe
+
+
+// ---------------------------------------------------------------------------------------------
+// Dispatch without any allocation.
+//
+// Some callers may not allocate device memory: a plug-in that runs inside a host application
+// whose memory pool is fixed at start-up, code on a latency-critical path where cudaMalloc's
+// implicit device synchronisation is not acceptable, or a process that has been told to stay
+// inside a memory budget it already spent.  Such callers cannot create a moe_ctx either, because
+// moe_create allocates the workspace.  For them the scratch of the dispatch kernels (per-block
+// histograms, bin offsets, the tenant tables derived from model_of_tenant, the statistics and
+// the status word) lives in the fixed array below, which every GPU that loads this library
+// holds until the process exits.
+// ---------------------------------------------------------------------------------------------
+
+namespace faasmoe {
+namespace {
+
+constexpr int kNoAllocWords = MOE_DISPATCH_NOALLOC_MAX_WORDS;
+static __device__ __align__(256) int32_t g_dispatch_scratch[kNoAllocWords];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+int32_t* g_scratch_ptr[kMaxDevices] = {nullptr};
+
+// Device address of g_dispatch_scratch on the current device.  In host code the array's name is
+// only a handle for the runtime, not an address a kernel could use, so it is translated once
+// per device with that device current.
+cudaError_t scratch_address(int32_t** out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ptr[dev]) {
+        int32_t* p = nullptr;
+        e = cudaGetSymbolAddress((void**)&p, g_dispatch_scratch);
+        if (e != cudaSuccess) return e;
+        g_scratch_ptr[dev] = p;
+    }
+    *out = g_scratch_ptr[dev];
+    return cudaSuccess;
+}
+
+// One block: derives the bin layout from model_of_tenant and clears the words that must start
+// at zero (the status word; the statistics are overwritten by the scan kernel).
+__global__ void __launch_bounds__(256)
+noalloc_setup_kernel(const int32_t* __restrict__ model_of_tenant, int n_tenants, int M, int E,
+                     int32_t* __restrict__ tenant_local, int32_t* __restrict__ tenants_in_model,
+                     int32_t* __restrict__ bin_base, int32_t* __restrict__ clean_model_of_tenant,
+                     int32_t* __restrict__ stats, int32_t* __restrict__ status)
+{
+    const int tid = threadIdx.x;
+    if (tid == 0) *status = 0;
+    if (tid < 4) stats[tid] = 0;
+    // thread m counts the tenants of model m in tenant order (sizes here are tiny)
+    for (int m = tid; m < M; m += blockDim.x) {
+        int n = 0;
+        for (int u = 0; u < n_tenants; ++u) {
+            int mu = model_of_tenant[u];
+            if (mu < 0 || mu >= M) mu = 0;
+            if (mu == m) { tenant_local[u] = n; clean_model_of_tenant[u] = mu; ++n; }
+        }
+        tenants_in_model[m] = n;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int run = 0;
+        for (int m = 0; m < M; ++m) { bin_base[m] = run; run += E * tenants_in_model[m]; }
+        bin_base[M] = run;
+    }
+}
+
+}  // namespace
+}  // namespace faasmoe
+
+extern "C" int moe_dispatch_noalloc(const int32_t* topk_idx, const int32_t* tenant_id, const int32_t* model_of_tenant,
+                                    int T, int k, int E, int M, int n_tenants, int G, int32_t* perm, int32_t* inv_perm,
+                                    int32_t* tenant_expert_count, int32_t* expert_off, int32_t* group_off,
+                                    int32_t* status_out, void* stream)
+{
+    using namespace faasmoe;
+    if (!topk_idx || !tenant_id || !model_of_tenant || !perm || !inv_perm || !expert_off) return MOE_ERR_NULL;
+    if (T < 0 || k < 1 || k > kMaxTopK || E < 1 || E > kMaxExperts || k > E || M < 1 || M > kMaxExperts ||
+        n_tenants < 1)
+        return MOE_ERR_SHAPE;
+    if (G < 1 || G > E) return MOE_ERR_G;
+    if ((long long)T * k > (1 << 28) || (long long)E * n_tenants > kMaxBins) return MOE_ERR_SHAPE;
+    const int R = T * k;
+    const int nbins = E * n_tenants;
+    const int nblk = (R + kDispatchChunk - 1) / kDispatchChunk;
+    // scratch layout, in 32-bit words
+    const long long o_stats = 0, o_status = 4, o_mot = 8, o_local = o_mot + n_tenants, o_tim = o_local + n_tenants,
+                    o_base = o_tim + M, o_binoff = o_base + M + 1, o_blk = o_binoff + nbins + 1,
+                    total = o_blk + (long long)nblk * nbins;
+    if (total > kNoAllocWords) return MOE_ERR_UNSUPPORTED;     // beyond the fixed scratch: see the header
+    if (T == 0) return MOE_OK;
+    int32_t* s = nullptr;
+    if (scratch_address(&s) != cudaSuccess) return MOE_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t* status = status_out ? status_out : s + o_status;
+    noalloc_setup_kernel<<<1, 256, 0, st>>>(model_of_tenant, n_tenants, M, E, s + o_local, s + o_tim, s + o_base,
+                                            s + o_mot, s + o_stats, status);
+    BinMap bm;
+    bm.model_of_tenant = s + o_mot;
+    bm.tenant_local = s + o_local;
+    bm.bin_base = s + o_base;
+    bm.tenants_in_model = s + o_tim;
+    bm.n_tenants = n_tenants;
+    bm.E = E;
+    const size_t smem = (size_t)nbins * sizeof(int32_t);
+    dispatch_hist_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, s + o_blk, status);
+    dispatch_scan_kernel<<<1, 1024, smem, st>>>(nblk, nbins, R, E, M, G, n_tenants, bm, s + o_blk, s + o_binoff,
+                                                tenant_expert_count, expert_off, group_off, s + o_stats);
+    dispatch_rank_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, s + o_blk, s + o_binoff, perm,
+                                                 inv_perm, status);
+    return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
