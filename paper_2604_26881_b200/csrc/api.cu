@@ -349,6 +349,7 @@ int moe_experts(moe_ctx* c, int layer, const void* x, const void* x_perm, const 
 {
     if (!c || !x_perm || !expert_off || !y_perm) return MOE_ERR_NULL;
     if (y_shared && (!x || !tenant_id)) return MOE_ERR_NULL;
+    if (((uintptr_t)x_perm | (uintptr_t)x | (uintptr_t)y_perm | (uintptr_t)y_shared) & 15) return MOE_ERR_SHAPE;
     if (T < 0 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
     if (G < 1 || G > c->cfg.n_experts) return MOE_ERR_G;
     const int rc = check_layer_ready(c, layer, true, y_shared != nullptr);
