@@ -58,9 +58,12 @@ enum {
     MOE_DEV_TIMEOUT = 8       /* a bounded wait inside a kernel ran out; outputs are invalid */
 };
 
-/* values of MOE_OPT_EXPERT_PATH */
+/* moe_set_option: which kernels run the expert FFNs (MOE_OPT_EXPERT_PATH) and the router
+ * (MOE_OPT_ROUTE_PATH).  AUTO takes the tcgen05 kernels whenever the shape allows
+ * (experts: hidden % 256 == 0; router: n_experts <= 64 and n_models * ceil16(n_experts) <= 256),
+ * FMA forces the CUDA-core kernels, TCGEN05 fails with MOE_ERR_UNSUPPORTED if not possible. */
 enum { MOE_PATH_AUTO = 0, MOE_PATH_FMA = 1, MOE_PATH_TCGEN05 = 2 };
-enum { MOE_OPT_EXPERT_PATH = 1 };
+enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2 };
 
 typedef struct {
     int32_t hidden;        /* H */

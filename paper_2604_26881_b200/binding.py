@@ -21,6 +21,7 @@ MOE_ERR_NULL, MOE_ERR_SHAPE, MOE_ERR_G, MOE_ERR_STATE = -1, -2, -3, -4
 MOE_ERR_CUDA, MOE_ERR_ALLOC, MOE_ERR_UNSUPPORTED = -5, -6, -7
 MOE_DEV_BAD_TENANT, MOE_DEV_BAD_EXPERT, MOE_DEV_TIMEOUT = 1, 2, 8
 MOE_OPT_EXPERT_PATH = 1
+MOE_OPT_ROUTE_PATH = 2
 MOE_PATH_AUTO, MOE_PATH_FMA, MOE_PATH_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["moe_create", "moe_destroy", "moe_set_expert_pool", "moe_set_model_weights", "moe_set_slot_table",

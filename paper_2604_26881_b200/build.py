@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "lib", "libfaasmoe.so")
-SOURCES = ["api.cu", "route.cu", "dispatch.cu", "plan.cu", "experts_fma.cu", "experts_tc.cu", "combine.cu"]
+SOURCES = ["api.cu", "route.cu", "route_tc.cu", "dispatch.cu", "plan.cu", "experts_fma.cu", "experts_tc.cu", "combine.cu"]
 
 
 def _newest_source_mtime() -> float:

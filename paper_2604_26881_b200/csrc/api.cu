@@ -195,6 +195,8 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->expert_path = MOE_PATH_AUTO;
     c->launches = 0;
     c->tmaps = nullptr;
+    c->rmaps = nullptr;
+    c->route_path = MOE_PATH_AUTO;
     c->timing = false;
     for (auto& e : c->ev) e = nullptr;
     c->errbuf[0] = 0;
@@ -240,6 +242,7 @@ int moe_destroy(moe_ctx* c)
     if (!c) return MOE_ERR_NULL;
     cudaDeviceSynchronize();
     tc_destroy(c);
+    route_tc_destroy(c);
     free_workspace(c);
     for (auto& e : c->ev) if (e) cudaEventDestroy(e);
     void* ptrs[] = {c->d_models, c->d_slot, c->d_model_of_tenant, c->d_tenant_local, c->d_bin_base,
@@ -281,6 +284,7 @@ int moe_set_model_weights(moe_ctx* c, int layer, int model, const void* router_w
     MOE_CUDA(c, cudaMemcpy(c->d_models + i, &mw, sizeof(mw), cudaMemcpyHostToDevice));
     c->model_set[i] = 1;
     tc_destroy(c);
+    route_tc_destroy(c);
     return MOE_OK;
 }
 
@@ -312,6 +316,12 @@ int moe_set_option(moe_ctx* c, int option, int value)
         if (value < MOE_PATH_AUTO || value > MOE_PATH_TCGEN05) return MOE_ERR_SHAPE;
         if (value == MOE_PATH_TCGEN05 && !tc_supported(c)) return MOE_ERR_UNSUPPORTED;
         c->expert_path = value;
+        return MOE_OK;
+    }
+    if (option == MOE_OPT_ROUTE_PATH) {
+        if (value < MOE_PATH_AUTO || value > MOE_PATH_TCGEN05) return MOE_ERR_SHAPE;
+        if (value == MOE_PATH_TCGEN05 && !route_tc_supported(c)) return MOE_ERR_UNSUPPORTED;
+        c->route_path = value;
         return MOE_OK;
     }
     return MOE_ERR_SHAPE;

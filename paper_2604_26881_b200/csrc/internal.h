@@ -121,6 +121,8 @@ struct moe_ctx {
     int32_t* d_tenants_in_model;  // [M]
     faasmoe::Workspace ws;
     faasmoe::TensorMaps* tmaps;   // TMA descriptors of the tensor-core path (host)
+    void* rmaps;                  // TMA descriptors of the tensor-core router
+    int route_path;
     bool timing;                  // record an event after every stage (moe_layer_forward_timed)
     cudaEvent_t ev[8];
     char errbuf[256];
@@ -144,6 +146,13 @@ cudaError_t launch_route(moe_ctx* c, int layer, const bf16* x, const int32_t* te
 cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, const int32_t* tenant_id, int T, int G,
                             int32_t* perm, int32_t* inv_perm, int32_t* tenant_expert_count, int32_t* expert_off,
                             int32_t* group_off, bf16* x_perm, cudaStream_t st);
+
+cudaError_t launch_route_fma(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,
+                             float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st);
+cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,
+                            float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st);
+bool route_tc_supported(const moe_ctx* c);
+void route_tc_destroy(moe_ctx* c);
 
 // Sorts tokens by (model, token) into ws.tok_perm / tok_inv / model_tok_off and gathers ws.xs_perm (M > 1).
 cudaError_t launch_token_sort(moe_ctx* c, const bf16* x, const int32_t* tenant_id, int T, cudaStream_t st);

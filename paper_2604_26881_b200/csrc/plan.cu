@@ -102,17 +102,20 @@ plan_kernel(const int32_t* __restrict__ expert_off, const int32_t* __restrict__ 
         const int su1 = n_stiles * snblk1, su2 = n_stiles * snblk2;
         for (int i = tid; i < su1; i += nth) { Unit u; u.colblock = i / n_stiles; u.tile = ~(i % n_stiles); units1[i] = u; }
         for (int i = tid; i < su2; i += nth) { Unit u; u.colblock = i / n_stiles; u.tile = ~(i % n_stiles); units2[i] = u; }
-        for (int gidx = 0; gidx < NG; ++gidx) {
+        __syncthreads();                      // the tiles written above are read back below
+        for (int i = tid; i < n_tiles * nblk1; i += nth) {
+            const int tile = i % n_tiles, cb = i / n_tiles;
+            const int gidx = tiles[tile].group;
             const int t0 = s_group_tile0[gidx], nt = s_group_tile0[gidx + 1] - t0;
-            if (nt == 0) continue;
-            for (int i = tid; i < nt * nblk1; i += nth) {
-                Unit u; u.colblock = i / nt; u.tile = t0 + i % nt;
-                units1[su1 + t0 * nblk1 + i] = u;
-            }
-            for (int i = tid; i < nt * nblk2; i += nth) {
-                Unit u; u.colblock = i / nt; u.tile = t0 + i % nt;
-                units2[su2 + t0 * nblk2 + i] = u;
-            }
+            Unit u; u.colblock = cb; u.tile = tile;
+            units1[su1 + t0 * nblk1 + cb * nt + (tile - t0)] = u;
+        }
+        for (int i = tid; i < n_tiles * nblk2; i += nth) {
+            const int tile = i % n_tiles, cb = i / n_tiles;
+            const int gidx = tiles[tile].group;
+            const int t0 = s_group_tile0[gidx], nt = s_group_tile0[gidx + 1] - t0;
+            Unit u; u.colblock = cb; u.tile = tile;
+            units2[su2 + t0 * nblk2 + cb * nt + (tile - t0)] = u;
         }
         if (tid == 0) {
             plan_counts[2] = su1 + n_tiles * nblk1;

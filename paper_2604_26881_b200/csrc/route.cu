@@ -185,6 +185,14 @@ route_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ tenant_id, 
 cudaError_t launch_route(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,
                          float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st)
 {
+    const bool tc = c->route_path != MOE_PATH_FMA && route_tc_supported(c) && ((uintptr_t)x & 15) == 0;
+    return tc ? launch_route_tc(c, layer, x, tenant_id, T, topk_idx, topk_w, shared_gate, tie_flag, st)
+              : launch_route_fma(c, layer, x, tenant_id, T, topk_idx, topk_w, shared_gate, tie_flag, st);
+}
+
+cudaError_t launch_route_fma(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,
+                             float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st)
+{
     const moe_config& g = c->cfg;
     const ModelWeights* models = c->d_models + (size_t)layer * g.n_models;
     // small batches: one token per warp so that the tokens spread over many SMs

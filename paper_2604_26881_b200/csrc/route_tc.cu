@@ -1,0 +1,291 @@
+// Gating network on the tensor cores (paper Sec. 2.1: the gate scores every expert and selects
+// the top-k per token).  One CTA scores 128 tokens against the routers of all tenant models at
+// once: the tokens are the M operand of tcgen05.mma (one TMEM lane per token), the router rows of
+// every model the N operand (E rows per model, padded to a multiple of 16).  The epilogue is one
+// thread per token: it picks the columns of its tenant's model out of TMEM and does the fp32
+// softmax and the top-k in registers.  While the MMA pipeline runs, the epilogue warps compute the
+// shared expert's sigmoid gate with plain FMAs.
+#include "internal.h"
+#include "tc_ptx.cuh"
+
+namespace faasmoe {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kRStages = 4;
+constexpr int kRBK = 64;
+constexpr int kRTokens = 128;
+constexpr int kRABytes = kRTokens * kRBK * 2;          // 16 KB of tokens per stage
+constexpr int kRMaxN = 256;                            // router rows of all models, padded
+constexpr int kRBBytes = kRMaxN * kRBK * 2;            // 32 KB
+constexpr int kRStageBytes = kRABytes + kRBBytes;
+constexpr int kRSmemBytes = kRStages * kRStageBytes + 1024 + 256;
+constexpr int kRThreads = 192;
+constexpr int kRMaxE = 64;                             // logits one thread keeps in registers
+
+struct RouteParams {
+    const bf16* x;
+    const int32_t* tenant_id;
+    int T, H, E, Epad, k, n_tenants, n_models;
+    const int32_t* model_of_tenant;
+    const ModelWeights* models;
+    const CUtensorMap* rmaps;      // one map per model over router_w [E,H], box Epad rows
+    int32_t* topk_idx;
+    float* topk_w;
+    float* shared_gate;
+    uint8_t* tie_flag;
+    int32_t* status;
+};
+
+__device__ __forceinline__ float dot8f(const uint4& a, const uint4& b, float acc)
+{
+    const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+    const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 fa = __bfloat1622float2(pa[i]), fb = __bfloat1622float2(pb[i]);
+        acc = fmaf(fa.x, fb.x, acc);
+        acc = fmaf(fa.y, fb.y, acc);
+    }
+    return acc;
+}
+
+__global__ void __launch_bounds__(kRThreads, 1)
+route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
+{
+    extern __shared__ unsigned char smem_dyn[];
+    const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    const uint32_t bars = smem_base + kRStages * kRStageBytes;
+    const uint32_t bar_full = bars, bar_empty = bars + 8 * kRStages, bar_tfull = bars + 16 * kRStages;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t0 = blockIdx.x * kRTokens;
+    const int ksteps = p.H / kRBK;
+    const int N = p.n_models * p.Epad;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kRStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        mbar_init(bar_tfull, 1);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                     "r"((uint32_t)kRMaxN)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, armed = 0, armed_phase = 0;
+            bool ok = true;
+            for (int ks = 0; ks < ksteps; ++ks) {
+                if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, &s_abort, p.status)) { ok = false; break; }
+                const uint32_t sa = smem_base + stage * kRStageBytes, sb = sa + kRABytes;
+                const uint32_t full = bar_full + 8 * stage;
+                mbar_expect_tx(full, kRABytes + N * kRBK * 2);
+                armed |= 1u << stage;
+                armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
+                tma_load_2d(sa, &xmap, full, ks * kRBK, t0);
+                for (int m = 0; m < p.n_models; ++m)
+                    tma_load_2d(sb + m * p.Epad * kRBK * 2, p.rmaps + m, full, ks * kRBK, 0);
+                if (++stage == kRStages) { stage = 0; phase ^= 1; }
+            }
+            if (!ok)
+                for (int s = 0; s < kRStages; ++s)
+                    if (armed & (1u << s)) mbar_wait(bar_full + 8 * s, (armed_phase >> s) & 1u, &s_abort, p.status);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((128u >> 4) << 24);
+            bool ok = true;
+            for (int ks = 0; ks < ksteps; ++ks) {
+                if (!mbar_wait(bar_full + 8 * stage, phase, &s_abort, p.status)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t sa = smem_base + stage * kRStageBytes, sb = sa + kRABytes;
+                const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+#pragma unroll
+                for (int kk = 0; kk < kRBK / 16; ++kk) {
+                    const uint64_t adv = (uint64_t)(kk * 32 >> 4);
+                    umma_bf16(tmem_base, da + adv, db + adv, idesc, (ks | kk) ? 1u : 0u);
+                }
+                umma_commit(bar_empty + 8 * stage);
+                if (++stage == kRStages) { stage = 0; phase ^= 1; }
+            }
+            if (ok) umma_commit(bar_tfull);
+        }
+    } else {
+        // ---- epilogue warps: thread <-> token (TMEM lane) ----
+        const int quarter = warp & 3;
+        const int t = t0 + quarter * 32 + lane;
+        const bool valid = t < p.T;
+        bool bad = false;
+        int model = 0;
+        if (valid) {
+            int u = p.tenant_id[t];
+            if (u < 0 || u >= p.n_tenants) { bad = true; u = 0; }
+            model = p.model_of_tenant[u];
+        }
+        // shared-expert gate, overlapped with the MMA pipeline: warp-wide dot products, lane j keeps token j's
+        float gate = 0.5f;
+        if (p.shared_gate) {
+            const int hv = p.H >> 3;
+            for (int j = 0; j < 32; ++j) {
+                const int tj = t0 + quarter * 32 + j;
+                if (tj >= p.T) break;                                    // warp-uniform
+                const int mj = __shfl_sync(0xffffffffu, model, j);
+                const bf16* sg = p.models[mj].shared_gate_w;
+                float acc = 0.f;
+                if (sg) {
+                    const uint4* xv = reinterpret_cast<const uint4*>(p.x + (size_t)tj * p.H);
+                    const uint4* wv = reinterpret_cast<const uint4*>(sg);
+                    for (int v = lane; v < hv; v += 32) acc = dot8f(__ldg(xv + v), __ldg(wv + v), acc);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+                }
+                if (lane == j) gate = sg ? 1.f / (1.f + expf(-acc)) : 0.5f;
+            }
+        }
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull, 0, &s_abort, p.status));
+        if (ok) {
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            // logits of this token's model: the column range depends on the model, the TMEM load is
+            // warp-wide, so every model's columns are loaded and each thread keeps its own
+            float z[kRMaxE];
+#pragma unroll
+            for (int e = 0; e < kRMaxE; ++e) z[e] = -INFINITY;
+            for (int m = 0; m < p.n_models; ++m) {
+#pragma unroll
+                for (int c = 0; c < kRMaxE / 16; ++c) {
+                    if (c * 16 < p.Epad) {                                // warp-uniform
+                        uint32_t r[16];
+                        tmem_ld16(taddr + m * p.Epad + c * 16, r);
+                        tmem_ld_wait();
+                        if (m == model) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) z[c * 16 + j] = __uint_as_float(r[j]);
+                        }
+                    }
+                }
+            }
+            if (valid) {
+                const float* rb = p.models[model].router_bias;
+                float zmax = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < kRMaxE; ++e) {
+                    if (e < p.E) { if (rb) z[e] += rb[e]; zmax = fmaxf(zmax, z[e]); }
+                    else z[e] = -INFINITY;
+                }
+                float den = 0.f;
+#pragma unroll
+                for (int e = 0; e < kRMaxE; ++e) { z[e] = (e < p.E) ? expf(z[e] - zmax) : 0.f; den += z[e]; }
+#pragma unroll
+                for (int e = 0; e < kRMaxE; ++e) z[e] = (e < p.E) ? z[e] / den : -1.f;
+                const int rounds = (p.k < p.E) ? p.k + 1 : p.k;
+                float prev = 0.f;
+                uint8_t flag = 0;
+                for (int j = 0; j < rounds; ++j) {
+                    float bv = -1.f;
+                    int bi = 0;
+#pragma unroll
+                    for (int e = 0; e < kRMaxE; ++e) if (z[e] > bv) { bv = z[e]; bi = e; }    // first maximum: lower id wins
+                    if (j > 0 && (prev - bv) < 1e-5f * prev) flag = 1;
+                    prev = bv;
+                    if (j < p.k) {
+                        p.topk_idx[(size_t)t * p.k + j] = bad ? j : bi;
+                        p.topk_w[(size_t)t * p.k + j] = bad ? 0.f : bv;
+                    }
+#pragma unroll
+                    for (int e = 0; e < kRMaxE; ++e) if (e == bi) z[e] = -1.f;
+                }
+                if (p.tie_flag) p.tie_flag[t] = flag;
+                if (p.shared_gate) p.shared_gate[t] = bad ? 0.f : gate;
+                if (bad) atomicOr(p.status, MOE_DEV_BAD_TENANT);
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kRMaxN) : "memory");
+    }
+}
+
+struct RouterMaps {
+    std::vector<CUtensorMap*> d_maps;     // per layer: device array of n_models maps
+};
+
+}  // namespace
+
+bool route_tc_supported(const moe_ctx* c)
+{
+    const moe_config& g = c->cfg;
+    const int epad = (g.n_experts + 15) & ~15;
+    return g.n_experts <= kRMaxE && g.n_models * epad <= kRMaxN && g.hidden % kRBK == 0;
+}
+
+void route_tc_destroy(moe_ctx* c)
+{
+    RouterMaps* rm = reinterpret_cast<RouterMaps*>(c->rmaps);
+    if (!rm) return;
+    cudaDeviceSynchronize();
+    for (CUtensorMap* p : rm->d_maps) if (p) cudaFree(p);
+    delete rm;
+    c->rmaps = nullptr;
+}
+
+cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,
+                            float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st)
+{
+    const moe_config& g = c->cfg;
+    const int M = g.n_models, E = g.n_experts, H = g.hidden;
+    const int epad = (E + 15) & ~15;
+    if (!c->rmaps) {
+        RouterMaps* rm = new RouterMaps();
+        rm->d_maps.assign(g.n_layers, nullptr);
+        c->rmaps = rm;
+    }
+    RouterMaps* rm = reinterpret_cast<RouterMaps*>(c->rmaps);
+    if (!rm->d_maps[layer]) {
+        std::vector<CUtensorMap> maps(M);
+        for (int m = 0; m < M; ++m)
+            if (!make_map(&maps[m], c->models[(size_t)layer * M + m].router_w, E, H, epad, false)) return cudaErrorInvalidValue;
+        cudaError_t e = cudaMalloc((void**)&rm->d_maps[layer], M * sizeof(CUtensorMap));
+        if (e != cudaSuccess) return e;
+        e = cudaMemcpy(rm->d_maps[layer], maps.data(), M * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) return e;
+    }
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(route_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes);
+        attr_set = true;
+    }
+    CUtensorMap xmap;
+    if (!make_map(&xmap, x, T, H, kRTokens, false)) return cudaErrorInvalidValue;
+    RouteParams p;
+    p.x = x; p.tenant_id = tenant_id; p.T = T; p.H = H; p.E = E; p.Epad = epad; p.k = g.top_k;
+    p.n_tenants = g.n_tenants; p.n_models = M; p.model_of_tenant = c->d_model_of_tenant;
+    p.models = c->d_models + (size_t)layer * M; p.rmaps = rm->d_maps[layer];
+    p.topk_idx = topk_idx; p.topk_w = topk_w; p.shared_gate = shared_gate; p.tie_flag = tie_flag;
+    p.status = c->ws.status;
+    route_tc_kernel<<<(T + kRTokens - 1) / kRTokens, kRThreads, kRSmemBytes, st>>>(p, xmap);
+    c->launches += 1;
+    return cudaGetLastError();
+}
+
+}  // namespace faasmoe

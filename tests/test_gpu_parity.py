@@ -23,6 +23,7 @@ def run_and_compare(wl, wts, x, tenant, mot, G, path, max_tokens=None):
     g = GpuLayer(wl, [wts], max_tokens or x.shape[0], model_of_tenant=mot)
     try:
         B.moe_set_option(g.ctx, B.MOE_OPT_EXPERT_PATH, path)
+        B.moe_set_option(g.ctx, B.MOE_OPT_ROUTE_PATH, path)
         o = g.four_calls(x, tenant, G)
         ref = oracle_layer(wl, wts, x, tenant, mot, G, o["topk_idx"].cpu().numpy(), o["topk_w"].cpu().numpy())
         compare_four_calls(o, ref, wl, x)
@@ -125,6 +126,7 @@ def test_pool_config_reduced_and_G_sweep(path):
     g = GpuLayer(wl, [wts], wl.T, model_of_tenant=mot)
     try:
         B.moe_set_option(g.ctx, B.MOE_OPT_EXPERT_PATH, path)
+        B.moe_set_option(g.ctx, B.MOE_OPT_ROUTE_PATH, path)
         base = g.forward(x, tenant, 1)
         assert torch.equal(base, o["out"])
         invocations = []
@@ -148,6 +150,7 @@ def test_stack_teacher_forced(path):
     g = GpuLayer(wl, layers, T, model_of_tenant=mot)
     try:
         B.moe_set_option(g.ctx, B.MOE_OPT_EXPERT_PATH, path)
+        B.moe_set_option(g.ctx, B.MOE_OPT_ROUTE_PATH, path)
         xd, td = x.to(g.dev).clone(), tenant.to(g.dev)
         dbg_in = torch.zeros((wl.n_layers, T, wl.H), dtype=torch.bfloat16, device=g.dev)
         dbg_out = torch.zeros_like(dbg_in)
