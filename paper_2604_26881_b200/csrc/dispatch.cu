@@ -47,30 +47,16 @@ dispatch_hist_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __rest
     for (int b = threadIdx.x; b < nbins; b += 32) dst[b] = s_cnt[b];
 }
 
-// D2: one block.  Totals per bin, exclusive scan in key order, per-block bases, and the
-// offset tables the caller sees.
-__global__ void __launch_bounds__(1024)
-dispatch_scan_kernel(int nblk, int nbins, int R, int E, int M, int G, int n_tenants, BinMap bm,
-                     int32_t* __restrict__ block_cnt, int32_t* __restrict__ bin_off,
-                     int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
-                     int32_t* __restrict__ group_off, int32_t* __restrict__ stats)
+// Block-wide: exclusive scan of the per-bin totals in s_tot (in key order), then the offset tables
+// the caller sees and the invocation statistics.  s_tot holds the offsets afterwards.
+__device__ void scan_and_tables(int32_t* s_tot, int32_t* s_part /* [blockDim.x] */, int32_t* s_count /* [2] */,
+                                int nbins, int R, int E, int M, int G, int n_tenants, const BinMap& bm,
+                                int32_t* __restrict__ bin_off /* may be null */,
+                                int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
+                                int32_t* __restrict__ group_off, int32_t* __restrict__ stats)
 {
-    extern __shared__ int32_t s_tot[];       // [nbins] totals, then exclusive offsets
-    __shared__ int32_t s_part[1024];
-    __shared__ int32_t s_count[2];
     const int tid = threadIdx.x, nth = blockDim.x;
-    // totals per bin; block_cnt becomes the exclusive prefix over blocks
-    for (int b = tid; b < nbins; b += nth) {
-        int run = 0;
-        for (int blk = 0; blk < nblk; ++blk) {
-            const int c = block_cnt[(size_t)blk * nbins + b];
-            block_cnt[(size_t)blk * nbins + b] = run;
-            run += c;
-        }
-        s_tot[b] = run;
-    }
     if (tid < 2) s_count[tid] = 0;
-    __syncthreads();
     if (tenant_expert_count) {
         for (int i = tid; i < n_tenants * E; i += nth) {
             const int u = i / E, e = i - u * E;
@@ -95,8 +81,10 @@ dispatch_scan_kernel(int nblk, int nbins, int R, int E, int M, int G, int n_tena
     int run = s_part[tid] - sum;
     for (int b = b0; b < b1; ++b) { const int c = s_tot[b]; s_tot[b] = run; run += c; }
     __syncthreads();
-    for (int b = tid; b < nbins; b += nth) bin_off[b] = s_tot[b];
-    if (tid == 0) bin_off[nbins] = R;
+    if (bin_off) {
+        for (int b = tid; b < nbins; b += nth) bin_off[b] = s_tot[b];
+        if (tid == 0) bin_off[nbins] = R;
+    }
     // expert_off[m*E + e] = offset of the first bin of (m, e); a model without tenants owns
     // no bins, so its experts start where the next model's bins start
     for (int i = tid; i <= M * E; i += nth) {
@@ -125,6 +113,84 @@ dispatch_scan_kernel(int nblk, int nbins, int R, int E, int M, int G, int n_tena
         if (expert_off[i + 1] > expert_off[i]) atomicAdd(&s_count[1], 1);
     __syncthreads();
     if (tid < 2) stats[tid] = s_count[tid];
+}
+
+// D2: one block.  Totals per bin, exclusive scan in key order, per-block bases, and the
+// offset tables the caller sees.
+__global__ void __launch_bounds__(1024)
+dispatch_scan_kernel(int nblk, int nbins, int R, int E, int M, int G, int n_tenants, BinMap bm,
+                     int32_t* __restrict__ block_cnt, int32_t* __restrict__ bin_off,
+                     int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
+                     int32_t* __restrict__ group_off, int32_t* __restrict__ stats)
+{
+    extern __shared__ int32_t s_tot[];       // [nbins] totals, then exclusive offsets
+    __shared__ int32_t s_part[1024];
+    __shared__ int32_t s_count[2];
+    const int tid = threadIdx.x, nth = blockDim.x;
+    // totals per bin; block_cnt becomes the exclusive prefix over blocks
+    for (int b = tid; b < nbins; b += nth) {
+        int run = 0;
+        for (int blk = 0; blk < nblk; ++blk) {
+            const int c = block_cnt[(size_t)blk * nbins + b];
+            block_cnt[(size_t)blk * nbins + b] = run;
+            run += c;
+        }
+        s_tot[b] = run;
+    }
+    __syncthreads();
+    scan_and_tables(s_tot, s_part, s_count, nbins, R, E, M, G, n_tenants, bm, bin_off, tenant_expert_count,
+                    expert_off, group_off, stats);
+}
+
+// Small batches: the whole dispatch in one block -- histogram, scan, tables, stable ranks (one warp
+// walks the rows in order), and the gather of the rows.  Same results as the multi-block kernels.
+constexpr int kSmallRows = 2048;
+
+__global__ void __launch_bounds__(1024)
+dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ tenant_id, int R, int k,
+                      BinMap bm, int nbins, int E, int M, int G, int n_tenants, int32_t* __restrict__ perm,
+                      int32_t* __restrict__ inv_perm, int32_t* __restrict__ tenant_expert_count,
+                      int32_t* __restrict__ expert_off, int32_t* __restrict__ group_off, int32_t* __restrict__ stats,
+                      int32_t* __restrict__ status, const bf16* __restrict__ x, bf16* __restrict__ x_perm, int H)
+{
+    extern __shared__ int32_t s_tot[];       // [nbins]
+    __shared__ int32_t s_part[1024];
+    __shared__ int32_t s_count[2];
+    const int tid = threadIdx.x, nth = blockDim.x;
+    for (int b = tid; b < nbins; b += nth) s_tot[b] = 0;
+    __syncthreads();
+    for (int r = tid; r < R; r += nth) atomicAdd(&s_tot[row_bin(bm, tenant_id[r / k], topk_idx[r], status)], 1);
+    __syncthreads();
+    scan_and_tables(s_tot, s_part, s_count, nbins, R, E, M, G, n_tenants, bm, nullptr, tenant_expert_count,
+                    expert_off, group_off, stats);
+    __syncthreads();
+    if (tid < 32) {                           // s_tot now holds the next free position of every bin
+        const int lane = tid;
+        for (int rr = 0; rr < R; rr += 32) {
+            const int r = rr + lane;
+            const bool live = r < R;
+            int bin = -1 - lane;
+            if (live) bin = row_bin(bm, tenant_id[r / k], topk_idx[r], status);
+            const unsigned peers = __match_any_sync(0xffffffffu, bin);
+            const int leader = __ffs(peers) - 1;
+            const int rank = __popc(peers & ((1u << lane) - 1u));
+            int start = 0;
+            if (live && lane == leader) { start = s_tot[bin]; s_tot[bin] = start + __popc(peers); }
+            start = __shfl_sync(0xffffffffu, start, leader);
+            if (live) { perm[start + rank] = r; inv_perm[r] = start + rank; }
+            __syncwarp();
+        }
+    }
+    if (x_perm) {
+        __syncthreads();                      // perm is complete and visible to the block
+        const int warp = tid >> 5, lane = tid & 31, nw = nth >> 5;
+        for (int pos = warp; pos < R; pos += nw) {
+            const int t = perm[pos] / k;
+            const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * H);
+            uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)pos * H);
+            for (int v = lane; v < (H >> 3); v += 32) dst[v] = src[v];
+        }
+    }
 }
 
 // D3: stable rank of every row inside its bin.  One warp per block walks its chunk in row
@@ -268,6 +334,20 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
     const int nbins = c->nbins;
     const BinMap bm = make_binmap(c);
     const size_t smem = (size_t)nbins * sizeof(int32_t);
+    if (R <= kSmallRows) {
+        // few rows: one block does everything; the gather rides along while it is small
+        const bool gather_inside = x_perm && (size_t)R * g.hidden * sizeof(bf16) <= (1u << 20);
+        dispatch_small_kernel<<<1, 1024, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, g.n_experts, g.n_models, G,
+                                                     g.n_tenants, perm, inv_perm, tenant_expert_count, expert_off,
+                                                     group_off, c->ws.stats, c->ws.status, x,
+                                                     gather_inside ? x_perm : nullptr, g.hidden);
+        c->launches += 1;
+        if (x_perm && !gather_inside) {
+            gather_rows_kernel<<<(R * 32 + 255) / 256, 256, 0, st>>>(x, perm, R, k, g.hidden, x_perm);
+            c->launches += 1;
+        }
+        return cudaGetLastError();
+    }
     dispatch_hist_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, c->ws.block_cnt, c->ws.status);
     dispatch_scan_kernel<<<1, 1024, smem, st>>>(nblk, nbins, R, g.n_experts, g.n_models, G, g.n_tenants, bm,
                                                 c->ws.block_cnt, c->ws.bin_off, tenant_expert_count, expert_off,

@@ -137,24 +137,26 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
             if (u < 0 || u >= p.n_tenants) { bad = true; u = 0; }
             model = p.model_of_tenant[u];
         }
-        // shared-expert gate, overlapped with the MMA pipeline: warp-wide dot products, lane j keeps token j's
+        // shared-expert gate, overlapped with the MMA pipeline: each thread walks its own token's row
+        // (independent 16-byte loads, four accumulators), so no cross-lane traffic is needed
         float gate = 0.5f;
-        if (p.shared_gate) {
-            const int hv = p.H >> 3;
-            for (int j = 0; j < 32; ++j) {
-                const int tj = t0 + quarter * 32 + j;
-                if (tj >= p.T) break;                                    // warp-uniform
-                const int mj = __shfl_sync(0xffffffffu, model, j);
-                const bf16* sg = p.models[mj].shared_gate_w;
-                float acc = 0.f;
-                if (sg) {
-                    const uint4* xv = reinterpret_cast<const uint4*>(p.x + (size_t)tj * p.H);
-                    const uint4* wv = reinterpret_cast<const uint4*>(sg);
-                    for (int v = lane; v < hv; v += 32) acc = dot8f(__ldg(xv + v), __ldg(wv + v), acc);
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (p.shared_gate && valid) {
+            const bf16* sg = p.models[model].shared_gate_w;
+            if (sg) {
+                const uint4* xv = reinterpret_cast<const uint4*>(p.x + (size_t)t * p.H);
+                const uint4* wv = reinterpret_cast<const uint4*>(sg);
+                const int hv = p.H >> 3;
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+                int v = 0;
+                for (; v + 4 <= hv; v += 4) {
+                    const uint4 x0 = __ldg(xv + v), x1 = __ldg(xv + v + 1), x2 = __ldg(xv + v + 2), x3 = __ldg(xv + v + 3);
+                    a0 = dot8f(x0, __ldg(wv + v), a0);
+                    a1 = dot8f(x1, __ldg(wv + v + 1), a1);
+                    a2 = dot8f(x2, __ldg(wv + v + 2), a2);
+                    a3 = dot8f(x3, __ldg(wv + v + 3), a3);
                 }
-                if (lane == j) gate = sg ? 1.f / (1.f + expf(-acc)) : 0.5f;
+                for (; v < hv; ++v) a0 = dot8f(__ldg(xv + v), __ldg(wv + v), a0);
+                gate = 1.f / (1.f + expf(-((a0 + a1) + (a2 + a3))));
             }
         }
         const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull, 0, &s_abort, p.status));
