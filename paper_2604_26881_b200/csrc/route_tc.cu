@@ -5,6 +5,8 @@
 // thread per token: it picks the columns of its tenant's model out of TMEM and does the fp32
 // softmax and the top-k in registers.  While the MMA pipeline runs, the epilogue warps compute the
 // shared expert's sigmoid gate with plain FMAs.
+#include <cstring>
+
 #include "internal.h"
 #include "tc_ptx.cuh"
 
@@ -14,13 +16,15 @@ namespace {
 
 using namespace tc;
 
-constexpr int kRStages = 4;
+constexpr int kRStages = 3;
 constexpr int kRBK = 64;
 constexpr int kRTokens = 128;
 constexpr int kRABytes = kRTokens * kRBK * 2;          // 16 KB of tokens per stage
 constexpr int kRMaxN = 256;                            // router rows of all models, padded
 constexpr int kRBBytes = kRMaxN * kRBK * 2;            // 32 KB
-constexpr int kRStageBytes = kRABytes + kRBBytes;
+constexpr int kRMaxGateN = 64;                         // 16 columns per model for the shared-expert gate (<= 4 models)
+constexpr int kRGBytes = kRMaxGateN * kRBK * 2;        // 8 KB
+constexpr int kRStageBytes = kRABytes + kRBBytes + kRGBytes;
 constexpr int kRSmemBytes = kRStages * kRStageBytes + 1024 + 256;
 constexpr int kRThreads = 192;
 constexpr int kRMaxE = 64;                             // logits one thread keeps in registers
@@ -32,6 +36,8 @@ struct RouteParams {
     const int32_t* model_of_tenant;
     const ModelWeights* models;
     const CUtensorMap* rmaps;      // one map per model over router_w [E,H], box Epad rows
+    const CUtensorMap* gmaps;      // one map per model over shared_gate_w [1,H], box 16 rows (15 read as zero)
+    int gate_mma;                  // 1: the gate logit is column m*16 of a second accumulator
     int32_t* topk_idx;
     float* topk_w;
     float* shared_gate;
@@ -76,7 +82,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
     if (warp == 1) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
-                     "r"((uint32_t)kRMaxN)
+                     "r"(512u)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -93,12 +99,15 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
                 if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, &s_abort, p.status)) { ok = false; break; }
                 const uint32_t sa = smem_base + stage * kRStageBytes, sb = sa + kRABytes;
                 const uint32_t full = bar_full + 8 * stage;
-                mbar_expect_tx(full, kRABytes + N * kRBK * 2);
+                mbar_expect_tx(full, kRABytes + N * kRBK * 2 + (p.gate_mma ? p.n_models * 16 * kRBK * 2 : 0));
                 armed |= 1u << stage;
                 armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
                 tma_load_2d(sa, &xmap, full, ks * kRBK, t0);
                 for (int m = 0; m < p.n_models; ++m)
                     tma_load_2d(sb + m * p.Epad * kRBK * 2, p.rmaps + m, full, ks * kRBK, 0);
+                if (p.gate_mma)
+                    for (int m = 0; m < p.n_models; ++m)
+                        tma_load_2d(sb + kRBBytes + m * 16 * kRBK * 2, p.gmaps + m, full, ks * kRBK, 0);
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
             }
             if (!ok)
@@ -109,16 +118,18 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t idesc_g = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_models * 16 >> 3) << 17) | ((128u >> 4) << 24);
             bool ok = true;
             for (int ks = 0; ks < ksteps; ++ks) {
                 if (!mbar_wait(bar_full + 8 * stage, phase, &s_abort, p.status)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t sa = smem_base + stage * kRStageBytes, sb = sa + kRABytes;
-                const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+                const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb), dg = smem_desc_sw128(sb + kRBBytes);
 #pragma unroll
                 for (int kk = 0; kk < kRBK / 16; ++kk) {
                     const uint64_t adv = (uint64_t)(kk * 32 >> 4);
                     umma_bf16(tmem_base, da + adv, db + adv, idesc, (ks | kk) ? 1u : 0u);
+                    if (p.gate_mma) umma_bf16(tmem_base + kRMaxN, da + adv, dg + adv, idesc_g, (ks | kk) ? 1u : 0u);
                 }
                 umma_commit(bar_empty + 8 * stage);
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
@@ -140,7 +151,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
         // shared-expert gate, overlapped with the MMA pipeline: each thread walks its own token's row
         // (independent 16-byte loads, four accumulators), so no cross-lane traffic is needed
         float gate = 0.5f;
-        if (p.shared_gate && valid) {
+        if (p.shared_gate && valid && !p.gate_mma) {
             const bf16* sg = p.models[model].shared_gate_w;
             if (sg) {
                 const uint4* xv = reinterpret_cast<const uint4*>(p.x + (size_t)t * p.H);
@@ -180,6 +191,14 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
                             for (int j = 0; j < 16; ++j) z[c * 16 + j] = __uint_as_float(r[j]);
                         }
                     }
+                }
+            }
+            if (p.gate_mma && p.shared_gate) {
+                for (int m = 0; m < p.n_models; ++m) {
+                    uint32_t r[16];
+                    tmem_ld16(taddr + kRMaxN + m * 16, r);
+                    tmem_ld_wait();
+                    if (m == model && valid && p.models[m].shared_gate_w) gate = 1.f / (1.f + expf(-__uint_as_float(r[0])));
                 }
             }
             if (valid) {
@@ -224,12 +243,13 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kRMaxN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
 }
 
 struct RouterMaps {
-    std::vector<CUtensorMap*> d_maps;     // per layer: device array of n_models maps
+    std::vector<CUtensorMap*> d_maps;     // per layer: device array of 2 * n_models maps (routers, then gates)
+    std::vector<int> gate_mma;            // per layer: every model has a gate vector and n_models <= 4
 };
 
 }  // namespace
@@ -260,17 +280,26 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     if (!c->rmaps) {
         RouterMaps* rm = new RouterMaps();
         rm->d_maps.assign(g.n_layers, nullptr);
+        rm->gate_mma.assign(g.n_layers, 0);
         c->rmaps = rm;
     }
     RouterMaps* rm = reinterpret_cast<RouterMaps*>(c->rmaps);
     if (!rm->d_maps[layer]) {
-        std::vector<CUtensorMap> maps(M);
-        for (int m = 0; m < M; ++m)
-            if (!make_map(&maps[m], c->models[(size_t)layer * M + m].router_w, E, H, epad, false)) return cudaErrorInvalidValue;
-        cudaError_t e = cudaMalloc((void**)&rm->d_maps[layer], M * sizeof(CUtensorMap));
+        std::vector<CUtensorMap> maps(2 * M);
+        memset(maps.data(), 0, maps.size() * sizeof(CUtensorMap));
+        int gate_mma = (M * 16 <= kRMaxGateN) ? 1 : 0;
+        for (int m = 0; m < M; ++m) {
+            const ModelWeights& mw = c->models[(size_t)layer * M + m];
+            if (!make_map(&maps[m], mw.router_w, E, H, epad, false)) return cudaErrorInvalidValue;
+            if (!mw.shared_gate_w) gate_mma = 0;
+        }
+        for (int m = 0; m < M && gate_mma; ++m)
+            if (!make_map(&maps[M + m], c->models[(size_t)layer * M + m].shared_gate_w, 1, H, 16, false)) gate_mma = 0;
+        cudaError_t e = cudaMalloc((void**)&rm->d_maps[layer], 2 * M * sizeof(CUtensorMap));
         if (e != cudaSuccess) return e;
-        e = cudaMemcpy(rm->d_maps[layer], maps.data(), M * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
+        e = cudaMemcpy(rm->d_maps[layer], maps.data(), 2 * M * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
         if (e != cudaSuccess) return e;
+        rm->gate_mma[layer] = gate_mma;
     }
     static bool attr_set = false;
     if (!attr_set) {
@@ -283,6 +312,7 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     p.x = x; p.tenant_id = tenant_id; p.T = T; p.H = H; p.E = E; p.Epad = epad; p.k = g.top_k;
     p.n_tenants = g.n_tenants; p.n_models = M; p.model_of_tenant = c->d_model_of_tenant;
     p.models = c->d_models + (size_t)layer * M; p.rmaps = rm->d_maps[layer];
+    p.gmaps = rm->d_maps[layer] + M; p.gate_mma = (shared_gate && rm->gate_mma[layer]) ? 1 : 0;
     p.topk_idx = topk_idx; p.topk_w = topk_w; p.shared_gate = shared_gate; p.tie_flag = tie_flag;
     p.status = c->ws.status;
     route_tc_kernel<<<(T + kRTokens - 1) / kRTokens, kRThreads, kRSmemBytes, st>>>(p, xmap);
