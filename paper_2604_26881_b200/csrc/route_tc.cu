@@ -16,7 +16,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int kRStages = 3;
+constexpr int kRMaxStages = 16;
 constexpr int kRBK = 64;
 constexpr int kRTokens = 128;
 constexpr int kRABytes = kRTokens * kRBK * 2;          // 16 KB of tokens per stage
@@ -24,8 +24,8 @@ constexpr int kRMaxN = 256;                            // router rows of all mod
 constexpr int kRBBytes = kRMaxN * kRBK * 2;            // 32 KB
 constexpr int kRMaxGateN = 64;                         // 16 columns per model for the shared-expert gate (<= 4 models)
 constexpr int kRGBytes = kRMaxGateN * kRBK * 2;        // 8 KB
-constexpr int kRStageBytes = kRABytes + kRBBytes + kRGBytes;
-constexpr int kRSmemBytes = kRStages * kRStageBytes + 1024 + 256;
+constexpr int kRTileBudget = 192 * 1024;               // shared memory for the pipeline stages
+constexpr int kRSmemBytes = kRTileBudget + kRABytes /* a short token tile is read as 128 rows */ + 1024 + 512;
 constexpr int kRThreads = 192;
 constexpr int kRMaxE = 64;                             // logits one thread keeps in registers
 
@@ -38,6 +38,7 @@ struct RouteParams {
     const CUtensorMap* rmaps;      // one map per model over router_w [E,H], box Epad rows
     const CUtensorMap* gmaps;      // one map per model over shared_gate_w [1,H], box 16 rows (15 read as zero)
     int gate_mma;                  // 1: the gate logit is column m*16 of a second accumulator
+    int a_bytes, b_bytes, stage_bytes, n_stages;   // pipeline geometry: small batches take more, smaller stages
     int32_t* topk_idx;
     float* topk_w;
     float* shared_gate;
@@ -63,8 +64,9 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
 {
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
-    const uint32_t bars = smem_base + kRStages * kRStageBytes;
-    const uint32_t bar_full = bars, bar_empty = bars + 8 * kRStages, bar_tfull = bars + 16 * kRStages;
+    const uint32_t bars = smem_base + kRTileBudget + kRABytes;
+    const uint32_t bar_full = bars, bar_empty = bars + 8 * kRMaxStages, bar_tfull = bars + 16 * kRMaxStages;
+    const int kRStages = p.n_stages;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
@@ -97,9 +99,9 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
             bool ok = true;
             for (int ks = 0; ks < ksteps; ++ks) {
                 if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, &s_abort, p.status)) { ok = false; break; }
-                const uint32_t sa = smem_base + stage * kRStageBytes, sb = sa + kRABytes;
+                const uint32_t sa = smem_base + stage * p.stage_bytes, sb = sa + p.a_bytes;
                 const uint32_t full = bar_full + 8 * stage;
-                mbar_expect_tx(full, kRABytes + N * kRBK * 2 + (p.gate_mma ? p.n_models * 16 * kRBK * 2 : 0));
+                mbar_expect_tx(full, p.a_bytes + N * kRBK * 2 + (p.gate_mma ? p.n_models * 16 * kRBK * 2 : 0));
                 armed |= 1u << stage;
                 armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
                 tma_load_2d(sa, &xmap, full, ks * kRBK, t0);
@@ -107,7 +109,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
                     tma_load_2d(sb + m * p.Epad * kRBK * 2, p.rmaps + m, full, ks * kRBK, 0);
                 if (p.gate_mma)
                     for (int m = 0; m < p.n_models; ++m)
-                        tma_load_2d(sb + kRBBytes + m * 16 * kRBK * 2, p.gmaps + m, full, ks * kRBK, 0);
+                        tma_load_2d(sb + p.b_bytes + m * 16 * kRBK * 2, p.gmaps + m, full, ks * kRBK, 0);
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
             }
             if (!ok)
@@ -123,8 +125,8 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
             for (int ks = 0; ks < ksteps; ++ks) {
                 if (!mbar_wait(bar_full + 8 * stage, phase, &s_abort, p.status)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t sa = smem_base + stage * kRStageBytes, sb = sa + kRABytes;
-                const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb), dg = smem_desc_sw128(sb + kRBBytes);
+                const uint32_t sa = smem_base + stage * p.stage_bytes, sb = sa + p.a_bytes;
+                const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb), dg = smem_desc_sw128(sb + p.b_bytes);
 #pragma unroll
                 for (int kk = 0; kk < kRBK / 16; ++kk) {
                     const uint64_t adv = (uint64_t)(kk * 32 >> 4);
@@ -306,8 +308,11 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
         cudaFuncSetAttribute(route_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes);
         attr_set = true;
     }
+    // token tile: only as many rows as the batch has (the MMA still reads 128 rows; the lanes of the
+    // rows that were not loaded are never looked at)
+    const int a_rows = T >= kRTokens ? kRTokens : ((T + 7) & ~7);
     CUtensorMap xmap;
-    if (!make_map(&xmap, x, T, H, kRTokens, false)) return cudaErrorInvalidValue;
+    if (!make_map(&xmap, x, T, H, a_rows, false)) return cudaErrorInvalidValue;
     RouteParams p;
     p.x = x; p.tenant_id = tenant_id; p.T = T; p.H = H; p.E = E; p.Epad = epad; p.k = g.top_k;
     p.n_tenants = g.n_tenants; p.n_models = M; p.model_of_tenant = c->d_model_of_tenant;
@@ -315,6 +320,11 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     p.gmaps = rm->d_maps[layer] + M; p.gate_mma = (shared_gate && rm->gate_mma[layer]) ? 1 : 0;
     p.topk_idx = topk_idx; p.topk_w = topk_w; p.shared_gate = shared_gate; p.tie_flag = tie_flag;
     p.status = c->ws.status;
+    p.a_bytes = (a_rows * kRBK * 2 + 1023) & ~1023;
+    p.b_bytes = (M * epad * kRBK * 2 + 1023) & ~1023;
+    p.stage_bytes = p.a_bytes + p.b_bytes + (p.gate_mma ? ((M * 16 * kRBK * 2 + 1023) & ~1023) : 0);
+    p.n_stages = kRTileBudget / p.stage_bytes;
+    if (p.n_stages > kRMaxStages) p.n_stages = kRMaxStages;
     route_tc_kernel<<<(T + kRTokens - 1) / kRTokens, kRThreads, kRSmemBytes, st>>>(p, xmap);
     c->launches += 1;
     return cudaGetLastError();
