@@ -144,6 +144,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap b_ro
                     if (armed & (1u << s)) mbar_wait(bar_full + 8 * s, (armed_phase >> s) & 1u, &s_abort, p.status);
             }
         }
+        __syncwarp();      // the whole warp reaches the block barrier below together
     } else if (warp == 1) {
         // ---------------- MMA issuer (one lane) ----------------
         if (lane == 0) {
@@ -176,6 +177,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap b_ro
                 if (++buf == 2) { buf = 0; bphase ^= 1; }
             }
         }
+        __syncwarp();
     } else {
         // ---------------- epilogue: 4 warps, one TMEM lane quarter each ----------------
         const int quarter = warp & 3;

@@ -35,8 +35,6 @@ struct RouteParams {
     int T, H, E, Epad, k, n_tenants, n_models;
     const int32_t* model_of_tenant;
     const ModelWeights* models;
-    const CUtensorMap* rmaps;      // one map per model over router_w [E,H], box Epad rows
-    const CUtensorMap* gmaps;      // one map per model over shared_gate_w [1,H], box 16 rows (15 read as zero)
     int gate_mma;                  // 1: the gate logit is column m*16 of a second accumulator
     int a_bytes, b_bytes, stage_bytes, n_stages;   // pipeline geometry: small batches take more, smaller stages
     int32_t* topk_idx;
@@ -44,6 +42,15 @@ struct RouteParams {
     float* shared_gate;
     uint8_t* tie_flag;
     int32_t* status;
+};
+
+constexpr int kRMaxModels = 4;
+
+// TMA descriptors, passed in kernel parameter space
+struct RouteMaps {
+    CUtensorMap x;                       // tokens [T,H], box a_rows
+    CUtensorMap r[kRMaxModels];          // router_w [E,H] of each model, box Epad rows
+    CUtensorMap g[kRMaxModels];          // shared_gate_w [1,H] of each model, box 16 rows (15 read as zero)
 };
 
 __device__ __forceinline__ float dot8f(const uint4& a, const uint4& b, float acc)
@@ -60,7 +67,7 @@ __device__ __forceinline__ float dot8f(const uint4& a, const uint4& b, float acc
 }
 
 __global__ void __launch_bounds__(kRThreads, 1)
-route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
+route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
 {
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -94,28 +101,34 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
     const uint32_t tmem_base = s_tmem_base;
 
     if (warp == 0) {
-        if (lane == 0) {
+        // three producer lanes (tokens / routers / gates) so that the TMA instructions of one stage are
+        // issued side by side; lane 0 also posts the byte count
+        if (lane < 3 && (lane < 2 || p.gate_mma)) {
             uint32_t stage = 0, phase = 0, armed = 0, armed_phase = 0;
             bool ok = true;
             for (int ks = 0; ks < ksteps; ++ks) {
                 if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, &s_abort, p.status)) { ok = false; break; }
                 const uint32_t sa = smem_base + stage * p.stage_bytes, sb = sa + p.a_bytes;
                 const uint32_t full = bar_full + 8 * stage;
-                mbar_expect_tx(full, p.a_bytes + N * kRBK * 2 + (p.gate_mma ? p.n_models * 16 * kRBK * 2 : 0));
                 armed |= 1u << stage;
                 armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
-                tma_load_2d(sa, &xmap, full, ks * kRBK, t0);
-                for (int m = 0; m < p.n_models; ++m)
-                    tma_load_2d(sb + m * p.Epad * kRBK * 2, p.rmaps + m, full, ks * kRBK, 0);
-                if (p.gate_mma)
+                if (lane == 0) {
+                    mbar_expect_tx(full, p.a_bytes + N * kRBK * 2 + (p.gate_mma ? p.n_models * 16 * kRBK * 2 : 0));
+                    tma_load_2d(sa, &maps.x, full, ks * kRBK, t0);
+                } else if (lane == 1) {
                     for (int m = 0; m < p.n_models; ++m)
-                        tma_load_2d(sb + p.b_bytes + m * 16 * kRBK * 2, p.gmaps + m, full, ks * kRBK, 0);
+                        tma_load_2d(sb + m * p.Epad * kRBK * 2, &maps.r[m], full, ks * kRBK, 0);
+                } else {
+                    for (int m = 0; m < p.n_models; ++m)
+                        tma_load_2d(sb + p.b_bytes + m * 16 * kRBK * 2, &maps.g[m], full, ks * kRBK, 0);
+                }
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
             }
             if (!ok)
                 for (int s = 0; s < kRStages; ++s)
                     if (armed & (1u << s)) mbar_wait(bar_full + 8 * s, (armed_phase >> s) & 1u, &s_abort, p.status);
         }
+        __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
@@ -138,6 +151,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
             }
             if (ok) umma_commit(bar_tfull);
         }
+        __syncwarp();
     } else {
         // ---- epilogue warps: thread <-> token (TMEM lane) ----
         const int quarter = warp & 3;
@@ -204,26 +218,49 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
                 }
             }
             if (valid) {
+                // Softmax is monotone, so the ranking is done on the logits themselves; the
+                // probabilities are exp2((z - zmax) * log2 e) / sum.  Four independent chains keep
+                // the one warp per scheduler busy.
                 const float* rb = p.models[model].router_bias;
-                float zmax = -INFINITY;
 #pragma unroll
                 for (int e = 0; e < kRMaxE; ++e) {
-                    if (e < p.E) { if (rb) z[e] += rb[e]; zmax = fmaxf(zmax, z[e]); }
+                    if (e < p.E) { if (rb) z[e] += rb[e]; }
                     else z[e] = -INFINITY;
                 }
-                float den = 0.f;
+                float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-                for (int e = 0; e < kRMaxE; ++e) { z[e] = (e < p.E) ? expf(z[e] - zmax) : 0.f; den += z[e]; }
+                for (int e = 0; e < kRMaxE; e += 4) {
+                    m0 = fmaxf(m0, z[e]); m1 = fmaxf(m1, z[e + 1]); m2 = fmaxf(m2, z[e + 2]); m3 = fmaxf(m3, z[e + 3]);
+                }
+                const float zmax = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+                const float kLog2e = 1.4426950408889634f;
+                float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
 #pragma unroll
-                for (int e = 0; e < kRMaxE; ++e) z[e] = (e < p.E) ? z[e] / den : -1.f;
+                for (int e = 0; e < kRMaxE; e += 4) {
+                    d0 += exp2f((z[e] - zmax) * kLog2e);     d1 += exp2f((z[e + 1] - zmax) * kLog2e);
+                    d2 += exp2f((z[e + 2] - zmax) * kLog2e); d3 += exp2f((z[e + 3] - zmax) * kLog2e);
+                }
+                const float inv_den = 1.f / ((d0 + d1) + (d2 + d3));
                 const int rounds = (p.k < p.E) ? p.k + 1 : p.k;
                 float prev = 0.f;
                 uint8_t flag = 0;
                 for (int j = 0; j < rounds; ++j) {
-                    float bv = -1.f;
-                    int bi = 0;
+                    // arg-max with ties to the lower id: each chain scans ids of one residue class in
+                    // ascending order, the merge prefers the larger value, then the smaller id
+                    float v0 = -INFINITY, v1 = -INFINITY, v2 = -INFINITY, v3 = -INFINITY;
+                    int i0 = 0, i1 = 1, i2 = 2, i3 = 3;
 #pragma unroll
-                    for (int e = 0; e < kRMaxE; ++e) if (z[e] > bv) { bv = z[e]; bi = e; }    // first maximum: lower id wins
+                    for (int e = 0; e < kRMaxE; e += 4) {
+                        if (z[e] > v0) { v0 = z[e]; i0 = e; }
+                        if (z[e + 1] > v1) { v1 = z[e + 1]; i1 = e + 1; }
+                        if (z[e + 2] > v2) { v2 = z[e + 2]; i2 = e + 2; }
+                        if (z[e + 3] > v3) { v3 = z[e + 3]; i3 = e + 3; }
+                    }
+                    if (v1 > v0 || (v1 == v0 && i1 < i0)) { v0 = v1; i0 = i1; }
+                    if (v3 > v2 || (v3 == v2 && i3 < i2)) { v2 = v3; i2 = i3; }
+                    if (v2 > v0 || (v2 == v0 && i2 < i0)) { v0 = v2; i0 = i2; }
+                    const int bi = i0;
+                    const float bv = exp2f((v0 - zmax) * kLog2e) * inv_den;
                     if (j > 0 && (prev - bv) < 1e-5f * prev) flag = 1;
                     prev = bv;
                     if (j < p.k) {
@@ -231,7 +268,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
                         p.topk_w[(size_t)t * p.k + j] = bad ? 0.f : bv;
                     }
 #pragma unroll
-                    for (int e = 0; e < kRMaxE; ++e) if (e == bi) z[e] = -1.f;
+                    for (int e = 0; e < kRMaxE; ++e) if (e == bi) z[e] = -INFINITY;
                 }
                 if (p.tie_flag) p.tie_flag[t] = flag;
                 if (p.shared_gate) p.shared_gate[t] = bad ? 0.f : gate;
@@ -250,8 +287,9 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ CUtensorMap xmap)
 }
 
 struct RouterMaps {
-    std::vector<CUtensorMap*> d_maps;     // per layer: device array of 2 * n_models maps (routers, then gates)
-    std::vector<int> gate_mma;            // per layer: every model has a gate vector and n_models <= 4
+    std::vector<RouteMaps> maps;          // per layer (the token map is filled per call)
+    std::vector<int> ready;
+    std::vector<int> gate_mma;            // per layer: every model has a gate vector
 };
 
 }  // namespace
@@ -260,15 +298,13 @@ bool route_tc_supported(const moe_ctx* c)
 {
     const moe_config& g = c->cfg;
     const int epad = (g.n_experts + 15) & ~15;
-    return g.n_experts <= kRMaxE && g.n_models * epad <= kRMaxN && g.hidden % kRBK == 0;
+    return g.n_experts <= kRMaxE && g.n_models <= kRMaxModels && g.n_models * epad <= kRMaxN && g.hidden % kRBK == 0;
 }
 
 void route_tc_destroy(moe_ctx* c)
 {
     RouterMaps* rm = reinterpret_cast<RouterMaps*>(c->rmaps);
     if (!rm) return;
-    cudaDeviceSynchronize();
-    for (CUtensorMap* p : rm->d_maps) if (p) cudaFree(p);
     delete rm;
     c->rmaps = nullptr;
 }
@@ -281,27 +317,25 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     const int epad = (E + 15) & ~15;
     if (!c->rmaps) {
         RouterMaps* rm = new RouterMaps();
-        rm->d_maps.assign(g.n_layers, nullptr);
+        rm->maps.resize(g.n_layers);
+        rm->ready.assign(g.n_layers, 0);
         rm->gate_mma.assign(g.n_layers, 0);
         c->rmaps = rm;
     }
     RouterMaps* rm = reinterpret_cast<RouterMaps*>(c->rmaps);
-    if (!rm->d_maps[layer]) {
-        std::vector<CUtensorMap> maps(2 * M);
-        memset(maps.data(), 0, maps.size() * sizeof(CUtensorMap));
-        int gate_mma = (M * 16 <= kRMaxGateN) ? 1 : 0;
+    if (!rm->ready[layer]) {
+        RouteMaps& mp = rm->maps[layer];
+        memset(&mp, 0, sizeof(mp));
+        int gate_mma = 1;
         for (int m = 0; m < M; ++m) {
             const ModelWeights& mw = c->models[(size_t)layer * M + m];
-            if (!make_map(&maps[m], mw.router_w, E, H, epad, false)) return cudaErrorInvalidValue;
+            if (!make_map(&mp.r[m], mw.router_w, E, H, epad, false)) return cudaErrorInvalidValue;
             if (!mw.shared_gate_w) gate_mma = 0;
         }
         for (int m = 0; m < M && gate_mma; ++m)
-            if (!make_map(&maps[M + m], c->models[(size_t)layer * M + m].shared_gate_w, 1, H, 16, false)) gate_mma = 0;
-        cudaError_t e = cudaMalloc((void**)&rm->d_maps[layer], 2 * M * sizeof(CUtensorMap));
-        if (e != cudaSuccess) return e;
-        e = cudaMemcpy(rm->d_maps[layer], maps.data(), 2 * M * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
-        if (e != cudaSuccess) return e;
+            if (!make_map(&mp.g[m], c->models[(size_t)layer * M + m].shared_gate_w, 1, H, 16, false)) gate_mma = 0;
         rm->gate_mma[layer] = gate_mma;
+        rm->ready[layer] = 1;
     }
     static bool attr_set = false;
     if (!attr_set) {
@@ -311,13 +345,13 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     // token tile: only as many rows as the batch has (the MMA still reads 128 rows; the lanes of the
     // rows that were not loaded are never looked at)
     const int a_rows = T >= kRTokens ? kRTokens : ((T + 7) & ~7);
-    CUtensorMap xmap;
-    if (!make_map(&xmap, x, T, H, a_rows, false)) return cudaErrorInvalidValue;
+    RouteMaps& mp = rm->maps[layer];
+    if (!make_map(&mp.x, x, T, H, a_rows, false)) return cudaErrorInvalidValue;
     RouteParams p;
     p.x = x; p.tenant_id = tenant_id; p.T = T; p.H = H; p.E = E; p.Epad = epad; p.k = g.top_k;
     p.n_tenants = g.n_tenants; p.n_models = M; p.model_of_tenant = c->d_model_of_tenant;
-    p.models = c->d_models + (size_t)layer * M; p.rmaps = rm->d_maps[layer];
-    p.gmaps = rm->d_maps[layer] + M; p.gate_mma = (shared_gate && rm->gate_mma[layer]) ? 1 : 0;
+    p.models = c->d_models + (size_t)layer * M;
+    p.gate_mma = (shared_gate && rm->gate_mma[layer]) ? 1 : 0;
     p.topk_idx = topk_idx; p.topk_w = topk_w; p.shared_gate = shared_gate; p.tie_flag = tie_flag;
     p.status = c->ws.status;
     p.a_bytes = (a_rows * kRBK * 2 + 1023) & ~1023;
@@ -325,7 +359,7 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     p.stage_bytes = p.a_bytes + p.b_bytes + (p.gate_mma ? ((M * 16 * kRBK * 2 + 1023) & ~1023) : 0);
     p.n_stages = kRTileBudget / p.stage_bytes;
     if (p.n_stages > kRMaxStages) p.n_stages = kRMaxStages;
-    route_tc_kernel<<<(T + kRTokens - 1) / kRTokens, kRThreads, kRSmemBytes, st>>>(p, xmap);
+    route_tc_kernel<<<(T + kRTokens - 1) / kRTokens, kRThreads, kRSmemBytes, st>>>(p, mp);
     c->launches += 1;
     return cudaGetLastError();
 }
