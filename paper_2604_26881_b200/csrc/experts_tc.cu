@@ -45,6 +45,7 @@ struct GemmParams {
     int ld_routed, ld_shared;
     const int32_t* shared_dst_rows;
     uint32_t idesc_fmt_routed, idesc_fmt_shared;   // operand format bits of the instruction descriptor
+    int stream_weights;           // 1: every weight tile is read once (small batch): mark it evict-first in L2
     int32_t* status;
 };
 
@@ -115,6 +116,8 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap b_ro
             uint32_t stage = 0, phase = 0;
             uint32_t armed = 0, armed_phase = 0;     // bit s: stage s has a load in flight / its phase
             bool ok = true;
+            const uint64_t pol_w = p.stream_weights ? l2_evict_first() : l2_evict_last();
+            const uint64_t pol_x = l2_evict_last();
             for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
                 const UnitInfo ui = decode_unit(p, u);
                 const CUtensorMap* ma0 = p.amaps + ui.amap0;
@@ -128,12 +131,13 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap b_ro
                     mbar_expect_tx(full, 2 * kABytes + ui.npad * kBK * 2);
                     armed |= 1u << stage;
                     armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
-                    tma_load_2d(sa0, ma0, full, ks * kBK, ui.a0_row);
-                    tma_load_2d(sa1, ma1, full, ks * kBK, ui.a1_row);
+                    tma_load_2d_hint(sa0, ma0, full, ks * kBK, ui.a0_row, pol_w);
+                    tma_load_2d_hint(sa1, ma1, full, ks * kBK, ui.a1_row, pol_w);
                     if (ui.npad == kTileRows) {
-                        tma_load_2d(sb, mb128, full, ks * kBK, ui.b_row0);
+                        tma_load_2d_hint(sb, mb128, full, ks * kBK, ui.b_row0, pol_x);
                     } else {
-                        for (int j = 0; j < ui.npad; j += 16) tma_load_2d(sb + j * kBK * 2, mb16, full, ks * kBK, ui.b_row0 + j);
+                        for (int j = 0; j < ui.npad; j += 16)
+                            tma_load_2d_hint(sb + j * kBK * 2, mb16, full, ks * kBK, ui.b_row0 + j, pol_x);
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
@@ -364,6 +368,7 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     p1.shared_dst_rows = nullptr;
     p1.idesc_fmt_routed = fmt_bf16; p1.idesc_fmt_shared = fmt_bf16;
     p1.status = c->ws.status;
+    p1.stream_weights = (R <= 2048) ? 1 : 0;
     grouped_gemm_kernel<0><<<c->sm_count, kThreads, kSmemBytes, st>>>(p1, br128, br16, bs128, bs16);
     stage_mark(c, st, kEvGateUp);
 

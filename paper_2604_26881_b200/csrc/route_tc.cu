@@ -106,6 +106,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
         if (lane < 3 && (lane < 2 || p.gate_mma)) {
             uint32_t stage = 0, phase = 0, armed = 0, armed_phase = 0;
             bool ok = true;
+            const uint64_t keep = l2_evict_last();      // router weights and tokens are read again soon
             for (int ks = 0; ks < ksteps; ++ks) {
                 if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, &s_abort, p.status)) { ok = false; break; }
                 const uint32_t sa = smem_base + stage * p.stage_bytes, sb = sa + p.a_bytes;
@@ -114,13 +115,13 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                 armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
                 if (lane == 0) {
                     mbar_expect_tx(full, p.a_bytes + N * kRBK * 2 + (p.gate_mma ? p.n_models * 16 * kRBK * 2 : 0));
-                    tma_load_2d(sa, &maps.x, full, ks * kRBK, t0);
+                    tma_load_2d_hint(sa, &maps.x, full, ks * kRBK, t0, keep);
                 } else if (lane == 1) {
                     for (int m = 0; m < p.n_models; ++m)
-                        tma_load_2d(sb + m * p.Epad * kRBK * 2, &maps.r[m], full, ks * kRBK, 0);
+                        tma_load_2d_hint(sb + m * p.Epad * kRBK * 2, &maps.r[m], full, ks * kRBK, 0, keep);
                 } else {
                     for (int m = 0; m < p.n_models; ++m)
-                        tma_load_2d(sb + p.b_bytes + m * 16 * kRBK * 2, &maps.g[m], full, ks * kRBK, 0);
+                        tma_load_2d_hint(sb + p.b_bytes + m * 16 * kRBK * 2, &maps.g[m], full, ks * kRBK, 0, keep);
                 }
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
             }
@@ -244,6 +245,8 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                 const int rounds = (p.k < p.E) ? p.k + 1 : p.k;
                 float prev = 0.f;
                 uint8_t flag = 0;
+                uint32_t taken_lo = 0, taken_hi = 0;      // experts already selected (a bit mask: writing to
+                                                          // z[bi] would be a data-dependent register index)
                 for (int j = 0; j < rounds; ++j) {
                     // arg-max with ties to the lower id: each chain scans ids of one residue class in
                     // ascending order, the merge prefers the larger value, then the smaller id
@@ -251,10 +254,11 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                     int i0 = 0, i1 = 1, i2 = 2, i3 = 3;
 #pragma unroll
                     for (int e = 0; e < kRMaxE; e += 4) {
-                        if (z[e] > v0) { v0 = z[e]; i0 = e; }
-                        if (z[e + 1] > v1) { v1 = z[e + 1]; i1 = e + 1; }
-                        if (z[e + 2] > v2) { v2 = z[e + 2]; i2 = e + 2; }
-                        if (z[e + 3] > v3) { v3 = z[e + 3]; i3 = e + 3; }
+                        const uint32_t tk = (e < 32) ? taken_lo : taken_hi;
+                        if (z[e] > v0 && !(tk & (1u << (e & 31)))) { v0 = z[e]; i0 = e; }
+                        if (z[e + 1] > v1 && !(tk & (1u << ((e + 1) & 31)))) { v1 = z[e + 1]; i1 = e + 1; }
+                        if (z[e + 2] > v2 && !(tk & (1u << ((e + 2) & 31)))) { v2 = z[e + 2]; i2 = e + 2; }
+                        if (z[e + 3] > v3 && !(tk & (1u << ((e + 3) & 31)))) { v3 = z[e + 3]; i3 = e + 3; }
                     }
                     if (v1 > v0 || (v1 == v0 && i1 < i0)) { v0 = v1; i0 = i1; }
                     if (v3 > v2 || (v3 == v2 && i3 < i2)) { v2 = v3; i2 = i3; }
@@ -267,8 +271,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                         p.topk_idx[(size_t)t * p.k + j] = bad ? j : bi;
                         p.topk_w[(size_t)t * p.k + j] = bad ? 0.f : bv;
                     }
-#pragma unroll
-                    for (int e = 0; e < kRMaxE; ++e) if (e == bi) z[e] = -INFINITY;
+                    if (bi < 32) taken_lo |= 1u << bi; else taken_hi |= 1u << (bi - 32);
                 }
                 if (p.tie_flag) p.tie_flag[t] = flag;
                 if (p.shared_gate) p.shared_gate[t] = bad ? 0.f : gate;
