@@ -63,7 +63,8 @@ enum {
  * (experts: hidden % 256 == 0; router: n_experts <= 64 and n_models * ceil16(n_experts) <= 256),
  * FMA forces the CUDA-core kernels, TCGEN05 fails with MOE_ERR_UNSUPPORTED if not possible. */
 enum { MOE_PATH_AUTO = 0, MOE_PATH_FMA = 1, MOE_PATH_TCGEN05 = 2 };
-enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2 };
+enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2,
+       MOE_OPT_PAIR_MODE = 3 /* 1 (default): long expert tiles use the 2-CTA tcgen05 shape; 0: never */ };
 
 typedef struct {
     int32_t hidden;        /* H */
@@ -158,12 +159,14 @@ int moe_dispatch(moe_ctx* ctx, const void* x, const int32_t* topk_idx, const int
  * routed experts and to fp16 for the shared expert before the down projection; the
  * results stay in fp32 so that the aggregation rounds only once)
  * G orders the work by expert block; results are bit-identical for every G.
- * x bf16 [T,H] and tenant_id are needed only when y_shared is requested.
- * x_perm must be readable for 128 rows past T*k (the tensor-core path loads whole
- * row tiles; what lies there is never used).
+ * x bf16 [T,H] and tenant_id are needed only when y_shared is requested.  perm (the
+ * output of moe_dispatch) may be NULL; with x and perm given and at most 128 tokens of a
+ * single model, the routed experts read the tokens in place instead of x_perm (same
+ * results).
  */
-int moe_experts(moe_ctx* ctx, int layer, const void* x, const void* x_perm, const int32_t* expert_off,
-                const int32_t* tenant_id, int T, int G, float* y_perm, float* y_shared, void* stream);
+int moe_experts(moe_ctx* ctx, int layer, const void* x, const void* x_perm, const int32_t* perm,
+                const int32_t* expert_off, const int32_t* tenant_id, int T, int G, float* y_perm, float* y_shared,
+                void* stream);
 
 /*
  * Aggregation (Sec. 3, Sec. 4.2):

@@ -22,6 +22,7 @@ MOE_ERR_CUDA, MOE_ERR_ALLOC, MOE_ERR_UNSUPPORTED = -5, -6, -7
 MOE_DEV_BAD_TENANT, MOE_DEV_BAD_EXPERT, MOE_DEV_TIMEOUT = 1, 2, 8
 MOE_OPT_EXPERT_PATH = 1
 MOE_OPT_ROUTE_PATH = 2
+MOE_OPT_PAIR_MODE = 3
 MOE_PATH_AUTO, MOE_PATH_FMA, MOE_PATH_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["moe_create", "moe_destroy", "moe_set_expert_pool", "moe_set_model_weights", "moe_set_slot_table",
@@ -71,7 +72,7 @@ def load_library(path: str | None = None):
         lib.moe_set_option.argtypes = [c_void_p, c_int, c_int]
         lib.moe_route.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int] + [c_void_p] * 5
         lib.moe_dispatch.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int] + [c_void_p] * 7
-        lib.moe_experts.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int,
+        lib.moe_experts.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int,
                                     c_void_p, c_void_p, c_void_p]
         lib.moe_combine.argtypes = [c_void_p] + [c_void_p] * 5 + [c_int, c_void_p, c_void_p]
         lib.moe_layer_forward.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p]
@@ -169,8 +170,8 @@ def moe_dispatch_noalloc(topk_idx, tenant_id, model_of_tenant, T, k, E, M, n_ten
         _ptr(tenant_expert_count), _ptr(expert_off), _ptr(group_off), _ptr(status_out), _stream(stream)))
 
 
-def moe_experts(ctx, layer, x, x_perm, expert_off, tenant_id, T, G, y_perm, y_shared=None, stream=None):
-    _check("moe_experts", load_library().moe_experts(ctx, layer, _ptr(x), _ptr(x_perm), _ptr(expert_off),
+def moe_experts(ctx, layer, x, x_perm, perm, expert_off, tenant_id, T, G, y_perm, y_shared=None, stream=None):
+    _check("moe_experts", load_library().moe_experts(ctx, layer, _ptr(x), _ptr(x_perm), _ptr(perm), _ptr(expert_off),
                                                      _ptr(tenant_id), T, G, _ptr(y_perm), _ptr(y_shared),
                                                      _stream(stream)))
 

@@ -42,7 +42,7 @@ int alloc_workspace(moe_ctx* c)
     c->nblk_tok = div_up((int)T, kDispatchChunk);
     c->max_tiles = div_up((int)R, kTileRows) + (int)ME;
     c->max_stiles = div_up((int)T, kTileRows) + g.n_models;
-    const int nblk1 = g.inter / 128, nblk2 = div_up(g.hidden, 256), snblk1 = g.shared_inter / 128;
+    const int nblk1 = g.inter / 64, nblk2 = div_up(g.hidden, 128), snblk1 = g.shared_inter / 64;
     c->max_units1 = c->max_tiles * nblk1 + c->max_stiles * snblk1;
     c->max_units2 = (c->max_tiles + c->max_stiles) * nblk2;
 
@@ -123,8 +123,9 @@ bool use_tc(const moe_ctx* c)
     return tc_supported(c);
 }
 
-int experts_impl(moe_ctx* c, int layer, const bf16* x, const bf16* x_perm, const int32_t* expert_off,
-                 const int32_t* tenant_id, int T, int G, float* y_perm, float* y_shared, cudaStream_t st)
+int experts_impl(moe_ctx* c, int layer, const bf16* x, const bf16* x_perm, const int32_t* perm,
+                 const int32_t* expert_off, const int32_t* tenant_id, int T, int G, float* y_perm, float* y_shared,
+                 cudaStream_t st)
 {
     const moe_config& g = c->cfg;
     const bool with_shared = y_shared != nullptr && g.shared_inter > 0;
@@ -140,7 +141,8 @@ int experts_impl(moe_ctx* c, int layer, const bf16* x, const bf16* x_perm, const
     if (use_tc(c)) {
         const int rc = tc_setup_layer(c, layer);
         if (rc != MOE_OK) return rc;
-        MOE_CUDA(c, launch_experts_tc(c, layer, xs, x_perm, T, y_perm, with_shared ? y_shared : nullptr, dst_rows, st));
+        MOE_CUDA(c, launch_experts_tc(c, layer, xs, x_perm, perm, T, y_perm, with_shared ? y_shared : nullptr, dst_rows,
+                                      st));
     } else {
         MOE_CUDA(c, launch_experts_fma(c, layer, xs, x_perm, T, y_perm, with_shared ? y_shared : nullptr, dst_rows, st));
     }
@@ -157,10 +159,12 @@ int layer_forward_impl(moe_ctx* c, int layer, const bf16* x, const int32_t* tena
     MOE_CUDA(c, launch_route(c, layer, x, tenant_id, T, w.topk_idx, w.topk_w, shared ? w.shared_gate : nullptr,
                              w.tie_flag, st));
     stage_mark(c, st, kEvRoute);
+    // with few tokens the tensor-core experts read the tokens in place: no permuted copy to make
+    const bool direct = use_tc(c) && tc_direct_mode(c, T);
     MOE_CUDA(c, launch_dispatch(c, x, w.topk_idx, tenant_id, T, G, w.perm, w.inv_perm, w.tenant_expert_count,
-                                w.expert_off, w.group_off, w.x_perm, st));
+                                w.expert_off, w.group_off, direct ? nullptr : w.x_perm, st));
     stage_mark(c, st, kEvDispatch);
-    const int rc = experts_impl(c, layer, x, w.x_perm, w.expert_off, tenant_id, T, G, w.y_perm,
+    const int rc = experts_impl(c, layer, x, w.x_perm, w.perm, w.expert_off, tenant_id, T, G, w.y_perm,
                                 shared ? w.y_shared : nullptr, st);
     if (rc != MOE_OK) return rc;
     MOE_CUDA(c, launch_combine(c, w.y_perm, w.inv_perm, w.topk_w, shared ? w.y_shared : nullptr,
@@ -197,6 +201,7 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->tmaps = nullptr;
     c->rmaps = nullptr;
     c->route_path = MOE_PATH_AUTO;
+    c->pair_mode_enabled = 1;
     c->timing = false;
     for (auto& e : c->ev) e = nullptr;
     c->errbuf[0] = 0;
@@ -318,6 +323,10 @@ int moe_set_option(moe_ctx* c, int option, int value)
         c->expert_path = value;
         return MOE_OK;
     }
+    if (option == MOE_OPT_PAIR_MODE) {
+        c->pair_mode_enabled = value ? 1 : 0;
+        return MOE_OK;
+    }
     if (option == MOE_OPT_ROUTE_PATH) {
         if (value < MOE_PATH_AUTO || value > MOE_PATH_TCGEN05) return MOE_ERR_SHAPE;
         if (value == MOE_PATH_TCGEN05 && !route_tc_supported(c)) return MOE_ERR_UNSUPPORTED;
@@ -354,7 +363,7 @@ int moe_dispatch(moe_ctx* c, const void* x, const int32_t* topk_idx, const int32
     return MOE_OK;
 }
 
-int moe_experts(moe_ctx* c, int layer, const void* x, const void* x_perm, const int32_t* expert_off,
+int moe_experts(moe_ctx* c, int layer, const void* x, const void* x_perm, const int32_t* perm, const int32_t* expert_off,
                 const int32_t* tenant_id, int T, int G, float* y_perm, float* y_shared, void* stream)
 {
     if (!c || !x_perm || !expert_off || !y_perm) return MOE_ERR_NULL;
@@ -365,8 +374,9 @@ int moe_experts(moe_ctx* c, int layer, const void* x, const void* x_perm, const 
     const int rc = check_layer_ready(c, layer, true, y_shared != nullptr);
     if (rc != MOE_OK) return rc;
     if (T == 0) return MOE_OK;
-    return experts_impl(c, layer, (const bf16*)x, (const bf16*)x_perm, expert_off, tenant_id, T, G, (float*)y_perm,
-                        (float*)y_shared, (cudaStream_t)stream);
+    // reading the tokens in place needs x and perm; without them the permuted copy is used
+    return experts_impl(c, layer, (const bf16*)x, (const bf16*)x_perm, x ? perm : nullptr, expert_off, tenant_id, T, G,
+                        (float*)y_perm, (float*)y_shared, (cudaStream_t)stream);
 }
 
 int moe_combine(moe_ctx* c, const float* y_perm, const int32_t* inv_perm, const float* topk_w, const float* y_shared,

@@ -3,10 +3,21 @@
 //   gate/up:  h[r, c]  = silu(W_g[c,:] . x[r,:]) * (W_u[c,:] . x[r,:])        (SwiGLU in the epilogue)
 //   down:     y[r, c]  = W_d[c,:] . h[r,:]
 // (paper Sec. 3: an expert block computes on the tokens assigned to it; only activated experts are
-// touched.)  The weight rows are the M operand of the MMA (128 rows per instruction, two
-// instructions per unit), the tokens of one expert tile are the N operand (16..128, a multiple of
-// 16), so a decode-sized tile streams each weight byte once through a narrow MMA and a prefill tile
-// uses the full 128x128 shape with no padding of ragged expert segments beyond 16 rows.
+// touched.)
+//
+// Orientation: the weight rows are the M operand of the MMA (128 rows per CTA), the tokens of one
+// expert tile are the N operand (16..256, a multiple of 16).  A decode-sized tile therefore streams
+// each weight byte once through a narrow MMA, and a prefill tile pads a ragged expert segment to 16
+// rows, not to 128.  For gate/up the 128 weight rows of a tile are 64 gate rows interleaved with
+// the 64 up rows of the same intermediate indices (a 3-D TMA box over the two weight arrays puts
+// them on neighbouring TMEM lanes), so SwiGLU needs one lane-pair shuffle and one accumulator.
+//
+// Two launch shapes of the same kernel:
+//   single (PAIR = false): one CTA per unit, units handed out through an atomic counter (longest
+//     units first), used when tiles are short (decode, many small experts);
+//   pair (PAIR = true): a cluster of two CTAs shares the token tile of a unit through
+//     tcgen05.mma.cta_group::2 -- each CTA loads half of the tokens and its own 128 weight rows, so
+//     the bytes fetched per FLOP drop by a third; used when tiles are long (prefill).
 // Routed-expert units and shared-expert units ride in the same launch.
 #include <cuda_fp16.h>
 
@@ -22,127 +33,249 @@ namespace {
 
 using namespace tc;
 
-constexpr int kStages = 4;
-constexpr int kBK = 64;                       // K elements per stage = one 128-byte swizzle row
-constexpr int kABytes = 128 * kBK * 2;        // one 128-row weight tile: 16 KB
-constexpr int kBBytes = kTileRows * kBK * 2;  // up to 128 token rows: 16 KB
-constexpr int kStageBytes = 2 * kABytes + kBBytes;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
-constexpr int kThreads = 192;                 // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: epilogue
-constexpr uint32_t kTmemCols = 512;           // 2 buffers x (2 accumulators x 128 columns)
+constexpr int kStages = 6;
+constexpr int kBK = 64;                        // K elements per stage = one 128-byte swizzle row
+constexpr int kABytes = 128 * kBK * 2;         // 128 weight rows: 16 KB
+constexpr int kBRows = 128;                    // token rows one CTA loads per stage (pair: half of the tile)
+constexpr int kBBytes = kBRows * kBK * 2;      // 16 KB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kQueue = 4;                      // depth of the unit queue of the dynamic scheduler
+constexpr int kNumBars = 2 * kStages + 4 + 2 * kQueue;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 8 * kNumBars + 64;
+constexpr int kThreads = 192;                  // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: epilogue
+constexpr uint32_t kTmemCols = 512;            // 2 accumulator buffers x 256 columns
 
 struct GemmParams {
     const Unit* units;
     const int32_t* n_units;
+    int32_t* counter;             // work counter of the dynamic scheduler (zeroed by the plan kernel)
     const Tile* tiles;
     const Tile* stiles;
-    const CUtensorMap* amaps;     // [0],[1]: routed A0/A1; [2+2m],[3+2m]: shared A0/A1 of model m
+    const int32_t* perm;          // direct mode: routed row -> flat (token, j) id
+    int top_k;
+    int direct;                   // 1: routed gate/up units read the tokens in place and pick their columns
+    int n_tokens_pad;             // direct mode: tokens rounded up to 16
     int k_routed, k_shared;       // contraction lengths
-    int rows_per_slot;            // weight rows per pool slot in the routed A maps
-    int cb_stride, a1_off;        // A0 row = base + cb*cb_stride, A1 row = A0 row + a1_off
+    int rows_per_slot;            // weight rows per pool slot in the routed A map
+    int cb_rows;                  // weight rows (gate/up: intermediate indices) per colblock: 64 or 128
     void* out_routed;
     void* out_shared;
     int ld_routed, ld_shared;
     const int32_t* shared_dst_rows;
     uint32_t idesc_fmt_routed, idesc_fmt_shared;   // operand format bits of the instruction descriptor
-    int stream_weights;           // 1: every weight tile is read once (small batch): mark it evict-first in L2
+    uint32_t gate_first_routed;   // bit 0: the gate row is the even TMEM lane of a pair (routed map)
+    uint32_t gate_first_shared;   // bit m: same for the shared expert of model m
+    int stream_weights;           // 1: every weight tile is read once: mark it evict-first in L2
     int32_t* status;
 };
 
-struct UnitInfo {
-    int a0_row, a1_row, amap0, amap1;
-    int b_row0, nrows, npad, ksteps, shared, cb;
+constexpr int kTcMaxModels = 8;
+
+// TMA descriptors in kernel-parameter space
+struct GemmMaps {
+    CUtensorMap a_routed;                  // gate/up: 3-D (K, {gate,up}, S*I); down: 2-D (K, S*H)
+    CUtensorMap a_shared[kTcMaxModels];    // same for the shared expert of each model
+    CUtensorMap b_routed128, b_routed16;   // activations of the routed units, boxes of 128 / 16 rows
+    CUtensorMap b_shared128, b_shared16;
 };
 
-__device__ __forceinline__ UnitInfo decode_unit(const GemmParams& p, int u)
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z,
+                                                 uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "l"(policy)
+        : "memory");
+}
+// pair mode: the load lands in this CTA's shared memory, its bytes are counted on the leader's barrier
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+                                                 uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(map), "r"(bar & 0xFEFFFFFFu), "r"(x), "r"(y), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z,
+                                                 uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+        ::"r"(dst), "l"(map), "r"(bar & 0xFEFFFFFFu), "r"(x), "r"(y), "r"(z), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrives on the barrier at the same offset in both CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((unsigned short)3)
+                 : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld1(uint32_t taddr, uint32_t& r)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr));
+}
+
+struct UnitInfo {
+    int a_row, amap;              // first weight row of the tile; -1: routed map, m: shared map of model m
+    int b_row0, nrows, npad, ksteps, shared, cb, model;
+    int direct;                   // routed gate/up unit in direct mode: B = all tokens
+};
+
+template <int MODE, bool PAIR>
+__device__ __forceinline__ UnitInfo decode_unit(const GemmParams& p, int u, uint32_t rank)
 {
     const Unit un = p.units[u];
     UnitInfo ui;
     ui.shared = un.tile < 0;
     const Tile t = ui.shared ? p.stiles[~un.tile] : p.tiles[un.tile];
-    ui.cb = un.colblock;
-    const int base = ui.shared ? 0 : t.slot * p.rows_per_slot;
-    ui.a0_row = base + un.colblock * p.cb_stride;
-    ui.a1_row = ui.a0_row + p.a1_off;
-    ui.amap0 = ui.shared ? 2 + 2 * t.slot : 0;
-    ui.amap1 = ui.amap0 + 1;
+    ui.cb = PAIR ? 2 * un.colblock + (int)rank : un.colblock;
+    ui.model = t.slot;
+    ui.amap = ui.shared ? t.slot : -1;
+    ui.a_row = (ui.shared ? 0 : t.slot * p.rows_per_slot) + ui.cb * p.cb_rows;
     ui.b_row0 = t.row0;
     ui.nrows = t.nrows;
-    ui.npad = (t.nrows + 15) & ~15;
+    ui.direct = (MODE == 0 && p.direct && !ui.shared) ? 1 : 0;
+    if (ui.direct) { ui.npad = p.n_tokens_pad; }
+    else if (PAIR) ui.npad = (t.nrows + 31) & ~31;
+    else ui.npad = (t.nrows + 15) & ~15;
     ui.ksteps = (ui.shared ? p.k_shared : p.k_routed) / kBK;
     return ui;
 }
 
 // MODE 0: gate/up + SwiGLU (output bf16 for routed units, fp16 for shared units)
 // MODE 1: down projection (output fp32)
-template <int MODE>
+template <int MODE, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
-grouped_gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap b_routed128,
-                    const __grid_constant__ CUtensorMap b_routed16, const __grid_constant__ CUtensorMap b_shared128,
-                    const __grid_constant__ CUtensorMap b_shared16)
+grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
 {
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
     const uint32_t bars = smem_base + kStages * kStageBytes;                   // 8-byte barriers after the tiles
     const uint32_t bar_full = bars, bar_empty = bars + 8 * kStages;
     const uint32_t bar_tfull = bars + 16 * kStages, bar_tempty = bar_tfull + 16;
+    const uint32_t bar_qfull = bar_tempty + 16, bar_qempty = bar_qfull + 8 * kQueue;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
+    __shared__ int s_queue[kQueue];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+    const bool leader = rank == 0;
     const int n_units = *p.n_units;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, PAIR ? 8 : 4); }
+        for (int q = 0; q < kQueue; ++q) { mbar_init(bar_qfull + 8 * q, 1); mbar_init(bar_qempty + 8 * q, 5); }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
         __syncwarp();
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
-                     "r"(kTmemCols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                         "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                         "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();          // the peer's barriers are initialised before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
 
+    // unit sequence: pair mode walks the list with a fixed stride; single mode pulls from a counter
+    const int stride = PAIR ? (int)(gridDim.x >> 1) : 0;
+    const int first = PAIR ? (int)(blockIdx.x >> 1) : 0;
+
     if (warp == 0) {
-        // ---------------- TMA producer (one lane) ----------------
+        // ---------------- TMA producer (one lane); in single mode also the scheduler ----------------
         if (lane == 0) {
-            uint32_t stage = 0, phase = 0;
-            uint32_t armed = 0, armed_phase = 0;     // bit s: stage s has a load in flight / its phase
+            uint32_t stage = 0, phase = 0, q = 0, qphase = 0;
+            uint32_t armed = 0, armed_phase = 0;
             bool ok = true;
             const uint64_t pol_w = p.stream_weights ? l2_evict_first() : l2_evict_last();
             const uint64_t pol_x = l2_evict_last();
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-                const UnitInfo ui = decode_unit(p, u);
-                const CUtensorMap* ma0 = p.amaps + ui.amap0;
-                const CUtensorMap* ma1 = p.amaps + ui.amap1;
-                const CUtensorMap* mb128 = ui.shared ? &b_shared128 : &b_routed128;
-                const CUtensorMap* mb16 = ui.shared ? &b_shared16 : &b_routed16;
+            int u = first;
+            while (ok) {
+                if (!PAIR) {
+                    if (!mbar_wait(bar_qempty + 8 * q, qphase ^ 1, &s_abort, p.status)) { ok = false; break; }
+                    u = atomicAdd(p.counter, 1);
+                    if (u >= n_units) u = -1;
+                    s_queue[q] = u;
+                    mbar_arrive(bar_qfull + 8 * q);
+                    if (++q == kQueue) { q = 0; qphase ^= 1; }
+                    if (u < 0) break;
+                } else if (u >= n_units) {
+                    break;
+                }
+                const UnitInfo ui = decode_unit<MODE, PAIR>(p, u, rank);
+                const CUtensorMap* ma = ui.amap < 0 ? &maps.a_routed : &maps.a_shared[ui.amap];
+                const bool bshared = ui.shared || ui.direct;
+                const CUtensorMap* mb128 = bshared ? &maps.b_shared128 : &maps.b_routed128;
+                const CUtensorMap* mb16 = bshared ? &maps.b_shared16 : &maps.b_routed16;
+                const int brow0 = ui.direct ? 0 : ui.b_row0;
+                const int my_rows = PAIR ? (ui.npad >> 1) : ui.npad;          // token rows this CTA loads
+                const int my_row0 = brow0 + (PAIR ? (int)rank * my_rows : 0);
                 for (int ks = 0; ks < ui.ksteps; ++ks) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, &s_abort, p.status)) { ok = false; break; }
-                    const uint32_t sa0 = smem_base + stage * kStageBytes, sa1 = sa0 + kABytes, sb = sa1 + kABytes;
+                    const uint32_t sa = smem_base + stage * kStageBytes, sb = sa + kABytes;
                     const uint32_t full = bar_full + 8 * stage;
-                    mbar_expect_tx(full, 2 * kABytes + ui.npad * kBK * 2);
+                    if (leader) mbar_expect_tx(full, (PAIR ? 2u : 1u) * (uint32_t)(kABytes + my_rows * kBK * 2));
                     armed |= 1u << stage;
                     armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
-                    tma_load_2d_hint(sa0, ma0, full, ks * kBK, ui.a0_row, pol_w);
-                    tma_load_2d_hint(sa1, ma1, full, ks * kBK, ui.a1_row, pol_w);
-                    if (ui.npad == kTileRows) {
-                        tma_load_2d_hint(sb, mb128, full, ks * kBK, ui.b_row0, pol_x);
+                    if (PAIR) {
+                        if (MODE == 0) tma_load_3d_pair(sa, ma, full, ks * kBK, 0, ui.a_row, pol_w);
+                        else tma_load_2d_pair(sa, ma, full, ks * kBK, ui.a_row, pol_w);
+                        int j = 0;
+                        for (; j + 128 <= my_rows; j += 128) tma_load_2d_pair(sb + j * kBK * 2, mb128, full, ks * kBK, my_row0 + j, pol_x);
+                        for (; j < my_rows; j += 16) tma_load_2d_pair(sb + j * kBK * 2, mb16, full, ks * kBK, my_row0 + j, pol_x);
                     } else {
-                        for (int j = 0; j < ui.npad; j += 16)
-                            tma_load_2d_hint(sb + j * kBK * 2, mb16, full, ks * kBK, ui.b_row0 + j, pol_x);
+                        if (MODE == 0) tma_load_3d_hint(sa, ma, full, ks * kBK, 0, ui.a_row, pol_w);
+                        else tma_load_2d_hint(sa, ma, full, ks * kBK, ui.a_row, pol_w);
+                        int j = 0;
+                        for (; j + 128 <= my_rows; j += 128) tma_load_2d_hint(sb + j * kBK * 2, mb128, full, ks * kBK, my_row0 + j, pol_x);
+                        for (; j < my_rows; j += 16) tma_load_2d_hint(sb + j * kBK * 2, mb16, full, ks * kBK, my_row0 + j, pol_x);
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
+                if (PAIR) u += stride;
             }
-            if (!ok) {
+            if (!ok && leader) {
                 // gave up: let the copies already in flight land before the block exits
                 for (int s = 0; s < kStages; ++s)
                     if (armed & (1u << s)) mbar_wait(bar_full + 8 * s, (armed_phase >> s) & 1u, &s_abort, p.status);
@@ -150,35 +283,47 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap b_ro
         }
         __syncwarp();      // the whole warp reaches the block barrier below together
     } else if (warp == 1) {
-        // ---------------- MMA issuer (one lane) ----------------
-        if (lane == 0) {
-            uint32_t stage = 0, phase = 0, buf = 0, bphase = 0;
+        // ---------------- MMA issuer (one lane; in pair mode only the leader CTA issues) ----------------
+        if (lane == 0 && leader) {
+            uint32_t stage = 0, phase = 0, buf = 0, bphase = 0, q = 0, qphase = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-                const UnitInfo ui = decode_unit(p, u);
+            int u = first;
+            while (ok) {
+                if (!PAIR) {
+                    if (!mbar_wait(bar_qfull + 8 * q, qphase, &s_abort, p.status)) { ok = false; break; }
+                    u = s_queue[q];
+                    mbar_arrive(bar_qempty + 8 * q);
+                    if (++q == kQueue) { q = 0; qphase ^= 1; }
+                    if (u < 0) break;
+                } else if (u >= n_units) {
+                    break;
+                }
+                const UnitInfo ui = decode_unit<MODE, PAIR>(p, u, rank);
                 const uint32_t fmt = ui.shared ? p.idesc_fmt_shared : p.idesc_fmt_routed;
-                const uint32_t idesc = (1u << 4) | fmt | ((uint32_t)(ui.npad >> 3) << 17) | ((128u >> 4) << 24);
+                const uint32_t idesc = (1u << 4) | fmt | ((uint32_t)(ui.npad >> 3) << 17) | (((PAIR ? 256u : 128u) >> 4) << 24);
                 if (!mbar_wait(bar_tempty + 8 * buf, bphase ^ 1, &s_abort, p.status)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d0 = tmem_base + buf * 256, d1 = d0 + 128;
+                const uint32_t d = tmem_base + buf * 256;
                 for (int ks = 0; ks < ui.ksteps; ++ks) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, &s_abort, p.status)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa0 = smem_base + stage * kStageBytes, sa1 = sa0 + kABytes, sb = sa1 + kABytes;
-                    const uint64_t da0 = smem_desc_sw128(sa0), da1 = smem_desc_sw128(sa1), db = smem_desc_sw128(sb);
+                    const uint32_t sa = smem_base + stage * kStageBytes, sb = sa + kABytes;
+                    const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
 #pragma unroll
                     for (int kk = 0; kk < kBK / 16; ++kk) {
                         const uint32_t acc = (ks | kk) ? 1u : 0u;
                         const uint64_t adv = (uint64_t)(kk * 32 >> 4);      // 16 elements = 32 bytes along K
-                        umma_bf16(d0, da0 + adv, db + adv, idesc, acc);
-                        umma_bf16(d1, da1 + adv, db + adv, idesc, acc);
+                        if (PAIR) umma_bf16_pair(d, da + adv, db + adv, idesc, acc);
+                        else umma_bf16(d, da + adv, db + adv, idesc, acc);
                     }
-                    umma_commit(bar_empty + 8 * stage);      // frees the stage when these MMAs have read it
+                    // frees the stage (in both CTAs of a pair) when these MMAs have read it
+                    if (PAIR) umma_commit_pair(bar_empty + 8 * stage); else umma_commit(bar_empty + 8 * stage);
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
-                umma_commit(bar_tfull + 8 * buf);            // accumulators complete
+                if (PAIR) umma_commit_pair(bar_tfull + 8 * buf); else umma_commit(bar_tfull + 8 * buf);
                 if (++buf == 2) { buf = 0; bphase ^= 1; }
+                if (PAIR) u += stride;
             }
         }
         __syncwarp();
@@ -186,63 +331,107 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap b_ro
         // ---------------- epilogue: 4 warps, one TMEM lane quarter each ----------------
         const int quarter = warp & 3;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-        const int row_in_block = quarter * 32 + lane;       // weight row inside the 128-row tile
-        uint32_t buf = 0, bphase = 0;
+        uint32_t buf = 0, bphase = 0, q = 0, qphase = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-            const UnitInfo ui = decode_unit(p, u);
+        int u = first;
+        const uint32_t tempty_leader = PAIR ? map_to_cta(bar_tempty, 0) : bar_tempty;
+        while (ok) {
+            if (!PAIR) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_qfull + 8 * q, qphase, &s_abort, p.status));
+                if (!ok) break;
+                u = s_queue[q];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_qempty + 8 * q);
+                if (++q == kQueue) { q = 0; qphase ^= 1; }
+                if (u < 0) break;
+            } else if (u >= n_units) {
+                break;
+            }
+            const UnitInfo ui = decode_unit<MODE, PAIR>(p, u, rank);
             // one decision for the whole warp: the TMEM loads below are warp-wide instructions
             ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, bphase, &s_abort, p.status));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t d0 = tmem_base + lane_addr + buf * 256, d1 = d0 + 128;
+            const uint32_t d = tmem_base + lane_addr + buf * 256;
             const int ld = ui.shared ? p.ld_shared : p.ld_routed;
-            for (int c0 = 0; c0 < ui.npad; c0 += 16) {
-                uint32_t r0[16], r1[16];
-                tmem_ld16(d0 + c0, r0);
-                tmem_ld16(d1 + c0, r1);
-                tmem_ld_wait();
-                if (MODE == 0) {
-                    const int col = ui.cb * 128 + row_in_block;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int n = c0 + j;
-                        if (n < ui.nrows) {
-                            const float g = __uint_as_float(r0[j]), up = __uint_as_float(r1[j]);
-                            const float v = (g / (1.f + __expf(-g))) * up;
-                            const size_t o = (size_t)(ui.b_row0 + n) * ld + col;
-                            if (ui.shared) reinterpret_cast<__half*>(p.out_shared)[o] = __float2half_rn(v);
-                            else reinterpret_cast<bf16*>(p.out_routed)[o] = __float2bfloat16_rn(v);
+            if (MODE == 0) {
+                // lanes 2i / 2i+1 hold the gate / up row (or up / gate) of intermediate index cb*64 + quarter*16 + i
+                const uint32_t gf = ui.shared ? (p.gate_first_shared >> ui.model) & 1u : p.gate_first_routed & 1u;
+                const bool even = (lane & 1) == 0;
+                const bool own_is_gate = even == (gf != 0);
+                const int col = ui.cb * 64 + quarter * 16 + (lane >> 1);
+                if (ui.direct) {
+                    for (int j = 0; j < ui.nrows; ++j) {
+                        const int tok = p.perm[ui.b_row0 + j] / p.top_k;            // warp-uniform
+                        uint32_t r;
+                        tmem_ld1(d + tok, r);
+                        tmem_ld_wait();
+                        const float own = __uint_as_float(r);
+                        const float other = __shfl_xor_sync(0xffffffffu, own, 1);
+                        if (even) {
+                            const float g = own_is_gate ? own : other, up = own_is_gate ? other : own;
+                            reinterpret_cast<bf16*>(p.out_routed)[(size_t)(ui.b_row0 + j) * ld + col] =
+                                __float2bfloat16_rn((g / (1.f + __expf(-g))) * up);
                         }
                     }
                 } else {
-                    const int col = ui.cb * 256 + row_in_block;
-                    float* out = reinterpret_cast<float*>(ui.shared ? p.out_shared : p.out_routed);
+                    for (int c0 = 0; c0 < ui.npad; c0 += 16) {
+                        uint32_t r[16];
+                        tmem_ld16(d + c0, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 16; j += 2) {
+                            // the even lane finishes token c0+j, the odd lane token c0+j+1
+                            const float send = __uint_as_float(even ? r[j + 1] : r[j]);
+                            const float recv = __shfl_xor_sync(0xffffffffu, send, 1);
+                            const float own = __uint_as_float(even ? r[j] : r[j + 1]);
+                            const int n = c0 + j + (even ? 0 : 1);
+                            if (n < ui.nrows) {
+                                const float g = own_is_gate ? own : recv, up = own_is_gate ? recv : own;
+                                const float v = (g / (1.f + __expf(-g))) * up;
+                                const size_t o = (size_t)(ui.b_row0 + n) * ld + col;
+                                if (ui.shared) reinterpret_cast<__half*>(p.out_shared)[o] = __float2half_rn(v);
+                                else reinterpret_cast<bf16*>(p.out_routed)[o] = __float2bfloat16_rn(v);
+                            }
+                        }
+                    }
+                }
+            } else {
+                const int col = ui.cb * 128 + quarter * 32 + lane;
+                float* out = reinterpret_cast<float*>(ui.shared ? p.out_shared : p.out_routed);
+                for (int c0 = 0; c0 < ui.npad; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld16(d + c0, r);
+                    tmem_ld_wait();
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int n = c0 + j;
                         if (n < ui.nrows) {
                             int row = ui.b_row0 + n;
                             if (ui.shared && p.shared_dst_rows) row = p.shared_dst_rows[row];
-                            out[(size_t)row * ld + col] = __uint_as_float(r0[j]);
-                            out[(size_t)row * ld + col + 128] = __uint_as_float(r1[j]);
+                            out[(size_t)row * ld + col] = __uint_as_float(r[j]);
                         }
                     }
                 }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+            if (lane == 0) {
+                if (PAIR) mbar_arrive_cluster(tempty_leader + 8 * buf); else mbar_arrive(bar_tempty + 8 * buf);
+            }
             if (++buf == 2) { buf = 0; bphase ^= 1; }
+            if (PAIR) u += stride;
         }
     }
 
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();      // nobody leaves while the peer may still read this CTA's memory or signal it
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -252,36 +441,59 @@ __global__ void bf16_to_fp16_kernel(const bf16* __restrict__ src, __half* __rest
     if (i < n) dst[i] = __float2half_rn(__bfloat162float(src[i]));
 }
 
-// ---- host side ----------------------------------------------------------------------------
+// 3-D map over two weight arrays of `rows` x `k` bf16 each: dimension 1 selects the array, so a box of
+// (64 K, 2, 64 rows) lands in shared memory as 128 rows that alternate between the two arrays.
+// Returns false on failure; *first_is_a tells whether index 0 of dimension 1 is array `a`.
+bool make_pair_map(CUtensorMap* m, const void* a, const void* b, uint64_t rows, uint64_t k, bool* first_is_a)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const uintptr_t pa = (uintptr_t)a, pb = (uintptr_t)b;
+    const uintptr_t lo = pa < pb ? pa : pb, hi = pa < pb ? pb : pa;
+    *first_is_a = pa <= pb;
+    const uint64_t diff = hi - lo;
+    if (diff == 0 || (diff & 15) || diff >= (1ull << 40)) return false;
+    cuuint64_t dims[3] = {k, 2, rows};
+    cuuint64_t strides[2] = {diff, k * 2};
+    cuuint32_t box[3] = {(cuuint32_t)kBK, 2, 64};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)lo, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 }  // namespace
 
 struct LayerMaps {
     bool ready = false;
-    CUtensorMap* d_amaps1 = nullptr;    // gate/up: [gate pool, up pool, (ws_gate, ws_up) per model]
-    CUtensorMap* d_amaps2 = nullptr;    // down:    [down pool, down pool, (ws_down fp16, same) per model]
+    GemmMaps m1, m2;                    // weight maps of the gate/up and down GEMMs (activation maps are per call)
+    uint32_t gate_first_routed = 1, gate_first_shared = 0;
     std::vector<__half*> ws_down_f16;   // per model
 };
 
 struct TensorMaps {
     std::vector<LayerMaps> layers;
+    int max_clusters = -1;              // co-resident 2-CTA clusters of the pair kernels
 };
 
 bool tc_supported(const moe_ctx* c)
 {
     const moe_config& g = c->cfg;
-    return g.hidden % 256 == 0 && g.inter % 128 == 0 && g.shared_inter % 128 == 0;
+    return g.hidden % 256 == 0 && g.inter % 128 == 0 && g.shared_inter % 128 == 0 && g.n_models <= kTcMaxModels;
+}
+
+// Long tiles: share the token tile between two CTAs.  The decision uses only host-side sizes.
+bool tc_pair_mode(const moe_ctx* c, int T)
+{
+    const moe_config& g = c->cfg;
+    return c->pair_mode_enabled && (long long)T * g.top_k >= 96ll * g.n_models * g.n_experts && T >= 512;
 }
 
 void tc_destroy(moe_ctx* c)
 {
     if (!c->tmaps) return;
     cudaDeviceSynchronize();
-    for (LayerMaps& lm : c->tmaps->layers) {
-        if (lm.d_amaps1) cudaFree(lm.d_amaps1);
-        if (lm.d_amaps2) cudaFree(lm.d_amaps2);
+    for (LayerMaps& lm : c->tmaps->layers)
         for (__half* p : lm.ws_down_f16) if (p) cudaFree(p);
-    }
     delete c->tmaps;
     c->tmaps = nullptr;
 }
@@ -297,95 +509,131 @@ int tc_setup_layer(moe_ctx* c, int layer)
     if (lm.ready) return MOE_OK;
     const int M = g.n_models, H = g.hidden, I = g.inter, Is = g.shared_inter;
     const PoolWeights& pw = c->pools[layer];
-    std::vector<CUtensorMap> m1(2 + 2 * M), m2(2 + 2 * M);
-    memset(m1.data(), 0, m1.size() * sizeof(CUtensorMap));
-    memset(m2.data(), 0, m2.size() * sizeof(CUtensorMap));
-    bool ok = true;
+    memset(&lm.m1, 0, sizeof(GemmMaps));
+    memset(&lm.m2, 0, sizeof(GemmMaps));
+    bool ok = true, first = true;
     const uint64_t S = g.n_slots;
-    ok &= make_map(&m1[0], pw.w_gate, S * I, H, 128, false);
-    ok &= make_map(&m1[1], pw.w_up, S * I, H, 128, false);
-    ok &= make_map(&m2[0], pw.w_down, S * H, I, 128, false);
-    m2[1] = m2[0];
+    ok &= make_pair_map(&lm.m1.a_routed, pw.w_gate, pw.w_up, S * I, H, &first);
+    lm.gate_first_routed = first ? 1u : 0u;
+    ok &= make_map(&lm.m2.a_routed, pw.w_down, S * H, I, 128, false);
     lm.ws_down_f16.assign(M, nullptr);
+    lm.gate_first_shared = 0;
     for (int m = 0; m < M && ok && Is > 0; ++m) {
         const ModelWeights& mw = c->models[(size_t)layer * M + m];
-        ok &= make_map(&m1[2 + 2 * m], mw.ws_gate, Is, H, 128, false);
-        ok &= make_map(&m1[3 + 2 * m], mw.ws_up, Is, H, 128, false);
+        ok &= make_pair_map(&lm.m1.a_shared[m], mw.ws_gate, mw.ws_up, Is, H, &first);
+        if (first) lm.gate_first_shared |= 1u << m;
         // fp16 copy of the shared expert's down projection (its activations are fp16 and one MMA takes
         // operands of one type); every bf16 weight of magnitude >= 2^-17 converts exactly
         const size_t n = (size_t)H * Is;
         if (cudaMalloc((void**)&lm.ws_down_f16[m], n * sizeof(__half)) != cudaSuccess) return MOE_ERR_ALLOC;
         bf16_to_fp16_kernel<<<(unsigned)((n + 255) / 256), 256>>>(mw.ws_down, lm.ws_down_f16[m], n);
-        ok &= make_map(&m2[2 + 2 * m], lm.ws_down_f16[m], H, Is, 128, true);
-        m2[3 + 2 * m] = m2[2 + 2 * m];
+        ok &= make_map(&lm.m2.a_shared[m], lm.ws_down_f16[m], H, Is, 128, true);
     }
     if (!ok) {
         snprintf(c->errbuf, sizeof(c->errbuf), "cuTensorMapEncodeTiled failed for a weight tensor");
         return MOE_ERR_CUDA;
     }
-    const size_t bytes = m1.size() * sizeof(CUtensorMap);
-    if (cudaMalloc((void**)&lm.d_amaps1, bytes) != cudaSuccess || cudaMalloc((void**)&lm.d_amaps2, bytes) != cudaSuccess)
-        return MOE_ERR_ALLOC;
-    if (cudaMemcpy(lm.d_amaps1, m1.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemcpy(lm.d_amaps2, m2.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaDeviceSynchronize() != cudaSuccess)
-        return MOE_ERR_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return MOE_ERR_CUDA;
     lm.ready = true;
     return MOE_OK;
 }
 
-cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, float* y_perm,
-                              float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st)
+namespace {
+
+template <int MODE, bool PAIR>
+cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, cudaStream_t st)
+{
+    auto kern = grouped_gemm_kernel<MODE, PAIR>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        attr_set = true;
+    }
+    if (!PAIR) {
+        kern<<<c->sm_count, kThreads, kSmemBytes, st>>>(p, maps);
+        return cudaGetLastError();
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (c->tmaps->max_clusters < 0) {
+        // a persistent kernel must not launch more clusters than can be resident at once
+        cfg.gridDim = dim3((unsigned)(c->sm_count & ~1));
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) n = 1;
+        if (n > c->sm_count / 2) n = c->sm_count / 2;
+        c->tmaps->max_clusters = n;
+    }
+    cfg.gridDim = dim3((unsigned)(2 * c->tmaps->max_clusters));
+    return cudaLaunchKernelEx(&cfg, kern, p, maps);
+}
+
+}  // namespace
+
+cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, const int32_t* perm, int T,
+                              float* y_perm, float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st)
 {
     const moe_config& g = c->cfg;
-    const LayerMaps& lm = c->tmaps->layers[layer];
+    LayerMaps& lm = c->tmaps->layers[layer];
     const int H = g.hidden, I = g.inter, Is = g.shared_inter;
     const uint64_t R = (uint64_t)T * g.top_k;
     const bool shared = y_shared != nullptr && Is > 0;
-
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(grouped_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        attr_set = true;
-    }
+    const bool pair = tc_pair_mode(c, T);
+    // direct mode: with few tokens the routed gate/up units read the tokens in place (no permuted copy)
+    const bool direct = tc_direct_mode(c, T) && perm != nullptr;
     const uint32_t fmt_bf16 = (1u << 7) | (1u << 10), fmt_fp16 = 0u;
 
-    // B operand maps are rebuilt per call: the activations' addresses and row counts are the call's
-    CUtensorMap br128, br16, bs128, bs16;
-    bool ok = make_map(&br128, x_perm, R, H, 128, false) && make_map(&br16, x_perm, R, H, 16, false);
-    if (shared) ok = ok && make_map(&bs128, x_or_xs, T, H, 128, false) && make_map(&bs16, x_or_xs, T, H, 16, false);
-    else { bs128 = br128; bs16 = br16; }
+    // activation maps are rebuilt per call: their addresses and row counts are the call's
+    GemmMaps& m1 = lm.m1;
+    bool ok = true;
+    if (!direct) ok = make_map(&m1.b_routed128, x_perm, R, H, 128, false) && make_map(&m1.b_routed16, x_perm, R, H, 16, false);
+    if (shared || direct) {
+        ok = ok && make_map(&m1.b_shared128, x_or_xs, T, H, 128, false) && make_map(&m1.b_shared16, x_or_xs, T, H, 16, false);
+        if (direct) { m1.b_routed128 = m1.b_shared128; m1.b_routed16 = m1.b_shared16; }
+    } else {
+        m1.b_shared128 = m1.b_routed128; m1.b_shared16 = m1.b_routed16;
+    }
     if (!ok) return cudaErrorInvalidValue;
 
     GemmParams p1;
-    p1.units = c->ws.units1; p1.n_units = c->ws.plan_counts + 2;
+    memset(&p1, 0, sizeof(p1));
+    p1.units = c->ws.units1; p1.n_units = c->ws.plan_counts + 2; p1.counter = c->ws.plan_counts + 4;
     p1.tiles = c->ws.tiles; p1.stiles = c->ws.stiles;
-    p1.amaps = lm.d_amaps1;
+    p1.perm = perm; p1.top_k = g.top_k; p1.direct = direct ? 1 : 0; p1.n_tokens_pad = (T + 15) & ~15;
     p1.k_routed = H; p1.k_shared = H;
-    p1.rows_per_slot = I; p1.cb_stride = 128; p1.a1_off = 0;
+    p1.rows_per_slot = I; p1.cb_rows = 64;
     p1.out_routed = c->ws.h; p1.out_shared = c->ws.hs; p1.ld_routed = I; p1.ld_shared = Is;
     p1.shared_dst_rows = nullptr;
     p1.idesc_fmt_routed = fmt_bf16; p1.idesc_fmt_shared = fmt_bf16;
+    p1.gate_first_routed = lm.gate_first_routed; p1.gate_first_shared = lm.gate_first_shared;
     p1.status = c->ws.status;
     p1.stream_weights = (R <= 2048) ? 1 : 0;
-    grouped_gemm_kernel<0><<<c->sm_count, kThreads, kSmemBytes, st>>>(p1, br128, br16, bs128, bs16);
+    cudaError_t e = pair ? launch_gemm<0, true>(c, p1, m1, st) : launch_gemm<0, false>(c, p1, m1, st);
+    if (e != cudaSuccess) return e;
     stage_mark(c, st, kEvGateUp);
 
-    CUtensorMap hr128, hr16, hs128, hs16;
-    ok = make_map(&hr128, c->ws.h, R, I, 128, false) && make_map(&hr16, c->ws.h, R, I, 16, false);
-    if (shared) ok = ok && make_map(&hs128, c->ws.hs, T, Is, 128, true) && make_map(&hs16, c->ws.hs, T, Is, 16, true);
-    else { hs128 = hr128; hs16 = hr16; }
+    GemmMaps& m2 = lm.m2;
+    ok = make_map(&m2.b_routed128, c->ws.h, R, I, 128, false) && make_map(&m2.b_routed16, c->ws.h, R, I, 16, false);
+    if (shared) ok = ok && make_map(&m2.b_shared128, c->ws.hs, T, Is, 128, true) && make_map(&m2.b_shared16, c->ws.hs, T, Is, 16, true);
+    else { m2.b_shared128 = m2.b_routed128; m2.b_shared16 = m2.b_routed16; }
     if (!ok) return cudaErrorInvalidValue;
     GemmParams p2 = p1;
-    p2.units = c->ws.units2; p2.n_units = c->ws.plan_counts + 3;
-    p2.amaps = lm.d_amaps2;
+    p2.units = c->ws.units2; p2.n_units = c->ws.plan_counts + 3; p2.counter = c->ws.plan_counts + 5;
+    p2.direct = 0;
     p2.k_routed = I; p2.k_shared = Is;
-    p2.rows_per_slot = H; p2.cb_stride = 256; p2.a1_off = 128;
+    p2.rows_per_slot = H; p2.cb_rows = 128;
     p2.out_routed = y_perm; p2.out_shared = y_shared; p2.ld_routed = H; p2.ld_shared = H;
     p2.shared_dst_rows = shared_dst_rows;
     p2.idesc_fmt_routed = fmt_bf16; p2.idesc_fmt_shared = fmt_fp16;
-    grouped_gemm_kernel<1><<<c->sm_count, kThreads, kSmemBytes, st>>>(p2, hr128, hr16, hs128, hs16);
+    e = pair ? launch_gemm<1, true>(c, p2, m2, st) : launch_gemm<1, false>(c, p2, m2, st);
+    if (e != cudaSuccess) return e;
     stage_mark(c, st, kEvDown);
     c->launches += 2;
     return cudaGetLastError();

@@ -123,6 +123,7 @@ struct moe_ctx {
     faasmoe::TensorMaps* tmaps;   // TMA descriptors of the tensor-core path (host)
     void* rmaps;                  // TMA descriptors of the tensor-core router
     int route_path;
+    int pair_mode_enabled;        // allow the 2-CTA (cta_group::2) shape of the grouped GEMM for long tiles
     bool timing;                  // record an event after every stage (moe_layer_forward_timed)
     cudaEvent_t ev[8];
     char errbuf[256];
@@ -163,8 +164,8 @@ cudaError_t launch_plan(moe_ctx* c, const int32_t* expert_off, int T, int G, boo
 cudaError_t launch_experts_fma(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, float* y_perm,
                                float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st);
 
-cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, float* y_perm,
-                              float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st);
+cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, const int32_t* perm, int T,
+                              float* y_perm, float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st);
 
 cudaError_t launch_combine(moe_ctx* c, const float* y_perm, const int32_t* inv_perm, const float* topk_w,
                            const float* y_shared, const float* shared_gate, const bf16* residual, int T, bf16* out,
@@ -177,5 +178,12 @@ cudaError_t launch_rmsnorm(moe_ctx* c, int layer, const bf16* x, const int32_t* 
 int tc_setup_layer(moe_ctx* c, int layer);
 void tc_destroy(moe_ctx* c);
 bool tc_supported(const moe_ctx* c);
+bool tc_pair_mode(const moe_ctx* c, int T);      // long tiles: two CTAs share a token tile
+
+// Few tokens of one model: the routed gate/up units read the tokens in place, no permuted copy is needed.
+static inline bool tc_direct_mode(const moe_ctx* c, int T)
+{
+    return tc_supported(c) && !tc_pair_mode(c, T) && T <= 128 && c->cfg.n_models == 1;
+}
 
 }  // namespace faasmoe

@@ -33,7 +33,7 @@ __device__ int block_exclusive_scan(int32_t* data, int n, int32_t* s_part /* [bl
 // One block.  ME = M*E experts; groups are blocks of G consecutive experts of one model.
 __global__ void __launch_bounds__(512)
 plan_kernel(const int32_t* __restrict__ expert_off, const int32_t* __restrict__ slot_table, int M, int E, int G, int T,
-            const int32_t* __restrict__ model_tok_off /* null when M == 1 */, bool with_shared,
+            int tile_rows, const int32_t* __restrict__ model_tok_off /* null when M == 1 */, bool with_shared,
             int nblk1 /* weight-row blocks of the gate/up GEMM, routed */, int nblk2 /* down GEMM */,
             int snblk1, int snblk2, Tile* __restrict__ tiles, Tile* __restrict__ stiles, Unit* __restrict__ units1,
             Unit* __restrict__ units2, int32_t* __restrict__ plan_counts)
@@ -49,7 +49,7 @@ plan_kernel(const int32_t* __restrict__ expert_off, const int32_t* __restrict__ 
 
     for (int i = tid; i < ME; i += nth) {
         const int cnt = expert_off[i + 1] - expert_off[i];
-        s_tile_base[i] = (cnt + kTileRows - 1) / kTileRows;
+        s_tile_base[i] = (cnt + tile_rows - 1) / tile_rows;
     }
     __syncthreads();
     const int n_tiles = block_exclusive_scan(s_tile_base, ME, s_part);
@@ -57,10 +57,10 @@ plan_kernel(const int32_t* __restrict__ expert_off, const int32_t* __restrict__ 
         const int m = i / E, e = i - m * E;
         const int row_begin = expert_off[i], row_end = expert_off[i + 1];
         int tix = s_tile_base[i];
-        for (int r = row_begin; r < row_end; r += kTileRows, ++tix) {
+        for (int r = row_begin; r < row_end; r += tile_rows, ++tix) {
             Tile t;
             t.row0 = r;
-            t.nrows = min(kTileRows, row_end - r);
+            t.nrows = min(tile_rows, row_end - r);
             t.slot = slot_table[i];
             t.group = m * B + e / G;
             tiles[tix] = t;
@@ -82,11 +82,11 @@ plan_kernel(const int32_t* __restrict__ expert_off, const int32_t* __restrict__ 
         for (int m = 0; m < M; ++m) {
             const int t_begin = model_tok_off ? model_tok_off[m] : 0;
             const int t_end = model_tok_off ? model_tok_off[m + 1] : T;
-            const int nt = (t_end - t_begin + kTileRows - 1) / kTileRows;
+            const int nt = (t_end - t_begin + tile_rows - 1) / tile_rows;
             for (int i = tid; i < nt; i += nth) {
                 Tile t;
-                t.row0 = t_begin + i * kTileRows;
-                t.nrows = min(kTileRows, t_end - t.row0);
+                t.row0 = t_begin + i * tile_rows;
+                t.nrows = min(tile_rows, t_end - t.row0);
                 t.slot = m;
                 t.group = m;
                 stiles[n_stiles + i] = t;
@@ -125,6 +125,8 @@ plan_kernel(const int32_t* __restrict__ expert_off, const int32_t* __restrict__ 
     if (tid == 0) {
         plan_counts[0] = n_tiles;
         plan_counts[1] = n_stiles;
+        plan_counts[4] = 0;           // work counters of the two grouped GEMM launches
+        plan_counts[5] = 0;
     }
 }
 
@@ -137,9 +139,13 @@ cudaError_t launch_plan(moe_ctx* c, const int32_t* expert_off, int T, int G, boo
     const int B = (g.n_experts + G - 1) / G;
     const size_t smem = (size_t)(ME + g.n_models * B + 1) * sizeof(int32_t);
     const bool tc = tc_supported(c);
-    const int nblk1 = g.inter / 128, nblk2 = g.hidden / 256;
-    const int snblk1 = g.shared_inter / 128, snblk2 = g.hidden / 256;
-    plan_kernel<<<1, 512, smem, st>>>(expert_off, c->d_slot, g.n_models, g.n_experts, G, T,
+    // weight-row blocks per unit: gate/up 64 intermediate indices, down 128 rows; a CTA pair takes two
+    const bool pair = tc && tc_pair_mode(c, T);
+    const int div1 = pair ? 128 : 64, div2 = pair ? 256 : 128;
+    const int nblk1 = g.inter / div1, nblk2 = g.hidden / div2;
+    const int snblk1 = g.shared_inter / div1, snblk2 = g.hidden / div2;
+    const int tile_rows = pair ? 256 : kTileRows;
+    plan_kernel<<<1, 512, smem, st>>>(expert_off, c->d_slot, g.n_models, g.n_experts, G, T, tile_rows,
                                       g.n_models > 1 ? c->ws.model_tok_off : nullptr, with_shared, nblk1, nblk2,
                                       snblk1, snblk2, c->ws.tiles, c->ws.stiles, tc ? c->ws.units1 : nullptr,
                                       tc ? c->ws.units2 : nullptr, c->ws.plan_counts);

@@ -76,7 +76,7 @@ class GpuLayer:
                     o["tie_flag"])
         B.moe_dispatch(self.ctx, xd, o["topk_idx"], td, T, G, o["perm"], o["inv_perm"], o["tenant_expert_count"],
                        o["expert_off"], o["group_off"], o["x_perm"])
-        B.moe_experts(self.ctx, layer, xd, o["x_perm"], o["expert_off"], td, T, G, o["y_perm"], o["y_shared"])
+        B.moe_experts(self.ctx, layer, xd, o["x_perm"], o["perm"], o["expert_off"], td, T, G, o["y_perm"], o["y_shared"])
         B.moe_combine(self.ctx, o["y_perm"], o["inv_perm"], o["topk_w"], o["y_shared"],
                       o["shared_gate"] if wl.Is else None, T, o["out"])
         torch.cuda.synchronize()
