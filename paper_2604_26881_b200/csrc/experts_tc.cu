@@ -42,7 +42,8 @@ constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kQueue = 4;                      // depth of the unit queue of the dynamic scheduler
 constexpr int kNumBars = 2 * kStages + 4 + 2 * kQueue;
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 8 * kNumBars + 64;
-constexpr int kThreads = 192;                  // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: epilogue
+constexpr int kEpiWarps = 8;                   // two warps per TMEM lane quarter, alternating 16-column chunks
+constexpr int kThreads = 64 + 32 * kEpiWarps;  // warp 0: TMA, warp 1: MMA + TMEM, warps 2..: epilogue
 constexpr uint32_t kTmemCols = 512;            // 2 accumulator buffers x 256 columns
 
 struct GemmParams {
@@ -195,8 +196,13 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, PAIR ? 8 : 4); }
-        for (int q = 0; q < kQueue; ++q) { mbar_init(bar_qfull + 8 * q, 1); mbar_init(bar_qempty + 8 * q, 5); }
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, (PAIR ? 2 : 1) * kEpiWarps); }
+        // unit queue: filled by the scheduler (the leader's producer lane); drained by the MMA lane and the
+        // epilogue warps of this CTA and, in pair mode, by the peer's producer lane and epilogue warps
+        for (int q = 0; q < kQueue; ++q) {
+            mbar_init(bar_qfull + 8 * q, 1);
+            mbar_init(bar_qempty + 8 * q, 1 + kEpiWarps + (PAIR ? 1 + kEpiWarps : 0));
+        }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -218,9 +224,10 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
 
-    // unit sequence: pair mode walks the list with a fixed stride; single mode pulls from a counter
-    const int stride = PAIR ? (int)(gridDim.x >> 1) : 0;
-    const int first = PAIR ? (int)(blockIdx.x >> 1) : 0;
+    // Units are pulled from a global counter by one scheduler lane per CTA (pair: per CTA pair, the leader's)
+    // and handed to the other roles through a small queue in shared memory; in pair mode the leader also
+    // writes the peer's queue and the peer's consumers release the slot on the leader's barrier.
+    const uint32_t qempty_leader = PAIR ? map_to_cta(bar_qempty, 0) : bar_qempty;
 
     if (warp == 0) {
         // ---------------- TMA producer (one lane); in single mode also the scheduler ----------------
@@ -230,19 +237,28 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
             bool ok = true;
             const uint64_t pol_w = p.stream_weights ? l2_evict_first() : l2_evict_last();
             const uint64_t pol_x = l2_evict_last();
-            int u = first;
+            int u = 0;
+            const uint32_t peer_queue = PAIR ? map_to_cta(smem_u32(&s_queue[0]), 1) : 0u;
+            const uint32_t peer_qfull = PAIR ? map_to_cta(bar_qfull, 1) : 0u;
             while (ok) {
-                if (!PAIR) {
-                    if (!mbar_wait(bar_qempty + 8 * q, qphase ^ 1, &s_abort, p.status)) { ok = false; break; }
+                if (leader) {
+                    if (!(PAIR ? mbar_wait_cluster(bar_qempty + 8 * q, qphase ^ 1, &s_abort, p.status)
+                               : mbar_wait(bar_qempty + 8 * q, qphase ^ 1, &s_abort, p.status))) { ok = false; break; }
                     u = atomicAdd(p.counter, 1);
                     if (u >= n_units) u = -1;
                     s_queue[q] = u;
                     mbar_arrive(bar_qfull + 8 * q);
-                    if (++q == kQueue) { q = 0; qphase ^= 1; }
-                    if (u < 0) break;
-                } else if (u >= n_units) {
-                    break;
+                    if (PAIR) {
+                        asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(peer_queue + 4 * q), "r"(u) : "memory");
+                        mbar_arrive_cluster(peer_qfull + 8 * q);
+                    }
+                } else {
+                    if (!mbar_wait_cluster(bar_qfull + 8 * q, qphase, &s_abort, p.status)) { ok = false; break; }
+                    u = s_queue[q];
+                    mbar_arrive_cluster(qempty_leader + 8 * q);
                 }
+                if (++q == kQueue) { q = 0; qphase ^= 1; }
+                if (u < 0) break;
                 const UnitInfo ui = decode_unit<MODE, PAIR>(p, u, rank);
                 const CUtensorMap* ma = ui.amap < 0 ? &maps.a_routed : &maps.a_shared[ui.amap];
                 const bool bshared = ui.shared || ui.direct;
@@ -273,7 +289,6 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
-                if (PAIR) u += stride;
             }
             if (!ok && leader) {
                 // gave up: let the copies already in flight land before the block exits
@@ -287,21 +302,18 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
         if (lane == 0 && leader) {
             uint32_t stage = 0, phase = 0, buf = 0, bphase = 0, q = 0, qphase = 0;
             bool ok = true;
-            int u = first;
+            int u = 0;
             while (ok) {
-                if (!PAIR) {
-                    if (!mbar_wait(bar_qfull + 8 * q, qphase, &s_abort, p.status)) { ok = false; break; }
-                    u = s_queue[q];
-                    mbar_arrive(bar_qempty + 8 * q);
-                    if (++q == kQueue) { q = 0; qphase ^= 1; }
-                    if (u < 0) break;
-                } else if (u >= n_units) {
-                    break;
-                }
+                if (!mbar_wait(bar_qfull + 8 * q, qphase, &s_abort, p.status)) { ok = false; break; }
+                u = s_queue[q];
+                mbar_arrive(bar_qempty + 8 * q);
+                if (++q == kQueue) { q = 0; qphase ^= 1; }
+                if (u < 0) break;
                 const UnitInfo ui = decode_unit<MODE, PAIR>(p, u, rank);
                 const uint32_t fmt = ui.shared ? p.idesc_fmt_shared : p.idesc_fmt_routed;
                 const uint32_t idesc = (1u << 4) | fmt | ((uint32_t)(ui.npad >> 3) << 17) | (((PAIR ? 256u : 128u) >> 4) << 24);
-                if (!mbar_wait(bar_tempty + 8 * buf, bphase ^ 1, &s_abort, p.status)) { ok = false; break; }
+                if (!(PAIR ? mbar_wait_cluster(bar_tempty + 8 * buf, bphase ^ 1, &s_abort, p.status)
+                           : mbar_wait(bar_tempty + 8 * buf, bphase ^ 1, &s_abort, p.status))) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d = tmem_base + buf * 256;
                 for (int ks = 0; ks < ui.ksteps; ++ks) {
@@ -323,30 +335,29 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 if (!ok) break;
                 if (PAIR) umma_commit_pair(bar_tfull + 8 * buf); else umma_commit(bar_tfull + 8 * buf);
                 if (++buf == 2) { buf = 0; bphase ^= 1; }
-                if (PAIR) u += stride;
             }
         }
         __syncwarp();
     } else {
-        // ---------------- epilogue: 4 warps, one TMEM lane quarter each ----------------
+        // ---------------- epilogue: two warps per TMEM lane quarter, alternating 16-column chunks ----------------
         const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;                  // 0 or 1: which chunks of 16 columns this warp takes
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         uint32_t buf = 0, bphase = 0, q = 0, qphase = 0;
         bool ok = true;
-        int u = first;
+        int u = 0;
         const uint32_t tempty_leader = PAIR ? map_to_cta(bar_tempty, 0) : bar_tempty;
         while (ok) {
-            if (!PAIR) {
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_qfull + 8 * q, qphase, &s_abort, p.status));
-                if (!ok) break;
-                u = s_queue[q];
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_qempty + 8 * q);
-                if (++q == kQueue) { q = 0; qphase ^= 1; }
-                if (u < 0) break;
-            } else if (u >= n_units) {
-                break;
+            ok = __all_sync(0xffffffffu, PAIR ? mbar_wait_cluster(bar_qfull + 8 * q, qphase, &s_abort, p.status)
+                                              : mbar_wait(bar_qfull + 8 * q, qphase, &s_abort, p.status));
+            if (!ok) break;
+            u = s_queue[q];
+            __syncwarp();
+            if (lane == 0) {
+                if (PAIR) mbar_arrive_cluster(qempty_leader + 8 * q); else mbar_arrive(bar_qempty + 8 * q);
             }
+            if (++q == kQueue) { q = 0; qphase ^= 1; }
+            if (u < 0) break;
             const UnitInfo ui = decode_unit<MODE, PAIR>(p, u, rank);
             // one decision for the whole warp: the TMEM loads below are warp-wide instructions
             ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, bphase, &s_abort, p.status));
@@ -361,7 +372,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 const bool own_is_gate = even == (gf != 0);
                 const int col = ui.cb * 64 + quarter * 16 + (lane >> 1);
                 if (ui.direct) {
-                    for (int j = 0; j < ui.nrows; ++j) {
+                    for (int j = half; j < ui.nrows; j += 2) {
                         const int tok = p.perm[ui.b_row0 + j] / p.top_k;            // warp-uniform
                         uint32_t r;
                         tmem_ld1(d + tok, r);
@@ -371,11 +382,14 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                         if (even) {
                             const float g = own_is_gate ? own : other, up = own_is_gate ? other : own;
                             reinterpret_cast<bf16*>(p.out_routed)[(size_t)(ui.b_row0 + j) * ld + col] =
-                                __float2bfloat16_rn((g / (1.f + __expf(-g))) * up);
+                                __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * up);
                         }
                     }
                 } else {
-                    for (int c0 = 0; c0 < ui.npad; c0 += 16) {
+                    // 16-bit outputs; this lane's element of row n sits at out16[(b_row0 + n) * ld + col]
+                    unsigned short* out16 = reinterpret_cast<unsigned short*>(ui.shared ? p.out_shared : p.out_routed) +
+                                            (size_t)ui.b_row0 * ld + col;
+                    for (int c0 = half * 16; c0 < ui.npad; c0 += 32) {
                         uint32_t r[16];
                         tmem_ld16(d + c0, r);
                         tmem_ld_wait();
@@ -388,18 +402,18 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                             const int n = c0 + j + (even ? 0 : 1);
                             if (n < ui.nrows) {
                                 const float g = own_is_gate ? own : recv, up = own_is_gate ? recv : own;
-                                const float v = (g / (1.f + __expf(-g))) * up;
-                                const size_t o = (size_t)(ui.b_row0 + n) * ld + col;
-                                if (ui.shared) reinterpret_cast<__half*>(p.out_shared)[o] = __float2half_rn(v);
-                                else reinterpret_cast<bf16*>(p.out_routed)[o] = __float2bfloat16_rn(v);
+                                const float v = __fdividef(g, 1.f + __expf(-g)) * up;
+                                out16[(size_t)n * ld] = ui.shared ? __half_as_ushort(__float2half_rn(v))
+                                                                  : __bfloat16_as_ushort(__float2bfloat16_rn(v));
                             }
                         }
                     }
                 }
             } else {
                 const int col = ui.cb * 128 + quarter * 32 + lane;
-                float* out = reinterpret_cast<float*>(ui.shared ? p.out_shared : p.out_routed);
-                for (int c0 = 0; c0 < ui.npad; c0 += 16) {
+                float* out = reinterpret_cast<float*>(ui.shared ? p.out_shared : p.out_routed) + col;
+                const bool remap = ui.shared && p.shared_dst_rows != nullptr;
+                for (int c0 = half * 16; c0 < ui.npad; c0 += 32) {
                     uint32_t r[16];
                     tmem_ld16(d + c0, r);
                     tmem_ld_wait();
@@ -408,8 +422,8 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                         const int n = c0 + j;
                         if (n < ui.nrows) {
                             int row = ui.b_row0 + n;
-                            if (ui.shared && p.shared_dst_rows) row = p.shared_dst_rows[row];
-                            out[(size_t)row * ld + col] = __uint_as_float(r[j]);
+                            if (remap) row = p.shared_dst_rows[row];
+                            out[(size_t)row * ld] = __uint_as_float(r[j]);
                         }
                     }
                 }
@@ -420,7 +434,6 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 if (PAIR) mbar_arrive_cluster(tempty_leader + 8 * buf); else mbar_arrive(bar_tempty + 8 * buf);
             }
             if (++buf == 2) { buf = 0; bphase ^= 1; }
-            if (PAIR) u += stride;
         }
     }
 
