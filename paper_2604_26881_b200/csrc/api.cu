@@ -125,7 +125,7 @@ bool use_tc(const moe_ctx* c)
 
 int experts_impl(moe_ctx* c, int layer, const bf16* x, const bf16* x_perm, const int32_t* perm,
                  const int32_t* expert_off, const int32_t* tenant_id, int T, int G, float* y_perm, float* y_shared,
-                 cudaStream_t st)
+                 cudaStream_t st, bool plan_done = false)
 {
     const moe_config& g = c->cfg;
     const bool with_shared = y_shared != nullptr && g.shared_inter > 0;
@@ -136,7 +136,7 @@ int experts_impl(moe_ctx* c, int layer, const bf16* x, const bf16* x_perm, const
         xs = c->ws.xs_perm;
         dst_rows = c->ws.tok_perm;
     }
-    MOE_CUDA(c, launch_plan(c, expert_off, T, G, with_shared, st));
+    if (!plan_done) MOE_CUDA(c, launch_plan(c, expert_off, T, G, with_shared, st));
     stage_mark(c, st, kEvPlan);
     if (use_tc(c)) {
         const int rc = tc_setup_layer(c, layer);
@@ -161,11 +161,12 @@ int layer_forward_impl(moe_ctx* c, int layer, const bf16* x, const int32_t* tena
     stage_mark(c, st, kEvRoute);
     // with few tokens the tensor-core experts read the tokens in place: no permuted copy to make
     const bool direct = use_tc(c) && tc_direct_mode(c, T);
+    bool plan_done = false;
     MOE_CUDA(c, launch_dispatch(c, x, w.topk_idx, tenant_id, T, G, w.perm, w.inv_perm, w.tenant_expert_count,
-                                w.expert_off, w.group_off, direct ? nullptr : w.x_perm, st));
+                                w.expert_off, w.group_off, direct ? nullptr : w.x_perm, st, true, shared, &plan_done));
     stage_mark(c, st, kEvDispatch);
     const int rc = experts_impl(c, layer, x, w.x_perm, w.perm, w.expert_off, tenant_id, T, G, w.y_perm,
-                                shared ? w.y_shared : nullptr, st);
+                                shared ? w.y_shared : nullptr, st, plan_done);
     if (rc != MOE_OK) return rc;
     MOE_CUDA(c, launch_combine(c, w.y_perm, w.inv_perm, w.topk_w, shared ? w.y_shared : nullptr,
                                shared ? w.shared_gate : nullptr, residual, T, out, st));

@@ -3,9 +3,12 @@
 // routing requests"; Sec. 4.1: all tokens routed to the same expert block become one batched
 // invocation).  Rows are ordered by (model, expert, tenant, token); the order is produced
 // without order-dependent atomics so that the permutation is reproducible bit for bit.
+#include <cstring>
 #include <mutex>
 
 #include "internal.h"
+#include "plan.cuh"
+#include "scan.cuh"
 
 namespace faasmoe {
 
@@ -49,7 +52,7 @@ dispatch_hist_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __rest
 
 // Block-wide: exclusive scan of the per-bin totals in s_tot (in key order), then the offset tables
 // the caller sees and the invocation statistics.  s_tot holds the offsets afterwards.
-__device__ void scan_and_tables(int32_t* s_tot, int32_t* s_part /* [blockDim.x] */, int32_t* s_count /* [2] */,
+__device__ void scan_and_tables(int32_t* s_tot, int32_t* s_part /* [33] */, int32_t* s_count /* [2] */,
                                 int nbins, int R, int E, int M, int G, int n_tenants, const BinMap& bm,
                                 int32_t* __restrict__ bin_off /* may be null */,
                                 int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
@@ -65,22 +68,7 @@ __device__ void scan_and_tables(int32_t* s_tot, int32_t* s_part /* [blockDim.x] 
         }
     }
     __syncthreads();
-    // exclusive scan over bins: each thread owns a contiguous run of bins
-    const int per = (nbins + nth - 1) / nth;
-    const int b0 = min(nbins, tid * per), b1 = min(nbins, b0 + per);
-    int sum = 0;
-    for (int b = b0; b < b1; ++b) sum += s_tot[b];
-    s_part[tid] = sum;
-    __syncthreads();
-    for (int off = 1; off < nth; off <<= 1) {          // Hillis-Steele inclusive scan of the partials
-        int v = (tid >= off) ? s_part[tid - off] : 0;
-        __syncthreads();
-        s_part[tid] += v;
-        __syncthreads();
-    }
-    int run = s_part[tid] - sum;
-    for (int b = b0; b < b1; ++b) { const int c = s_tot[b]; s_tot[b] = run; run += c; }
-    __syncthreads();
+    block_scan_exclusive(s_tot, nbins, s_part);
     if (bin_off) {
         for (int b = tid; b < nbins; b += nth) bin_off[b] = s_tot[b];
         if (tid == 0) bin_off[nbins] = R;
@@ -124,7 +112,7 @@ dispatch_scan_kernel(int nblk, int nbins, int R, int E, int M, int G, int n_tena
                      int32_t* __restrict__ group_off, int32_t* __restrict__ stats)
 {
     extern __shared__ int32_t s_tot[];       // [nbins] totals, then exclusive offsets
-    __shared__ int32_t s_part[1024];
+    __shared__ int32_t s_part[33];
     __shared__ int32_t s_count[2];
     const int tid = threadIdx.x, nth = blockDim.x;
     // totals per bin; block_cnt becomes the exclusive prefix over blocks
@@ -151,10 +139,11 @@ dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
                       BinMap bm, int nbins, int E, int M, int G, int n_tenants, int32_t* __restrict__ perm,
                       int32_t* __restrict__ inv_perm, int32_t* __restrict__ tenant_expert_count,
                       int32_t* __restrict__ expert_off, int32_t* __restrict__ group_off, int32_t* __restrict__ stats,
-                      int32_t* __restrict__ status, const bf16* __restrict__ x, bf16* __restrict__ x_perm, int H)
+                      int32_t* __restrict__ status, const bf16* __restrict__ x, bf16* __restrict__ x_perm, int H,
+                      int do_plan, PlanArgs pa)
 {
-    extern __shared__ int32_t s_tot[];       // [nbins]
-    __shared__ int32_t s_part[1024];
+    extern __shared__ int32_t s_tot[];       // [nbins], then the plan's scratch
+    __shared__ int32_t s_part[33];
     __shared__ int32_t s_count[2];
     const int tid = threadIdx.x, nth = blockDim.x;
     for (int b = tid; b < nbins; b += nth) s_tot[b] = 0;
@@ -180,6 +169,10 @@ dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
             if (live) { perm[start + rank] = r; inv_perm[r] = start + rank; }
             __syncwarp();
         }
+    }
+    if (do_plan) {
+        __syncthreads();                      // expert_off (written above) is visible to the block
+        plan_body(expert_off, pa, s_tot + nbins, s_part);
     }
     if (x_perm) {
         __syncthreads();                      // perm is complete and visible to the block
@@ -326,8 +319,10 @@ BinMap make_binmap(const moe_ctx* c)
 
 cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, const int32_t* tenant_id, int T, int G,
                             int32_t* perm, int32_t* inv_perm, int32_t* tenant_expert_count, int32_t* expert_off,
-                            int32_t* group_off, bf16* x_perm, cudaStream_t st)
+                            int32_t* group_off, bf16* x_perm, cudaStream_t st, bool with_plan, bool plan_shared,
+                            bool* plan_done)
 {
+    if (plan_done) *plan_done = false;
     const moe_config& g = c->cfg;
     const int k = g.top_k, R = T * k;
     const int nblk = (R + kDispatchChunk - 1) / kDispatchChunk;
@@ -337,10 +332,18 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
     if (R <= kSmallRows) {
         // few rows: one block does everything; the gather rides along while it is small
         const bool gather_inside = x_perm && (size_t)R * g.hidden * sizeof(bf16) <= (1u << 20);
-        dispatch_small_kernel<<<1, 1024, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, g.n_experts, g.n_models, G,
-                                                     g.n_tenants, perm, inv_perm, tenant_expert_count, expert_off,
-                                                     group_off, c->ws.stats, c->ws.status, x,
-                                                     gather_inside ? x_perm : nullptr, g.hidden);
+        // the expert work plan rides along when the shared-expert tiles need no token sort (one model)
+        const bool do_plan = with_plan && g.n_models == 1;
+        PlanArgs pa;
+        memset(&pa, 0, sizeof(pa));
+        size_t plan_ints = 0;
+        if (do_plan) { pa = make_plan_args(c, T, G, plan_shared); plan_ints = plan_smem_ints(c, G); }
+        const int threads = (R <= 512 && nbins <= 1024) ? 256 : 1024;
+        dispatch_small_kernel<<<1, threads, smem + plan_ints * sizeof(int32_t), st>>>(
+            topk_idx, tenant_id, R, k, bm, nbins, g.n_experts, g.n_models, G, g.n_tenants, perm, inv_perm,
+            tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, x, gather_inside ? x_perm : nullptr,
+            g.hidden, do_plan ? 1 : 0, pa);
+        if (plan_done) *plan_done = do_plan;
         c->launches += 1;
         if (x_perm && !gather_inside) {
             gather_rows_kernel<<<(R * 32 + 255) / 256, 256, 0, st>>>(x, perm, R, k, g.hidden, x_perm);

@@ -146,7 +146,8 @@ cudaError_t launch_route(moe_ctx* c, int layer, const bf16* x, const int32_t* te
 
 cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, const int32_t* tenant_id, int T, int G,
                             int32_t* perm, int32_t* inv_perm, int32_t* tenant_expert_count, int32_t* expert_off,
-                            int32_t* group_off, bf16* x_perm, cudaStream_t st);
+                            int32_t* group_off, bf16* x_perm, cudaStream_t st, bool with_plan = false,
+                            bool plan_shared = false, bool* plan_done = nullptr);
 
 cudaError_t launch_route_fma(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,
                              float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st);
@@ -157,6 +158,10 @@ void route_tc_destroy(moe_ctx* c);
 
 // Sorts tokens by (model, token) into ws.tok_perm / tok_inv / model_tok_off and gathers ws.xs_perm (M > 1).
 cudaError_t launch_token_sort(moe_ctx* c, const bf16* x, const int32_t* tenant_id, int T, cudaStream_t st);
+
+struct PlanArgs;
+PlanArgs make_plan_args(moe_ctx* c, int T, int G, bool with_shared);
+size_t plan_smem_ints(const moe_ctx* c, int G);
 
 // Builds the tile lists (and the unit lists of the tensor-core path) from expert_off.
 cudaError_t launch_plan(moe_ctx* c, const int32_t* expert_off, int T, int G, bool with_shared, cudaStream_t st);
