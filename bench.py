@@ -123,6 +123,12 @@ def algorithmic_work(wl, active_experts: int, T: int):
     return dict(total_bytes=total_bytes, flops=flops, gateup_bytes=gateup_bytes, gateup_flops=gateup_flops)
 
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
+# ncu capture summarised in profiles/grouped_gemm_decode_ncu.md; None where no capture of the current
+# kernel exists.
+NCU_TRAFFIC_BYTES = {"decode": 657.641728e6 + 3.782912e6}
+
+
 def run_reference(args, wl, rank):
     """The oracle, as it stands, on the host cores: each step is a bounded sample of the workload."""
     import oracle
@@ -280,7 +286,9 @@ def main():
             achieved = work["gateup_flops"] / (gu_ms * 1e-3) / 1e12 if gu_ms else None
             peak, runit = peaks["bf16_tflops"], "TFLOP/s"
         roofline = {"bound": bound, "kernel": "moe_experts gate/up grouped GEMM", "achieved": achieved, "peak": peak,
-                    "unit": runit, "frac": (achieved / peak) if achieved else None, "traffic": None,
+                    "unit": runit, "frac": (achieved / peak) if achieved else None,
+                    "traffic": NCU_TRAFFIC_BYTES.get(wl.name) if args.path == "auto" else None,
+                    "algorithmic": work["gateup_bytes"] if bound == "hbm" else work["gateup_flops"],
                     "peak_source": peaks["source"],
                     "path": {"roofline_ms": 1e3 * max(t_hbm, t_tc), "measured_ms": ms_step,
                              "frac": 1e3 * max(t_hbm, t_tc) / ms_step, "algorithmic_bytes": work["total_bytes"],
