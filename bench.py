@@ -25,6 +25,7 @@ if ROOT not in sys.path:
 
 import torch
 
+from paper_2604_26881_b200 import replicas
 from paper_2604_26881_b200 import workloads as W
 
 METRIC = "MoE-layer tokens/s at Qwen1.5-MoE shape on 1 B200"
@@ -206,7 +207,7 @@ def main():
 
     # every rank is an independent replica with its own batch (different seed), same weights recipe
     wts = W.make_weights(wl, seed=0)
-    x, tenant, mot = W.make_tokens(wl, seed=rank)
+    x, tenant, mot = W.make_tokens(wl, seed=replicas.rank_seed(0, rank))
     T = x.shape[0]
     layer = B.MoELayer(H=wl.H, E=wl.E, I=wl.I, k=wl.k, Is=wl.Is, M=wl.M, n_tenants=wl.n_tenants, max_tokens=T,
                        device=str(dev))
@@ -219,9 +220,7 @@ def main():
     stream = torch.cuda.current_stream()
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(world, torch.cuda.synchronize)
 
     # ---- device-resident throughput -----------------------------------------------------------
     for _ in range(warmup):
@@ -264,10 +263,7 @@ def main():
     e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0))
     barrier()
 
-    if world > 1:
-        t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, e2e_ms = float(t[0]), float(t[1])
+    ms_total, e2e_ms = replicas.max_over_ranks([ms_total, e2e_ms], world, dev)
 
     if rank == 0:
         peaks = measured_peaks()

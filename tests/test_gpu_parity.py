@@ -189,6 +189,27 @@ def test_stack_teacher_forced(path):
         g.close()
 
 
+def test_pair_shape_and_single_shape_agree_bit_for_bit(qwen_weights):
+    # the 2-CTA (cta_group::2) and the 1-CTA shape of the grouped GEMM tile the work differently but
+    # accumulate every output element over K in the same order
+    wl = W.scaled(W.WORKLOADS["prefill"], T=1024)
+    x, tenant, mot = W.make_tokens(wl, seed=2)
+    g = GpuLayer(wl, [qwen_weights], wl.T, model_of_tenant=mot)
+    try:
+        B.moe_set_option(g.ctx, B.MOE_OPT_PAIR_MODE, 1)
+        pair = g.forward(x, tenant, wl.G)
+        B.moe_set_option(g.ctx, B.MOE_OPT_PAIR_MODE, 0)
+        single = g.forward(x, tenant, wl.G)
+        assert B.moe_last_status(g.ctx)[0] == 0
+        assert torch.equal(pair, single)
+        # and both are the CUDA-core path within the tolerance
+        B.moe_set_option(g.ctx, B.MOE_OPT_EXPERT_PATH, B.MOE_PATH_FMA)
+        fma = g.forward(x, tenant, wl.G)
+        assert_close("pair vs fma", bf16_to_f64(pair), bf16_to_f64(fma))
+    finally:
+        g.close()
+
+
 def test_host_entry_point_matches_device_entry_point():
     wl = W.WORKLOADS["tiny"]
     wts = W.make_weights(wl, seed=0)
