@@ -210,6 +210,110 @@ def test_pair_shape_and_single_shape_agree_bit_for_bit(qwen_weights):
         g.close()
 
 
+def _sampled_check(g, wl, wts, x, tenant, mot, G, out, n_sample=32, layer_inputs=None):
+    """Routing/dispatch of the last layer call in full, layer outputs on sampled tokens."""
+    ws = B.moe_get_workspace(g.ctx)
+    T, k, E, M = x.shape[0], wl.k, wl.E, wl.M
+    idx = B.wrap_device_pointer(ws["topk_idx"], (T, k), torch.int32, g.dev).cpu().numpy()
+    wgt = B.wrap_device_pointer(ws["topk_w"], (T, k), torch.float32, g.dev).cpu().numpy()
+    perm = B.wrap_device_pointer(ws["perm"], (T * k,), torch.int32, g.dev).cpu().numpy()
+    eoff = B.wrap_device_pointer(ws["expert_off"], (M * E + 1,), torch.int32, g.dev).cpu().numpy()
+    wn = W.weights_as_numpy(wts)
+    r = oracle.route(W.as_u16(x), tenant.numpy(), mot.numpy(), wn["router_w"], wn["router_bias"],
+                     wn["shared_gate_w"], k=k)
+    idx_o, mask = check_routing(idx, wgt, r, k)
+    ref_idx = np.where(mask[:, None], idx_o, r.topk_idx)
+    assert np.array_equal(idx, ref_idx)
+    d = oracle.dispatch(ref_idx, tenant.numpy(), mot.numpy(), n_models=M, E=E, G=G)
+    assert np.array_equal(perm, d.perm) and np.array_equal(eoff, d.expert_off)
+    sample = np.sort(np.random.default_rng(1).choice(T, min(n_sample, T), replace=False))
+    ref = oracle.layer_forward(W.as_u16(x[sample].contiguous()), tenant[sample].contiguous().numpy(), mot.numpy(), wn,
+                               k=k, G=G, topk_override=(idx[sample], np.ones(len(sample), bool)))
+    return sample, ref, d
+
+
+def test_pool_full_size_G_sweep_sampled():
+    # 4 tenant models, 240 routed slots + 4 shared experts in one pool (4.4 GB), 2048 tokens with uniform
+    # tenant ids, shuffled slot table: outputs bit-identical for every G, sampled tokens against the oracle
+    wl = W.WORKLOADS["pool"]
+    wts = W.make_weights(wl, seed=0, shuffle_slots=True)
+    x, tenant, mot = W.make_tokens(wl, seed=0)
+    g = GpuLayer(wl, [wts], wl.T, model_of_tenant=mot)
+    try:
+        base = g.forward(x, tenant, 1)
+        sample, ref, d = _sampled_check(g, wl, wts, x, tenant, mot, 1, base)
+        assert_close("pool out[sample]", bf16_to_f64(base[sample]), ref.out)
+        inv = []
+        for G in (1, 2, 4, 6, 12, 60):
+            out = g.forward(x, tenant, G)
+            st = B.moe_last_status(g.ctx)
+            assert st[0] == 0 and torch.equal(out, base), f"G={G}"
+            inv.append(st[1])
+        assert inv[0] == st[2] and inv[-1] == 4 and inv == sorted(inv, reverse=True)
+    finally:
+        g.close()
+
+
+def test_stack_full_size_teacher_forced_sampled():
+    # 24 blocks, 26.6 GB of weights resident, 16 tenants with ragged request lengths, G = 6.  Blocks 0, 11
+    # and 23 have CPU twins of their weights and are checked against the oracle from the GPU's own block
+    # inputs; the other blocks get device-generated weights of the same distribution.
+    wl = W.WORKLOADS["stack"]
+    if torch.cuda.mem_get_info()[0] < 40e9:
+        pytest.skip("needs about 30 GB of free device memory")
+    x, tenant, mot = W.make_tokens(wl, seed=0)
+    T = x.shape[0]
+    checked = {0: None, 11: None, 23: None}
+    dev = torch.device("cuda:0")
+    layers = []
+    gen = torch.Generator(device=dev).manual_seed(1234)
+    for l in range(wl.n_layers):
+        if l in checked:
+            checked[l] = W.make_weights(wl, seed=0, layer=l)
+            layers.append(checked[l])
+        else:
+            def rnd(*shape, std=0.02):
+                return (torch.randn(*shape, generator=gen, device=dev, dtype=torch.float32) * std).to(torch.bfloat16)
+            S = wl.n_slots
+            layers.append({
+                "router_w": rnd(1, wl.E, wl.H), "router_bias": None,
+                "pool_gate": rnd(S, wl.I, wl.H), "pool_up": rnd(S, wl.I, wl.H), "pool_down": rnd(S, wl.H, wl.I),
+                "shared_gate_w": rnd(1, wl.H), "ws_gate": rnd(1, wl.Is, wl.H), "ws_up": rnd(1, wl.Is, wl.H),
+                "ws_down": rnd(1, wl.H, wl.Is), "slot_table": torch.arange(S, dtype=torch.int32),
+                "rms_w": (1.0 + torch.randn(wl.H, generator=gen, device=dev) * 0.02).to(torch.bfloat16)})
+    g = GpuLayer(wl, layers, T, model_of_tenant=mot)
+    try:
+        xd, td = x.to(dev).clone(), tenant.to(dev)
+        dbg_in = torch.zeros((wl.n_layers, T, wl.H), dtype=torch.bfloat16, device=dev)
+        dbg_out = torch.zeros_like(dbg_in)
+        B.moe_stack_forward(g.ctx, xd, td, T, wl.G, dbg_in, dbg_out)
+        torch.cuda.synchronize()
+        assert B.moe_last_status(g.ctx)[0] == 0
+        assert torch.isfinite(xd.float()).all()
+        sample = np.sort(np.random.default_rng(2).choice(T, 24, replace=False))
+        for l, wts in checked.items():
+            wn = W.weights_as_numpy(wts)
+            x_in = (x if l == 0 else dbg_out[l - 1].cpu())
+            xn_gpu = dbg_in[l].cpu()
+            xs, xns, ts = x_in[sample].contiguous(), xn_gpu[sample].contiguous(), tenant[sample].contiguous()
+            xn_ref = oracle.rmsnorm(W.as_u16(xs), wn["rms_w"], wl.rms_eps)
+            ulp = 2.0 ** (np.floor(np.log2(np.abs(xn_ref) + 1e-300)) - 7)
+            assert (np.abs(bf16_to_f64(xns) - xn_ref) / ulp).max() <= 1.0
+            tk_i = torch.zeros((T, wl.k), dtype=torch.int32, device=dev)
+            tk_w = torch.zeros((T, wl.k), dtype=torch.float32, device=dev)
+            B.moe_route(g.ctx, l, dbg_in[l], td, T, tk_i, tk_w)
+            torch.cuda.synchronize()
+            r = oracle.route(W.as_u16(xns), ts.numpy(), mot.numpy(), wn["router_w"], wn["router_bias"],
+                             wn["shared_gate_w"], k=wl.k)
+            ov = check_routing(tk_i.cpu().numpy()[sample], tk_w.cpu().numpy()[sample], r, wl.k)
+            _, _, res = oracle.block_forward(W.as_u16(xs), ts.numpy(), mot.numpy(), wn, k=wl.k, G=wl.G, eps=wl.rms_eps,
+                                             xn_override=W.as_u16(xns), topk_override=ov)
+            assert_close(f"block {l} residual stream (sample)", bf16_to_f64(dbg_out[l][sample]),
+                         bf16_to_f64(xs) + res.out)
+    finally:
+        g.close()
+
+
 def test_host_entry_point_matches_device_entry_point():
     wl = W.WORKLOADS["tiny"]
     wts = W.make_weights(wl, seed=0)
