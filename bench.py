@@ -37,9 +37,10 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "pool"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "pool", "stack"])
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "fma", "tcgen05"])
+    ap.add_argument("--pair", default="auto", choices=["auto", "never"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -180,6 +181,83 @@ def cpu_baseline(wl, wts, x, tenant, mot):
             "sample": f"first {n} tokens of the {wl.name} batch, {reps} passes, {dt:.1f} s"}
 
 
+def run_stack(args, wl, rank, local_rank, world):
+    """The 24-block configuration: RMSNorm -> MoE layer (+shared expert) -> residual, 26.6 GB of weights resident."""
+    from paper_2604_26881_b200 import binding as B
+    import torch.distributed as dist
+    dev = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(dev)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    steps = args.steps if args.steps is not None else 30
+    warmup = max(args.warmup if args.warmup is not None else 3, 3)
+    x, tenant, mot = W.make_tokens(wl, seed=replicas.rank_seed(0, rank))
+    T = x.shape[0]
+    gen = torch.Generator(device=dev).manual_seed(1234)
+
+    def rnd(*shape, std=0.02):
+        return (torch.randn(*shape, generator=gen, device=dev, dtype=torch.float32) * std).to(torch.bfloat16)
+    layer = B.MoELayer(H=wl.H, E=wl.E, I=wl.I, k=wl.k, Is=wl.Is, M=1, n_tenants=wl.n_tenants, max_tokens=T,
+                       n_layers=wl.n_layers, device=str(dev))
+    S = wl.n_slots
+    for l in range(wl.n_layers):
+        layer.set_layer_weights(l, {
+            "router_w": rnd(1, wl.E, wl.H), "router_bias": None, "pool_gate": rnd(S, wl.I, wl.H),
+            "pool_up": rnd(S, wl.I, wl.H), "pool_down": rnd(S, wl.H, wl.I), "shared_gate_w": rnd(1, wl.H),
+            "ws_gate": rnd(1, wl.Is, wl.H), "ws_up": rnd(1, wl.Is, wl.H), "ws_down": rnd(1, wl.H, wl.Is),
+            "rms_w": (1.0 + torch.randn(wl.H, generator=gen, device=dev) * 0.02).to(torch.bfloat16)})
+    layer.set_tables(model_of_tenant=mot)
+    ctx = layer.ctx
+    B.moe_set_option(ctx, B.MOE_OPT_PAIR_MODE, {"auto": 1, "never": 0}[args.pair])
+    xd, td = x.to(dev), tenant.to(dev)
+    xw = xd.clone()
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        xw.copy_(xd)
+        B.moe_stack_forward(ctx, xw, td, T, wl.G, None, None, stream)
+    torch.cuda.synchronize()
+    if B.moe_last_status(ctx)[0] != 0:
+        raise SystemExit("device status set after warm-up")
+    sampler = ClockSampler(local_rank)
+    replicas.barrier(world, torch.cuda.synchronize)
+    sampler.start()
+    l0 = B.moe_launch_count(ctx)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(steps):
+        xw.copy_(xd)
+        B.moe_stack_forward(ctx, xw, td, T, wl.G, None, None, stream)
+    ev1.record(stream)
+    replicas.barrier(world, torch.cuda.synchronize)
+    clocks = sampler.stop()
+    launches = B.moe_launch_count(ctx) - l0
+    ms_total = replicas.max_over_ranks([ev0.elapsed_time(ev1)], world, dev)[0]
+    if rank == 0:
+        peaks = measured_peaks()
+        layer_bytes = wl.E * 3 * wl.H * wl.I * 2 + 3 * wl.H * wl.Is * 2 + (wl.E + 1) * wl.H * 2 + wl.H * 2
+        total_bytes = wl.n_layers * (layer_bytes + 4 * T * wl.H)          # upper bound: all experts active
+        flops = wl.n_layers * T * (wl.k * 6 * wl.H * wl.I + 6 * wl.H * wl.Is + 2 * wl.H * wl.E)
+        t_hbm, t_tc = total_bytes / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)
+        ms_step = ms_total / steps
+        line = {"metric": METRIC, "value": world * T * steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+                "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": wl.name, "blocks": wl.n_layers, "tokens_per_step_per_gpu": T, "tenants": wl.n_tenants,
+                           "G": wl.G, "weights_gb": wl.n_layers * layer_bytes / 1e9,
+                           "l2": "26.6 GB of weights per pass exceed the 126 MB L2; no flush",
+                           "parallelism": f"replicas x{world}"},
+                "clocks": clocks, "gpu_launches": int(launches),
+                "roofline": {"bound": "hbm" if t_hbm >= t_tc else "tensor", "kernel": "whole stack",
+                             "achieved": total_bytes / (ms_step * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                             "frac": 1e3 * max(t_hbm, t_tc) / ms_step, "traffic": None, "peak_source": peaks["source"],
+                             "note": "bytes assume every expert of every block is active"}}
+        print(json.dumps(line), flush=True)
+    layer.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -202,6 +280,9 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
 
+    if wl.n_layers > 1:
+        run_stack(args, wl, rank, local_rank, world)
+        return
     steps = args.steps if args.steps is not None else {"decode": 3000, "prefill": 200, "pool": 200}[args.workload]
     warmup = max(args.warmup if args.warmup is not None else 20, 3)
 
@@ -215,6 +296,7 @@ def main():
     layer.set_tables(slot_table=wts["slot_table"], model_of_tenant=mot)
     ctx = layer.ctx
     B.moe_set_option(ctx, B.MOE_OPT_EXPERT_PATH, {"auto": 0, "fma": 1, "tcgen05": 2}[args.path])
+    B.moe_set_option(ctx, B.MOE_OPT_PAIR_MODE, {"auto": 1, "never": 0}[args.pair])
     xd, td = x.to(dev), tenant.to(dev)
     out = torch.zeros_like(xd)
     stream = torch.cuda.current_stream()

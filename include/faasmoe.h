@@ -64,7 +64,8 @@ enum {
  * FMA forces the CUDA-core kernels, TCGEN05 fails with MOE_ERR_UNSUPPORTED if not possible. */
 enum { MOE_PATH_AUTO = 0, MOE_PATH_FMA = 1, MOE_PATH_TCGEN05 = 2 };
 enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2,
-       MOE_OPT_PAIR_MODE = 3 /* 1 (default): long expert tiles use the 2-CTA tcgen05 shape; 0: never */ };
+       MOE_OPT_PAIR_MODE = 3 /* 1 (default): batches of more than 128 tokens use the 2-CTA tcgen05 shape;
+                                0: never */ };
 
 typedef struct {
     int32_t hidden;        /* H */

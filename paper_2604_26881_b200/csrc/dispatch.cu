@@ -109,30 +109,42 @@ __global__ void __launch_bounds__(1024)
 dispatch_scan_kernel(int nblk, int nbins, int R, int E, int M, int G, int n_tenants, BinMap bm,
                      int32_t* __restrict__ block_cnt, int32_t* __restrict__ bin_off,
                      int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
-                     int32_t* __restrict__ group_off, int32_t* __restrict__ stats)
+                     int32_t* __restrict__ group_off, int32_t* __restrict__ stats, int do_plan, PlanArgs pa)
 {
-    extern __shared__ int32_t s_tot[];       // [nbins] totals, then exclusive offsets
+    extern __shared__ int32_t s_tot[];       // [nbins] totals, then exclusive offsets; then the plan's scratch
     __shared__ int32_t s_part[33];
     __shared__ int32_t s_count[2];
-    const int tid = threadIdx.x, nth = blockDim.x;
-    // totals per bin; block_cnt becomes the exclusive prefix over blocks
-    for (int b = tid; b < nbins; b += nth) {
+    const int tid = threadIdx.x, nth = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nth >> 5;
+    // totals per bin; block_cnt becomes the exclusive prefix over blocks.  One warp per bin: the lanes
+    // take the blocks 32 at a time and scan them with shuffles.
+    for (int b = warp; b < nbins; b += nw) {
         int run = 0;
-        for (int blk = 0; blk < nblk; ++blk) {
-            const int c = block_cnt[(size_t)blk * nbins + b];
-            block_cnt[(size_t)blk * nbins + b] = run;
-            run += c;
+        for (int blk0 = 0; blk0 < nblk; blk0 += 32) {
+            const int blk = blk0 + lane;
+            const int c = blk < nblk ? block_cnt[(size_t)blk * nbins + b] : 0;
+            int incl = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            if (blk < nblk) block_cnt[(size_t)blk * nbins + b] = run + incl - c;
+            run += __shfl_sync(0xffffffffu, incl, 31);
         }
-        s_tot[b] = run;
+        if (lane == 0) s_tot[b] = run;
     }
     __syncthreads();
     scan_and_tables(s_tot, s_part, s_count, nbins, R, E, M, G, n_tenants, bm, bin_off, tenant_expert_count,
                     expert_off, group_off, stats);
+    if (do_plan) {
+        __syncthreads();
+        plan_body(expert_off, pa, s_tot + nbins, s_part);
+    }
 }
 
 // Small batches: the whole dispatch in one block -- histogram, scan, tables, stable ranks (one warp
 // walks the rows in order), and the gather of the rows.  Same results as the multi-block kernels.
-constexpr int kSmallRows = 2048;
+constexpr int kSmallRows = 8192;
 
 __global__ void __launch_bounds__(1024)
 dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ tenant_id, int R, int k,
@@ -351,10 +363,16 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
         }
         return cudaGetLastError();
     }
+    const bool do_plan = with_plan && g.n_models == 1;
+    PlanArgs pa;
+    memset(&pa, 0, sizeof(pa));
+    size_t plan_ints = 0;
+    if (do_plan) { pa = make_plan_args(c, T, G, plan_shared); plan_ints = plan_smem_ints(c, G); }
     dispatch_hist_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, c->ws.block_cnt, c->ws.status);
-    dispatch_scan_kernel<<<1, 1024, smem, st>>>(nblk, nbins, R, g.n_experts, g.n_models, G, g.n_tenants, bm,
-                                                c->ws.block_cnt, c->ws.bin_off, tenant_expert_count, expert_off,
-                                                group_off, c->ws.stats);
+    dispatch_scan_kernel<<<1, 1024, smem + plan_ints * sizeof(int32_t), st>>>(
+        nblk, nbins, R, g.n_experts, g.n_models, G, g.n_tenants, bm, c->ws.block_cnt, c->ws.bin_off,
+        tenant_expert_count, expert_off, group_off, c->ws.stats, do_plan ? 1 : 0, pa);
+    if (plan_done) *plan_done = do_plan;
     dispatch_rank_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, c->ws.block_cnt, c->ws.bin_off,
                                                  perm, inv_perm, c->ws.status);
     c->launches += 3;
@@ -496,7 +514,7 @@ extern "C" int moe_dispatch_noalloc(const int32_t* topk_idx, const int32_t* tena
     const size_t smem = (size_t)nbins * sizeof(int32_t);
     dispatch_hist_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, s + o_blk, status);
     dispatch_scan_kernel<<<1, 1024, smem, st>>>(nblk, nbins, R, E, M, G, n_tenants, bm, s + o_blk, s + o_binoff,
-                                                tenant_expert_count, expert_off, group_off, s + o_stats);
+                                                tenant_expert_count, expert_off, group_off, s + o_stats, 0, PlanArgs());
     dispatch_rank_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, s + o_blk, s + o_binoff, perm,
                                                  inv_perm, status);
     return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
