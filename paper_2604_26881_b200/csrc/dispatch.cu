@@ -144,7 +144,7 @@ dispatch_scan_kernel(int nblk, int nbins, int R, int E, int M, int G, int n_tena
 
 // Small batches: the whole dispatch in one block -- histogram, scan, tables, stable ranks (one warp
 // walks the rows in order), and the gather of the rows.  Same results as the multi-block kernels.
-constexpr int kSmallRows = 8192;
+constexpr int kSmallRows = 2048;   // above this the serial ranking pass of one warp costs more than the extra launches
 
 __global__ void __launch_bounds__(1024)
 dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ tenant_id, int R, int k,
@@ -152,15 +152,20 @@ dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
                       int32_t* __restrict__ inv_perm, int32_t* __restrict__ tenant_expert_count,
                       int32_t* __restrict__ expert_off, int32_t* __restrict__ group_off, int32_t* __restrict__ stats,
                       int32_t* __restrict__ status, const bf16* __restrict__ x, bf16* __restrict__ x_perm, int H,
-                      int do_plan, PlanArgs pa)
+                      int do_plan, int plan_ints, PlanArgs pa)
 {
-    extern __shared__ int32_t s_tot[];       // [nbins], then the plan's scratch
+    extern __shared__ int32_t s_tot[];       // [nbins], then the plan's scratch, then the bin of every row (u16)
     __shared__ int32_t s_part[33];
     __shared__ int32_t s_count[2];
     const int tid = threadIdx.x, nth = blockDim.x;
+    unsigned short* s_bin = reinterpret_cast<unsigned short*>(s_tot + nbins + plan_ints);
     for (int b = tid; b < nbins; b += nth) s_tot[b] = 0;
     __syncthreads();
-    for (int r = tid; r < R; r += nth) atomicAdd(&s_tot[row_bin(bm, tenant_id[r / k], topk_idx[r], status)], 1);
+    for (int r = tid; r < R; r += nth) {
+        const int bin = row_bin(bm, tenant_id[r / k], topk_idx[r], status);
+        s_bin[r] = (unsigned short)bin;      // nbins <= 8192: fits; the ranking pass below reads it back
+        atomicAdd(&s_tot[bin], 1);
+    }
     __syncthreads();
     scan_and_tables(s_tot, s_part, s_count, nbins, R, E, M, G, n_tenants, bm, nullptr, tenant_expert_count,
                     expert_off, group_off, stats);
@@ -171,7 +176,7 @@ dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
             const int r = rr + lane;
             const bool live = r < R;
             int bin = -1 - lane;
-            if (live) bin = row_bin(bm, tenant_id[r / k], topk_idx[r], status);
+            if (live) bin = s_bin[r];
             const unsigned peers = __match_any_sync(0xffffffffu, bin);
             const int leader = __ffs(peers) - 1;
             const int rank = __popc(peers & ((1u << lane) - 1u));
@@ -351,10 +356,13 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
         size_t plan_ints = 0;
         if (do_plan) { pa = make_plan_args(c, T, G, plan_shared); plan_ints = plan_smem_ints(c, G); }
         const int threads = (R <= 512 && nbins <= 1024) ? 256 : 1024;
-        dispatch_small_kernel<<<1, threads, smem + plan_ints * sizeof(int32_t), st>>>(
+        const size_t smem_small = smem + plan_ints * sizeof(int32_t) + (((size_t)R * 2 + 15) & ~(size_t)15);
+        if (smem_small > 48 * 1024)
+            cudaFuncSetAttribute(dispatch_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_small);
+        dispatch_small_kernel<<<1, threads, smem_small, st>>>(
             topk_idx, tenant_id, R, k, bm, nbins, g.n_experts, g.n_models, G, g.n_tenants, perm, inv_perm,
             tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, x, gather_inside ? x_perm : nullptr,
-            g.hidden, do_plan ? 1 : 0, pa);
+            g.hidden, do_plan ? 1 : 0, (int)plan_ints, pa);
         if (plan_done) *plan_done = do_plan;
         c->launches += 1;
         if (x_perm && !gather_inside) {
