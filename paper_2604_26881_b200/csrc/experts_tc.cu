@@ -40,10 +40,12 @@ constexpr int kBRows = 128;                    // token rows one CTA loads per s
 constexpr int kBBytes = kBRows * kBK * 2;      // 16 KB
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kQueue = 4;                      // depth of the unit queue of the dynamic scheduler
-constexpr int kNumBars = 2 * kStages + 4 + 2 * kQueue;
+constexpr int kNumBars = 2 * kStages + 4 + 2 * kQueue + 1;
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 8 * kNumBars + 64;
 constexpr int kEpiWarps = 8;                   // two warps per TMEM lane quarter, alternating 16-column chunks
-constexpr int kThreads = 64 + 32 * kEpiWarps;  // warp 0: TMA, warp 1: MMA + TMEM, warps 2..: epilogue
+constexpr int kSchedWarp = 2 + kEpiWarps;      // warp 0: TMA, warp 1: MMA + TMEM, warps 2..9: epilogue, warp 10: scheduler
+constexpr int kThreads = 32 * (kSchedWarp + 1);
+constexpr int kClaimAhead = 8;                 // the next unit is claimed this many K steps before the current one is loaded
 constexpr uint32_t kTmemCols = 512;            // 2 accumulator buffers x 256 columns
 
 struct GemmParams {
@@ -152,25 +154,39 @@ struct UnitInfo {
     int direct;                   // routed gate/up unit in direct mode: B = all tokens
 };
 
+// One slot of the unit queue: the unit as the scheduler decoded it for cluster rank 0, so that no other role
+// has to chase the unit and tile tables through global memory.  u < 0: no more work.
+struct __align__(16) QEntry {
+    int u, tile_slot, b_row0, nrows;
+    int colblock, shared, pad0, pad1;
+};
+
 template <int MODE, bool PAIR>
-__device__ __forceinline__ UnitInfo decode_unit(const GemmParams& p, int u, uint32_t rank)
+__device__ __forceinline__ UnitInfo unit_info(const GemmParams& p, const QEntry& e, uint32_t rank)
 {
-    const Unit un = p.units[u];
     UnitInfo ui;
-    ui.shared = un.tile < 0;
-    const Tile t = ui.shared ? p.stiles[~un.tile] : p.tiles[un.tile];
-    ui.cb = PAIR ? 2 * un.colblock + (int)rank : un.colblock;
-    ui.model = t.slot;
-    ui.amap = ui.shared ? t.slot : -1;
-    ui.a_row = (ui.shared ? 0 : t.slot * p.rows_per_slot) + ui.cb * p.cb_rows;
-    ui.b_row0 = t.row0;
-    ui.nrows = t.nrows;
+    ui.shared = e.shared;
+    ui.cb = PAIR ? 2 * e.colblock + (int)rank : e.colblock;
+    ui.model = e.tile_slot;
+    ui.amap = ui.shared ? e.tile_slot : -1;
+    ui.a_row = (ui.shared ? 0 : e.tile_slot * p.rows_per_slot) + ui.cb * p.cb_rows;
+    ui.b_row0 = e.b_row0;
+    ui.nrows = e.nrows;
     ui.direct = (MODE == 0 && p.direct && !ui.shared) ? 1 : 0;
     if (ui.direct) { ui.npad = p.n_tokens_pad; }
-    else if (PAIR) ui.npad = (t.nrows + 31) & ~31;
-    else ui.npad = (t.nrows + 15) & ~15;
+    else if (PAIR) ui.npad = (e.nrows + 31) & ~31;
+    else ui.npad = (e.nrows + 15) & ~15;
     ui.ksteps = (ui.shared ? p.k_shared : p.k_routed) / kBK;
     return ui;
+}
+
+__device__ __forceinline__ QEntry read_entry(const QEntry* q)
+{
+    const int4 a = *reinterpret_cast<const int4*>(q);
+    const int2 b = *reinterpret_cast<const int2*>(&q->colblock);
+    QEntry e;
+    e.u = a.x; e.tile_slot = a.y; e.b_row0 = a.z; e.nrows = a.w; e.colblock = b.x; e.shared = b.y; e.pad0 = e.pad1 = 0;
+    return e;
 }
 
 // MODE 0: gate/up + SwiGLU (output bf16 for routed units, fp16 for shared units)
@@ -185,9 +201,10 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     const uint32_t bar_full = bars, bar_empty = bars + 8 * kStages;
     const uint32_t bar_tfull = bars + 16 * kStages, bar_tempty = bar_tfull + 16;
     const uint32_t bar_qfull = bar_tempty + 16, bar_qempty = bar_qfull + 8 * kQueue;
+    const uint32_t bar_sched = bar_qempty + 8 * kQueue;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
-    __shared__ int s_queue[kQueue];
+    __shared__ QEntry s_queue[kQueue];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
@@ -197,12 +214,13 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, (PAIR ? 2 : 1) * kEpiWarps); }
-        // unit queue: filled by the scheduler (the leader's producer lane); drained by the MMA lane and the
-        // epilogue warps of this CTA and, in pair mode, by the peer's producer lane and epilogue warps
+        // unit queue: filled by the scheduler lane (of the leader CTA); drained by the producer lane, the MMA lane
+        // and the epilogue warps of this CTA and, in pair mode, by the peer's producer lane and epilogue warps
         for (int q = 0; q < kQueue; ++q) {
             mbar_init(bar_qfull + 8 * q, 1);
-            mbar_init(bar_qempty + 8 * q, 1 + kEpiWarps + (PAIR ? 1 + kEpiWarps : 0));
+            mbar_init(bar_qempty + 8 * q, 2 + kEpiWarps + (PAIR ? 1 + kEpiWarps : 0));
         }
+        mbar_init(bar_sched, 1);
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -224,9 +242,11 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
 
-    // Units are pulled from a global counter by one scheduler lane per CTA (pair: per CTA pair, the leader's)
-    // and handed to the other roles through a small queue in shared memory; in pair mode the leader also
-    // writes the peer's queue and the peer's consumers release the slot on the leader's barrier.
+    // Units are pulled from a global counter by one scheduler lane per CTA (pair: per CTA pair, the leader's),
+    // decoded, and handed to the other roles through a small queue in shared memory; in pair mode the scheduler
+    // also writes the peer's queue and the peer's consumers release the slot on the leader's barrier.  The
+    // scheduler is a warp of its own: a global load or atomic issued by the lane that feeds the TMA unit
+    // queues behind the tile requests and was measured to cost thousands of cycles per unit.
     const uint32_t qempty_leader = PAIR ? map_to_cta(bar_qempty, 0) : bar_qempty;
 
     if (warp == 0) {
@@ -237,29 +257,15 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
             bool ok = true;
             const uint64_t pol_w = p.stream_weights ? l2_evict_first() : l2_evict_last();
             const uint64_t pol_x = l2_evict_last();
-            int u = 0;
-            const uint32_t peer_queue = PAIR ? map_to_cta(smem_u32(&s_queue[0]), 1) : 0u;
-            const uint32_t peer_qfull = PAIR ? map_to_cta(bar_qfull, 1) : 0u;
             while (ok) {
-                if (leader) {
-                    if (!(PAIR ? mbar_wait_cluster(bar_qempty + 8 * q, qphase ^ 1, &s_abort, p.status)
-                               : mbar_wait(bar_qempty + 8 * q, qphase ^ 1, &s_abort, p.status))) { ok = false; break; }
-                    u = atomicAdd(p.counter, 1);
-                    if (u >= n_units) u = -1;
-                    s_queue[q] = u;
-                    mbar_arrive(bar_qfull + 8 * q);
-                    if (PAIR) {
-                        asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(peer_queue + 4 * q), "r"(u) : "memory");
-                        mbar_arrive_cluster(peer_qfull + 8 * q);
-                    }
-                } else {
-                    if (!mbar_wait_cluster(bar_qfull + 8 * q, qphase, &s_abort, p.status)) { ok = false; break; }
-                    u = s_queue[q];
-                    mbar_arrive_cluster(qempty_leader + 8 * q);
-                }
+                if (!(leader ? mbar_wait(bar_qfull + 8 * q, qphase, &s_abort, p.status)
+                             : mbar_wait_cluster(bar_qfull + 8 * q, qphase, &s_abort, p.status))) { ok = false; break; }
+                const QEntry e = read_entry(&s_queue[q]);
+                if (leader) mbar_arrive(bar_qempty + 8 * q); else mbar_arrive_cluster(qempty_leader + 8 * q);
                 if (++q == kQueue) { q = 0; qphase ^= 1; }
-                if (u < 0) break;
-                const UnitInfo ui = decode_unit<MODE, PAIR>(p, u, rank);
+                if (e.u < 0) break;
+                const UnitInfo ui = unit_info<MODE, PAIR>(p, e, rank);
+                const int claim_ks = ui.ksteps > kClaimAhead ? ui.ksteps - kClaimAhead : 0;
                 const CUtensorMap* ma = ui.amap < 0 ? &maps.a_routed : &maps.a_shared[ui.amap];
                 const bool bshared = ui.shared || ui.direct;
                 const CUtensorMap* mb128 = bshared ? &maps.b_shared128 : &maps.b_routed128;
@@ -268,6 +274,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 const int my_rows = PAIR ? (ui.npad >> 1) : ui.npad;          // token rows this CTA loads
                 const int my_row0 = brow0 + (PAIR ? (int)rank * my_rows : 0);
                 for (int ks = 0; ks < ui.ksteps; ++ks) {
+                    if (leader && ks == claim_ks) mbar_arrive(bar_sched);      // time to claim the next unit
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, &s_abort, p.status)) { ok = false; break; }
                     const uint32_t sa = smem_base + stage * kStageBytes, sb = sa + kABytes;
                     const uint32_t full = bar_full + 8 * stage;
@@ -302,14 +309,13 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
         if (lane == 0 && leader) {
             uint32_t stage = 0, phase = 0, buf = 0, bphase = 0, q = 0, qphase = 0;
             bool ok = true;
-            int u = 0;
             while (ok) {
                 if (!mbar_wait(bar_qfull + 8 * q, qphase, &s_abort, p.status)) { ok = false; break; }
-                u = s_queue[q];
+                const QEntry e = read_entry(&s_queue[q]);
                 mbar_arrive(bar_qempty + 8 * q);
                 if (++q == kQueue) { q = 0; qphase ^= 1; }
-                if (u < 0) break;
-                const UnitInfo ui = decode_unit<MODE, PAIR>(p, u, rank);
+                if (e.u < 0) break;
+                const UnitInfo ui = unit_info<MODE, PAIR>(p, e, rank);
                 const uint32_t fmt = ui.shared ? p.idesc_fmt_shared : p.idesc_fmt_routed;
                 const uint32_t idesc = (1u << 4) | fmt | ((uint32_t)(ui.npad >> 3) << 17) | (((PAIR ? 256u : 128u) >> 4) << 24);
                 if (!(PAIR ? mbar_wait_cluster(bar_tempty + 8 * buf, bphase ^ 1, &s_abort, p.status)
@@ -338,27 +344,26 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
             }
         }
         __syncwarp();
-    } else {
+    } else if (warp < kSchedWarp) {
         // ---------------- epilogue: two warps per TMEM lane quarter, alternating 16-column chunks ----------------
         const int quarter = warp & 3;
         const int half = (warp - 2) >> 2;                  // 0 or 1: which chunks of 16 columns this warp takes
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         uint32_t buf = 0, bphase = 0, q = 0, qphase = 0;
         bool ok = true;
-        int u = 0;
         const uint32_t tempty_leader = PAIR ? map_to_cta(bar_tempty, 0) : bar_tempty;
         while (ok) {
             ok = __all_sync(0xffffffffu, PAIR ? mbar_wait_cluster(bar_qfull + 8 * q, qphase, &s_abort, p.status)
                                               : mbar_wait(bar_qfull + 8 * q, qphase, &s_abort, p.status));
             if (!ok) break;
-            u = s_queue[q];
+            const QEntry e = read_entry(&s_queue[q]);
             __syncwarp();
             if (lane == 0) {
                 if (PAIR) mbar_arrive_cluster(qempty_leader + 8 * q); else mbar_arrive(bar_qempty + 8 * q);
             }
             if (++q == kQueue) { q = 0; qphase ^= 1; }
-            if (u < 0) break;
-            const UnitInfo ui = decode_unit<MODE, PAIR>(p, u, rank);
+            if (e.u < 0) break;
+            const UnitInfo ui = unit_info<MODE, PAIR>(p, e, rank);
             // one decision for the whole warp: the TMEM loads below are warp-wide instructions
             ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, bphase, &s_abort, p.status));
             if (!ok) break;
@@ -435,6 +440,48 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
             }
             if (++buf == 2) { buf = 0; bphase ^= 1; }
         }
+    } else {
+        // ---------------- scheduler (one lane of the leader CTA) ----------------
+        if (lane == 0 && leader) {
+            uint32_t q = 0, qphase = 0, sphase = 0;
+            bool first = true;
+            const uint32_t peer_queue = PAIR ? map_to_cta(smem_u32(&s_queue[0]), 1) : 0u;
+            const uint32_t peer_qfull = PAIR ? map_to_cta(bar_qfull, 1) : 0u;
+            for (;;) {
+                // the first unit at once, every further one when the producer nears the end of its current unit
+                if (!first) {
+                    if (!mbar_wait(bar_sched, sphase, &s_abort, p.status)) break;
+                    sphase ^= 1;
+                }
+                first = false;
+                if (!(PAIR ? mbar_wait_cluster(bar_qempty + 8 * q, qphase ^ 1, &s_abort, p.status)
+                           : mbar_wait(bar_qempty + 8 * q, qphase ^ 1, &s_abort, p.status))) break;
+                int u = atomicAdd(p.counter, 1);
+                int4 e0 = make_int4(-1, 0, 0, 0);
+                int2 e1 = make_int2(0, 0);
+                if (u < n_units) {
+                    const Unit un = p.units[u];
+                    const Tile t = un.tile < 0 ? p.stiles[~un.tile] : p.tiles[un.tile];
+                    e0 = make_int4(u, t.slot, t.row0, t.nrows);
+                    e1 = make_int2(un.colblock, un.tile < 0 ? 1 : 0);
+                } else {
+                    u = -1;
+                }
+                *reinterpret_cast<int4*>(&s_queue[q]) = e0;
+                *reinterpret_cast<int2*>(&s_queue[q].colblock) = e1;
+                mbar_arrive(bar_qfull + 8 * q);
+                if (PAIR) {
+                    const uint32_t dst = peer_queue + (uint32_t)sizeof(QEntry) * q;
+                    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(e0.x), "r"(e0.y), "r"(e0.z),
+                                 "r"(e0.w) : "memory");
+                    asm volatile("st.shared::cluster.v2.b32 [%0], {%1, %2};" ::"r"(dst + 16), "r"(e1.x), "r"(e1.y) : "memory");
+                    mbar_arrive_cluster(peer_qfull + 8 * q);
+                }
+                if (++q == kQueue) { q = 0; qphase ^= 1; }
+                if (u < 0) break;
+            }
+        }
+        __syncwarp();
     }
 
     tc_fence_before();
