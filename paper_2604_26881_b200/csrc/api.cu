@@ -203,6 +203,7 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->rmaps = nullptr;
     c->route_path = MOE_PATH_AUTO;
     c->pair_mode_enabled = 1;
+    c->wide_tiles_enabled = 1;
     c->timing = false;
     for (auto& e : c->ev) e = nullptr;
     c->errbuf[0] = 0;
@@ -326,6 +327,11 @@ int moe_set_option(moe_ctx* c, int option, int value)
     }
     if (option == MOE_OPT_PAIR_MODE) {
         c->pair_mode_enabled = value ? 1 : 0;
+        return MOE_OK;
+    }
+    if (option == MOE_OPT_WIDE_TILES) {
+        if (value < 0 || value > 2) return MOE_ERR_SHAPE;
+        c->wide_tiles_enabled = value;
         return MOE_OK;
     }
     if (option == MOE_OPT_ROUTE_PATH) {

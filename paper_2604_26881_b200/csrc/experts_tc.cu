@@ -33,15 +33,25 @@ namespace {
 
 using namespace tc;
 
-constexpr int kStages = 6;
+constexpr int kMaxStages = 6;
 constexpr int kBK = 64;                        // K elements per stage = one 128-byte swizzle row
 constexpr int kABytes = 128 * kBK * 2;         // 128 weight rows: 16 KB
-constexpr int kBRows = 128;                    // token rows one CTA loads per stage (pair: half of the tile)
+constexpr int kBRows = 128;                    // token rows one CTA loads per accumulator and stage (pair: half of them)
 constexpr int kBBytes = kBRows * kBK * 2;      // 16 KB
-constexpr int kStageBytes = kABytes + kBBytes;
+// Two pipeline geometries over the same 192 KB: 6 stages of (weights + one token tile), or 4 stages of
+// (weights + two token tiles) when a unit may feed both accumulators from one weight tile ("wide" units).
+constexpr int kRingBytes = kMaxStages * (kABytes + kBBytes);
+constexpr int kWideStages = kRingBytes / (kABytes + 2 * kBBytes);
 constexpr int kQueue = 4;                      // depth of the unit queue of the dynamic scheduler
-constexpr int kNumBars = 2 * kStages + 4 + 2 * kQueue + 1;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 8 * kNumBars + 64;
+constexpr int kNumBars = 2 * kMaxStages + 4 + 2 * kQueue + 1;
+constexpr int kBarBytes = 256;                 // >= 8 * kNumBars, keeps the staging area 128-byte aligned
+// Output staging of the epilogue: results go to shared memory and leave as bulk copies of one row each,
+// so that the epilogue warps never wait on the global store path (which the operand loads saturate).
+// The two groups of four epilogue warps own one half each.
+constexpr int kOutStageBytes = 32768;
+constexpr int kOutGroupBytes = kOutStageBytes / 2;
+constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + kBarBytes + kOutStageBytes;
+static_assert(8 * kNumBars <= kBarBytes, "barrier area too small");
 constexpr int kEpiWarps = 8;                   // two warps per TMEM lane quarter, alternating 16-column chunks
 constexpr int kSchedWarp = 2 + kEpiWarps;      // warp 0: TMA, warp 1: MMA + TMEM, warps 2..9: epilogue, warp 10: scheduler
 constexpr int kThreads = 32 * (kSchedWarp + 1);
@@ -69,6 +79,8 @@ struct GemmParams {
     uint32_t gate_first_routed;   // bit 0: the gate row is the even TMEM lane of a pair (routed map)
     uint32_t gate_first_shared;   // bit m: same for the shared expert of model m
     int stream_weights;           // 1: every weight tile is read once: mark it evict-first in L2
+    int group;                    // stages handed back to the producer per commit (divides the stage count)
+    int wide;                     // 1: tiles of up to 512 rows (pair shape only): 4 stages of 48 KB instead of 6 of 32 KB
     int32_t* status;
 };
 
@@ -148,9 +160,33 @@ __device__ __forceinline__ void tmem_ld1(uint32_t taddr, uint32_t& r)
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr));
 }
 
+// bulk copy shared -> global of one output row (16-byte aligned on both sides, size a multiple of 16)
+__device__ __forceinline__ void bulk_store(void* gdst, uint32_t ssrc, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(ssrc), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// barrier of one epilogue group (128 threads) that also ANDs a flag over the group
+__device__ __forceinline__ bool group_and(int id, bool v)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, %2, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"((uint32_t)v), "r"(id) : "memory");
+    return r != 0;
+}
+__device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+
 struct UnitInfo {
     int a_row, amap;              // first weight row of the tile; -1: routed map, m: shared map of model m
     int b_row0, nrows, npad, ksteps, shared, cb, model;
+    int npad1;                    // wide unit: padded rows of the second accumulator (rows 256..), else 0
     int direct;                   // routed gate/up unit in direct mode: B = all tokens
 };
 
@@ -173,8 +209,14 @@ __device__ __forceinline__ UnitInfo unit_info(const GemmParams& p, const QEntry&
     ui.b_row0 = e.b_row0;
     ui.nrows = e.nrows;
     ui.direct = (MODE == 0 && p.direct && !ui.shared) ? 1 : 0;
+    ui.npad1 = 0;
     if (ui.direct) { ui.npad = p.n_tokens_pad; }
-    else if (PAIR) ui.npad = (e.nrows + 31) & ~31;
+    else if (PAIR) {
+        // up to 512 rows: the first 256 go to one accumulator, the rest to the other
+        const int n0 = e.nrows < 256 ? e.nrows : 256;
+        ui.npad = (n0 + 31) & ~31;
+        ui.npad1 = (e.nrows - n0 + 31) & ~31;
+    }
     else ui.npad = (e.nrows + 15) & ~15;
     ui.ksteps = (ui.shared ? p.k_shared : p.k_routed) / kBK;
     return ui;
@@ -197,9 +239,14 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
 {
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
-    const uint32_t bars = smem_base + kStages * kStageBytes;                   // 8-byte barriers after the tiles
-    const uint32_t bar_full = bars, bar_empty = bars + 8 * kStages;
-    const uint32_t bar_tfull = bars + 16 * kStages, bar_tempty = bar_tfull + 16;
+    const uint32_t bars = smem_base + kRingBytes;                              // 8-byte barriers after the tiles
+    const uint32_t bar_full = bars, bar_empty = bars + 8 * kMaxStages;
+    const uint32_t bar_tfull = bars + 16 * kMaxStages, bar_tempty = bar_tfull + 16;
+    const uint32_t n_stages = (PAIR && p.wide) ? kWideStages : kMaxStages;
+    const uint32_t stage_bytes = kRingBytes / n_stages;
+    // Stages are handed back to the producer in groups: a tcgen05.commit costs the issuing lane about as much
+    // as two MMAs, so with four MMAs per stage one commit per stage would starve the tensor pipe.
+    const uint32_t group = (uint32_t)p.group;
     const uint32_t bar_qfull = bar_tempty + 16, bar_qempty = bar_qfull + 8 * kQueue;
     const uint32_t bar_sched = bar_qempty + 8 * kQueue;
     __shared__ uint32_t s_tmem_base;
@@ -212,7 +259,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     const int n_units = *p.n_units;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, (PAIR ? 2 : 1) * kEpiWarps); }
         // unit queue: filled by the scheduler lane (of the leader CTA); drained by the producer lane, the MMA lane
         // and the epilogue warps of this CTA and, in pair mode, by the peer's producer lane and epilogue warps
@@ -273,12 +320,15 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 const int brow0 = ui.direct ? 0 : ui.b_row0;
                 const int my_rows = PAIR ? (ui.npad >> 1) : ui.npad;          // token rows this CTA loads
                 const int my_row0 = brow0 + (PAIR ? (int)rank * my_rows : 0);
+                const int my_rows1 = ui.npad1 >> 1;                           // same for the second accumulator
+                const int my_row1 = brow0 + 256 + (int)rank * my_rows1;
                 for (int ks = 0; ks < ui.ksteps; ++ks) {
                     if (leader && ks == claim_ks) mbar_arrive(bar_sched);      // time to claim the next unit
-                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, &s_abort, p.status)) { ok = false; break; }
-                    const uint32_t sa = smem_base + stage * kStageBytes, sb = sa + kABytes;
+                    if (stage % group == 0 &&
+                        !mbar_wait(bar_empty + 8 * (stage / group), phase ^ 1, &s_abort, p.status)) { ok = false; break; }
+                    const uint32_t sa = smem_base + stage * stage_bytes, sb = sa + kABytes;
                     const uint32_t full = bar_full + 8 * stage;
-                    if (leader) mbar_expect_tx(full, (PAIR ? 2u : 1u) * (uint32_t)(kABytes + my_rows * kBK * 2));
+                    if (leader) mbar_expect_tx(full, (PAIR ? 2u : 1u) * (uint32_t)(kABytes + (my_rows + my_rows1) * kBK * 2));
                     armed |= 1u << stage;
                     armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
                     if (PAIR) {
@@ -287,6 +337,9 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                         int j = 0;
                         for (; j + 128 <= my_rows; j += 128) tma_load_2d_pair(sb + j * kBK * 2, mb128, full, ks * kBK, my_row0 + j, pol_x);
                         for (; j < my_rows; j += 16) tma_load_2d_pair(sb + j * kBK * 2, mb16, full, ks * kBK, my_row0 + j, pol_x);
+                        const uint32_t sb1 = sb + kBBytes;
+                        for (j = 0; j + 128 <= my_rows1; j += 128) tma_load_2d_pair(sb1 + j * kBK * 2, mb128, full, ks * kBK, my_row1 + j, pol_x);
+                        for (; j < my_rows1; j += 16) tma_load_2d_pair(sb1 + j * kBK * 2, mb16, full, ks * kBK, my_row1 + j, pol_x);
                     } else {
                         if (MODE == 0) tma_load_3d_hint(sa, ma, full, ks * kBK, 0, ui.a_row, pol_w);
                         else tma_load_2d_hint(sa, ma, full, ks * kBK, ui.a_row, pol_w);
@@ -294,12 +347,12 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                         for (; j + 128 <= my_rows; j += 128) tma_load_2d_hint(sb + j * kBK * 2, mb128, full, ks * kBK, my_row0 + j, pol_x);
                         for (; j < my_rows; j += 16) tma_load_2d_hint(sb + j * kBK * 2, mb16, full, ks * kBK, my_row0 + j, pol_x);
                     }
-                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                    if (++stage == n_stages) { stage = 0; phase ^= 1; }
                 }
             }
             if (!ok && leader) {
                 // gave up: let the copies already in flight land before the block exits
-                for (int s = 0; s < kStages; ++s)
+                for (int s = 0; s < kMaxStages; ++s)
                     if (armed & (1u << s)) mbar_wait(bar_full + 8 * s, (armed_phase >> s) & 1u, &s_abort, p.status);
             }
         }
@@ -317,15 +370,21 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 if (e.u < 0) break;
                 const UnitInfo ui = unit_info<MODE, PAIR>(p, e, rank);
                 const uint32_t fmt = ui.shared ? p.idesc_fmt_shared : p.idesc_fmt_routed;
-                const uint32_t idesc = (1u << 4) | fmt | ((uint32_t)(ui.npad >> 3) << 17) | (((PAIR ? 256u : 128u) >> 4) << 24);
+                const uint32_t idesc_m = (1u << 4) | fmt | (((PAIR ? 256u : 128u) >> 4) << 24);
+                const uint32_t idesc = idesc_m | ((uint32_t)(ui.npad >> 3) << 17);
+                const uint32_t idesc1 = idesc_m | ((uint32_t)(ui.npad1 >> 3) << 17);
+                const bool wide = PAIR && ui.npad1 > 0;
+                // a wide unit takes both accumulator buffers, in the order the epilogue drains them
                 if (!(PAIR ? mbar_wait_cluster(bar_tempty + 8 * buf, bphase ^ 1, &s_abort, p.status)
                            : mbar_wait(bar_tempty + 8 * buf, bphase ^ 1, &s_abort, p.status))) { ok = false; break; }
-                tc_fence_after();
                 const uint32_t d = tmem_base + buf * 256;
+                const uint32_t buf1 = buf ^ 1u, bphase1 = buf ? (bphase ^ 1u) : bphase;
+                const uint32_t d1 = tmem_base + buf1 * 256;
+                tc_fence_after();
                 for (int ks = 0; ks < ui.ksteps; ++ks) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, &s_abort, p.status)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = smem_base + stage * kStageBytes, sb = sa + kABytes;
+                    const uint32_t sa = smem_base + stage * stage_bytes, sb = sa + kABytes;
                     const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
 #pragma unroll
                     for (int kk = 0; kk < kBK / 16; ++kk) {
@@ -334,22 +393,48 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                         if (PAIR) umma_bf16_pair(d, da + adv, db + adv, idesc, acc);
                         else umma_bf16(d, da + adv, db + adv, idesc, acc);
                     }
-                    // frees the stage (in both CTAs of a pair) when these MMAs have read it
-                    if (PAIR) umma_commit_pair(bar_empty + 8 * stage); else umma_commit(bar_empty + 8 * stage);
-                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                    if (wide) {
+                        if (ks == ui.ksteps - 1) umma_commit_pair(bar_tfull + 8 * buf);      // first half done: its epilogue may start
+                        if (ks == 0) {
+                            if (!mbar_wait_cluster(bar_tempty + 8 * buf1, bphase1 ^ 1, &s_abort, p.status)) { ok = false; break; }
+                            tc_fence_after();
+                        }
+                        const uint64_t db1 = smem_desc_sw128(sb + kBBytes);
+#pragma unroll
+                        for (int kk = 0; kk < kBK / 16; ++kk) {
+                            const uint32_t acc = (ks | kk) ? 1u : 0u;
+                            const uint64_t adv = (uint64_t)(kk * 32 >> 4);
+                            umma_bf16_pair(d1, da + adv, db1 + adv, idesc1, acc);
+                        }
+                    }
+                    // frees the stage group (in both CTAs of a pair) when these MMAs have read it
+                    if (stage % group == group - 1) {
+                        if (PAIR) umma_commit_pair(bar_empty + 8 * (stage / group)); else umma_commit(bar_empty + 8 * (stage / group));
+                    }
+                    if (++stage == n_stages) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
-                if (PAIR) umma_commit_pair(bar_tfull + 8 * buf); else umma_commit(bar_tfull + 8 * buf);
-                if (++buf == 2) { buf = 0; bphase ^= 1; }
+                if (wide) {
+                    umma_commit_pair(bar_tfull + 8 * buf1);
+                    bphase ^= 1;                                   // two buffers taken: same buffer next, other phase
+                } else {
+                    if (PAIR) umma_commit_pair(bar_tfull + 8 * buf); else umma_commit(bar_tfull + 8 * buf);
+                    if (++buf == 2) { buf = 0; bphase ^= 1; }
+                }
             }
         }
         __syncwarp();
     } else if (warp < kSchedWarp) {
-        // ---------------- epilogue: two warps per TMEM lane quarter, alternating 16-column chunks ----------------
+        // ---------------- epilogue: two groups of four warps (one warp per TMEM lane quarter), ----------------
+        // ---------------- the groups alternate over the 16-column chunks of an accumulator     ----------------
         const int quarter = warp & 3;
-        const int half = (warp - 2) >> 2;                  // 0 or 1: which chunks of 16 columns this warp takes
+        const int half = (warp - 2) >> 2;                  // group: 0 or 1
+        const int gbar = 1 + half;                         // named barrier of the group
+        const int gtid = quarter * 32 + lane;              // thread index inside the group
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        const uint32_t stg = bars + kBarBytes + half * kOutGroupBytes;      // this group's staging area
         uint32_t buf = 0, bphase = 0, q = 0, qphase = 0;
+        uint32_t rnd = 0;                                  // MODE 1: staging slot = rnd & 1
         bool ok = true;
         const uint32_t tempty_leader = PAIR ? map_to_cta(bar_tempty, 0) : bar_tempty;
         while (ok) {
@@ -364,21 +449,26 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
             if (++q == kQueue) { q = 0; qphase ^= 1; }
             if (e.u < 0) break;
             const UnitInfo ui = unit_info<MODE, PAIR>(p, e, rank);
-            // one decision for the whole warp: the TMEM loads below are warp-wide instructions
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull + 8 * buf, bphase, &s_abort, p.status));
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t d = tmem_base + lane_addr + buf * 256;
             const int ld = ui.shared ? p.ld_shared : p.ld_routed;
-            if (MODE == 0) {
-                // lanes 2i / 2i+1 hold the gate / up row (or up / gate) of intermediate index cb*64 + quarter*16 + i
-                const uint32_t gf = ui.shared ? (p.gate_first_shared >> ui.model) & 1u : p.gate_first_routed & 1u;
-                const bool even = (lane & 1) == 0;
-                const bool own_is_gate = even == (gf != 0);
-                const int col = ui.cb * 64 + quarter * 16 + (lane >> 1);
-                if (ui.direct) {
-                    for (int j = half; j < ui.nrows; j += 2) {
-                        const int tok = p.perm[ui.b_row0 + j] / p.top_k;            // warp-uniform
+            const int n_acc = (PAIR && ui.npad1 > 0) ? 2 : 1;
+            for (int hh = 0; hh < n_acc && ok; ++hh) {
+                // rows of this accumulator: a wide unit keeps rows 256.. in its second one
+                const int row0 = ui.b_row0 + hh * 256;
+                const int nrows = hh ? ui.nrows - 256 : (n_acc == 2 ? 256 : ui.nrows);
+                const int npad = hh ? ui.npad1 : ui.npad;
+                ok = mbar_wait(bar_tfull + 8 * buf, bphase, &s_abort, p.status);
+                const uint32_t d = tmem_base + lane_addr + buf * 256;
+                if (MODE == 0 && ui.direct) {
+                    // one decision for the whole warp: the TMEM loads below are warp-wide instructions
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    // lanes 2i / 2i+1 hold the gate / up row (or up / gate) of intermediate index cb*64 + quarter*16 + i
+                    const bool even = (lane & 1) == 0;
+                    const bool own_is_gate = even == ((p.gate_first_routed & 1u) != 0);
+                    const int col = ui.cb * 64 + quarter * 16 + (lane >> 1);
+                    for (int j = half; j < nrows; j += 2) {
+                        const int tok = p.perm[row0 + j] / p.top_k;            // warp-uniform
                         uint32_t r;
                         tmem_ld1(d + tok, r);
                         tmem_ld_wait();
@@ -386,15 +476,28 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                         const float other = __shfl_xor_sync(0xffffffffu, own, 1);
                         if (even) {
                             const float g = own_is_gate ? own : other, up = own_is_gate ? other : own;
-                            reinterpret_cast<bf16*>(p.out_routed)[(size_t)(ui.b_row0 + j) * ld + col] =
+                            reinterpret_cast<bf16*>(p.out_routed)[(size_t)(row0 + j) * ld + col] =
                                 __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * up);
                         }
                     }
-                } else {
-                    // 16-bit outputs; this lane's element of row n sits at out16[(b_row0 + n) * ld + col]
-                    unsigned short* out16 = reinterpret_cast<unsigned short*>(ui.shared ? p.out_shared : p.out_routed) +
-                                            (size_t)ui.b_row0 * ld + col;
-                    for (int c0 = half * 16; c0 < ui.npad; c0 += 32) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+                } else if (MODE == 0) {
+                    // The group's staging area holds its 8 chunks of 16 tokens as rows of 64 outputs (128 bytes).
+                    // Its previous contents must have left (every thread waits for the rows it sent itself), and the
+                    // whole group takes one decision on the accumulator wait.
+                    bulk_wait_read<0>();
+                    ok = group_and(gbar, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t gf = ui.shared ? (p.gate_first_shared >> ui.model) & 1u : p.gate_first_routed & 1u;
+                    const bool even = (lane & 1) == 0;
+                    const bool own_is_gate = even == (gf != 0);
+                    // lanes 2i / 2i+1 hold the gate / up row (or up / gate) of intermediate index cb*64 + quarter*16 + i
+                    const uint32_t my_col = stg + (uint32_t)(quarter * 32 + (lane >> 1) * 2);
+                    int i = 0;
+                    for (int c0 = half * 16; c0 < npad; c0 += 32, ++i) {
                         uint32_t r[16];
                         tmem_ld16(d + c0, r);
                         tmem_ld_wait();
@@ -404,42 +507,87 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                             const float send = __uint_as_float(even ? r[j + 1] : r[j]);
                             const float recv = __shfl_xor_sync(0xffffffffu, send, 1);
                             const float own = __uint_as_float(even ? r[j] : r[j + 1]);
-                            const int n = c0 + j + (even ? 0 : 1);
-                            if (n < ui.nrows) {
-                                const float g = own_is_gate ? own : recv, up = own_is_gate ? recv : own;
-                                const float v = __fdividef(g, 1.f + __expf(-g)) * up;
-                                out16[(size_t)n * ld] = ui.shared ? __half_as_ushort(__float2half_rn(v))
-                                                                  : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+                            const float g = own_is_gate ? own : recv, up = own_is_gate ? recv : own;
+                            const float v = __fdividef(g, 1.f + __expf(-g)) * up;
+                            const unsigned short o = ui.shared ? __half_as_ushort(__float2half_rn(v))
+                                                               : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+                            const uint32_t a = my_col + (uint32_t)(i * 16 + j + (even ? 0 : 1)) * 128u;
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "h"(o) : "memory");
+                        }
+                    }
+                    // the accumulator is free as soon as it has been read
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (PAIR) mbar_arrive_cluster(tempty_leader + 8 * buf); else mbar_arrive(bar_tempty + 8 * buf);
+                    }
+                    fence_async_smem();
+                    group_sync(gbar);
+                    // thread t of the group sends staged row t: token (t / 16) * 32 + half * 16 + t % 16
+                    {
+                        const int n = (gtid >> 4) * 32 + half * 16 + (gtid & 15);
+                        if (n < nrows) {
+                            unsigned short* out16 = reinterpret_cast<unsigned short*>(ui.shared ? p.out_shared : p.out_routed);
+                            bulk_store(out16 + (size_t)(row0 + n) * ld + ui.cb * 64, stg + (uint32_t)gtid * 128u, 128u);
+                        }
+                        bulk_commit();
+                    }
+                } else {
+                    // fp32 rows of 128 outputs (512 bytes); a chunk of 16 tokens fills one of the group's two slots
+                    const bool remap = ui.shared && p.shared_dst_rows != nullptr;
+                    float* outp = reinterpret_cast<float*>(ui.shared ? p.out_shared : p.out_routed) + ui.cb * 128;
+                    bool first = true;
+                    for (int c0 = half * 16; c0 < npad; c0 += 32, ++rnd) {
+                        const uint32_t slot = stg + (rnd & 1u) * 8192u;
+                        bulk_wait_read<1>();                       // the rows this thread sent from this slot have left
+                        if (first) {
+                            ok = group_and(gbar, ok);
+                            if (!ok) break;
+                            tc_fence_after();
+                            first = false;
+                        } else {
+                            group_sync(gbar);
+                        }
+                        uint32_t r[16];
+                        tmem_ld16(d + c0, r);
+                        tmem_ld_wait();
+                        const uint32_t a = slot + (uint32_t)(quarter * 128 + lane * 4);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) asm volatile("st.shared.b32 [%0], %1;" ::"r"(a + j * 512u), "r"(r[j]) : "memory");
+                        if (c0 + 32 >= npad) {
+                            // last chunk of this group: the accumulator has been read
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) {
+                                if (PAIR) mbar_arrive_cluster(tempty_leader + 8 * buf); else mbar_arrive(bar_tempty + 8 * buf);
                             }
                         }
+                        fence_async_smem();
+                        group_sync(gbar);
+                        if (lane < 4) {
+                            const int j = quarter * 4 + lane, n = c0 + j;
+                            if (n < nrows) {
+                                int row = row0 + n;
+                                if (remap) row = p.shared_dst_rows[row];
+                                bulk_store(outp + (size_t)row * ld, slot + (uint32_t)j * 512u, 512u);
+                            }
+                        }
+                        bulk_commit();
                     }
-                }
-            } else {
-                const int col = ui.cb * 128 + quarter * 32 + lane;
-                float* out = reinterpret_cast<float*>(ui.shared ? p.out_shared : p.out_routed) + col;
-                const bool remap = ui.shared && p.shared_dst_rows != nullptr;
-                for (int c0 = half * 16; c0 < ui.npad; c0 += 32) {
-                    uint32_t r[16];
-                    tmem_ld16(d + c0, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int n = c0 + j;
-                        if (n < ui.nrows) {
-                            int row = ui.b_row0 + n;
-                            if (remap) row = p.shared_dst_rows[row];
-                            out[(size_t)row * ld] = __uint_as_float(r[j]);
+                    if (!ok) break;
+                    if (first) {
+                        // no chunk for this group (a tile of at most 16 columns): only release the accumulator
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        if (lane == 0) {
+                            if (PAIR) mbar_arrive_cluster(tempty_leader + 8 * buf); else mbar_arrive(bar_tempty + 8 * buf);
                         }
                     }
                 }
+                if (++buf == 2) { buf = 0; bphase ^= 1; }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if (PAIR) mbar_arrive_cluster(tempty_leader + 8 * buf); else mbar_arrive(bar_tempty + 8 * buf);
-            }
-            if (++buf == 2) { buf = 0; bphase ^= 1; }
         }
+        bulk_wait_read<0>();       // staged rows are read before the block's shared memory goes away
     } else {
         // ---------------- scheduler (one lane of the leader CTA) ----------------
         if (lane == 0 && leader) {
@@ -549,6 +697,18 @@ bool tc_pair_mode(const moe_ctx* c, int T)
     // measured: above 128 tokens the pair shape wins for every workload tried (prefill 4096 tokens, the
     // 240-expert pool with ~34 rows per expert, the 24-block stack with ~1100 tokens)
     return c->pair_mode_enabled != 0 && T > 128;
+}
+
+// Tiles of up to 512 rows pay when the segments are long enough to fill them: the weight tile of a K step then
+// feeds two accumulators, so a CTA fetches 48 KB instead of 64 KB per 512 tokens.  The price is a shallower
+// pipeline (4 stages) and an epilogue that is not hidden behind the next unit.
+bool tc_wide_mode(const moe_ctx* c, int T)
+{
+    if (!tc_pair_mode(c, T) || c->wide_tiles_enabled == 0) return false;
+    if (c->wide_tiles_enabled == 2) return true;
+    // measured: pays from about 2048 tokens per tenant model (shared-expert tiles and the hot routed experts
+    // fill 512 rows); below that the units are short and want the deeper pipeline
+    return T / c->cfg.n_models >= 2048;
 }
 
 void tc_destroy(moe_ctx* c)
@@ -678,6 +838,8 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     p1.gate_first_routed = lm.gate_first_routed; p1.gate_first_shared = lm.gate_first_shared;
     p1.status = c->ws.status;
     p1.stream_weights = (R <= 2048) ? 1 : 0;
+    p1.wide = tc_wide_mode(c, T) ? 1 : 0;
+    p1.group = p1.wide ? 1 : 2;
     cudaError_t e = pair ? launch_gemm<0, true>(c, p1, m1, st) : launch_gemm<0, false>(c, p1, m1, st);
     if (e != cudaSuccess) return e;
     stage_mark(c, st, kEvGateUp);

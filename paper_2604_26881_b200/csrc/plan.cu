@@ -28,7 +28,7 @@ PlanArgs make_plan_args(moe_ctx* c, int T, int G, bool with_shared)
     PlanArgs a;
     a.slot_table = c->d_slot;
     a.M = g.n_models; a.E = g.n_experts; a.G = G; a.T = T;
-    a.tile_rows = pair ? 256 : kTileRows;
+    a.tile_rows = pair ? (tc_wide_mode(c, T) ? 512 : 256) : kTileRows;
     a.model_tok_off = g.n_models > 1 ? c->ws.model_tok_off : nullptr;
     a.with_shared = with_shared ? 1 : 0;
     a.nblk1 = g.inter / div1; a.nblk2 = g.hidden / div2;

@@ -210,6 +210,25 @@ def test_pair_shape_and_single_shape_agree_bit_for_bit(qwen_weights):
         g.close()
 
 
+@pytest.mark.parametrize("T", [1024, 1500, 4096])
+def test_wide_tiles_and_narrow_tiles_agree_bit_for_bit(qwen_weights, T):
+    # tiles of up to 512 rows feed two accumulators from one weight tile; every output element is
+    # still accumulated over K in the same order as with 256-row tiles.  The Zipf-skewed router
+    # gives segments of every length: shorter than 256, between 256 and 512, and several tiles long.
+    wl = W.scaled(W.WORKLOADS["prefill"], T=T)
+    x, tenant, mot = W.make_tokens(wl, seed=4)
+    g = GpuLayer(wl, [qwen_weights], wl.T, model_of_tenant=mot)
+    try:
+        B.moe_set_option(g.ctx, B.MOE_OPT_WIDE_TILES, 2)
+        wide = g.forward(x, tenant, wl.G)
+        B.moe_set_option(g.ctx, B.MOE_OPT_WIDE_TILES, 0)
+        narrow = g.forward(x, tenant, wl.G)
+        assert B.moe_last_status(g.ctx)[0] == 0
+        assert torch.equal(wide, narrow)
+    finally:
+        g.close()
+
+
 def _sampled_check(g, wl, wts, x, tenant, mot, G, out, n_sample=32, layer_inputs=None):
     """Routing/dispatch of the last layer call in full, layer outputs on sampled tokens."""
     ws = B.moe_get_workspace(g.ctx)
