@@ -67,13 +67,14 @@ int alloc_workspace(moe_ctx* c)
     }
     A(&w.xn, (T + kTileRows) * H);
     A(&w.x_stage, (T + kTileRows) * H); A(&w.tenant_stage, T); A(&w.out_stage, T * H);
-    A(&w.status, 1); A(&w.stats, 4);
+    A(&w.status, 1); A(&w.stats, 4); A(&w.dispatch_done, 1);
     if (e != cudaSuccess) {
         snprintf(c->errbuf, sizeof(c->errbuf), "workspace allocation: %s", cudaGetErrorString(e));
         return MOE_ERR_ALLOC;
     }
     cudaMemset(w.status, 0, sizeof(int32_t));
     cudaMemset(w.stats, 0, 4 * sizeof(int32_t));
+    cudaMemset(w.dispatch_done, 0, sizeof(int32_t));
     cudaMemset(w.plan_counts, 0, 8 * sizeof(int32_t));
     return MOE_OK;
 }
@@ -84,7 +85,7 @@ void free_workspace(moe_ctx* c)
     void* ptrs[] = {w.topk_idx, w.topk_w, w.shared_gate, w.tie_flag, w.perm, w.inv_perm, w.tenant_expert_count,
                     w.expert_off, w.group_off, w.block_cnt, w.bin_off, w.tok_block_cnt, w.model_tok_off, w.tok_perm,
                     w.tok_inv, w.tiles, w.stiles, w.plan_counts, w.units1, w.units2, w.x_perm, w.xs_perm, w.h, w.hs,
-                    w.y_perm, w.y_shared, w.xn, w.x_stage, w.tenant_stage, w.out_stage, w.status, w.stats};
+                    w.y_perm, w.y_shared, w.xn, w.x_stage, w.tenant_stage, w.out_stage, w.status, w.stats, w.dispatch_done};
     for (void* p : ptrs) if (p) cudaFree(p);
     w = Workspace();
 }

@@ -31,25 +31,6 @@ __device__ __forceinline__ int row_bin(const BinMap& bm, int tenant, int expert,
     return bm.bin_base[m] + expert * bm.tenants_in_model[m] + bm.tenant_local[tenant];
 }
 
-// D1: each block counts the rows of its chunk per bin.  One warp per block.
-__global__ void __launch_bounds__(32)
-dispatch_hist_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ tenant_id, int R, int k,
-                     BinMap bm, int nbins, int32_t* __restrict__ block_cnt, int32_t* __restrict__ status)
-{
-    extern __shared__ int32_t s_cnt[];
-    for (int b = threadIdx.x; b < nbins; b += 32) s_cnt[b] = 0;
-    __syncwarp();
-    const int r0 = blockIdx.x * kDispatchChunk;
-    const int r1 = min(R, r0 + kDispatchChunk);
-    for (int r = r0 + threadIdx.x; r < r1; r += 32) {
-        const int bin = row_bin(bm, tenant_id[r / k], topk_idx[r], status);
-        atomicAdd(&s_cnt[bin], 1);      // counts only: the result does not depend on the order
-    }
-    __syncwarp();
-    int32_t* dst = block_cnt + (size_t)blockIdx.x * nbins;
-    for (int b = threadIdx.x; b < nbins; b += 32) dst[b] = s_cnt[b];
-}
-
 // Block-wide: exclusive scan of the per-bin totals in s_tot (in key order), then the offset tables
 // the caller sees and the invocation statistics.  s_tot holds the offsets afterwards.
 __device__ void scan_and_tables(int32_t* s_tot, int32_t* s_part /* [33] */, int32_t* s_count /* [2] */,
@@ -103,35 +84,73 @@ __device__ void scan_and_tables(int32_t* s_tot, int32_t* s_part /* [33] */, int3
     if (tid < 2) stats[tid] = s_count[tid];
 }
 
-// D2: one block.  Totals per bin, exclusive scan in key order, per-block bases, and the
-// offset tables the caller sees.
-__global__ void __launch_bounds__(1024)
-dispatch_scan_kernel(int nblk, int nbins, int R, int E, int M, int G, int n_tenants, BinMap bm,
-                     int32_t* __restrict__ block_cnt, int32_t* __restrict__ bin_off,
-                     int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
-                     int32_t* __restrict__ group_off, int32_t* __restrict__ stats, int do_plan, PlanArgs pa)
+// D1 (large batches): every block ranks the rows of its chunk.  One warp walks the chunk in row order; rows
+// that share a bin inside one step are ranked by lane order (= row order), so the rank of a row inside
+// (block, bin) does not depend on timing.  The pair (bin, rank in block) is parked in inv_perm[r] for D2.
+// The block that finishes last turns the per-block counts into offsets: totals per bin, exclusive scan in key
+// order, per-block bases, the offset tables the caller sees, and (optionally) the expert work plan.
+constexpr int kCountThreads = 512;
+
+__global__ void __launch_bounds__(kCountThreads)
+dispatch_count_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ tenant_id, int nblk, int nbins,
+                      int R, int k, int E, int M, int G, int n_tenants, BinMap bm, int32_t* __restrict__ block_cnt,
+                      int32_t* __restrict__ bin_off, int32_t* __restrict__ inv_perm,
+                      int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
+                      int32_t* __restrict__ group_off, int32_t* __restrict__ stats, int32_t* __restrict__ status,
+                      int32_t* __restrict__ done_counter, int do_plan, PlanArgs pa)
 {
-    extern __shared__ int32_t s_tot[];       // [nbins] totals, then exclusive offsets; then the plan's scratch
+    extern __shared__ int32_t s_tot[];       // [nbins] counts of this block; in the last block: totals, then offsets,
+                                             // followed by the plan's scratch
     __shared__ int32_t s_part[33];
     __shared__ int32_t s_count[2];
+    __shared__ int s_last;
     const int tid = threadIdx.x, nth = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nth >> 5;
-    // totals per bin; block_cnt becomes the exclusive prefix over blocks.  One warp per bin: the lanes
-    // take the blocks 32 at a time and scan them with shuffles.
-    for (int b = warp; b < nbins; b += nw) {
-        int run = 0;
-        for (int blk0 = 0; blk0 < nblk; blk0 += 32) {
-            const int blk = blk0 + lane;
-            const int c = blk < nblk ? block_cnt[(size_t)blk * nbins + b] : 0;
-            int incl = c;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int v = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += v;
-            }
-            if (blk < nblk) block_cnt[(size_t)blk * nbins + b] = run + incl - c;
-            run += __shfl_sync(0xffffffffu, incl, 31);
+    for (int b = tid; b < nbins; b += nth) s_tot[b] = 0;
+    __syncthreads();
+    if (warp == 0) {
+        const int r0 = blockIdx.x * kDispatchChunk;
+        const int r1 = min(R, r0 + kDispatchChunk);
+        for (int rr = r0; rr < r1; rr += 32) {
+            const int r = rr + lane;
+            const bool live = r < r1;
+            int bin = -1 - lane;                 // distinct dummy keys for idle lanes
+            if (live) bin = row_bin(bm, tenant_id[r / k], topk_idx[r], status);
+            const unsigned peers = __match_any_sync(0xffffffffu, bin);
+            const int leader = __ffs(peers) - 1;
+            const int rank = __popc(peers & ((1u << lane) - 1u));
+            int start = 0;
+            if (live && lane == leader) { start = s_tot[bin]; s_tot[bin] = start + __popc(peers); }
+            start = __shfl_sync(0xffffffffu, start, leader);
+            if (live) inv_perm[r] = bin | ((start + rank) << 16);      // bin < 8192, rank < kDispatchChunk
+            __syncwarp();
         }
-        if (lane == 0) s_tot[b] = run;
+    }
+    __syncthreads();
+    int32_t* mine = block_cnt + (size_t)blockIdx.x * nbins;
+    for (int b = tid; b < nbins; b += nth) mine[b] = s_tot[b];
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(done_counter, 1) == nblk - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (tid == 0) *done_counter = 0;             // ready for the next call on this stream
+    // totals per bin; block_cnt becomes the exclusive prefix over blocks.  One thread per bin (neighbouring
+    // threads read neighbouring counters); the counts of 16 blocks are fetched before any is replaced, so the
+    // loads of a round are in flight together.
+    for (int b = tid; b < nbins; b += nth) {
+        int run = 0;
+        for (int blk0 = 0; blk0 < nblk; blk0 += 16) {
+            int cnt[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) cnt[j] = blk0 + j < nblk ? __ldcg(block_cnt + (size_t)(blk0 + j) * nbins + b) : 0;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                if (blk0 + j < nblk) block_cnt[(size_t)(blk0 + j) * nbins + b] = run;
+                run += cnt[j];
+            }
+        }
+        s_tot[b] = run;
     }
     __syncthreads();
     scan_and_tables(s_tot, s_part, s_count, nbins, R, E, M, G, n_tenants, bm, bin_off, tenant_expert_count,
@@ -139,6 +158,34 @@ dispatch_scan_kernel(int nblk, int nbins, int R, int E, int M, int G, int n_tena
     if (do_plan) {
         __syncthreads();
         plan_body(expert_off, pa, s_tot + nbins, s_part);
+    }
+}
+
+// D2 (large batches): position of every row = offset of its bin + rows of that bin in earlier blocks + rank in
+// its block; writes perm / inv_perm and, with GATHER, copies the token's row to its place in x_perm (one warp
+// per row, 16-byte vectors).
+template <bool GATHER>
+__global__ void __launch_bounds__(256)
+dispatch_place_kernel(int R, int k, int nbins, const int32_t* __restrict__ block_cnt, const int32_t* __restrict__ bin_off,
+                      int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, const bf16* __restrict__ x,
+                      bf16* __restrict__ x_perm, int H)
+{
+    const int gtid = blockIdx.x * blockDim.x + threadIdx.x;
+    const int r = GATHER ? gtid >> 5 : gtid;
+    if (r >= R) return;
+    const int lane = threadIdx.x & 31;
+    const int packed = inv_perm[r];
+    const int bin = packed & 0xffff, lrank = packed >> 16;
+    const int pos = bin_off[bin] + block_cnt[(size_t)(r / kDispatchChunk) * nbins + bin] + lrank;
+    if (GATHER) {
+        __syncwarp();                            // every lane has read the parked value before lane 0 replaces it
+        if (lane == 0) { perm[pos] = r; inv_perm[r] = pos; }
+        const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)(r / k) * H);
+        uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)pos * H);
+        for (int v = lane; v < (H >> 3); v += 32) dst[v] = src[v];
+    } else {
+        perm[pos] = r;
+        inv_perm[r] = pos;
     }
 }
 
@@ -200,40 +247,6 @@ dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
             uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)pos * H);
             for (int v = lane; v < (H >> 3); v += 32) dst[v] = src[v];
         }
-    }
-}
-
-// D3: stable rank of every row inside its bin.  One warp per block walks its chunk in row
-// order; rows that share a bin inside one step are ranked by lane order (= row order).
-__global__ void __launch_bounds__(32)
-dispatch_rank_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ tenant_id, int R, int k,
-                     BinMap bm, int nbins, const int32_t* __restrict__ block_cnt, const int32_t* __restrict__ bin_off,
-                     int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, int32_t* __restrict__ status)
-{
-    extern __shared__ int32_t s_next[];      // next free position of each bin for this block
-    const int lane = threadIdx.x;
-    const int32_t* base = block_cnt + (size_t)blockIdx.x * nbins;
-    for (int b = lane; b < nbins; b += 32) s_next[b] = bin_off[b] + base[b];
-    __syncwarp();
-    const int r0 = blockIdx.x * kDispatchChunk;
-    const int r1 = min(R, r0 + kDispatchChunk);
-    for (int rr = r0; rr < r1; rr += 32) {
-        const int r = rr + lane;
-        const bool live = r < r1;
-        int bin = -1 - lane;                 // distinct dummy keys for idle lanes
-        if (live) bin = row_bin(bm, tenant_id[r / k], topk_idx[r], status);
-        const unsigned peers = __match_any_sync(0xffffffffu, bin);
-        const int leader = __ffs(peers) - 1;
-        const int rank = __popc(peers & ((1u << lane) - 1u));
-        int start = 0;
-        if (live && lane == leader) { start = s_next[bin]; s_next[bin] = start + __popc(peers); }
-        start = __shfl_sync(0xffffffffu, start, leader);
-        if (live) {
-            const int pos = start + rank;
-            perm[pos] = r;
-            inv_perm[r] = pos;
-        }
-        __syncwarp();
     }
 }
 
@@ -376,19 +389,21 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
     memset(&pa, 0, sizeof(pa));
     size_t plan_ints = 0;
     if (do_plan) { pa = make_plan_args(c, T, G, plan_shared); plan_ints = plan_smem_ints(c, G); }
-    dispatch_hist_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, c->ws.block_cnt, c->ws.status);
-    dispatch_scan_kernel<<<1, 1024, smem + plan_ints * sizeof(int32_t), st>>>(
-        nblk, nbins, R, g.n_experts, g.n_models, G, g.n_tenants, bm, c->ws.block_cnt, c->ws.bin_off,
-        tenant_expert_count, expert_off, group_off, c->ws.stats, do_plan ? 1 : 0, pa);
+    const size_t smem_count = smem + plan_ints * sizeof(int32_t);
+    if (smem_count > 48 * 1024)
+        cudaFuncSetAttribute(dispatch_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_count);
+    dispatch_count_kernel<<<nblk, kCountThreads, smem_count, st>>>(
+        topk_idx, tenant_id, nblk, nbins, R, k, g.n_experts, g.n_models, G, g.n_tenants, bm, c->ws.block_cnt, c->ws.bin_off,
+        inv_perm, tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, c->ws.dispatch_done,
+        do_plan ? 1 : 0, pa);
     if (plan_done) *plan_done = do_plan;
-    dispatch_rank_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, c->ws.block_cnt, c->ws.bin_off,
-                                                 perm, inv_perm, c->ws.status);
-    c->launches += 3;
-    if (x_perm) {
-        const int blocks = (R * 32 + 255) / 256;
-        gather_rows_kernel<<<blocks, 256, 0, st>>>(x, perm, R, k, g.hidden, x_perm);
-        c->launches += 1;
-    }
+    if (x_perm)
+        dispatch_place_kernel<true><<<(R * 32 + 255) / 256, 256, 0, st>>>(R, k, nbins, c->ws.block_cnt, c->ws.bin_off, perm,
+                                                                          inv_perm, x, x_perm, g.hidden);
+    else
+        dispatch_place_kernel<false><<<(R + 255) / 256, 256, 0, st>>>(R, k, nbins, c->ws.block_cnt, c->ws.bin_off, perm,
+                                                                      inv_perm, nullptr, nullptr, g.hidden);
+    c->launches += 2;
     return cudaGetLastError();
 }
 
@@ -520,10 +535,12 @@ extern "C" int moe_dispatch_noalloc(const int32_t* topk_idx, const int32_t* tena
     bm.n_tenants = n_tenants;
     bm.E = E;
     const size_t smem = (size_t)nbins * sizeof(int32_t);
-    dispatch_hist_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, s + o_blk, status);
-    dispatch_scan_kernel<<<1, 1024, smem, st>>>(nblk, nbins, R, E, M, G, n_tenants, bm, s + o_blk, s + o_binoff,
-                                                tenant_expert_count, expert_off, group_off, s + o_stats, 0, PlanArgs());
-    dispatch_rank_kernel<<<nblk, 32, smem, st>>>(topk_idx, tenant_id, R, k, bm, nbins, s + o_blk, s + o_binoff, perm,
-                                                 inv_perm, status);
+    // stats[2] (cleared by the set-up kernel) counts the blocks that have finished
+    dispatch_count_kernel<<<nblk, kCountThreads, smem, st>>>(topk_idx, tenant_id, nblk, nbins, R, k, E, M, G, n_tenants, bm,
+                                                             s + o_blk, s + o_binoff, inv_perm, tenant_expert_count,
+                                                             expert_off, group_off, s + o_stats, status, s + o_stats + 2, 0,
+                                                             PlanArgs());
+    dispatch_place_kernel<false><<<(R + 255) / 256, 256, 0, st>>>(R, k, nbins, s + o_blk, s + o_binoff, perm, inv_perm,
+                                                                  nullptr, nullptr, 0);
     return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

@@ -53,8 +53,9 @@ constexpr int kOutGroupBytes = kOutStageBytes / 2;
 constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + kBarBytes + kOutStageBytes;
 static_assert(8 * kNumBars <= kBarBytes, "barrier area too small");
 constexpr int kEpiWarps = 8;                   // two warps per TMEM lane quarter, alternating 16-column chunks
-constexpr int kSchedWarp = 2 + kEpiWarps;      // warp 0: TMA, warp 1: MMA + TMEM, warps 2..9: epilogue, warp 10: scheduler
-constexpr int kThreads = 32 * (kSchedWarp + 1);
+constexpr int kSchedWarp = 2 + kEpiWarps;      // warp 0: TMA (weights), warp 1: MMA + TMEM, warps 2..9: epilogue, warp 10: scheduler,
+constexpr int kTokWarp = kSchedWarp + 1;       // warp 11: TMA (tokens)
+constexpr int kThreads = 32 * (kTokWarp + 1);
 constexpr int kClaimAhead = 8;                 // the next unit is claimed this many K steps before the current one is loaded
 constexpr uint32_t kTmemCols = 512;            // 2 accumulator buffers x 256 columns
 
@@ -90,8 +91,8 @@ constexpr int kTcMaxModels = 8;
 struct GemmMaps {
     CUtensorMap a_routed;                  // gate/up: 3-D (K, {gate,up}, S*I); down: 2-D (K, S*H)
     CUtensorMap a_shared[kTcMaxModels];    // same for the shared expert of each model
-    CUtensorMap b_routed128, b_routed16;   // activations of the routed units, boxes of 128 / 16 rows
-    CUtensorMap b_shared128, b_shared16;
+    CUtensorMap b_routed[4];               // activations of the routed units, boxes of 128 / 64 / 32 / 16 rows
+    CUtensorMap b_shared[4];
 };
 
 __device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z,
@@ -261,11 +262,11 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(bar_tfull + 8 * b, 1); mbar_init(bar_tempty + 8 * b, (PAIR ? 2 : 1) * kEpiWarps); }
-        // unit queue: filled by the scheduler lane (of the leader CTA); drained by the producer lane, the MMA lane
-        // and the epilogue warps of this CTA and, in pair mode, by the peer's producer lane and epilogue warps
+        // unit queue: filled by the scheduler lane (of the leader CTA); drained by the two producer lanes, the MMA lane
+        // and the epilogue warps of this CTA and, in pair mode, by the peer's producer lanes and epilogue warps
         for (int q = 0; q < kQueue; ++q) {
             mbar_init(bar_qfull + 8 * q, 1);
-            mbar_init(bar_qempty + 8 * q, 2 + kEpiWarps + (PAIR ? 1 + kEpiWarps : 0));
+            mbar_init(bar_qempty + 8 * q, 3 + kEpiWarps + (PAIR ? 2 + kEpiWarps : 0));
         }
         mbar_init(bar_sched, 1);
         s_abort = 0;
@@ -296,8 +297,12 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     // queues behind the tile requests and was measured to cost thousands of cycles per unit.
     const uint32_t qempty_leader = PAIR ? map_to_cta(bar_qempty, 0) : bar_qempty;
 
-    if (warp == 0) {
-        // ---------------- TMA producer (one lane); in single mode also the scheduler ----------------
+    if (warp == 0 || warp == kTokWarp) {
+        // ---------------- TMA producers: one lane of warp 0 posts the byte count of a stage and loads the weight tile,
+        // one lane of another warp loads the token tiles.  A tile load costs its issuing lane about 140 cycles and
+        // the barrier handshake of a stage about 290, whatever the tile's size; in one lane that was more per K step
+        // than the MMAs of a full tile take.  Lanes of one warp would not help: their branches run one after the other.
+        const bool wrole = warp == 0;
         if (lane == 0) {
             uint32_t stage = 0, phase = 0, q = 0, qphase = 0;
             uint32_t armed = 0, armed_phase = 0;
@@ -315,42 +320,52 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 const int claim_ks = ui.ksteps > kClaimAhead ? ui.ksteps - kClaimAhead : 0;
                 const CUtensorMap* ma = ui.amap < 0 ? &maps.a_routed : &maps.a_shared[ui.amap];
                 const bool bshared = ui.shared || ui.direct;
-                const CUtensorMap* mb128 = bshared ? &maps.b_shared128 : &maps.b_routed128;
-                const CUtensorMap* mb16 = bshared ? &maps.b_shared16 : &maps.b_routed16;
+                const CUtensorMap* mb = bshared ? maps.b_shared : maps.b_routed;
                 const int brow0 = ui.direct ? 0 : ui.b_row0;
                 const int my_rows = PAIR ? (ui.npad >> 1) : ui.npad;          // token rows this CTA loads
                 const int my_row0 = brow0 + (PAIR ? (int)rank * my_rows : 0);
                 const int my_rows1 = ui.npad1 >> 1;                           // same for the second accumulator
                 const int my_row1 = brow0 + 256 + (int)rank * my_rows1;
                 for (int ks = 0; ks < ui.ksteps; ++ks) {
-                    if (leader && ks == claim_ks) mbar_arrive(bar_sched);      // time to claim the next unit
+                    if (wrole && leader && ks == claim_ks) mbar_arrive(bar_sched);      // time to claim the next unit
                     if (stage % group == 0 &&
                         !mbar_wait(bar_empty + 8 * (stage / group), phase ^ 1, &s_abort, p.status)) { ok = false; break; }
                     const uint32_t sa = smem_base + stage * stage_bytes, sb = sa + kABytes;
                     const uint32_t full = bar_full + 8 * stage;
-                    if (leader) mbar_expect_tx(full, (PAIR ? 2u : 1u) * (uint32_t)(kABytes + (my_rows + my_rows1) * kBK * 2));
-                    armed |= 1u << stage;
-                    armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
-                    if (PAIR) {
-                        if (MODE == 0) tma_load_3d_pair(sa, ma, full, ks * kBK, 0, ui.a_row, pol_w);
-                        else tma_load_2d_pair(sa, ma, full, ks * kBK, ui.a_row, pol_w);
-                        int j = 0;
-                        for (; j + 128 <= my_rows; j += 128) tma_load_2d_pair(sb + j * kBK * 2, mb128, full, ks * kBK, my_row0 + j, pol_x);
-                        for (; j < my_rows; j += 16) tma_load_2d_pair(sb + j * kBK * 2, mb16, full, ks * kBK, my_row0 + j, pol_x);
-                        const uint32_t sb1 = sb + kBBytes;
-                        for (j = 0; j + 128 <= my_rows1; j += 128) tma_load_2d_pair(sb1 + j * kBK * 2, mb128, full, ks * kBK, my_row1 + j, pol_x);
-                        for (; j < my_rows1; j += 16) tma_load_2d_pair(sb1 + j * kBK * 2, mb16, full, ks * kBK, my_row1 + j, pol_x);
+                    if (wrole) {
+                        // the token lane's bytes may be counted before this is posted: the phase still cannot complete
+                        // without this arrival
+                        if (leader) mbar_expect_tx(full, (PAIR ? 2u : 1u) * (uint32_t)(kABytes + (my_rows + my_rows1) * kBK * 2));
+                        armed |= 1u << stage;
+                        armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
+                        if (PAIR) {
+                            if (MODE == 0) tma_load_3d_pair(sa, ma, full, ks * kBK, 0, ui.a_row, pol_w);
+                            else tma_load_2d_pair(sa, ma, full, ks * kBK, ui.a_row, pol_w);
+                        } else {
+                            if (MODE == 0) tma_load_3d_hint(sa, ma, full, ks * kBK, 0, ui.a_row, pol_w);
+                            else tma_load_2d_hint(sa, ma, full, ks * kBK, ui.a_row, pol_w);
+                        }
                     } else {
-                        if (MODE == 0) tma_load_3d_hint(sa, ma, full, ks * kBK, 0, ui.a_row, pol_w);
-                        else tma_load_2d_hint(sa, ma, full, ks * kBK, ui.a_row, pol_w);
-                        int j = 0;
-                        for (; j + 128 <= my_rows; j += 128) tma_load_2d_hint(sb + j * kBK * 2, mb128, full, ks * kBK, my_row0 + j, pol_x);
-                        for (; j < my_rows; j += 16) tma_load_2d_hint(sb + j * kBK * 2, mb16, full, ks * kBK, my_row0 + j, pol_x);
+                        // token rows in boxes of 128 / 64 / 32 / 16 rows
+                        for (int acc = 0; acc < 2; ++acc) {
+                            const int rows = acc ? my_rows1 : my_rows, r0 = acc ? my_row1 : my_row0;
+                            const uint32_t dst = sb + acc * kBBytes;
+                            int j = 0;
+#pragma unroll
+                            for (int bx = 0; bx < 4; ++bx) {
+                                const int n = 128 >> bx;
+                                while (j + n <= rows) {
+                                    if (PAIR) tma_load_2d_pair(dst + j * kBK * 2, mb + bx, full, ks * kBK, r0 + j, pol_x);
+                                    else tma_load_2d_hint(dst + j * kBK * 2, mb + bx, full, ks * kBK, r0 + j, pol_x);
+                                    j += n;
+                                }
+                            }
+                        }
                     }
                     if (++stage == n_stages) { stage = 0; phase ^= 1; }
                 }
             }
-            if (!ok && leader) {
+            if (!ok && leader && wrole) {
                 // gave up: let the copies already in flight land before the block exits
                 for (int s = 0; s < kMaxStages; ++s)
                     if (armed & (1u << s)) mbar_wait(bar_full + 8 * s, (armed_phase >> s) & 1u, &s_abort, p.status);
@@ -816,12 +831,18 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     // activation maps are rebuilt per call: their addresses and row counts are the call's
     GemmMaps& m1 = lm.m1;
     bool ok = true;
-    if (!direct) ok = make_map(&m1.b_routed128, x_perm, R, H, 128, false) && make_map(&m1.b_routed16, x_perm, R, H, 16, false);
+    auto make_b = [](CUtensorMap* m, const void* base, uint64_t rows, uint64_t k, bool fp16) {
+        bool good = true;
+        for (int bx = 0; bx < 4; ++bx) good = good && make_map(m + bx, base, rows, k, 128u >> bx, fp16);
+        return good;
+    };
+    auto copy_b = [](CUtensorMap* dst, const CUtensorMap* src) { for (int bx = 0; bx < 4; ++bx) dst[bx] = src[bx]; };
+    if (!direct) ok = make_b(m1.b_routed, x_perm, R, H, false);
     if (shared || direct) {
-        ok = ok && make_map(&m1.b_shared128, x_or_xs, T, H, 128, false) && make_map(&m1.b_shared16, x_or_xs, T, H, 16, false);
-        if (direct) { m1.b_routed128 = m1.b_shared128; m1.b_routed16 = m1.b_shared16; }
+        ok = ok && make_b(m1.b_shared, x_or_xs, T, H, false);
+        if (direct) copy_b(m1.b_routed, m1.b_shared);
     } else {
-        m1.b_shared128 = m1.b_routed128; m1.b_shared16 = m1.b_routed16;
+        copy_b(m1.b_shared, m1.b_routed);
     }
     if (!ok) return cudaErrorInvalidValue;
 
@@ -845,9 +866,9 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     stage_mark(c, st, kEvGateUp);
 
     GemmMaps& m2 = lm.m2;
-    ok = make_map(&m2.b_routed128, c->ws.h, R, I, 128, false) && make_map(&m2.b_routed16, c->ws.h, R, I, 16, false);
-    if (shared) ok = ok && make_map(&m2.b_shared128, c->ws.hs, T, Is, 128, true) && make_map(&m2.b_shared16, c->ws.hs, T, Is, 16, true);
-    else { m2.b_shared128 = m2.b_routed128; m2.b_shared16 = m2.b_routed16; }
+    ok = make_b(m2.b_routed, c->ws.h, R, I, false);
+    if (shared) ok = ok && make_b(m2.b_shared, c->ws.hs, T, Is, true);
+    else copy_b(m2.b_shared, m2.b_routed);
     if (!ok) return cudaErrorInvalidValue;
     GemmParams p2 = p1;
     p2.units = c->ws.units2; p2.n_units = c->ws.plan_counts + 3; p2.counter = c->ws.plan_counts + 5;

@@ -69,6 +69,7 @@ struct Workspace {
     // dispatch scratch
     int32_t* block_cnt = nullptr;  // [nblk, nbins]
     int32_t* bin_off = nullptr;    // [nbins+1]
+    int32_t* dispatch_done = nullptr;  // [1] blocks of the counting kernel that have finished (zero between calls)
     int32_t* tok_block_cnt = nullptr;  // [nblk_tok, M]
     int32_t* model_tok_off = nullptr;  // [M+1]
     int32_t* tok_perm = nullptr;   // [T] tokens sorted by (model, token)

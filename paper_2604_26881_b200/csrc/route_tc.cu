@@ -26,7 +26,7 @@ constexpr int kRMaxGateN = 64;                         // 16 columns per model f
 constexpr int kRGBytes = kRMaxGateN * kRBK * 2;        // 8 KB
 constexpr int kRTileBudget = 192 * 1024;               // shared memory for the pipeline stages
 constexpr int kRSmemBytes = kRTileBudget + kRABytes /* a short token tile is read as 128 rows */ + 1024 + 512;
-constexpr int kRThreads = 192;
+constexpr int kRThreads = 256;                         // warp 0: TMA (tokens), 1: MMA, 2..5: epilogue, 6 / 7: TMA (routers / gates)
 constexpr int kRMaxE = 64;                             // logits one thread keeps in registers
 
 struct RouteParams {
@@ -35,7 +35,10 @@ struct RouteParams {
     int T, H, E, Epad, k, n_tenants, n_models;
     const int32_t* model_of_tenant;
     const ModelWeights* models;
-    int gate_mma;                  // 1: the gate logit is column m*16 of a second accumulator
+    int gate_mma;                  // 1: the gate logit of model m is accumulator column gate_col + m*16
+    int gate_col;                  // first gate column: right after the router columns when one MMA covers both
+    int gate_merged;               // 1: router rows and gate rows are one N operand (n_models * (Epad + 16) <= 256)
+    int group;                     // stages handed back to the producer per commit (divides n_stages)
     int a_bytes, b_bytes, stage_bytes, n_stages;   // pipeline geometry: small batches take more, smaller stages
     int32_t* topk_idx;
     float* topk_w;
@@ -100,23 +103,27 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
 
-    if (warp == 0) {
-        // three producer lanes (tokens / routers / gates) so that the TMA instructions of one stage are
-        // issued side by side; lane 0 also posts the byte count
-        if (lane < 3 && (lane < 2 || p.gate_mma)) {
+    if (warp == 0 || warp >= 6) {
+        // three producer lanes (tokens / routers / gates) in three warps, so that the TMA instructions of one stage
+        // are issued side by side (a tile load costs its issuing lane about 140 cycles, the barrier handshake about
+        // 290; lanes of one warp would run their branches one after the other); the token lane also posts the
+        // byte count
+        const int role = warp == 0 ? 0 : warp - 5;
+        if (lane == 0 && (role < 2 || p.gate_mma)) {
             uint32_t stage = 0, phase = 0, armed = 0, armed_phase = 0;
             bool ok = true;
             const uint64_t keep = l2_evict_last();      // router weights and tokens are read again soon
             for (int ks = 0; ks < ksteps; ++ks) {
-                if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, &s_abort, p.status)) { ok = false; break; }
+                if (stage % p.group == 0 &&
+                    !mbar_wait(bar_empty + 8 * (stage / p.group), phase ^ 1, &s_abort, p.status)) { ok = false; break; }
                 const uint32_t sa = smem_base + stage * p.stage_bytes, sb = sa + p.a_bytes;
                 const uint32_t full = bar_full + 8 * stage;
                 armed |= 1u << stage;
                 armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
-                if (lane == 0) {
+                if (role == 0) {
                     mbar_expect_tx(full, p.a_bytes + N * kRBK * 2 + (p.gate_mma ? p.n_models * 16 * kRBK * 2 : 0));
                     tma_load_2d_hint(sa, &maps.x, full, ks * kRBK, t0, keep);
-                } else if (lane == 1) {
+                } else if (role == 1) {
                     for (int m = 0; m < p.n_models; ++m)
                         tma_load_2d_hint(sb + m * p.Epad * kRBK * 2, &maps.r[m], full, ks * kRBK, 0, keep);
                 } else {
@@ -125,7 +132,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                 }
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
             }
-            if (!ok)
+            if (!ok && role == 0)
                 for (int s = 0; s < kRStages; ++s)
                     if (armed & (1u << s)) mbar_wait(bar_full + 8 * s, (armed_phase >> s) & 1u, &s_abort, p.status);
         }
@@ -133,7 +140,10 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
     } else if (warp == 1) {
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((128u >> 4) << 24);
+            // a tcgen05.mma costs its issuing lane about 100 cycles whatever its width, a commit about 200: the gate
+            // rows ride in the router's MMA when they fit, and stages go back to the producer in groups
+            const int n_main = p.gate_merged ? N + p.n_models * 16 : N;
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_main >> 3) << 17) | ((128u >> 4) << 24);
             const uint32_t idesc_g = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_models * 16 >> 3) << 17) | ((128u >> 4) << 24);
             bool ok = true;
             for (int ks = 0; ks < ksteps; ++ks) {
@@ -145,15 +155,15 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                 for (int kk = 0; kk < kRBK / 16; ++kk) {
                     const uint64_t adv = (uint64_t)(kk * 32 >> 4);
                     umma_bf16(tmem_base, da + adv, db + adv, idesc, (ks | kk) ? 1u : 0u);
-                    if (p.gate_mma) umma_bf16(tmem_base + kRMaxN, da + adv, dg + adv, idesc_g, (ks | kk) ? 1u : 0u);
+                    if (p.gate_mma && !p.gate_merged) umma_bf16(tmem_base + p.gate_col, da + adv, dg + adv, idesc_g, (ks | kk) ? 1u : 0u);
                 }
-                umma_commit(bar_empty + 8 * stage);
+                if (stage % p.group == p.group - 1) umma_commit(bar_empty + 8 * (stage / p.group));
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
             }
             if (ok) umma_commit(bar_tfull);
         }
         __syncwarp();
-    } else {
+    } else if (warp < 6) {
         // ---- epilogue warps: thread <-> token (TMEM lane) ----
         const int quarter = warp & 3;
         const int t = t0 + quarter * 32 + lane;
@@ -213,7 +223,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
             if (p.gate_mma && p.shared_gate) {
                 for (int m = 0; m < p.n_models; ++m) {
                     uint32_t r[16];
-                    tmem_ld16(taddr + kRMaxN + m * 16, r);
+                    tmem_ld16(taddr + p.gate_col + m * 16, r);
                     tmem_ld_wait();
                     if (m == model && valid && p.models[m].shared_gate_w) gate = 1.f / (1.f + expf(-__uint_as_float(r[0])));
                 }
@@ -362,6 +372,11 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     p.stage_bytes = p.a_bytes + p.b_bytes + (p.gate_mma ? ((M * 16 * kRBK * 2 + 1023) & ~1023) : 0);
     p.n_stages = kRTileBudget / p.stage_bytes;
     if (p.n_stages > kRMaxStages) p.n_stages = kRMaxStages;
+    p.group = p.n_stages >= 8 ? 4 : (p.n_stages >= 4 ? 2 : 1);
+    p.n_stages -= p.n_stages % p.group;
+    // the gate rows follow the router rows in shared memory (b_bytes has no padding: Epad is a multiple of 16)
+    p.gate_merged = (p.gate_mma && M * (epad + 16) <= kRMaxN && p.b_bytes == M * epad * kRBK * 2) ? 1 : 0;
+    p.gate_col = p.gate_merged ? M * epad : kRMaxN;
     route_tc_kernel<<<(T + kRTokens - 1) / kRTokens, kRThreads, kRSmemBytes, st>>>(p, mp);
     c->launches += 1;
     return cudaGetLastError();
