@@ -43,8 +43,9 @@ int alloc_workspace(moe_ctx* c)
     c->max_tiles = div_up((int)R, kTileRows) + (int)ME;
     c->max_stiles = div_up((int)T, kTileRows) + g.n_models;
     const int nblk1 = g.inter / 64, nblk2 = div_up(g.hidden, 128), snblk1 = g.shared_inter / 64;
-    c->max_units1 = c->max_tiles * nblk1 + c->max_stiles * snblk1;
-    c->max_units2 = (c->max_tiles + c->max_stiles) * nblk2;
+    // (+256: the token-major plan splits up to half a round of units in two; its shared units are up to 4x narrower)
+    c->max_units1 = c->max_tiles * nblk1 + c->max_stiles * snblk1 + 256;
+    c->max_units2 = (c->max_tiles + 4 * c->max_stiles) * nblk2 + 256;
 
     cudaError_t e = cudaSuccess;
     auto A = [&](auto** p, size_t n) { if (e == cudaSuccess) e = dev_alloc(p, n); };
@@ -205,6 +206,7 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->route_path = MOE_PATH_AUTO;
     c->pair_mode_enabled = 1;
     c->wide_tiles_enabled = 1;
+    c->token_major_enabled = 1;
     c->timing = false;
     for (auto& e : c->ev) e = nullptr;
     c->errbuf[0] = 0;
@@ -327,7 +329,12 @@ int moe_set_option(moe_ctx* c, int option, int value)
         return MOE_OK;
     }
     if (option == MOE_OPT_PAIR_MODE) {
-        c->pair_mode_enabled = value ? 1 : 0;
+        if (value < 0 || value > 2) return MOE_ERR_SHAPE;
+        c->pair_mode_enabled = value;
+        return MOE_OK;
+    }
+    if (option == MOE_OPT_TOKEN_MAJOR) {
+        c->token_major_enabled = value ? 1 : 0;
         return MOE_OK;
     }
     if (option == MOE_OPT_WIDE_TILES) {

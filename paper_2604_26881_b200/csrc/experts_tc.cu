@@ -89,8 +89,8 @@ constexpr int kTcMaxModels = 8;
 
 // TMA descriptors in kernel-parameter space
 struct GemmMaps {
-    CUtensorMap a_routed;                  // gate/up: 3-D (K, {gate,up}, S*I); down: 2-D (K, S*H)
-    CUtensorMap a_shared[kTcMaxModels];    // same for the shared expert of each model
+    CUtensorMap a_routed[3];               // gate/up: 3-D (K, {gate,up}, S*I); down: 2-D (K, S*H); [1], [2]: boxes of a half
+    CUtensorMap a_shared[kTcMaxModels][3]; //   and a quarter of the weight rows (token-major shape); same for the shared experts
     CUtensorMap b_routed[4];               // activations of the routed units, boxes of 128 / 64 / 32 / 16 rows
     CUtensorMap b_shared[4];
 };
@@ -188,6 +188,8 @@ struct UnitInfo {
     int a_row, amap;              // first weight row of the tile; -1: routed map, m: shared map of model m
     int b_row0, nrows, npad, ksteps, shared, cb, model;
     int npad1;                    // wide unit: padded rows of the second accumulator (rows 256..), else 0
+    int width;                    // token-major shape: weight rows of the unit: 256, 128 or 64; a stage then holds 1, 2 or 4
+    int kb;                       //   slices of 64 K elements (always 32 KB of weights), so that narrow units stream as fast
     int direct;                   // routed gate/up unit in direct mode: B = all tokens
 };
 
@@ -198,12 +200,14 @@ struct __align__(16) QEntry {
     int colblock, shared, pad0, pad1;
 };
 
-template <int MODE, bool PAIR>
+template <int MODE, bool PAIR, bool SWAP>
 __device__ __forceinline__ UnitInfo unit_info(const GemmParams& p, const QEntry& e, uint32_t rank)
 {
     UnitInfo ui;
     ui.shared = e.shared;
-    ui.cb = PAIR ? 2 * e.colblock + (int)rank : e.colblock;
+    ui.cb = PAIR ? 2 * e.colblock + (int)rank : e.colblock;      // (token-major shape: in steps of 64 weight rows)
+    ui.width = SWAP ? e.pad0 : 0;
+    ui.kb = SWAP ? 256 / e.pad0 : 1;
     ui.model = e.tile_slot;
     ui.amap = ui.shared ? e.tile_slot : -1;
     ui.a_row = (ui.shared ? 0 : e.tile_slot * p.rows_per_slot) + ui.cb * p.cb_rows;
@@ -218,8 +222,8 @@ __device__ __forceinline__ UnitInfo unit_info(const GemmParams& p, const QEntry&
         ui.npad = (n0 + 31) & ~31;
         ui.npad1 = (e.nrows - n0 + 31) & ~31;
     }
-    else ui.npad = (e.nrows + 15) & ~15;
-    ui.ksteps = (ui.shared ? p.k_shared : p.k_routed) / kBK;
+    else ui.npad = (e.nrows + 15) & ~15;      // (token-major shape: rows of the token tile that are loaded)
+    ui.ksteps = (ui.shared ? p.k_shared : p.k_routed) / (kBK * ui.kb);
     return ui;
 }
 
@@ -228,22 +232,28 @@ __device__ __forceinline__ QEntry read_entry(const QEntry* q)
     const int4 a = *reinterpret_cast<const int4*>(q);
     const int2 b = *reinterpret_cast<const int2*>(&q->colblock);
     QEntry e;
-    e.u = a.x; e.tile_slot = a.y; e.b_row0 = a.z; e.nrows = a.w; e.colblock = b.x; e.shared = b.y; e.pad0 = e.pad1 = 0;
+    e.u = a.x; e.tile_slot = a.y; e.b_row0 = a.z; e.nrows = a.w; e.colblock = b.x; e.shared = b.y; e.pad0 = q->pad0; e.pad1 = 0;
     return e;
 }
 
 // MODE 0: gate/up + SwiGLU (output bf16 for routed units, fp16 for shared units)
 // MODE 1: down projection (output fp32)
-template <int MODE, bool PAIR>
+// SWAP (one CTA per unit only): the tokens are the M operand (one TMEM lane per token, up to 128) and up to 256
+// weight rows the N operand.  One MMA then covers twice the weight bytes of the other orientation, which is what
+// counts for short tiles: an MMA costs its issuing lane about 100 cycles however narrow it is, so with weights as M
+// a tile of a few tokens is bound by MMA issue, not by the weight stream.
+template <int MODE, bool PAIR, bool SWAP>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
 {
+    static_assert(!(PAIR && SWAP), "the token-major shape is a one-CTA shape");
+    constexpr uint32_t kWBytes = SWAP ? 2 * kABytes : kABytes;               // weight tile of one stage
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
     const uint32_t bars = smem_base + kRingBytes;                              // 8-byte barriers after the tiles
     const uint32_t bar_full = bars, bar_empty = bars + 8 * kMaxStages;
     const uint32_t bar_tfull = bars + 16 * kMaxStages, bar_tempty = bar_tfull + 16;
-    const uint32_t n_stages = (PAIR && p.wide) ? kWideStages : kMaxStages;
+    const uint32_t n_stages = ((PAIR && p.wide) || SWAP) ? kWideStages : kMaxStages;
     const uint32_t stage_bytes = kRingBytes / n_stages;
     // Stages are handed back to the producer in groups: a tcgen05.commit costs the issuing lane about as much
     // as two MMAs, so with four MMAs per stage one commit per stage would starve the tensor pipe.
@@ -316,9 +326,10 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 if (leader) mbar_arrive(bar_qempty + 8 * q); else mbar_arrive_cluster(qempty_leader + 8 * q);
                 if (++q == kQueue) { q = 0; qphase ^= 1; }
                 if (e.u < 0) break;
-                const UnitInfo ui = unit_info<MODE, PAIR>(p, e, rank);
+                const UnitInfo ui = unit_info<MODE, PAIR, SWAP>(p, e, rank);
                 const int claim_ks = ui.ksteps > kClaimAhead ? ui.ksteps - kClaimAhead : 0;
-                const CUtensorMap* ma = ui.amap < 0 ? &maps.a_routed : &maps.a_shared[ui.amap];
+                const int wsel = SWAP ? (ui.width == 256 ? 0 : (ui.width == 128 ? 1 : 2)) : 0;
+                const CUtensorMap* ma = ui.amap < 0 ? &maps.a_routed[wsel] : &maps.a_shared[ui.amap][wsel];
                 const bool bshared = ui.shared || ui.direct;
                 const CUtensorMap* mb = bshared ? maps.b_shared : maps.b_routed;
                 const int brow0 = ui.direct ? 0 : ui.b_row0;
@@ -330,33 +341,39 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     if (wrole && leader && ks == claim_ks) mbar_arrive(bar_sched);      // time to claim the next unit
                     if (stage % group == 0 &&
                         !mbar_wait(bar_empty + 8 * (stage / group), phase ^ 1, &s_abort, p.status)) { ok = false; break; }
-                    const uint32_t sa = smem_base + stage * stage_bytes, sb = sa + kABytes;
+                    const uint32_t sa = smem_base + stage * stage_bytes, sb = sa + kWBytes;
                     const uint32_t full = bar_full + 8 * stage;
                     if (wrole) {
                         // the token lane's bytes may be counted before this is posted: the phase still cannot complete
                         // without this arrival
-                        if (leader) mbar_expect_tx(full, (PAIR ? 2u : 1u) * (uint32_t)(kABytes + (my_rows + my_rows1) * kBK * 2));
+                        if (leader) mbar_expect_tx(full, (PAIR ? 2u : 1u) * (uint32_t)(kWBytes + ui.kb * (my_rows + my_rows1) * kBK * 2));
                         armed |= 1u << stage;
                         armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
                         if (PAIR) {
                             if (MODE == 0) tma_load_3d_pair(sa, ma, full, ks * kBK, 0, ui.a_row, pol_w);
                             else tma_load_2d_pair(sa, ma, full, ks * kBK, ui.a_row, pol_w);
                         } else {
-                            if (MODE == 0) tma_load_3d_hint(sa, ma, full, ks * kBK, 0, ui.a_row, pol_w);
-                            else tma_load_2d_hint(sa, ma, full, ks * kBK, ui.a_row, pol_w);
+                            // (token-major: kb slices of 64 K elements, each `width` rows high, one after the other)
+                            for (int a = 0; a < ui.kb; ++a) {
+                                const uint32_t dst = sa + (uint32_t)(a * ui.width) * kBK * 2;
+                                if (MODE == 0) tma_load_3d_hint(dst, ma, full, (ks * ui.kb + a) * kBK, 0, ui.a_row, pol_w);
+                                else tma_load_2d_hint(dst, ma, full, (ks * ui.kb + a) * kBK, ui.a_row, pol_w);
+                            }
                         }
                     } else {
                         // token rows in boxes of 128 / 64 / 32 / 16 rows
-                        for (int acc = 0; acc < 2; ++acc) {
-                            const int rows = acc ? my_rows1 : my_rows, r0 = acc ? my_row1 : my_row0;
-                            const uint32_t dst = sb + acc * kBBytes;
+                        for (int acc = 0; acc < (PAIR ? 2 : ui.kb); ++acc) {
+                            // pair shape: the two accumulators' tiles; token-major shape: the K slices of the stage
+                            const int rows = (PAIR && acc) ? my_rows1 : my_rows, r0 = (PAIR && acc) ? my_row1 : my_row0;
+                            const uint32_t dst = sb + (PAIR ? acc * kBBytes : acc * my_rows * kBK * 2);
+                            const int kx = (PAIR ? ks : ks * ui.kb + acc) * kBK;
                             int j = 0;
 #pragma unroll
                             for (int bx = 0; bx < 4; ++bx) {
                                 const int n = 128 >> bx;
                                 while (j + n <= rows) {
-                                    if (PAIR) tma_load_2d_pair(dst + j * kBK * 2, mb + bx, full, ks * kBK, r0 + j, pol_x);
-                                    else tma_load_2d_hint(dst + j * kBK * 2, mb + bx, full, ks * kBK, r0 + j, pol_x);
+                                    if (PAIR) tma_load_2d_pair(dst + j * kBK * 2, mb + bx, full, kx, r0 + j, pol_x);
+                                    else tma_load_2d_hint(dst + j * kBK * 2, mb + bx, full, kx, r0 + j, pol_x);
                                     j += n;
                                 }
                             }
@@ -383,10 +400,10 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 mbar_arrive(bar_qempty + 8 * q);
                 if (++q == kQueue) { q = 0; qphase ^= 1; }
                 if (e.u < 0) break;
-                const UnitInfo ui = unit_info<MODE, PAIR>(p, e, rank);
+                const UnitInfo ui = unit_info<MODE, PAIR, SWAP>(p, e, rank);
                 const uint32_t fmt = ui.shared ? p.idesc_fmt_shared : p.idesc_fmt_routed;
                 const uint32_t idesc_m = (1u << 4) | fmt | (((PAIR ? 256u : 128u) >> 4) << 24);
-                const uint32_t idesc = idesc_m | ((uint32_t)(ui.npad >> 3) << 17);
+                const uint32_t idesc = idesc_m | ((uint32_t)((SWAP ? ui.width : ui.npad) >> 3) << 17);
                 const uint32_t idesc1 = idesc_m | ((uint32_t)(ui.npad1 >> 3) << 17);
                 const bool wide = PAIR && ui.npad1 > 0;
                 // a wide unit takes both accumulator buffers, in the order the epilogue drains them
@@ -399,14 +416,19 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 for (int ks = 0; ks < ui.ksteps; ++ks) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, &s_abort, p.status)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = smem_base + stage * stage_bytes, sb = sa + kABytes;
-                    const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+                    const uint32_t sa = smem_base + stage * stage_bytes, sb = sa + kWBytes;
+                    // M operand first: the weight tile, or the token tile in the token-major shape
+                    const uint64_t da = smem_desc_sw128(SWAP ? sb : sa), db = smem_desc_sw128(SWAP ? sa : sb);
+                    for (int a = 0; a < ui.kb; ++a) {
+                        // (token-major: slice a of the stage; its token rows and weight rows follow those of slice a - 1)
+                        const uint64_t oa = (uint64_t)((a * ui.npad * kBK * 2) >> 4), ob = (uint64_t)((a * ui.width * kBK * 2) >> 4);
 #pragma unroll
-                    for (int kk = 0; kk < kBK / 16; ++kk) {
-                        const uint32_t acc = (ks | kk) ? 1u : 0u;
-                        const uint64_t adv = (uint64_t)(kk * 32 >> 4);      // 16 elements = 32 bytes along K
-                        if (PAIR) umma_bf16_pair(d, da + adv, db + adv, idesc, acc);
-                        else umma_bf16(d, da + adv, db + adv, idesc, acc);
+                        for (int kk = 0; kk < kBK / 16; ++kk) {
+                            const uint32_t acc = (ks | a | kk) ? 1u : 0u;
+                            const uint64_t adv = (uint64_t)(kk * 32 >> 4);      // 16 elements = 32 bytes along K
+                            if (PAIR) umma_bf16_pair(d, da + adv, db + adv, idesc, acc);
+                            else umma_bf16(d, da + oa + adv, db + ob + adv, idesc, acc);
+                        }
                     }
                     if (wide) {
                         if (ks == ui.ksteps - 1) umma_commit_pair(bar_tfull + 8 * buf);      // first half done: its epilogue may start
@@ -463,7 +485,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
             }
             if (++q == kQueue) { q = 0; qphase ^= 1; }
             if (e.u < 0) break;
-            const UnitInfo ui = unit_info<MODE, PAIR>(p, e, rank);
+            const UnitInfo ui = unit_info<MODE, PAIR, SWAP>(p, e, rank);
             const int ld = ui.shared ? p.ld_shared : p.ld_routed;
             const int n_acc = (PAIR && ui.npad1 > 0) ? 2 : 1;
             for (int hh = 0; hh < n_acc && ok; ++hh) {
@@ -473,7 +495,85 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 const int npad = hh ? ui.npad1 : ui.npad;
                 ok = mbar_wait(bar_tfull + 8 * buf, bphase, &s_abort, p.status);
                 const uint32_t d = tmem_base + lane_addr + buf * 256;
-                if (MODE == 0 && ui.direct) {
+                if (SWAP) {
+                    // Token-major accumulator: this thread's TMEM lane is token `gtid` of the tile, the columns are the
+                    // unit's weight rows (256, 128 or 64); each group takes half of them.  Every thread stages and sends
+                    // only its own token's outputs, so the group needs no barrier.
+                    const int gcols = ui.width >> 1;          // columns of this group
+                    const int c_first = half * gcols;
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    // destination row of this thread's token, -1: none
+                    int drow = -1;
+                    if (ui.direct) {
+                        // the tile holds all tokens; this expert's rows name theirs through perm
+                        for (int j = 0; j < nrows; ++j)
+                            if (p.perm[row0 + j] / p.top_k == gtid) drow = row0 + j;
+                    } else if (gtid < nrows) {
+                        drow = row0 + gtid;
+                    }
+                    if (MODE == 0) {
+                        // columns 2i / 2i+1 hold the gate / up row (or up / gate) of intermediate index cb*32 + i
+                        const uint32_t gf = ui.shared ? (p.gate_first_shared >> ui.model) & 1u : p.gate_first_routed & 1u;
+                        const uint32_t mine = stg + (uint32_t)gtid * 128u;       // up to 64 outputs of 16 bits
+                        bulk_wait_read<0>();                                     // the row sent for the previous tile has left
+#pragma unroll 2
+                        for (int i = 0; i < (gcols >> 4); ++i) {
+                            uint32_t r[16];
+                            tmem_ld16(d + c_first + i * 16, r);
+                            tmem_ld_wait();
+                            uint32_t o[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                unsigned short h2[2];
+#pragma unroll
+                                for (int t = 0; t < 2; ++t) {
+                                    const float a = __uint_as_float(r[4 * j + 2 * t]), b = __uint_as_float(r[4 * j + 2 * t + 1]);
+                                    const float g = gf ? a : b, up = gf ? b : a;
+                                    const float v = __fdividef(g, 1.f + __expf(-g)) * up;
+                                    h2[t] = ui.shared ? __half_as_ushort(__float2half_rn(v)) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+                                }
+                                o[j] = (uint32_t)h2[0] | ((uint32_t)h2[1] << 16);
+                            }
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(mine + i * 16), "r"(o[0]), "r"(o[1]), "r"(o[2]),
+                                         "r"(o[3]) : "memory");
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+                        fence_async_smem();
+                        if (drow >= 0) {
+                            unsigned short* out16 = reinterpret_cast<unsigned short*>(ui.shared ? p.out_shared : p.out_routed);
+                            bulk_store(out16 + (size_t)drow * ld + ui.cb * 32 + (c_first >> 1), mine, (uint32_t)gcols);
+                        }
+                        bulk_commit();
+                    } else {
+                        // fp32 outputs, 16 at a time through one of this thread's two 64-byte slots
+                        if (drow >= 0 && ui.shared && p.shared_dst_rows != nullptr) drow = p.shared_dst_rows[drow];
+                        float* outp = reinterpret_cast<float*>(ui.shared ? p.out_shared : p.out_routed) + ui.cb * 64 + c_first;
+                        const int nchunk = gcols >> 4;
+                        for (int i = 0; i < nchunk; ++i, ++rnd) {
+                            const uint32_t slot = stg + (uint32_t)gtid * 128u + (rnd & 1u) * 64u;
+                            bulk_wait_read<1>();
+                            uint32_t r[16];
+                            tmem_ld16(d + c_first + i * 16, r);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slot + j * 16), "r"(r[4 * j]), "r"(r[4 * j + 1]),
+                                             "r"(r[4 * j + 2]), "r"(r[4 * j + 3]) : "memory");
+                            if (i == nchunk - 1) {
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+                            }
+                            fence_async_smem();
+                            if (drow >= 0) bulk_store(outp + (size_t)drow * ld + i * 16, slot, 64u);
+                            bulk_commit();
+                        }
+                    }
+                } else if (MODE == 0 && ui.direct) {
                     // one decision for the whole warp: the TMEM loads below are warp-wide instructions
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
@@ -622,22 +722,26 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 int u = atomicAdd(p.counter, 1);
                 int4 e0 = make_int4(-1, 0, 0, 0);
                 int2 e1 = make_int2(0, 0);
+                int e0w = 0;                  // token-major shape: weight rows of the unit
                 if (u < n_units) {
                     const Unit un = p.units[u];
                     const Tile t = un.tile < 0 ? p.stiles[~un.tile] : p.tiles[un.tile];
                     e0 = make_int4(u, t.slot, t.row0, t.nrows);
-                    e1 = make_int2(un.colblock, un.tile < 0 ? 1 : 0);
+                    e1 = make_int2(un.colblock & 0xffffff, un.tile < 0 ? 1 : 0);
+                    e0w = 256 >> (un.colblock >> 24);
                 } else {
                     u = -1;
                 }
                 *reinterpret_cast<int4*>(&s_queue[q]) = e0;
                 *reinterpret_cast<int2*>(&s_queue[q].colblock) = e1;
+                s_queue[q].pad0 = e0w;
                 mbar_arrive(bar_qfull + 8 * q);
                 if (PAIR) {
                     const uint32_t dst = peer_queue + (uint32_t)sizeof(QEntry) * q;
                     asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(e0.x), "r"(e0.y), "r"(e0.z),
                                  "r"(e0.w) : "memory");
                     asm volatile("st.shared::cluster.v2.b32 [%0], {%1, %2};" ::"r"(dst + 16), "r"(e1.x), "r"(e1.y) : "memory");
+                    asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(dst + 24), "r"(e0w) : "memory");
                     mbar_arrive_cluster(peer_qfull + 8 * q);
                 }
                 if (++q == kQueue) { q = 0; qphase ^= 1; }
@@ -667,7 +771,7 @@ __global__ void bf16_to_fp16_kernel(const bf16* __restrict__ src, __half* __rest
 // 3-D map over two weight arrays of `rows` x `k` bf16 each: dimension 1 selects the array, so a box of
 // (64 K, 2, 64 rows) lands in shared memory as 128 rows that alternate between the two arrays.
 // Returns false on failure; *first_is_a tells whether index 0 of dimension 1 is array `a`.
-bool make_pair_map(CUtensorMap* m, const void* a, const void* b, uint64_t rows, uint64_t k, bool* first_is_a)
+bool make_pair_map(CUtensorMap* m, const void* a, const void* b, uint64_t rows, uint64_t k, uint32_t box_rows, bool* first_is_a)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
@@ -678,7 +782,7 @@ bool make_pair_map(CUtensorMap* m, const void* a, const void* b, uint64_t rows, 
     if (diff == 0 || (diff & 15) || diff >= (1ull << 40)) return false;
     cuuint64_t dims[3] = {k, 2, rows};
     cuuint64_t strides[2] = {diff, k * 2};
-    cuuint32_t box[3] = {(cuuint32_t)kBK, 2, 64};
+    cuuint32_t box[3] = {(cuuint32_t)kBK, 2, box_rows};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)lo, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -689,6 +793,7 @@ bool make_pair_map(CUtensorMap* m, const void* a, const void* b, uint64_t rows, 
 struct LayerMaps {
     bool ready = false;
     GemmMaps m1, m2;                    // weight maps of the gate/up and down GEMMs (activation maps are per call)
+    GemmMaps m1t, m2t;                  // the same for the token-major shape (boxes of 256 / 128 / 64 weight rows)
     uint32_t gate_first_routed = 1, gate_first_shared = 0;
     std::vector<__half*> ws_down_f16;   // per model
 };
@@ -709,9 +814,11 @@ bool tc_pair_mode(const moe_ctx* c, int T)
 {
     const moe_config& g = c->cfg;
     (void)g;
-    // measured: above 128 tokens the pair shape wins for every workload tried (prefill 4096 tokens, the
-    // 240-expert pool with ~34 rows per expert, the 24-block stack with ~1100 tokens)
-    return c->pair_mode_enabled != 0 && T > 128;
+    // measured: the pair shape (with 512-row tiles) wins where the hot experts and the shared expert fill long tiles
+    // (prefill, 4096 tokens of one model); the 240-expert pool (~34 rows per expert) and the 24-block stack (~1100
+    // tokens) are faster with one-CTA token-major units.  2 forces the pair shape for every batch above 128 tokens.
+    if (c->pair_mode_enabled == 2) return T > 128;
+    return c->pair_mode_enabled != 0 && T / g.n_models >= 2048;
 }
 
 // Tiles of up to 512 rows pay when the segments are long enough to fill them: the weight tile of a K step then
@@ -724,6 +831,12 @@ bool tc_wide_mode(const moe_ctx* c, int T)
     // measured: pays from about 2048 tokens per tenant model (shared-expert tiles and the hot routed experts
     // fill 512 rows); below that the units are short and want the deeper pipeline
     return T / c->cfg.n_models >= 2048;
+}
+
+// One-CTA units with the tokens as the M operand: every batch that does not take the pair shape.
+bool tc_token_major(const moe_ctx* c, int T)
+{
+    return !tc_pair_mode(c, T) && c->token_major_enabled != 0;
 }
 
 void tc_destroy(moe_ctx* c)
@@ -749,23 +862,31 @@ int tc_setup_layer(moe_ctx* c, int layer)
     const PoolWeights& pw = c->pools[layer];
     memset(&lm.m1, 0, sizeof(GemmMaps));
     memset(&lm.m2, 0, sizeof(GemmMaps));
+    memset(&lm.m1t, 0, sizeof(GemmMaps));
+    memset(&lm.m2t, 0, sizeof(GemmMaps));
     bool ok = true, first = true;
     const uint64_t S = g.n_slots;
-    ok &= make_pair_map(&lm.m1.a_routed, pw.w_gate, pw.w_up, S * I, H, &first);
+    ok &= make_pair_map(&lm.m1.a_routed[0], pw.w_gate, pw.w_up, S * I, H, 64, &first);
     lm.gate_first_routed = first ? 1u : 0u;
-    ok &= make_map(&lm.m2.a_routed, pw.w_down, S * H, I, 128, false);
+    ok &= make_map(&lm.m2.a_routed[0], pw.w_down, S * H, I, 128, false);
+    for (int w = 0; w < 3; ++w) {       // token-major shape: 256, 128 and 64 weight rows per box
+        ok &= make_pair_map(&lm.m1t.a_routed[w], pw.w_gate, pw.w_up, S * I, H, 128u >> w, &first);
+        ok &= make_map(&lm.m2t.a_routed[w], pw.w_down, S * H, I, 256u >> w, false);
+    }
     lm.ws_down_f16.assign(M, nullptr);
     lm.gate_first_shared = 0;
     for (int m = 0; m < M && ok && Is > 0; ++m) {
         const ModelWeights& mw = c->models[(size_t)layer * M + m];
-        ok &= make_pair_map(&lm.m1.a_shared[m], mw.ws_gate, mw.ws_up, Is, H, &first);
+        ok &= make_pair_map(&lm.m1.a_shared[m][0], mw.ws_gate, mw.ws_up, Is, H, 64, &first);
+        for (int w = 0; w < 3; ++w) ok &= make_pair_map(&lm.m1t.a_shared[m][w], mw.ws_gate, mw.ws_up, Is, H, 128u >> w, &first);
         if (first) lm.gate_first_shared |= 1u << m;
         // fp16 copy of the shared expert's down projection (its activations are fp16 and one MMA takes
         // operands of one type); every bf16 weight of magnitude >= 2^-17 converts exactly
         const size_t n = (size_t)H * Is;
         if (cudaMalloc((void**)&lm.ws_down_f16[m], n * sizeof(__half)) != cudaSuccess) return MOE_ERR_ALLOC;
         bf16_to_fp16_kernel<<<(unsigned)((n + 255) / 256), 256>>>(mw.ws_down, lm.ws_down_f16[m], n);
-        ok &= make_map(&lm.m2.a_shared[m], lm.ws_down_f16[m], H, Is, 128, true);
+        ok &= make_map(&lm.m2.a_shared[m][0], lm.ws_down_f16[m], H, Is, 128, true);
+        for (int w = 0; w < 3; ++w) ok &= make_map(&lm.m2t.a_shared[m][w], lm.ws_down_f16[m], H, Is, 256u >> w, true);
     }
     if (!ok) {
         snprintf(c->errbuf, sizeof(c->errbuf), "cuTensorMapEncodeTiled failed for a weight tensor");
@@ -778,10 +899,10 @@ int tc_setup_layer(moe_ctx* c, int layer)
 
 namespace {
 
-template <int MODE, bool PAIR>
+template <int MODE, bool PAIR, bool SWAP>
 cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, cudaStream_t st)
 {
-    auto kern = grouped_gemm_kernel<MODE, PAIR>;
+    auto kern = grouped_gemm_kernel<MODE, PAIR, SWAP>;
     static bool attr_set = false;
     if (!attr_set) {
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
@@ -824,12 +945,13 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     const uint64_t R = (uint64_t)T * g.top_k;
     const bool shared = y_shared != nullptr && Is > 0;
     const bool pair = tc_pair_mode(c, T);
+    const bool swap = tc_token_major(c, T);
     // direct mode: with few tokens the routed gate/up units read the tokens in place (no permuted copy)
     const bool direct = tc_direct_mode(c, T) && perm != nullptr;
     const uint32_t fmt_bf16 = (1u << 7) | (1u << 10), fmt_fp16 = 0u;
 
     // activation maps are rebuilt per call: their addresses and row counts are the call's
-    GemmMaps& m1 = lm.m1;
+    GemmMaps& m1 = swap ? lm.m1t : lm.m1;
     bool ok = true;
     auto make_b = [](CUtensorMap* m, const void* base, uint64_t rows, uint64_t k, bool fp16) {
         bool good = true;
@@ -852,7 +974,7 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     p1.tiles = c->ws.tiles; p1.stiles = c->ws.stiles;
     p1.perm = perm; p1.top_k = g.top_k; p1.direct = direct ? 1 : 0; p1.n_tokens_pad = (T + 15) & ~15;
     p1.k_routed = H; p1.k_shared = H;
-    p1.rows_per_slot = I; p1.cb_rows = 64;
+    p1.rows_per_slot = I; p1.cb_rows = swap ? 32 : 64;      // token-major: colblocks count steps of 64 weight rows
     p1.out_routed = c->ws.h; p1.out_shared = c->ws.hs; p1.ld_routed = I; p1.ld_shared = Is;
     p1.shared_dst_rows = nullptr;
     p1.idesc_fmt_routed = fmt_bf16; p1.idesc_fmt_shared = fmt_bf16;
@@ -861,11 +983,12 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     p1.stream_weights = (R <= 2048) ? 1 : 0;
     p1.wide = tc_wide_mode(c, T) ? 1 : 0;
     p1.group = p1.wide ? 1 : 2;
-    cudaError_t e = pair ? launch_gemm<0, true>(c, p1, m1, st) : launch_gemm<0, false>(c, p1, m1, st);
+    cudaError_t e = pair ? launch_gemm<0, true, false>(c, p1, m1, st)
+                         : (swap ? launch_gemm<0, false, true>(c, p1, m1, st) : launch_gemm<0, false, false>(c, p1, m1, st));
     if (e != cudaSuccess) return e;
     stage_mark(c, st, kEvGateUp);
 
-    GemmMaps& m2 = lm.m2;
+    GemmMaps& m2 = swap ? lm.m2t : lm.m2;
     ok = make_b(m2.b_routed, c->ws.h, R, I, false);
     if (shared) ok = ok && make_b(m2.b_shared, c->ws.hs, T, Is, true);
     else copy_b(m2.b_shared, m2.b_routed);
@@ -874,11 +997,12 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     p2.units = c->ws.units2; p2.n_units = c->ws.plan_counts + 3; p2.counter = c->ws.plan_counts + 5;
     p2.direct = 0;
     p2.k_routed = I; p2.k_shared = Is;
-    p2.rows_per_slot = H; p2.cb_rows = 128;
+    p2.rows_per_slot = H; p2.cb_rows = swap ? 64 : 128;
     p2.out_routed = y_perm; p2.out_shared = y_shared; p2.ld_routed = H; p2.ld_shared = H;
     p2.shared_dst_rows = shared_dst_rows;
     p2.idesc_fmt_routed = fmt_bf16; p2.idesc_fmt_shared = fmt_fp16;
-    e = pair ? launch_gemm<1, true>(c, p2, m2, st) : launch_gemm<1, false>(c, p2, m2, st);
+    e = pair ? launch_gemm<1, true, false>(c, p2, m2, st)
+             : (swap ? launch_gemm<1, false, true>(c, p2, m2, st) : launch_gemm<1, false, false>(c, p2, m2, st));
     if (e != cudaSuccess) return e;
     stage_mark(c, st, kEvDown);
     c->launches += 2;

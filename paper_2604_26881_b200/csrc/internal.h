@@ -125,6 +125,7 @@ struct moe_ctx {
     void* rmaps;                  // TMA descriptors of the tensor-core router
     int route_path;
     int pair_mode_enabled;        // allow the 2-CTA (cta_group::2) shape of the grouped GEMM for long tiles
+    int token_major_enabled;      // one-CTA units take the tokens as the M operand of the MMA (up to 256 weight rows per tile)
     int wide_tiles_enabled;       // allow 512-row tiles (two accumulators per weight tile) in the 2-CTA shape
     bool timing;                  // record an event after every stage (moe_layer_forward_timed)
     cudaEvent_t ev[8];
@@ -187,6 +188,7 @@ void tc_destroy(moe_ctx* c);
 bool tc_supported(const moe_ctx* c);
 bool tc_pair_mode(const moe_ctx* c, int T);      // long tiles: two CTAs share a token tile
 bool tc_wide_mode(const moe_ctx* c, int T);      // pair shape with tiles of up to 512 rows
+bool tc_token_major(const moe_ctx* c, int T);    // one-CTA shape with the tokens as the M operand
 
 // Few tokens of one model: the routed gate/up units read the tokens in place, no permuted copy is needed.
 static inline bool tc_direct_mode(const moe_ctx* c, int T)

@@ -24,7 +24,8 @@ PlanArgs make_plan_args(moe_ctx* c, int T, int G, bool with_shared)
     const bool tc = tc_supported(c);
     // weight-row blocks per unit: gate/up 64 intermediate indices, down 128 rows; a CTA pair takes two
     const bool pair = tc && tc_pair_mode(c, T);
-    const int div1 = pair ? 128 : 64, div2 = pair ? 256 : 128;
+    const bool wide_rows = pair || (tc && tc_token_major(c, T));      // 256 weight rows per unit
+    const int div1 = wide_rows ? 128 : 64, div2 = wide_rows ? 256 : 128;
     PlanArgs a;
     a.slot_table = c->d_slot;
     a.M = g.n_models; a.E = g.n_experts; a.G = G; a.T = T;
@@ -33,6 +34,17 @@ PlanArgs make_plan_args(moe_ctx* c, int T, int G, bool with_shared)
     a.with_shared = with_shared ? 1 : 0;
     a.nblk1 = g.inter / div1; a.nblk2 = g.hidden / div2;
     a.snblk1 = g.shared_inter / div1; a.snblk2 = g.hidden / div2;
+    a.token_major = (tc && tc_token_major(c, T)) ? 1 : 0;
+    a.n_ctas = c->sm_count;
+    a.shared_down_width = 256;
+    if (a.token_major && g.shared_inter > 0) {
+        // few tokens: the shared expert's down units get narrower (their K slices per stage must divide K / 64)
+        const int want = T <= 32 ? 64 : (T <= 64 ? 128 : 256);
+        if ((g.shared_inter / 64) % (256 / want) == 0) a.shared_down_width = want;
+        a.snblk2 = g.hidden / a.shared_down_width;
+    }
+    a.split_ok[0] = (g.hidden / 64) % 2 == 0; a.split_ok[1] = (g.inter / 64) % 2 == 0;
+    a.direct = tc_direct_mode(c, T) ? 1 : 0;
     a.tiles = c->ws.tiles; a.stiles = c->ws.stiles;
     a.units1 = tc ? c->ws.units1 : nullptr; a.units2 = tc ? c->ws.units2 : nullptr;
     a.plan_counts = c->ws.plan_counts;

@@ -14,6 +14,11 @@ struct PlanArgs {
     const int32_t* model_tok_off;     // null when M == 1
     int with_shared;
     int nblk1, nblk2, snblk1, snblk2; // weight-row blocks of the gate/up and down GEMMs (routed, shared)
+    int token_major;                  // 1: units of the one-CTA token-major shape (see the end of plan_body)
+    int n_ctas;                       // CTAs of the grouped GEMM launches
+    int shared_down_width;            // token-major: weight rows of a shared-expert unit of the down projection
+    int split_ok[2];                  // token-major: K / 64 of the routed units is even (gate/up, down)
+    int direct;                       // the routed gate/up units read all T tokens in place
     Tile* tiles;
     Tile* stiles;
     Unit* units1;                     // null: no unit lists (CUDA-core path)
@@ -102,6 +107,60 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
         if (tid == 0) {
             a.plan_counts[2] = su1 + n_tiles * a.nblk1;
             a.plan_counts[3] = su2 + n_tiles * a.nblk2;
+        }
+        if (a.token_major) {
+            // Token-major units: the colblock becomes (first weight row / 64) with a width code in the top byte
+            // (0: 256 weight rows, 1: 128, 2: 64); narrower units pack 2 or 4 K slices into a stage, so a unit of
+            // half the rows is half as long.  Two uses:
+            //  - the shared expert's down projection contracts over 4x more elements than a routed expert's; with
+            //    few tokens its units are made 4x (2x) narrower so that they are as long as the routed ones;
+            //  - U equally long units on S CTAs take ceil(U / S) rounds; when the last round is less than half
+            //    full, its units are split in two (where the tile has at most 64 rows), so that round costs half.
+            __shared__ int s_split[128];
+            for (int l = 0; l < 2; ++l) {
+                Unit* list = l ? a.units2 : a.units1;
+                const int n_shared = l ? su2 : su1;
+                const int routed = n_tiles * (l ? a.nblk2 : a.nblk1);
+                const int total = n_shared + routed;
+                const int wsh = l ? a.shared_down_width : 256;
+                const int sh_step = wsh / 64, sh_code = wsh == 256 ? 0 : (wsh == 128 ? 1 : 2);
+                int r = total % a.n_ctas;
+                if (2 * r > a.n_ctas || r > routed || r > 128 || !a.split_ok[l]) r = 0;     // (the tail of a list is routed units)
+                __syncthreads();                                            // the list is complete
+                Unit mine;
+                int cnt = 0;
+                if (tid < r) {
+                    mine = list[total - r + tid];
+                    const int rows = a.direct ? a.T : a.tiles[mine.tile].nrows;
+                    cnt = rows <= 64 ? 2 : 1;
+                    s_split[tid] = cnt;
+                }
+                for (int i = tid; i < total - r; i += nth) {
+                    const int cb = list[i].colblock;
+                    list[i].colblock = i < n_shared ? (cb * sh_step) | (sh_code << 24) : cb * 4;
+                }
+                __syncthreads();
+                if (tid < r) {
+                    int off = 0;
+                    for (int j = 0; j < tid; ++j) off += s_split[j];
+                    Unit u = mine;
+                    if (cnt == 2) {
+                        u.colblock = (mine.colblock * 4) | (1 << 24);
+                        list[total - r + off] = u;
+                        u.colblock = (mine.colblock * 4 + 2) | (1 << 24);
+                        list[total - r + off + 1] = u;
+                    } else {
+                        u.colblock = mine.colblock * 4;
+                        list[total - r + off] = u;
+                    }
+                }
+                if (tid == 0) {
+                    int extra = 0;
+                    for (int j = 0; j < r; ++j) extra += s_split[j] - 1;
+                    a.plan_counts[2 + l] = total + extra;
+                }
+                __syncthreads();
+            }
         }
     }
     if (tid == 0) {

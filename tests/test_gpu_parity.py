@@ -196,12 +196,14 @@ def test_pair_shape_and_single_shape_agree_bit_for_bit(qwen_weights):
     x, tenant, mot = W.make_tokens(wl, seed=2)
     g = GpuLayer(wl, [qwen_weights], wl.T, model_of_tenant=mot)
     try:
-        B.moe_set_option(g.ctx, B.MOE_OPT_PAIR_MODE, 1)
+        B.moe_set_option(g.ctx, B.MOE_OPT_PAIR_MODE, 2)
         pair = g.forward(x, tenant, wl.G)
         B.moe_set_option(g.ctx, B.MOE_OPT_PAIR_MODE, 0)
-        single = g.forward(x, tenant, wl.G)
+        single = g.forward(x, tenant, wl.G)              # one CTA per unit, tokens as the M operand
+        B.moe_set_option(g.ctx, B.MOE_OPT_TOKEN_MAJOR, 0)
+        single_wm = g.forward(x, tenant, wl.G)           # one CTA per unit, weight rows as the M operand
         assert B.moe_last_status(g.ctx)[0] == 0
-        assert torch.equal(pair, single)
+        assert torch.equal(pair, single) and torch.equal(pair, single_wm)
         # and both are the CUDA-core path within the tolerance
         B.moe_set_option(g.ctx, B.MOE_OPT_EXPERT_PATH, B.MOE_PATH_FMA)
         fma = g.forward(x, tenant, wl.G)
