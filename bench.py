@@ -126,9 +126,9 @@ def algorithmic_work(wl, active_experts: int, T: int):
 
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
-# ncu capture summarised in profiles/grouped_gemm_decode_ncu.md; None where no capture of the current
-# kernel exists.
-NCU_TRAFFIC_BYTES = {"decode": 657.641728e6 + 3.782912e6}
+# ncu captures summarised in profiles/grouped_gemm_decode_ncu.md and profiles/grouped_gemm_prefill_ncu.md; None where
+# no capture of the current kernel exists.
+NCU_TRAFFIC_BYTES = {"decode": 657.655808e6 + 3.741696e6, "prefill": 814.875648e6 + 92.275712e6}
 
 
 def run_reference(args, wl, rank):
