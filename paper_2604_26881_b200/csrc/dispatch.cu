@@ -105,16 +105,20 @@ dispatch_count_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
     __shared__ int32_t s_count[2];
     __shared__ int s_last;
     const int tid = threadIdx.x, nth = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nth >> 5;
+    // every thread looks up the bin of one row of the chunk (the lookups are chains of dependent loads: all of them
+    // in flight at once), then one warp walks the bins in row order out of shared memory
+    __shared__ unsigned short s_bin[kDispatchChunk];
+    const int r0 = blockIdx.x * kDispatchChunk;
+    const int r1 = min(R, r0 + kDispatchChunk);
     for (int b = tid; b < nbins; b += nth) s_tot[b] = 0;
+    for (int r = r0 + tid; r < r1; r += nth) s_bin[r - r0] = (unsigned short)row_bin(bm, tenant_id[r / k], topk_idx[r], status);
     __syncthreads();
     if (warp == 0) {
-        const int r0 = blockIdx.x * kDispatchChunk;
-        const int r1 = min(R, r0 + kDispatchChunk);
         for (int rr = r0; rr < r1; rr += 32) {
             const int r = rr + lane;
             const bool live = r < r1;
             int bin = -1 - lane;                 // distinct dummy keys for idle lanes
-            if (live) bin = row_bin(bm, tenant_id[r / k], topk_idx[r], status);
+            if (live) bin = s_bin[r - r0];
             const unsigned peers = __match_any_sync(0xffffffffu, bin);
             const int leader = __ffs(peers) - 1;
             const int rank = __popc(peers & ((1u << lane) - 1u));
