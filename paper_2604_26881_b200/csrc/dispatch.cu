@@ -104,7 +104,7 @@ dispatch_count_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
     __shared__ int32_t s_part[33];
     __shared__ int32_t s_count[2];
     __shared__ int s_last;
-    const int tid = threadIdx.x, nth = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nth >> 5;
+    const int tid = threadIdx.x, nth = blockDim.x, lane = tid & 31, warp = tid >> 5;
     // every thread looks up the bin of one row of the chunk (the lookups are chains of dependent loads: all of them
     // in flight at once), then one warp walks the bins in row order out of shared memory
     __shared__ unsigned short s_bin[kDispatchChunk];

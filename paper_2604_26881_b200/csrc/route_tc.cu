@@ -21,9 +21,6 @@ constexpr int kRBK = 64;
 constexpr int kRTokens = 128;
 constexpr int kRABytes = kRTokens * kRBK * 2;          // 16 KB of tokens per stage
 constexpr int kRMaxN = 256;                            // router rows of all models, padded
-constexpr int kRBBytes = kRMaxN * kRBK * 2;            // 32 KB
-constexpr int kRMaxGateN = 64;                         // 16 columns per model for the shared-expert gate (<= 4 models)
-constexpr int kRGBytes = kRMaxGateN * kRBK * 2;        // 8 KB
 constexpr int kRTileBudget = 192 * 1024;               // shared memory for the pipeline stages
 constexpr int kRSmemBytes = kRTileBudget + kRABytes /* a short token tile is read as 128 rows */ + 1024 + 512;
 constexpr int kRThreads = 256;                         // warp 0: TMA (tokens), 1: MMA, 2..5: epilogue, 6 / 7: TMA (routers / gates)

@@ -66,6 +66,17 @@ def test_decode_config(qwen_weights, path):
     assert 30 <= o["active_experts"] <= 60
 
 
+@pytest.mark.parametrize("T", [1, 5, 33, 64, 100, 128])
+def test_small_batches_token_major_units(qwen_weights, T):
+    # batch sizes around the switches of the token-major plan: the shared expert's down units are 64 weight rows
+    # wide up to 32 tokens, 128 up to 64 tokens, 256 above; the last round of units is split in two while the tiles
+    # have at most 64 rows; up to 128 tokens the routed gate/up units read the tokens in place
+    wl = W.scaled(W.WORKLOADS["decode"], T=T)
+    wts = dict(qwen_weights, router_bias=None)
+    x, tenant, mot = W.make_tokens(wl, seed=11)
+    run_and_compare(wl, wts, x, tenant, mot, wl.G, B.MOE_PATH_AUTO)
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_prefill_reduced(qwen_weights, path):
     # the prefill layer (Zipf-skewed router) on 300 tokens: every element against the oracle
