@@ -62,6 +62,8 @@ constexpr uint32_t kTmemCols = 512;            // 2 accumulator buffers x 256 co
 struct GemmParams {
     const Unit* units;
     const int32_t* n_units;
+    const int32_t* n_shared;      // shared-expert units at the head of the list that are to be spread evenly over the
+                                  // launch (0: take the list in order)
     int32_t* counter;             // work counter of the dynamic scheduler (zeroed by the plan kernel)
     const Tile* tiles;
     const Tile* stiles;
@@ -268,6 +270,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
     const bool leader = rank == 0;
     const int n_units = *p.n_units;
+    const int n_shared = *p.n_shared;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
@@ -317,7 +320,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
             uint32_t stage = 0, phase = 0, q = 0, qphase = 0;
             uint32_t armed = 0, armed_phase = 0;
             bool ok = true;
-            const uint64_t pol_w = p.stream_weights ? l2_evict_first() : l2_evict_last();
+            const uint64_t pol_first = l2_evict_first(), pol_last = l2_evict_last();
             const uint64_t pol_x = l2_evict_last();
             while (ok) {
                 if (!(leader ? mbar_wait(bar_qfull + 8 * q, qphase, &s_abort, p.status)
@@ -328,6 +331,10 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 if (e.u < 0) break;
                 const UnitInfo ui = unit_info<MODE, PAIR, SWAP>(p, e, rank);
                 const int claim_ks = ui.ksteps > kClaimAhead ? ui.ksteps - kClaimAhead : 0;
+                // L2 policy of the weight tiles: a routed expert with at most 128 rows is read by one tile only, so its
+                // weights stream through (evict-first) and leave the cache to what is read again -- the shared expert's
+                // weights (every token tile of the model reads them) and the weights of the experts with several tiles
+                const uint64_t pol_w = (p.stream_weights || (!ui.shared && ui.nrows <= 128)) ? pol_first : pol_last;
                 const int wsel = SWAP ? (ui.width == 256 ? 0 : (ui.width == 128 ? 1 : 2)) : 0;
                 const CUtensorMap* ma = ui.amap < 0 ? &maps.a_routed[wsel] : &maps.a_shared[ui.amap][wsel];
                 const bool bshared = ui.shared || ui.direct;
@@ -724,7 +731,15 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 int2 e1 = make_int2(0, 0);
                 int e0w = 0;                  // token-major shape: weight rows of the unit
                 if (u < n_units) {
-                    const Unit un = p.units[u];
+                    // The list holds the shared expert's units first.  They are fed from L2 (every token tile of the
+                    // model reads the same weights) while the routed units stream theirs from HBM, so the two kinds are
+                    // dealt out alternately, in proportion: HBM then stays busy for the whole launch.
+                    int ix = u;
+                    if (n_shared > 0) {
+                        const int a = (int)((long long)u * n_shared / n_units), b = (int)((long long)(u + 1) * n_shared / n_units);
+                        ix = b > a ? a : n_shared + (u - a);
+                    }
+                    const Unit un = p.units[ix];
                     const Tile t = un.tile < 0 ? p.stiles[~un.tile] : p.tiles[un.tile];
                     e0 = make_int4(u, t.slot, t.row0, t.nrows);
                     e1 = make_int2(un.colblock & 0xffffff, un.tile < 0 ? 1 : 0);
@@ -971,6 +986,7 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     GemmParams p1;
     memset(&p1, 0, sizeof(p1));
     p1.units = c->ws.units1; p1.n_units = c->ws.plan_counts + 2; p1.counter = c->ws.plan_counts + 4;
+    p1.n_shared = c->ws.plan_counts + 6;
     p1.tiles = c->ws.tiles; p1.stiles = c->ws.stiles;
     p1.perm = perm; p1.top_k = g.top_k; p1.direct = direct ? 1 : 0; p1.n_tokens_pad = (T + 15) & ~15;
     p1.k_routed = H; p1.k_shared = H;
@@ -983,6 +999,7 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     p1.stream_weights = (R <= 2048) ? 1 : 0;
     p1.wide = tc_wide_mode(c, T) ? 1 : 0;
     p1.group = p1.wide ? 1 : 2;
+    if (swap) p1.group = 1;
     cudaError_t e = pair ? launch_gemm<0, true, false>(c, p1, m1, st)
                          : (swap ? launch_gemm<0, false, true>(c, p1, m1, st) : launch_gemm<0, false, false>(c, p1, m1, st));
     if (e != cudaSuccess) return e;
@@ -995,6 +1012,7 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     if (!ok) return cudaErrorInvalidValue;
     GemmParams p2 = p1;
     p2.units = c->ws.units2; p2.n_units = c->ws.plan_counts + 3; p2.counter = c->ws.plan_counts + 5;
+    p2.n_shared = c->ws.plan_counts + 7;
     p2.direct = 0;
     p2.k_routed = I; p2.k_shared = Is;
     p2.rows_per_slot = H; p2.cb_rows = swap ? 64 : 128;

@@ -45,6 +45,8 @@ PlanArgs make_plan_args(moe_ctx* c, int T, int G, bool with_shared)
     }
     a.split_ok[0] = (g.hidden / 64) % 2 == 0; a.split_ok[1] = (g.inter / 64) % 2 == 0;
     a.direct = tc_direct_mode(c, T) ? 1 : 0;
+    a.interleave_down = (a.token_major && g.shared_inter > 0 &&
+                         (long long)a.shared_down_width * g.shared_inter == 256ll * g.inter) ? 1 : 0;
     a.tiles = c->ws.tiles; a.stiles = c->ws.stiles;
     a.units1 = tc ? c->ws.units1 : nullptr; a.units2 = tc ? c->ws.units2 : nullptr;
     a.plan_counts = c->ws.plan_counts;

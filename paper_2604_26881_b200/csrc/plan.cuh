@@ -19,6 +19,7 @@ struct PlanArgs {
     int shared_down_width;            // token-major: weight rows of a shared-expert unit of the down projection
     int split_ok[2];                  // token-major: K / 64 of the routed units is even (gate/up, down)
     int direct;                       // the routed gate/up units read all T tokens in place
+    int interleave_down;              // the shared units of the down projection are as long as the routed ones
     Tile* tiles;
     Tile* stiles;
     Unit* units1;                     // null: no unit lists (CUDA-core path)
@@ -107,6 +108,12 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
         if (tid == 0) {
             a.plan_counts[2] = su1 + n_tiles * a.nblk1;
             a.plan_counts[3] = su2 + n_tiles * a.nblk2;
+            // shared units that the scheduler spreads over the launch: only where a model's tokens fill several tiles
+            // (its shared weights are then read again and again out of L2, while a single tile streams them from HBM
+            // like any routed expert), and only equally long units (longer ones go first)
+            const bool reread = n_stiles > a.M;
+            a.plan_counts[6] = reread ? su1 : 0;
+            a.plan_counts[7] = (reread && a.interleave_down) ? su2 : 0;
         }
         if (a.token_major) {
             // Token-major units: the colblock becomes (first weight row / 64) with a width code in the top byte
