@@ -225,7 +225,11 @@ __device__ __forceinline__ UnitInfo unit_info(const GemmParams& p, const QEntry&
         ui.npad1 = (e.nrows - n0 + 31) & ~31;
     }
     else ui.npad = (e.nrows + 15) & ~15;      // (token-major shape: rows of the token tile that are loaded)
-    ui.ksteps = (ui.shared ? p.k_shared : p.k_routed) / (kBK * ui.kb);
+    const int k_len = ui.shared ? p.k_shared : p.k_routed;
+    // pair shape with 48 KB stages: a unit of at most 128 tokens puts two K slices into a stage (2 x 16 KB of weights
+    // and 2 x at most 8 KB of tokens per CTA), which halves the waits and commits of its MMA lane -- all a short unit costs
+    if (PAIR && p.wide && ui.npad1 == 0 && ui.npad <= 128 && (k_len / kBK) % 2 == 0) ui.kb = 2;
+    ui.ksteps = k_len / (kBK * ui.kb);
     return ui;
 }
 
@@ -353,12 +357,15 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     if (wrole) {
                         // the token lane's bytes may be counted before this is posted: the phase still cannot complete
                         // without this arrival
-                        if (leader) mbar_expect_tx(full, (PAIR ? 2u : 1u) * (uint32_t)(kWBytes + ui.kb * (my_rows + my_rows1) * kBK * 2));
+                        if (leader) mbar_expect_tx(full, (PAIR ? 2u : 1u) * (uint32_t)((PAIR ? ui.kb * kABytes : kWBytes) +
+                                                                                       ui.kb * (my_rows + my_rows1) * kBK * 2));
                         armed |= 1u << stage;
                         armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
                         if (PAIR) {
-                            if (MODE == 0) tma_load_3d_pair(sa, ma, full, ks * kBK, 0, ui.a_row, pol_w);
-                            else tma_load_2d_pair(sa, ma, full, ks * kBK, ui.a_row, pol_w);
+                            for (int a = 0; a < ui.kb; ++a) {
+                                if (MODE == 0) tma_load_3d_pair(sa + a * kABytes, ma, full, (ks * ui.kb + a) * kBK, 0, ui.a_row, pol_w);
+                                else tma_load_2d_pair(sa + a * kABytes, ma, full, (ks * ui.kb + a) * kBK, ui.a_row, pol_w);
+                            }
                         } else {
                             // (token-major: kb slices of 64 K elements, each `width` rows high, one after the other)
                             for (int a = 0; a < ui.kb; ++a) {
@@ -369,11 +376,14 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                         }
                     } else {
                         // token rows in boxes of 128 / 64 / 32 / 16 rows
-                        for (int acc = 0; acc < (PAIR ? 2 : ui.kb); ++acc) {
-                            // pair shape: the two accumulators' tiles; token-major shape: the K slices of the stage
-                            const int rows = (PAIR && acc) ? my_rows1 : my_rows, r0 = (PAIR && acc) ? my_row1 : my_row0;
-                            const uint32_t dst = sb + (PAIR ? acc * kBBytes : acc * my_rows * kBK * 2);
-                            const int kx = (PAIR ? ks : ks * ui.kb + acc) * kBK;
+                        const bool by_acc = PAIR && ui.kb == 1;
+                        for (int acc = 0; acc < (by_acc ? 2 : ui.kb); ++acc) {
+                            // pair shape: the two accumulators' tiles, or the K slices of a short unit (behind its two weight
+                            // slices); token-major shape: the K slices of the stage
+                            const int rows = (by_acc && acc) ? my_rows1 : my_rows, r0 = (by_acc && acc) ? my_row1 : my_row0;
+                            const uint32_t dst = by_acc ? sb + acc * kBBytes
+                                                        : (PAIR ? sa + ui.kb * kABytes : sb) + acc * my_rows * kBK * 2;
+                            const int kx = (by_acc ? ks : ks * ui.kb + acc) * kBK;
                             int j = 0;
 #pragma unroll
                             for (int bx = 0; bx < 4; ++bx) {
@@ -429,11 +439,14 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     for (int a = 0; a < ui.kb; ++a) {
                         // (token-major: slice a of the stage; its token rows and weight rows follow those of slice a - 1)
                         const uint64_t oa = (uint64_t)((a * ui.npad * kBK * 2) >> 4), ob = (uint64_t)((a * ui.width * kBK * 2) >> 4);
+                        // (pair shape, short unit: weight slice a, and the token slices behind the two weight slices)
+                        const uint64_t pa = (uint64_t)((a * kABytes) >> 4);
+                        const uint64_t pb = (uint64_t)((((ui.kb - 1) * kABytes) + a * (ui.npad >> 1) * kBK * 2) >> 4);
 #pragma unroll
                         for (int kk = 0; kk < kBK / 16; ++kk) {
                             const uint32_t acc = (ks | a | kk) ? 1u : 0u;
                             const uint64_t adv = (uint64_t)(kk * 32 >> 4);      // 16 elements = 32 bytes along K
-                            if (PAIR) umma_bf16_pair(d, da + adv, db + adv, idesc, acc);
+                            if (PAIR) umma_bf16_pair(d, da + pa + adv, db + pb + adv, idesc, acc);
                             else umma_bf16(d, da + oa + adv, db + ob + adv, idesc, acc);
                         }
                     }
