@@ -747,9 +747,14 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     // The list holds the shared expert's units first.  They are fed from L2 (every token tile of the
                     // model reads the same weights) while the routed units stream theirs from HBM, so the two kinds are
                     // dealt out alternately, in proportion: HBM then stays busy for the whole launch.
+                    // The last sixth of the launch is kept for routed units: the shared ones are full-length, and a
+                    // long unit handed out at the very end is what the other CTAs then wait for.
                     int ix = u;
                     if (n_shared > 0) {
-                        const int a = (int)((long long)u * n_shared / n_units), b = (int)((long long)(u + 1) * n_shared / n_units);
+                        const int routed = n_units - n_shared;
+                        const int cut = n_units - min(routed, n_units / 6);
+                        const int uc = min(u, cut), uc1 = min(u + 1, cut);
+                        const int a = (int)((long long)uc * n_shared / cut), b = (int)((long long)uc1 * n_shared / cut);
                         ix = b > a ? a : n_shared + (u - a);
                     }
                     const Unit un = p.units[ix];
