@@ -263,7 +263,8 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     const uint32_t stage_bytes = kRingBytes / n_stages;
     // Stages are handed back to the producer in groups: a tcgen05.commit costs the issuing lane about as much
     // as two MMAs, so with four MMAs per stage one commit per stage would starve the tensor pipe.
-    const uint32_t group = (uint32_t)p.group;
+    const uint32_t group = (uint32_t)p.group;                                  // 1 or 2: masks and shifts below, a
+    const uint32_t gmask = group - 1, gshift = group >> 1;                     // division per K step would be felt
     const uint32_t bar_qfull = bar_tempty + 16, bar_qempty = bar_qfull + 8 * kQueue;
     const uint32_t bar_sched = bar_qempty + 8 * kQueue;
     __shared__ uint32_t s_tmem_base;
@@ -350,8 +351,8 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 const int my_row1 = brow0 + 256 + (int)rank * my_rows1;
                 for (int ks = 0; ks < ui.ksteps; ++ks) {
                     if (wrole && leader && ks == claim_ks) mbar_arrive(bar_sched);      // time to claim the next unit
-                    if (stage % group == 0 &&
-                        !mbar_wait(bar_empty + 8 * (stage / group), phase ^ 1, &s_abort, p.status)) { ok = false; break; }
+                    if ((stage & gmask) == 0 &&
+                        !mbar_wait(bar_empty + 8 * (stage >> gshift), phase ^ 1, &s_abort, p.status)) { ok = false; break; }
                     const uint32_t sa = smem_base + stage * stage_bytes, sb = sa + kWBytes;
                     const uint32_t full = bar_full + 8 * stage;
                     if (wrole) {
@@ -465,8 +466,8 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                         }
                     }
                     // frees the stage group (in both CTAs of a pair) when these MMAs have read it
-                    if (stage % group == group - 1) {
-                        if (PAIR) umma_commit_pair(bar_empty + 8 * (stage / group)); else umma_commit(bar_empty + 8 * (stage / group));
+                    if ((stage & gmask) == gmask) {
+                        if (PAIR) umma_commit_pair(bar_empty + 8 * (stage >> gshift)); else umma_commit(bar_empty + 8 * (stage >> gshift));
                     }
                     if (++stage == n_stages) { stage = 0; phase ^= 1; }
                 }

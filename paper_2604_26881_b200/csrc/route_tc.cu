@@ -74,6 +74,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
     const uint32_t bars = smem_base + kRTileBudget + kRABytes;
     const uint32_t bar_full = bars, bar_empty = bars + 8 * kRMaxStages, bar_tfull = bars + 16 * kRMaxStages;
     const int kRStages = p.n_stages;
+    const uint32_t gmask = (uint32_t)p.group - 1, gshift = p.group == 4 ? 2u : (p.group == 2 ? 1u : 0u);      // group: 1, 2 or 4
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
@@ -111,8 +112,8 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
             bool ok = true;
             const uint64_t keep = l2_evict_last();      // router weights and tokens are read again soon
             for (int ks = 0; ks < ksteps; ++ks) {
-                if (stage % p.group == 0 &&
-                    !mbar_wait(bar_empty + 8 * (stage / p.group), phase ^ 1, &s_abort, p.status)) { ok = false; break; }
+                if ((stage & gmask) == 0 &&
+                    !mbar_wait(bar_empty + 8 * (stage >> gshift), phase ^ 1, &s_abort, p.status)) { ok = false; break; }
                 const uint32_t sa = smem_base + stage * p.stage_bytes, sb = sa + p.a_bytes;
                 const uint32_t full = bar_full + 8 * stage;
                 armed |= 1u << stage;
@@ -154,7 +155,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                     umma_bf16(tmem_base, da + adv, db + adv, idesc, (ks | kk) ? 1u : 0u);
                     if (p.gate_mma && !p.gate_merged) umma_bf16(tmem_base + p.gate_col, da + adv, dg + adv, idesc_g, (ks | kk) ? 1u : 0u);
                 }
-                if (stage % p.group == p.group - 1) umma_commit(bar_empty + 8 * (stage / p.group));
+                if ((stage & gmask) == gmask) umma_commit(bar_empty + 8 * (stage >> gshift));
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
             }
             if (ok) umma_commit(bar_tfull);
