@@ -42,6 +42,8 @@ combine_kernel(const float* __restrict__ y_perm, const int32_t* __restrict__ inv
                const float* __restrict__ y_shared, const float* __restrict__ shared_gate,
                const bf16* residual, int T, int H, int k, bf16* out)
 {
+    pdl_wait();
+    pdl_launch_dependents();
     const int hv = H >> 3;
     const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (gid >= (long long)T * hv) return;
@@ -72,6 +74,8 @@ rmsnorm_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ tenant_id
                int n_tenants, const int32_t* __restrict__ model_of_tenant, const ModelWeights* __restrict__ models,
                bf16* __restrict__ xn)
 {
+    pdl_wait();
+    pdl_launch_dependents();
     const int t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (t >= T) return;
     int u = tenant_id[t];
@@ -107,7 +111,7 @@ cudaError_t launch_combine(moe_ctx* c, const float* y_perm, const int32_t* inv_p
     const moe_config& g = c->cfg;
     const long long n = (long long)T * (g.hidden >> 3);
     const int blocks = (int)((n + 255) / 256);
-    combine_kernel<<<blocks, 256, 0, st>>>(y_perm, inv_perm, topk_w, y_shared, shared_gate, residual, T, g.hidden,
+    launch_pdl(combine_kernel, dim3(blocks), dim3(256), 0, st, y_perm, inv_perm, topk_w, y_shared, shared_gate, residual, T, g.hidden,
                                            g.top_k, out);
     c->launches += 1;
     return cudaGetLastError();
@@ -118,7 +122,7 @@ cudaError_t launch_rmsnorm(moe_ctx* c, int layer, const bf16* x, const int32_t* 
 {
     const moe_config& g = c->cfg;
     const int blocks = (T * 32 + 255) / 256;
-    rmsnorm_kernel<<<blocks, 256, 0, st>>>(x, tenant_id, T, g.hidden, g.rms_eps, g.n_tenants, c->d_model_of_tenant,
+    launch_pdl(rmsnorm_kernel, dim3(blocks), dim3(256), 0, st, x, tenant_id, T, g.hidden, g.rms_eps, g.n_tenants, c->d_model_of_tenant,
                                            c->d_models + (size_t)layer * g.n_models, xn);
     c->launches += 1;
     return cudaGetLastError();

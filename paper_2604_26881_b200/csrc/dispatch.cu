@@ -104,6 +104,8 @@ dispatch_count_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
     __shared__ int32_t s_part[33];
     __shared__ int32_t s_count[2];
     __shared__ int s_last;
+    pdl_wait();
+    pdl_launch_dependents();
     const int tid = threadIdx.x, nth = blockDim.x, lane = tid & 31, warp = tid >> 5;
     // every thread looks up the bin of one row of the chunk (the lookups are chains of dependent loads: all of them
     // in flight at once), then one warp walks the bins in row order out of shared memory
@@ -174,6 +176,8 @@ dispatch_place_kernel(int R, int k, int nbins, const int32_t* __restrict__ block
                       int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, const bf16* __restrict__ x,
                       bf16* __restrict__ x_perm, int H)
 {
+    pdl_wait();
+    pdl_launch_dependents();
     const int gtid = blockIdx.x * blockDim.x + threadIdx.x;
     const int r = GATHER ? gtid >> 5 : gtid;
     if (r >= R) return;
@@ -208,6 +212,8 @@ dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
     extern __shared__ int32_t s_tot[];       // [nbins], then the plan's scratch, then the bin of every row (u16)
     __shared__ int32_t s_part[33];
     __shared__ int32_t s_count[2];
+    pdl_wait();
+    pdl_launch_dependents();
     const int tid = threadIdx.x, nth = blockDim.x;
     unsigned short* s_bin = reinterpret_cast<unsigned short*>(s_tot + nbins + plan_ints);
     for (int b = tid; b < nbins; b += nth) s_tot[b] = 0;
@@ -376,7 +382,7 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
         const size_t smem_small = smem + plan_ints * sizeof(int32_t) + (((size_t)R * 2 + 15) & ~(size_t)15);
         if (smem_small > 48 * 1024)
             cudaFuncSetAttribute(dispatch_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_small);
-        dispatch_small_kernel<<<1, threads, smem_small, st>>>(
+        launch_pdl(dispatch_small_kernel, dim3(1), dim3(threads), smem_small, st,
             topk_idx, tenant_id, R, k, bm, nbins, g.n_experts, g.n_models, G, g.n_tenants, perm, inv_perm,
             tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, x, gather_inside ? x_perm : nullptr,
             g.hidden, do_plan ? 1 : 0, (int)plan_ints, pa);
@@ -396,16 +402,16 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
     const size_t smem_count = smem + plan_ints * sizeof(int32_t);
     if (smem_count > 48 * 1024)
         cudaFuncSetAttribute(dispatch_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_count);
-    dispatch_count_kernel<<<nblk, kCountThreads, smem_count, st>>>(
+    launch_pdl(dispatch_count_kernel, dim3(nblk), dim3(kCountThreads), smem_count, st,
         topk_idx, tenant_id, nblk, nbins, R, k, g.n_experts, g.n_models, G, g.n_tenants, bm, c->ws.block_cnt, c->ws.bin_off,
         inv_perm, tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, c->ws.dispatch_done,
         do_plan ? 1 : 0, pa);
     if (plan_done) *plan_done = do_plan;
     if (x_perm)
-        dispatch_place_kernel<true><<<(R * 32 + 255) / 256, 256, 0, st>>>(R, k, nbins, c->ws.block_cnt, c->ws.bin_off, perm,
+        launch_pdl(dispatch_place_kernel<true>, dim3((R * 32 + 255) / 256), dim3(256), 0, st, R, k, nbins, c->ws.block_cnt, c->ws.bin_off, perm,
                                                                           inv_perm, x, x_perm, g.hidden);
     else
-        dispatch_place_kernel<false><<<(R + 255) / 256, 256, 0, st>>>(R, k, nbins, c->ws.block_cnt, c->ws.bin_off, perm,
+        launch_pdl(dispatch_place_kernel<false>, dim3((R + 255) / 256), dim3(256), 0, st, R, k, nbins, c->ws.block_cnt, c->ws.bin_off, perm,
                                                                       inv_perm, nullptr, nullptr, g.hidden);
     c->launches += 2;
     return cudaGetLastError();

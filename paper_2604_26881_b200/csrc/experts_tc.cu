@@ -274,8 +274,6 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
     const bool leader = rank == 0;
-    const int n_units = *p.n_units;
-    const int n_shared = *p.n_shared;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
@@ -307,6 +305,10 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     if (PAIR) cluster_sync_all();          // the peer's barriers are initialised before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
+    pdl_wait();                            // set-up above overlaps the previous kernel; its results are read from here on
+    pdl_launch_dependents();
+    const int n_units = *p.n_units;
+    const int n_shared = *p.n_shared;
 
     // Units are pulled from a global counter by one scheduler lane per CTA (pair: per CTA pair, the leader's),
     // decoded, and handed to the other roles through a small queue in shared memory; in pair mode the scheduler
@@ -943,19 +945,20 @@ cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, c
         attr_set = true;
     }
     if (!PAIR) {
-        kern<<<c->sm_count, kThreads, kSmemBytes, st>>>(p, maps);
-        return cudaGetLastError();
+        return launch_pdl(kern, dim3(c->sm_count), dim3(kThreads), kSmemBytes, st, p, maps);
     }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     if (c->tmaps->max_clusters < 0) {
         // a persistent kernel must not launch more clusters than can be resident at once
         cfg.gridDim = dim3((unsigned)(c->sm_count & ~1));

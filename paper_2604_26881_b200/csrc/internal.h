@@ -142,6 +142,27 @@ static inline void stage_mark(moe_ctx* c, cudaStream_t st, int i)
 
 namespace faasmoe {
 
+// Programmatic dependent launch: the kernels of a layer pass are launched so that each may be set up (block
+// scheduling, barrier initialisation, TMEM allocation) while its predecessor in the stream is still running.  Every
+// such kernel calls pdl_wait() before it reads anything a predecessor wrote, and every block passes through it
+// before it exits, so completion of a kernel implies completion of all earlier ones.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg;
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+#endif
+
 // --- launchers (each returns a cudaError_t from the launch) -------------------------------
 
 cudaError_t launch_route(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,

@@ -13,6 +13,8 @@ plan_kernel(const int32_t* __restrict__ expert_off, PlanArgs a)
 {
     extern __shared__ int32_t s_mem[];
     __shared__ int32_t s_warp[33];
+    pdl_wait();
+    pdl_launch_dependents();
     plan_body(expert_off, a, s_mem, s_warp);
 }
 
@@ -63,7 +65,7 @@ size_t plan_smem_ints(const moe_ctx* c, int G)
 cudaError_t launch_plan(moe_ctx* c, const int32_t* expert_off, int T, int G, bool with_shared, cudaStream_t st)
 {
     const PlanArgs a = make_plan_args(c, T, G, with_shared);
-    plan_kernel<<<1, 512, plan_smem_ints(c, G) * sizeof(int32_t), st>>>(expert_off, a);
+    launch_pdl(plan_kernel, dim3(1), dim3(512), plan_smem_ints(c, G) * sizeof(int32_t), st, expert_off, a);
     c->launches += 1;
     return cudaGetLastError();
 }

@@ -100,6 +100,8 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
+    pdl_wait();                     // set-up above overlaps the previous kernel; its results are read from here on
+    pdl_launch_dependents();
 
     if (warp == 0 || warp >= 6) {
         // three producer lanes (tokens / routers / gates) in three warps, so that the TMA instructions of one stage
@@ -375,7 +377,7 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     // the gate rows follow the router rows in shared memory (b_bytes has no padding: Epad is a multiple of 16)
     p.gate_merged = (p.gate_mma && M * (epad + 16) <= kRMaxN && p.b_bytes == M * epad * kRBK * 2) ? 1 : 0;
     p.gate_col = p.gate_merged ? M * epad : kRMaxN;
-    route_tc_kernel<<<(T + kRTokens - 1) / kRTokens, kRThreads, kRSmemBytes, st>>>(p, mp);
+    launch_pdl(route_tc_kernel, dim3((T + kRTokens - 1) / kRTokens), dim3(kRThreads), kRSmemBytes, st, p, mp);
     c->launches += 1;
     return cudaGetLastError();
 }
