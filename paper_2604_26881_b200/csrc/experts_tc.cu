@@ -5,19 +5,20 @@
 // (paper Sec. 3: an expert block computes on the tokens assigned to it; only activated experts are
 // touched.)
 //
-// Orientation: the weight rows are the M operand of the MMA (128 rows per CTA), the tokens of one
-// expert tile are the N operand (16..256, a multiple of 16).  A decode-sized tile therefore streams
-// each weight byte once through a narrow MMA, and a prefill tile pads a ragged expert segment to 16
-// rows, not to 128.  For gate/up the 128 weight rows of a tile are 64 gate rows interleaved with
-// the 64 up rows of the same intermediate indices (a 3-D TMA box over the two weight arrays puts
-// them on neighbouring TMEM lanes), so SwiGLU needs one lane-pair shuffle and one accumulator.
-//
-// Two launch shapes of the same kernel:
-//   single (PAIR = false): one CTA per unit, units handed out through an atomic counter (longest
-//     units first), used when tiles are short (decode, many small experts);
-//   pair (PAIR = true): a cluster of two CTAs shares the token tile of a unit through
-//     tcgen05.mma.cta_group::2 -- each CTA loads half of the tokens and its own 128 weight rows, so
-//     the bytes fetched per FLOP drop by a third; used when tiles are long (prefill).
+// Three shapes of the same kernel (all give bit-identical results: every output element is accumulated over K
+// in the same order):
+//   token-major (SWAP): one CTA per unit; the tokens of an expert tile (at most 128) are the M operand, one
+//     TMEM lane per token, and 256 weight rows the N operand (128 or 64 for the narrow units of the plan).
+//     For gate/up a 3-D TMA box over the two weight arrays interleaves gate and up rows, which land on
+//     neighbouring TMEM columns of a token's lane: SwiGLU needs no cross-lane traffic.  This is the
+//     weight-streaming shape: every batch below 2048 tokens per tenant model (decode, pools of many small
+//     experts).  One MMA covers 256 weight rows, and an MMA costs its issuing lane about 100 cycles whatever
+//     its width, so few tokens are bound by HBM, not by MMA issue.
+//   pair (PAIR): a cluster of two CTAs works on one unit through tcgen05.mma.cta_group::2; the weight rows
+//     are the M operand (128 per CTA), the tokens N: up to 512 per unit in two 256-column accumulators fed from
+//     the same weight tile, each CTA loading half of the tokens.  Used when tiles are long (prefill).
+//   weight-major, one CTA (neither flag): 128 weight rows as M, at most 128 tokens as N; kept as the A/B
+//     reference of the other two.
 // Routed-expert units and shared-expert units ride in the same launch.
 #include <cuda_fp16.h>
 
