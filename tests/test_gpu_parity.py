@@ -77,6 +77,18 @@ def test_small_batches_token_major_units(qwen_weights, T):
     run_and_compare(wl, wts, x, tenant, mot, wl.G, B.MOE_PATH_AUTO)
 
 
+@pytest.mark.parametrize("T", [2048, 2600])
+def test_pair_shape_at_another_layer_shape(T):
+    # the 2-CTA shape (512-row tiles, short units with two K slices per stage, shared units dealt out between the
+    # routed ones) away from the Qwen sizes: 8 K steps, skewed loads from an empty expert to several tiles, every
+    # element against the oracle
+    wl = W.MoEWorkload("pair-small", T=T, H=512, E=8, I=256, k=2, Is=512, M=1, n_tenants=3, G=3,
+                       zipf_bias=True, tenant_layout="uniform")
+    wts = W.make_weights(wl, seed=21)
+    x, tenant, mot = W.make_tokens(wl, seed=21)
+    run_and_compare(wl, wts, x, tenant, mot, wl.G, B.MOE_PATH_AUTO)
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_prefill_reduced(qwen_weights, path):
     # the prefill layer (Zipf-skewed router) on 300 tokens: every element against the oracle
