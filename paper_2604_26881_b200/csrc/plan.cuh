@@ -91,8 +91,21 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
     // experts of a block advance through the same weight-row block together.
     if (a.units1) {
         const int su1 = n_stiles * a.snblk1, su2 = n_stiles * a.snblk2;
-        for (int i = tid; i < su1; i += nth) { Unit u; u.colblock = i / n_stiles; u.tile = ~(i % n_stiles); a.units1[i] = u; }
-        for (int i = tid; i < su2; i += nth) { Unit u; u.colblock = i / n_stiles; u.tile = ~(i % n_stiles); a.units2[i] = u; }
+        // Token-major units: the colblock is (first weight row / 64) with a width code in the top byte (0: 256 weight
+        // rows, 1: 128, 2: 64); narrower units pack 2 or 4 K slices into a stage, so a unit of half the rows is half
+        // as long.  The shared expert's down projection contracts over 4x more elements than a routed expert's; with
+        // few tokens its units are made 4x (2x) narrower so that they are as long as the routed ones.
+        const int tm = a.token_major;
+        const int wsh = a.shared_down_width;
+        const int sh_step = wsh / 64, sh_code = wsh == 256 ? 0 : (wsh == 128 ? 1 : 2);
+        for (int i = tid; i < su1; i += nth) { Unit u; u.colblock = (i / n_stiles) * (tm ? 4 : 1); u.tile = ~(i % n_stiles); a.units1[i] = u; }
+        for (int i = tid; i < su2; i += nth) {
+            Unit u;
+            const int cb = i / n_stiles;
+            u.colblock = tm ? (cb * sh_step) | (sh_code << 24) : cb;
+            u.tile = ~(i % n_stiles);
+            a.units2[i] = u;
+        }
         const int nmax = n_tiles * max(a.nblk1, a.nblk2);
         for (int i = tid; i < nmax; i += nth) {
             const int tile = i % n_tiles, cb = i / n_tiles;
@@ -101,7 +114,7 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
             while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (s_group_tile0[mid] <= tile) lo = mid; else hi = mid; }
             // empty blocks share their first tile with the next one: step to the last of them
             const int t0 = s_group_tile0[lo], nt = s_group_tile0[lo + 1] - t0;
-            Unit u; u.colblock = cb; u.tile = tile;
+            Unit u; u.colblock = cb * (tm ? 4 : 1); u.tile = tile;
             if (cb < a.nblk1) a.units1[su1 + t0 * a.nblk1 + cb * nt + (tile - t0)] = u;
             if (cb < a.nblk2) a.units2[su2 + t0 * a.nblk2 + cb * nt + (tile - t0)] = u;
         }
@@ -116,23 +129,23 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
             a.plan_counts[7] = (reread && a.interleave_down) ? su2 : 0;
         }
         if (a.token_major) {
-            // Token-major units: the colblock becomes (first weight row / 64) with a width code in the top byte
-            // (0: 256 weight rows, 1: 128, 2: 64); narrower units pack 2 or 4 K slices into a stage, so a unit of
-            // half the rows is half as long.  Two uses:
-            //  - the shared expert's down projection contracts over 4x more elements than a routed expert's; with
-            //    few tokens its units are made 4x (2x) narrower so that they are as long as the routed ones;
-            //  - U equally long units on S CTAs take ceil(U / S) rounds; when the last round is less than half
-            //    full, its units are split in two (where the tile has at most 64 rows), so that round costs half.
+            // U equally long units on S CTAs take ceil(U / S) rounds; when the last round is less than half full, its
+            // units (the tail of the list: routed ones) are split into two units of half the weight rows each, where
+            // the tile has at most 64 rows, so that round costs half.
             __shared__ int s_split[128];
+            int r2[2];
             for (int l = 0; l < 2; ++l) {
-                Unit* list = l ? a.units2 : a.units1;
-                const int n_shared = l ? su2 : su1;
                 const int routed = n_tiles * (l ? a.nblk2 : a.nblk1);
-                const int total = n_shared + routed;
-                const int wsh = l ? a.shared_down_width : 256;
-                const int sh_step = wsh / 64, sh_code = wsh == 256 ? 0 : (wsh == 128 ? 1 : 2);
+                const int total = (l ? su2 : su1) + routed;
                 int r = total % a.n_ctas;
-                if (2 * r > a.n_ctas || r > routed || r > 128 || !a.split_ok[l]) r = 0;     // (the tail of a list is routed units)
+                if (2 * r > a.n_ctas || r > routed || r > 128 || !a.split_ok[l]) r = 0;
+                r2[l] = r;
+            }
+            for (int l = 0; l < 2; ++l) {
+                const int r = r2[l];
+                if (r == 0) continue;                                       // (the same decision in every thread)
+                Unit* list = l ? a.units2 : a.units1;
+                const int total = (l ? su2 : su1) + n_tiles * (l ? a.nblk2 : a.nblk1);
                 __syncthreads();                                            // the list is complete
                 Unit mine;
                 int cnt = 0;
@@ -142,22 +155,17 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
                     cnt = rows <= 64 ? 2 : 1;
                     s_split[tid] = cnt;
                 }
-                for (int i = tid; i < total - r; i += nth) {
-                    const int cb = list[i].colblock;
-                    list[i].colblock = i < n_shared ? (cb * sh_step) | (sh_code << 24) : cb * 4;
-                }
                 __syncthreads();
                 if (tid < r) {
                     int off = 0;
                     for (int j = 0; j < tid; ++j) off += s_split[j];
                     Unit u = mine;
                     if (cnt == 2) {
-                        u.colblock = (mine.colblock * 4) | (1 << 24);
+                        u.colblock = mine.colblock | (1 << 24);
                         list[total - r + off] = u;
-                        u.colblock = (mine.colblock * 4 + 2) | (1 << 24);
+                        u.colblock = (mine.colblock + 2) | (1 << 24);
                         list[total - r + off + 1] = u;
                     } else {
-                        u.colblock = mine.colblock * 4;
                         list[total - r + off] = u;
                     }
                 }
