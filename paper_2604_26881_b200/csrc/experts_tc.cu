@@ -434,25 +434,31 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 const uint32_t buf1 = buf ^ 1u, bphase1 = buf ? (bphase ^ 1u) : bphase;
                 const uint32_t d1 = tmem_base + buf1 * 256;
                 tc_fence_after();
+                // This lane is alone in its warp: every instruction of the loop below is paid in full, so whatever
+                // does not change inside a unit is worked out here, and the descriptors are put together from two
+                // 32-bit words (only the start-address field in the low word changes).
+                //   slice step of the M operand / of the N operand inside a stage, in 16-byte units:
+                const uint32_t m_step = (PAIR ? kABytes : (SWAP ? ui.npad * kBK * 2 : 0)) >> 4;
+                const uint32_t n_step = (PAIR ? (ui.npad >> 1) * kBK * 2 : (SWAP ? ui.width * kBK * 2 : 0)) >> 4;
+                //   pair shape, short unit: the token slices sit behind the two weight slices
+                const uint32_t n_base = PAIR ? ((ui.kb - 1) * kABytes) >> 4 : 0;
+                const uint32_t m_off = (SWAP ? kWBytes : 0) >> 4, n_off = (SWAP ? 0 : kWBytes) >> 4;
+                uint32_t acc = 0;                                 // the first MMA of a unit overwrites the accumulator
+                uint32_t acc1 = 0;
                 for (int ks = 0; ks < ui.ksteps; ++ks) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, &s_abort, p.status)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = smem_base + stage * stage_bytes, sb = sa + kWBytes;
-                    // M operand first: the weight tile, or the token tile in the token-major shape
-                    const uint64_t da = smem_desc_sw128(SWAP ? sb : sa), db = smem_desc_sw128(SWAP ? sa : sb);
+                    const uint32_t lo = smem_desc_lo(smem_base + stage * stage_bytes);
+                    uint32_t lo_m = lo + m_off, lo_n = lo + n_off + n_base;
                     for (int a = 0; a < ui.kb; ++a) {
-                        // (token-major: slice a of the stage; its token rows and weight rows follow those of slice a - 1)
-                        const uint64_t oa = (uint64_t)((a * ui.npad * kBK * 2) >> 4), ob = (uint64_t)((a * ui.width * kBK * 2) >> 4);
-                        // (pair shape, short unit: weight slice a, and the token slices behind the two weight slices)
-                        const uint64_t pa = (uint64_t)((a * kABytes) >> 4);
-                        const uint64_t pb = (uint64_t)((((ui.kb - 1) * kABytes) + a * (ui.npad >> 1) * kBK * 2) >> 4);
 #pragma unroll
                         for (int kk = 0; kk < kBK / 16; ++kk) {
-                            const uint32_t acc = (ks | a | kk) ? 1u : 0u;
-                            const uint64_t adv = (uint64_t)(kk * 32 >> 4);      // 16 elements = 32 bytes along K
-                            if (PAIR) umma_bf16_pair(d, da + pa + adv, db + pb + adv, idesc, acc);
-                            else umma_bf16(d, da + oa + adv, db + ob + adv, idesc, acc);
+                            // 16 elements = 32 bytes along K = 2 address units
+                            if (PAIR) umma_bf16_pair(d, smem_desc_pack(lo_m + 2 * kk), smem_desc_pack(lo_n + 2 * kk), idesc, acc);
+                            else umma_bf16(d, smem_desc_pack(lo_m + 2 * kk), smem_desc_pack(lo_n + 2 * kk), idesc, acc);
+                            acc = 1;
                         }
+                        lo_m += m_step; lo_n += n_step;
                     }
                     if (wide) {
                         if (ks == ui.ksteps - 1) umma_commit_pair(bar_tfull + 8 * buf);      // first half done: its epilogue may start
@@ -460,12 +466,11 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                             if (!mbar_wait_cluster(bar_tempty + 8 * buf1, bphase1 ^ 1, &s_abort, p.status)) { ok = false; break; }
                             tc_fence_after();
                         }
-                        const uint64_t db1 = smem_desc_sw128(sb + kBBytes);
+                        const uint32_t lo_m1 = lo + m_off, lo_n1 = lo + n_off + (kBBytes >> 4);
 #pragma unroll
                         for (int kk = 0; kk < kBK / 16; ++kk) {
-                            const uint32_t acc = (ks | kk) ? 1u : 0u;
-                            const uint64_t adv = (uint64_t)(kk * 32 >> 4);
-                            umma_bf16_pair(d1, da + adv, db1 + adv, idesc1, acc);
+                            umma_bf16_pair(d1, smem_desc_pack(lo_m1 + 2 * kk), smem_desc_pack(lo_n1 + 2 * kk), idesc1, acc1);
+                            acc1 = 1;
                         }
                     }
                     // frees the stage group (in both CTAs of a pair) when these MMAs have read it

@@ -167,6 +167,17 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
 }
 
 
+// The same descriptor in two 32-bit words, for loops that only move the start address: the low word holds the start
+// address field (offsets in 16-byte units can simply be added to it), the high word is constant.
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr) { return ((addr >> 4) & 0x3FFFu) | (1u << 16); }
+__device__ __forceinline__ uint64_t smem_desc_pack(uint32_t lo)
+{
+    constexpr uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
