@@ -146,16 +146,20 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_main >> 3) << 17) | ((128u >> 4) << 24);
             const uint32_t idesc_g = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_models * 16 >> 3) << 17) | ((128u >> 4) << 24);
             bool ok = true;
+            const uint32_t b_off = (uint32_t)p.a_bytes >> 4, g_off = (uint32_t)p.b_bytes >> 4;
+            const bool two_mmas = p.gate_mma && !p.gate_merged;
+            uint32_t acc = 0;                   // the first MMA overwrites the accumulators
             for (int ks = 0; ks < ksteps; ++ks) {
                 if (!mbar_wait(bar_full + 8 * stage, phase, &s_abort, p.status)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t sa = smem_base + stage * p.stage_bytes, sb = sa + p.a_bytes;
-                const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb), dg = smem_desc_sw128(sb + p.b_bytes);
+                // (this lane is alone in its warp and pays for every instruction: descriptors from 32-bit words)
+                const uint32_t lo_a = smem_desc_lo(smem_base + stage * p.stage_bytes);
+                const uint32_t lo_b = lo_a + b_off, lo_g = lo_b + g_off;
 #pragma unroll
                 for (int kk = 0; kk < kRBK / 16; ++kk) {
-                    const uint64_t adv = (uint64_t)(kk * 32 >> 4);
-                    umma_bf16(tmem_base, da + adv, db + adv, idesc, (ks | kk) ? 1u : 0u);
-                    if (p.gate_mma && !p.gate_merged) umma_bf16(tmem_base + p.gate_col, da + adv, dg + adv, idesc_g, (ks | kk) ? 1u : 0u);
+                    umma_bf16(tmem_base, smem_desc_pack(lo_a + 2 * kk), smem_desc_pack(lo_b + 2 * kk), idesc, acc);
+                    if (two_mmas) umma_bf16(tmem_base + p.gate_col, smem_desc_pack(lo_a + 2 * kk), smem_desc_pack(lo_g + 2 * kk), idesc_g, acc);
+                    acc = 1;
                 }
                 if ((stage & gmask) == gmask) umma_commit(bar_empty + 8 * (stage >> gshift));
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
