@@ -36,6 +36,9 @@ struct RouteParams {
     int gate_col;                  // first gate column: right after the router columns when one MMA covers both
     int gate_merged;               // 1: router rows and gate rows are one N operand (n_models * (Epad + 16) <= 256)
     int group;                     // stages handed back to the producer per commit (divides n_stages)
+    int kb;                        // slices of 64 K elements per stage (1, 2 or 4): a wait, a fence and a commit per stage
+                                   // cost the MMA lane as much as several of these narrow MMAs
+    int bg_bytes;                  // router rows + gate rows of one slice
     int a_bytes, b_bytes, stage_bytes, n_stages;   // pipeline geometry: small batches take more, smaller stages
     int32_t* topk_idx;
     float* topk_w;
@@ -80,7 +83,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t0 = blockIdx.x * kRTokens;
-    const int ksteps = p.H / kRBK;
+    const int ksteps = p.H / (kRBK * p.kb);        // stages to go through
     const int N = p.n_models * p.Epad;
 
     if (threadIdx.x == 0) {
@@ -116,19 +119,23 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
             for (int ks = 0; ks < ksteps; ++ks) {
                 if ((stage & gmask) == 0 &&
                     !mbar_wait(bar_empty + 8 * (stage >> gshift), phase ^ 1, &s_abort, p.status)) { ok = false; break; }
-                const uint32_t sa = smem_base + stage * p.stage_bytes, sb = sa + p.a_bytes;
+                // stage: kb token slices, then kb slices of (router rows, gate rows)
+                const uint32_t sa = smem_base + stage * p.stage_bytes, sb = sa + p.kb * p.a_bytes;
                 const uint32_t full = bar_full + 8 * stage;
                 armed |= 1u << stage;
                 armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
                 if (role == 0) {
-                    mbar_expect_tx(full, p.a_bytes + N * kRBK * 2 + (p.gate_mma ? p.n_models * 16 * kRBK * 2 : 0));
-                    tma_load_2d_hint(sa, &maps.x, full, ks * kRBK, t0, keep);
+                    mbar_expect_tx(full, p.kb * (p.a_bytes + N * kRBK * 2 + (p.gate_mma ? p.n_models * 16 * kRBK * 2 : 0)));
+                    for (int a = 0; a < p.kb; ++a) tma_load_2d_hint(sa + a * p.a_bytes, &maps.x, full, (ks * p.kb + a) * kRBK, t0, keep);
                 } else if (role == 1) {
-                    for (int m = 0; m < p.n_models; ++m)
-                        tma_load_2d_hint(sb + m * p.Epad * kRBK * 2, &maps.r[m], full, ks * kRBK, 0, keep);
+                    for (int a = 0; a < p.kb; ++a)
+                        for (int m = 0; m < p.n_models; ++m)
+                            tma_load_2d_hint(sb + a * p.bg_bytes + m * p.Epad * kRBK * 2, &maps.r[m], full, (ks * p.kb + a) * kRBK, 0, keep);
                 } else {
-                    for (int m = 0; m < p.n_models; ++m)
-                        tma_load_2d_hint(sb + p.b_bytes + m * 16 * kRBK * 2, &maps.g[m], full, ks * kRBK, 0, keep);
+                    for (int a = 0; a < p.kb; ++a)
+                        for (int m = 0; m < p.n_models; ++m)
+                            tma_load_2d_hint(sb + a * p.bg_bytes + p.b_bytes + m * 16 * kRBK * 2, &maps.g[m], full, (ks * p.kb + a) * kRBK, 0,
+                                             keep);
                 }
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
             }
@@ -146,20 +153,25 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_main >> 3) << 17) | ((128u >> 4) << 24);
             const uint32_t idesc_g = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_models * 16 >> 3) << 17) | ((128u >> 4) << 24);
             bool ok = true;
-            const uint32_t b_off = (uint32_t)p.a_bytes >> 4, g_off = (uint32_t)p.b_bytes >> 4;
+            const uint32_t a_step = (uint32_t)p.a_bytes >> 4, bg_step = (uint32_t)p.bg_bytes >> 4;
+            const uint32_t b_off = (uint32_t)(p.kb * p.a_bytes) >> 4, g_off = (uint32_t)p.b_bytes >> 4;
             const bool two_mmas = p.gate_mma && !p.gate_merged;
             uint32_t acc = 0;                   // the first MMA overwrites the accumulators
             for (int ks = 0; ks < ksteps; ++ks) {
                 if (!mbar_wait(bar_full + 8 * stage, phase, &s_abort, p.status)) { ok = false; break; }
                 tc_fence_after();
                 // (this lane is alone in its warp and pays for every instruction: descriptors from 32-bit words)
-                const uint32_t lo_a = smem_desc_lo(smem_base + stage * p.stage_bytes);
-                const uint32_t lo_b = lo_a + b_off, lo_g = lo_b + g_off;
+                uint32_t lo_a = smem_desc_lo(smem_base + stage * p.stage_bytes);
+                uint32_t lo_b = lo_a + b_off;
+                for (int a = 0; a < p.kb; ++a) {
+                    const uint32_t lo_g = lo_b + g_off;
 #pragma unroll
-                for (int kk = 0; kk < kRBK / 16; ++kk) {
-                    umma_bf16(tmem_base, smem_desc_pack(lo_a + 2 * kk), smem_desc_pack(lo_b + 2 * kk), idesc, acc);
-                    if (two_mmas) umma_bf16(tmem_base + p.gate_col, smem_desc_pack(lo_a + 2 * kk), smem_desc_pack(lo_g + 2 * kk), idesc_g, acc);
-                    acc = 1;
+                    for (int kk = 0; kk < kRBK / 16; ++kk) {
+                        umma_bf16(tmem_base, smem_desc_pack(lo_a + 2 * kk), smem_desc_pack(lo_b + 2 * kk), idesc, acc);
+                        if (two_mmas) umma_bf16(tmem_base + p.gate_col, smem_desc_pack(lo_a + 2 * kk), smem_desc_pack(lo_g + 2 * kk), idesc_g, acc);
+                        acc = 1;
+                    }
+                    lo_a += a_step; lo_b += bg_step;
                 }
                 if ((stage & gmask) == gmask) umma_commit(bar_empty + 8 * (stage >> gshift));
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
@@ -373,7 +385,12 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     p.status = c->ws.status;
     p.a_bytes = (a_rows * kRBK * 2 + 1023) & ~1023;
     p.b_bytes = (M * epad * kRBK * 2 + 1023) & ~1023;
-    p.stage_bytes = p.a_bytes + p.b_bytes + (p.gate_mma ? ((M * 16 * kRBK * 2 + 1023) & ~1023) : 0);
+    p.bg_bytes = p.b_bytes + (p.gate_mma ? ((M * 16 * kRBK * 2 + 1023) & ~1023) : 0);
+    const int slice_bytes = p.a_bytes + p.bg_bytes;
+    p.kb = 1;
+    for (int kb = 4; kb > 1; kb >>= 1)
+        if ((H / kRBK) % kb == 0 && kRTileBudget / (kb * slice_bytes) >= 3) { p.kb = kb; break; }
+    p.stage_bytes = p.kb * slice_bytes;
     p.n_stages = kRTileBudget / p.stage_bytes;
     if (p.n_stages > kRMaxStages) p.n_stages = kRMaxStages;
     p.group = p.n_stages >= 8 ? 4 : (p.n_stages >= 4 ? 2 : 1);
