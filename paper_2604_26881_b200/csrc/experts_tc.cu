@@ -11,12 +11,13 @@
 //     TMEM lane per token, and 256 weight rows the N operand (128 or 64 for the narrow units of the plan).
 //     For gate/up a 3-D TMA box over the two weight arrays interleaves gate and up rows, which land on
 //     neighbouring TMEM columns of a token's lane: SwiGLU needs no cross-lane traffic.  This is the
-//     weight-streaming shape: every batch below 2048 tokens per tenant model (decode, pools of many small
-//     experts).  One MMA covers 256 weight rows, and an MMA costs its issuing lane about 100 cycles whatever
+//     weight-streaming shape of small batches: up to 128 tokens (decode), where the routed units also read
+//     the tokens in place.  One MMA covers 256 weight rows, and an MMA costs its issuing lane about 100 cycles whatever
 //     its width, so few tokens are bound by HBM, not by MMA issue.
 //   pair (PAIR): a cluster of two CTAs works on one unit through tcgen05.mma.cta_group::2; the weight rows
 //     are the M operand (128 per CTA), the tokens N: up to 512 per unit in two 256-column accumulators fed from
-//     the same weight tile, each CTA loading half of the tokens.  Used when tiles are long (prefill).
+//     the same weight tile, each CTA loading half of the tokens; short units put two K slices into a stage.
+//     Used for every batch above 128 tokens.
 //   weight-major, one CTA (neither flag): 128 weight rows as M, at most 128 tokens as N; kept as the A/B
 //     reference of the other two.
 // Routed-expert units and shared-expert units ride in the same launch.
@@ -856,23 +857,19 @@ bool tc_pair_mode(const moe_ctx* c, int T)
 {
     const moe_config& g = c->cfg;
     (void)g;
-    // measured: the pair shape (with 512-row tiles) wins where the hot experts and the shared expert fill long tiles
-    // (prefill, 4096 tokens of one model); the 240-expert pool (~34 rows per expert) and the 24-block stack (~1100
-    // tokens) are faster with one-CTA token-major units.  2 forces the pair shape for every batch above 128 tokens.
-    if (c->pair_mode_enabled == 2) return T > 128;
-    return c->pair_mode_enabled != 0 && T / g.n_models >= 2048;
+    // measured (with 512-row tiles, two K slices per stage for the short units and the shared units dealt out between
+    // the routed ones): the pair shape wins for every batch above 128 tokens -- prefill, the 240-expert pool with ~34
+    // rows per expert, the 24-block stack, 256..2048 tokens of one model.  Up to 128 tokens the token-major shape
+    // reads the tokens in place.
+    return c->pair_mode_enabled != 0 && T > 128;
 }
 
-// Tiles of up to 512 rows pay when the segments are long enough to fill them: the weight tile of a K step then
-// feeds two accumulators, so a CTA fetches 48 KB instead of 64 KB per 512 tokens.  The price is a shallower
-// pipeline (4 stages) and an epilogue that is not hidden behind the next unit.
+// Tiles of up to 512 rows: the weight tile of a K step feeds two accumulators, so a CTA fetches 48 KB instead of
+// 64 KB per 512 tokens; the 48 KB stages also let a short unit put two K slices into a stage.  The price is a
+// shallower pipeline (4 stages) and, for full tiles, an epilogue that is not hidden behind the next unit.
 bool tc_wide_mode(const moe_ctx* c, int T)
 {
-    if (!tc_pair_mode(c, T) || c->wide_tiles_enabled == 0) return false;
-    if (c->wide_tiles_enabled == 2) return true;
-    // measured: pays from about 2048 tokens per tenant model (shared-expert tiles and the hot routed experts
-    // fill 512 rows); below that the units are short and want the deeper pipeline
-    return T / c->cfg.n_models >= 2048;
+    return tc_pair_mode(c, T) && c->wide_tiles_enabled != 0;
 }
 
 // One-CTA units with the tokens as the M operand: every batch that does not take the pair shape.
