@@ -64,9 +64,9 @@ enum {
  * FMA forces the CUDA-core kernels, TCGEN05 fails with MOE_ERR_UNSUPPORTED if not possible. */
 enum { MOE_PATH_AUTO = 0, MOE_PATH_FMA = 1, MOE_PATH_TCGEN05 = 2 };
 enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2,
-       MOE_OPT_PAIR_MODE = 3, /* 1 (default; 2 means the same): batches of more than 128 tokens use the 2-CTA tcgen05
-                                 shape; 0: never */
-       MOE_OPT_TOKEN_MAJOR = 5, /* 1 (default): batches outside the 2-CTA shape (at most 128 tokens) run their expert tiles with the tokens
+       MOE_OPT_PAIR_MODE = 3, /* 1 (default): batches of more than 64 tokens use the 2-CTA tcgen05 shape; 0: never;
+                                 2: every batch */
+       MOE_OPT_TOKEN_MAJOR = 5, /* 1 (default): batches outside the 2-CTA shape (at most 64 tokens) run their expert tiles with the tokens
                                    as the M operand of the MMA and the weight rows as N; 0: weight rows as M.  Results
                                    are bit-identical (the accumulation order over K is the same). */
        MOE_OPT_WIDE_TILES = 4 /* 1 (default; 2 means the same): the 2-CTA shape uses expert tiles of up to 512 rows whose

@@ -11,13 +11,13 @@
 //     TMEM lane per token, and 256 weight rows the N operand (128 or 64 for the narrow units of the plan).
 //     For gate/up a 3-D TMA box over the two weight arrays interleaves gate and up rows, which land on
 //     neighbouring TMEM columns of a token's lane: SwiGLU needs no cross-lane traffic.  This is the
-//     weight-streaming shape of small batches: up to 128 tokens (decode), where the routed units also read
+//     weight-streaming shape of small batches: up to 64 tokens (decode), where the routed units also read
 //     the tokens in place.  One MMA covers 256 weight rows, and an MMA costs its issuing lane about 100 cycles whatever
 //     its width, so few tokens are bound by HBM, not by MMA issue.
 //   pair (PAIR): a cluster of two CTAs works on one unit through tcgen05.mma.cta_group::2; the weight rows
 //     are the M operand (128 per CTA), the tokens N: up to 512 per unit in two 256-column accumulators fed from
 //     the same weight tile, each CTA loading half of the tokens; short units put two K slices into a stage.
-//     Used for every batch above 128 tokens.
+//     Used for every batch above 64 tokens.
 //   weight-major, one CTA (neither flag): 128 weight rows as M, at most 128 tokens as N; kept as the A/B
 //     reference of the other two.
 // Routed-expert units and shared-expert units ride in the same launch.
@@ -858,10 +858,11 @@ bool tc_pair_mode(const moe_ctx* c, int T)
     const moe_config& g = c->cfg;
     (void)g;
     // measured (with 512-row tiles, two K slices per stage for the short units and the shared units dealt out between
-    // the routed ones): the pair shape wins for every batch above 128 tokens -- prefill, the 240-expert pool with ~34
-    // rows per expert, the 24-block stack, 256..2048 tokens of one model.  Up to 128 tokens the token-major shape
-    // reads the tokens in place.
-    return c->pair_mode_enabled != 0 && T > 128;
+    // the routed ones): the pair shape wins for every batch above 64 tokens -- prefill, the 240-expert pool with ~34
+    // rows per expert, the 24-block stack, 96..2048 tokens of one model.  Up to 64 tokens the token-major shape, which
+    // reads the tokens in place and needs no permuted copy, is faster (189.8 against 196.9 us at 32 tokens).
+    if (c->pair_mode_enabled == 2) return true;        // (for measurements: the pair shape whatever the batch size)
+    return c->pair_mode_enabled != 0 && T > 64;
 }
 
 // Tiles of up to 512 rows: the weight tile of a K step feeds two accumulators, so a CTA fetches 48 KB instead of
