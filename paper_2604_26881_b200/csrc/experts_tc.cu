@@ -49,14 +49,15 @@ constexpr int kNumBars = 2 * kMaxStages + 4 + 2 * kQueue + 1;
 constexpr int kBarBytes = 256;                 // >= 8 * kNumBars, keeps the staging area 128-byte aligned
 // Output staging of the epilogue: results go to shared memory and leave as bulk copies of one row each,
 // so that the epilogue warps never wait on the global store path (which the operand loads saturate).
-// The two groups of four epilogue warps own one half each.
+// Each group of four epilogue warps owns a quarter of it.
 constexpr int kOutStageBytes = 32768;
-constexpr int kOutGroupBytes = kOutStageBytes / 2;
+constexpr int kEpiGroups = 4;                  // groups of four epilogue warps (one warp per TMEM lane quarter)
+constexpr int kOutGroupBytes = kOutStageBytes / kEpiGroups;
 constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + kBarBytes + kOutStageBytes;
 static_assert(8 * kNumBars <= kBarBytes, "barrier area too small");
-constexpr int kEpiWarps = 8;                   // two warps per TMEM lane quarter, alternating 16-column chunks
-constexpr int kSchedWarp = 2 + kEpiWarps;      // warp 0: TMA (weights), warp 1: MMA + TMEM, warps 2..9: epilogue, warp 10: scheduler,
-constexpr int kTokWarp = kSchedWarp + 1;       // warp 11: TMA (tokens)
+constexpr int kEpiWarps = 4 * kEpiGroups;      // four warps per TMEM lane quarter, taking the 16-column chunks in turn
+constexpr int kSchedWarp = 2 + kEpiWarps;      // warp 0: TMA (weights), warp 1: MMA + TMEM, warps 2..17: epilogue, warp 18: scheduler,
+constexpr int kTokWarp = kSchedWarp + 1;       // warp 19: TMA (tokens)
 constexpr int kThreads = 32 * (kTokWarp + 1);
 constexpr int kClaimAhead = 8;                 // the next unit is claimed this many K steps before the current one is loaded
 constexpr uint32_t kTmemCols = 512;            // 2 accumulator buffers x 256 columns
@@ -495,13 +496,12 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
         // ---------------- epilogue: two groups of four warps (one warp per TMEM lane quarter), ----------------
         // ---------------- the groups alternate over the 16-column chunks of an accumulator     ----------------
         const int quarter = warp & 3;
-        const int half = (warp - 2) >> 2;                  // group: 0 or 1
+        const int half = (warp - 2) >> 2;                  // group: 0 .. kEpiGroups - 1
         const int gbar = 1 + half;                         // named barrier of the group
         const int gtid = quarter * 32 + lane;              // thread index inside the group
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const uint32_t stg = bars + kBarBytes + half * kOutGroupBytes;      // this group's staging area
         uint32_t buf = 0, bphase = 0, q = 0, qphase = 0;
-        uint32_t rnd = 0;                                  // MODE 1: staging slot = rnd & 1
         bool ok = true;
         const uint32_t tempty_leader = PAIR ? map_to_cta(bar_tempty, 0) : bar_tempty;
         while (ok) {
@@ -527,9 +527,9 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 const uint32_t d = tmem_base + lane_addr + buf * 256;
                 if (SWAP) {
                     // Token-major accumulator: this thread's TMEM lane is token `gtid` of the tile, the columns are the
-                    // unit's weight rows (256, 128 or 64); each group takes half of them.  Every thread stages and sends
-                    // only its own token's outputs, so the group needs no barrier.
-                    const int gcols = ui.width >> 1;          // columns of this group
+                    // unit's weight rows (256, 128 or 64); each group takes a quarter of them.  Every thread stages and
+                    // sends only its own token's outputs (a 64-byte slot), so the group needs no barrier.
+                    const int gcols = ui.width / kEpiGroups;  // columns of this group: 64, 32 or 16
                     const int c_first = half * gcols;
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
@@ -546,7 +546,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     if (MODE == 0) {
                         // columns 2i / 2i+1 hold the gate / up row (or up / gate) of intermediate index cb*32 + i
                         const uint32_t gf = ui.shared ? (p.gate_first_shared >> ui.model) & 1u : p.gate_first_routed & 1u;
-                        const uint32_t mine = stg + (uint32_t)gtid * 128u;       // up to 64 outputs of 16 bits
+                        const uint32_t mine = stg + (uint32_t)gtid * 64u;        // up to 32 outputs of 16 bits
                         bulk_wait_read<0>();                                     // the row sent for the previous tile has left
 #pragma unroll 2
                         for (int i = 0; i < (gcols >> 4); ++i) {
@@ -579,13 +579,13 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                         }
                         bulk_commit();
                     } else {
-                        // fp32 outputs, 16 at a time through one of this thread's two 64-byte slots
+                        // fp32 outputs, 16 at a time through this thread's 64-byte slot
                         if (drow >= 0 && ui.shared && p.shared_dst_rows != nullptr) drow = p.shared_dst_rows[drow];
                         float* outp = reinterpret_cast<float*>(ui.shared ? p.out_shared : p.out_routed) + ui.cb * 64 + c_first;
                         const int nchunk = gcols >> 4;
-                        for (int i = 0; i < nchunk; ++i, ++rnd) {
-                            const uint32_t slot = stg + (uint32_t)gtid * 128u + (rnd & 1u) * 64u;
-                            bulk_wait_read<1>();
+                        const uint32_t slot = stg + (uint32_t)gtid * 64u;
+                        for (int i = 0; i < nchunk; ++i) {
+                            bulk_wait_read<0>();
                             uint32_t r[16];
                             tmem_ld16(d + c_first + i * 16, r);
                             tmem_ld_wait();
@@ -612,7 +612,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     const bool even = (lane & 1) == 0;
                     const bool own_is_gate = even == ((p.gate_first_routed & 1u) != 0);
                     const int col = ui.cb * 64 + quarter * 16 + (lane >> 1);
-                    for (int j = half; j < nrows; j += 2) {
+                    for (int j = half; j < nrows; j += kEpiGroups) {
                         const int tok = p.perm[row0 + j] / p.top_k;            // warp-uniform
                         uint32_t r;
                         tmem_ld1(d + tok, r);
@@ -629,7 +629,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
                 } else if (MODE == 0) {
-                    // The group's staging area holds its 8 chunks of 16 tokens as rows of 64 outputs (128 bytes).
+                    // The group's staging area holds its 4 chunks of 16 tokens as rows of 64 outputs (128 bytes).
                     // Its previous contents must have left (every thread waits for the rows it sent itself), and the
                     // whole group takes one decision on the accumulator wait.
                     bulk_wait_read<0>();
@@ -642,7 +642,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     // lanes 2i / 2i+1 hold the gate / up row (or up / gate) of intermediate index cb*64 + quarter*16 + i
                     const uint32_t my_col = stg + (uint32_t)(quarter * 32 + (lane >> 1) * 2);
                     int i = 0;
-                    for (int c0 = half * 16; c0 < npad; c0 += 32, ++i) {
+                    for (int c0 = half * 16; c0 < npad; c0 += 16 * kEpiGroups, ++i) {
                         uint32_t r[16];
                         tmem_ld16(d + c0, r);
                         tmem_ld_wait();
@@ -668,23 +668,23 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     }
                     fence_async_smem();
                     group_sync(gbar);
-                    // thread t of the group sends staged row t: token (t / 16) * 32 + half * 16 + t % 16
+                    // thread t < 64 of the group sends staged row t: token (t / 16) * 64 + group * 16 + t % 16
                     {
-                        const int n = (gtid >> 4) * 32 + half * 16 + (gtid & 15);
-                        if (n < nrows) {
+                        const int n = (gtid >> 4) * (16 * kEpiGroups) + half * 16 + (gtid & 15);
+                        if (gtid < 64 && n < nrows) {
                             unsigned short* out16 = reinterpret_cast<unsigned short*>(ui.shared ? p.out_shared : p.out_routed);
                             bulk_store(out16 + (size_t)(row0 + n) * ld + ui.cb * 64, stg + (uint32_t)gtid * 128u, 128u);
                         }
                         bulk_commit();
                     }
                 } else {
-                    // fp32 rows of 128 outputs (512 bytes); a chunk of 16 tokens fills one of the group's two slots
+                    // fp32 rows of 128 outputs (512 bytes); a chunk of 16 tokens fills the group's staging area
                     const bool remap = ui.shared && p.shared_dst_rows != nullptr;
                     float* outp = reinterpret_cast<float*>(ui.shared ? p.out_shared : p.out_routed) + ui.cb * 128;
                     bool first = true;
-                    for (int c0 = half * 16; c0 < npad; c0 += 32, ++rnd) {
-                        const uint32_t slot = stg + (rnd & 1u) * 8192u;
-                        bulk_wait_read<1>();                       // the rows this thread sent from this slot have left
+                    const uint32_t slot = stg;
+                    for (int c0 = half * 16; c0 < npad; c0 += 16 * kEpiGroups) {
+                        bulk_wait_read<0>();                       // the rows this thread sent from the area have left
                         if (first) {
                             ok = group_and(gbar, ok);
                             if (!ok) break;
@@ -699,7 +699,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                         const uint32_t a = slot + (uint32_t)(quarter * 128 + lane * 4);
 #pragma unroll
                         for (int j = 0; j < 16; ++j) asm volatile("st.shared.b32 [%0], %1;" ::"r"(a + j * 512u), "r"(r[j]) : "memory");
-                        if (c0 + 32 >= npad) {
+                        if (c0 + 16 * kEpiGroups >= npad) {
                             // last chunk of this group: the accumulator has been read
                             tc_fence_before();
                             __syncwarp();
@@ -721,7 +721,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     }
                     if (!ok) break;
                     if (first) {
-                        // no chunk for this group (a tile of at most 16 columns): only release the accumulator
+                        // no chunk for this group (a tile with few columns): only release the accumulator
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) break;
                         if (lane == 0) {
