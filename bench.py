@@ -128,7 +128,7 @@ def algorithmic_work(wl, active_experts: int, T: int):
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
 # ncu captures summarised in profiles/grouped_gemm_decode_ncu.md and profiles/grouped_gemm_prefill_ncu.md; None where
 # no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"decode": 657.659136e6 + 4.009728e6, "prefill": 859.891712e6 + 87.351808e6}
+NCU_TRAFFIC_BYTES = {"decode": 657.657600e6 + 3.586304e6, "prefill": 858.381312e6 + 84.442624e6}
 
 
 def run_reference(args, wl, rank):
