@@ -69,9 +69,15 @@ enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2,
        MOE_OPT_TOKEN_MAJOR = 5, /* 1 (default): batches outside the 2-CTA shape (at most 64 tokens) run their expert tiles with the tokens
                                    as the M operand of the MMA and the weight rows as N; 0: weight rows as M.  Results
                                    are bit-identical (the accumulation order over K is the same). */
-       MOE_OPT_WIDE_TILES = 4 /* 1 (default; 2 means the same): the 2-CTA shape uses expert tiles of up to 512 rows whose
+       MOE_OPT_WIDE_TILES = 4, /* 1 (default; 2 means the same): the 2-CTA shape uses expert tiles of up to 512 rows whose
                                  two 256-column accumulators are fed from one weight tile; 0: tiles of at most 256
-                                 rows.  Results are bit-identical either way. */ };
+                                 rows.  Results are bit-identical either way. */
+       MOE_OPT_EARLY_SHARED = 6, /* one model with a shared expert, moe_layer_forward and the calls built on it: the
+                                    shared expert's two launches go to a second stream of the context, beside the
+                                    router and the dispatch; the combine waits for both.  2 (default): every batch;
+                                    1: batches of at most 64 tokens; 0: never.  Results are bit-identical. */
+       MOE_OPT_EARLY_SHARED_SMS = 7 /* SMs that the shared expert's CTA pairs may hold while they run beside other
+                                       kernels (batches of more than 64 tokens; default: no limit) */ };
 
 typedef struct {
     int32_t hidden;        /* H */

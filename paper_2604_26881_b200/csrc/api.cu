@@ -57,6 +57,10 @@ int alloc_workspace(moe_ctx* c)
     A(&w.tok_perm, T); A(&w.tok_inv, T);
     A(&w.tiles, (size_t)c->max_tiles); A(&w.stiles, (size_t)c->max_stiles); A(&w.plan_counts, 8);
     A(&w.units1, (size_t)c->max_units1); A(&w.units2, (size_t)c->max_units2);
+    if (Is > 0 && g.n_models == 1) {
+        A(&w.stiles_sh, (size_t)c->max_stiles); A(&w.plan_counts_sh, 8);
+        A(&w.units1_sh, (size_t)c->max_stiles * snblk1); A(&w.units2_sh, (size_t)4 * c->max_stiles * nblk2);
+    }
     // activations: one extra tile of rows so that a whole-tile load never leaves the buffer
     A(&w.x_perm, (R + kTileRows) * H); A(&w.h, (R + kTileRows) * I); A(&w.y_perm, R * H);
     if (g.n_models > 1) A(&w.xs_perm, (T + kTileRows) * H);
@@ -77,6 +81,7 @@ int alloc_workspace(moe_ctx* c)
     cudaMemset(w.stats, 0, 4 * sizeof(int32_t));
     cudaMemset(w.dispatch_done, 0, sizeof(int32_t));
     cudaMemset(w.plan_counts, 0, 8 * sizeof(int32_t));
+    if (w.plan_counts_sh) cudaMemset(w.plan_counts_sh, 0, 8 * sizeof(int32_t));
     return MOE_OK;
 }
 
@@ -85,7 +90,8 @@ void free_workspace(moe_ctx* c)
     Workspace& w = c->ws;
     void* ptrs[] = {w.topk_idx, w.topk_w, w.shared_gate, w.tie_flag, w.perm, w.inv_perm, w.tenant_expert_count,
                     w.expert_off, w.group_off, w.block_cnt, w.bin_off, w.tok_block_cnt, w.model_tok_off, w.tok_perm,
-                    w.tok_inv, w.tiles, w.stiles, w.plan_counts, w.units1, w.units2, w.x_perm, w.xs_perm, w.h, w.hs,
+                    w.tok_inv, w.tiles, w.stiles, w.plan_counts, w.units1, w.units2, w.stiles_sh, w.plan_counts_sh, w.units1_sh,
+                    w.units2_sh, w.x_perm, w.xs_perm, w.h, w.hs,
                     w.y_perm, w.y_shared, w.xn, w.x_stage, w.tenant_stage, w.out_stage, w.status, w.stats, w.dispatch_done};
     for (void* p : ptrs) if (p) cudaFree(p);
     w = Workspace();
@@ -157,6 +163,20 @@ int layer_forward_impl(moe_ctx* c, int layer, const bf16* x, const int32_t* tena
     const moe_config& g = c->cfg;
     Workspace& w = c->ws;
     const bool shared = g.shared_inter > 0;
+    // One model: the shared expert's work does not depend on the routing.  Its two launches go to a second stream, where
+    // they run beside the router and the dispatch (HBM- or tensor-bound work beside latency-bound work); the combine
+    // waits for both streams.  Not while the stages are being timed one by one.
+    const bool early = shared && g.n_models == 1 && use_tc(c) && !c->timing && c->side != nullptr &&
+                       (c->early_shared_enabled == 2 || (c->early_shared_enabled == 1 && tc_token_major(c, T)));
+    if (early) {
+        const int rc = tc_setup_layer(c, layer);
+        if (rc != MOE_OK) return rc;
+        MOE_CUDA(c, cudaEventRecord(c->ev_fork, st));
+        MOE_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+        MOE_CUDA(c, launch_plan_shared(c, T, c->side));
+        MOE_CUDA(c, launch_experts_tc(c, layer, x, nullptr, nullptr, T, nullptr, w.y_shared, nullptr, c->side, true));
+        MOE_CUDA(c, cudaEventRecord(c->ev_join, c->side));
+    }
     stage_mark(c, st, kEvBegin);
     MOE_CUDA(c, launch_route(c, layer, x, tenant_id, T, w.topk_idx, w.topk_w, shared ? w.shared_gate : nullptr,
                              w.tie_flag, st));
@@ -165,11 +185,12 @@ int layer_forward_impl(moe_ctx* c, int layer, const bf16* x, const int32_t* tena
     const bool direct = use_tc(c) && tc_direct_mode(c, T);
     bool plan_done = false;
     MOE_CUDA(c, launch_dispatch(c, x, w.topk_idx, tenant_id, T, G, w.perm, w.inv_perm, w.tenant_expert_count,
-                                w.expert_off, w.group_off, direct ? nullptr : w.x_perm, st, true, shared, &plan_done));
+                                w.expert_off, w.group_off, direct ? nullptr : w.x_perm, st, true, shared && !early, &plan_done));
     stage_mark(c, st, kEvDispatch);
     const int rc = experts_impl(c, layer, x, w.x_perm, w.perm, w.expert_off, tenant_id, T, G, w.y_perm,
-                                shared ? w.y_shared : nullptr, st, plan_done);
+                                (shared && !early) ? w.y_shared : nullptr, st, plan_done);
     if (rc != MOE_OK) return rc;
+    if (early) MOE_CUDA(c, cudaStreamWaitEvent(st, c->ev_join, 0));
     MOE_CUDA(c, launch_combine(c, w.y_perm, w.inv_perm, w.topk_w, shared ? w.y_shared : nullptr,
                                shared ? w.shared_gate : nullptr, residual, T, out, st));
     stage_mark(c, st, kEvCombine);
@@ -208,6 +229,9 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->wide_tiles_enabled = 1;
     c->token_major_enabled = 1;
     c->timing = false;
+    c->early_shared_enabled = 2;
+    c->early_shared_sms = 1 << 20;      // no limit
+    c->side = nullptr; c->ev_fork = nullptr; c->ev_join = nullptr;
     for (auto& e : c->ev) e = nullptr;
     c->errbuf[0] = 0;
     c->d_models = nullptr; c->d_slot = nullptr; c->d_model_of_tenant = nullptr; c->d_tenant_local = nullptr;
@@ -238,6 +262,15 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     }
     if (rc == MOE_OK) rc = upload_tenant_tables(c);
     if (rc == MOE_OK) rc = alloc_workspace(c);
+    if (rc == MOE_OK && g.shared_inter > 0 && g.n_models == 1) {
+        e = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
+        if (e != cudaSuccess) {
+            snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "moe_create: %s", cudaGetErrorString(e));
+            rc = MOE_ERR_CUDA;
+        }
+    }
     if (rc != MOE_OK) {
         if (c->errbuf[0]) snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "%s", c->errbuf);
         moe_destroy(c);
@@ -255,6 +288,9 @@ int moe_destroy(moe_ctx* c)
     route_tc_destroy(c);
     free_workspace(c);
     for (auto& e : c->ev) if (e) cudaEventDestroy(e);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    if (c->side) cudaStreamDestroy(c->side);
     void* ptrs[] = {c->d_models, c->d_slot, c->d_model_of_tenant, c->d_tenant_local, c->d_bin_base,
                     c->d_tenants_in_model};
     for (void* p : ptrs) if (p) cudaFree(p);
@@ -331,6 +367,16 @@ int moe_set_option(moe_ctx* c, int option, int value)
     if (option == MOE_OPT_PAIR_MODE) {
         if (value < 0 || value > 2) return MOE_ERR_SHAPE;
         c->pair_mode_enabled = value;
+        return MOE_OK;
+    }
+    if (option == MOE_OPT_EARLY_SHARED) {
+        if (value < 0 || value > 2) return MOE_ERR_SHAPE;
+        c->early_shared_enabled = value;
+        return MOE_OK;
+    }
+    if (option == MOE_OPT_EARLY_SHARED_SMS) {
+        if (value < 2) return MOE_ERR_SHAPE;
+        c->early_shared_sms = value & ~1;
         return MOE_OK;
     }
     if (option == MOE_OPT_TOKEN_MAJOR) {

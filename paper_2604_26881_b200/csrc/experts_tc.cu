@@ -23,6 +23,7 @@
 // Routed-expert units and shared-expert units ride in the same launch.
 #include <cuda_fp16.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 
@@ -940,7 +941,7 @@ int tc_setup_layer(moe_ctx* c, int layer)
 namespace {
 
 template <int MODE, bool PAIR, bool SWAP>
-cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, cudaStream_t st)
+cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, cudaStream_t st, int grid_cap)
 {
     auto kern = grouped_gemm_kernel<MODE, PAIR, SWAP>;
     static bool attr_set = false;
@@ -949,7 +950,7 @@ cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, c
         attr_set = true;
     }
     if (!PAIR) {
-        return launch_pdl(kern, dim3(c->sm_count), dim3(kThreads), kSmemBytes, st, p, maps);
+        return launch_pdl(kern, dim3(std::max(1, std::min(c->sm_count, grid_cap))), dim3(kThreads), kSmemBytes, st, p, maps);
     }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -971,14 +972,15 @@ cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, c
         if (n > c->sm_count / 2) n = c->sm_count / 2;
         c->tmaps->max_clusters = n;
     }
-    cfg.gridDim = dim3((unsigned)(2 * c->tmaps->max_clusters));
+    cfg.gridDim = dim3((unsigned)(2 * std::max(1, std::min(c->tmaps->max_clusters, grid_cap / 2))));
     return cudaLaunchKernelEx(&cfg, kern, p, maps);
 }
 
 }  // namespace
 
 cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, const int32_t* perm, int T,
-                              float* y_perm, float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st)
+                              float* y_perm, float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st,
+                              bool shared_only)
 {
     const moe_config& g = c->cfg;
     LayerMaps& lm = c->tmaps->layers[layer];
@@ -988,7 +990,7 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     const bool pair = tc_pair_mode(c, T);
     const bool swap = tc_token_major(c, T);
     // direct mode: with few tokens the routed gate/up units read the tokens in place (no permuted copy)
-    const bool direct = tc_direct_mode(c, T) && perm != nullptr;
+    const bool direct = tc_direct_mode(c, T) && perm != nullptr && !shared_only;
     const uint32_t fmt_bf16 = (1u << 7) | (1u << 10), fmt_fp16 = 0u;
 
     // activation maps are rebuilt per call: their addresses and row counts are the call's
@@ -1000,10 +1002,10 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
         return good;
     };
     auto copy_b = [](CUtensorMap* dst, const CUtensorMap* src) { for (int bx = 0; bx < 4; ++bx) dst[bx] = src[bx]; };
-    if (!direct) ok = make_b(m1.b_routed, x_perm, R, H, false);
+    if (!direct && !shared_only) ok = make_b(m1.b_routed, x_perm, R, H, false);
     if (shared || direct) {
         ok = ok && make_b(m1.b_shared, x_or_xs, T, H, false);
-        if (direct) copy_b(m1.b_routed, m1.b_shared);
+        if (direct || shared_only) copy_b(m1.b_routed, m1.b_shared);
     } else {
         copy_b(m1.b_shared, m1.b_routed);
     }
@@ -1011,9 +1013,17 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
 
     GemmParams p1;
     memset(&p1, 0, sizeof(p1));
-    p1.units = c->ws.units1; p1.n_units = c->ws.plan_counts + 2; p1.counter = c->ws.plan_counts + 4;
-    p1.n_shared = c->ws.plan_counts + 6;
-    p1.tiles = c->ws.tiles; p1.stiles = c->ws.stiles;
+    // the shared expert alone runs from unit lists of its own (it may be in flight beside the routed launches)
+    int32_t* counts = shared_only ? c->ws.plan_counts_sh : c->ws.plan_counts;
+    p1.units = shared_only ? c->ws.units1_sh : c->ws.units1;
+    p1.n_units = counts + 2; p1.counter = counts + 4; p1.n_shared = counts + 6;
+    p1.tiles = c->ws.tiles; p1.stiles = shared_only ? c->ws.stiles_sh : c->ws.stiles;
+    int cap1 = c->sm_count, cap2 = c->sm_count;
+    if (shared_only) {
+        // its unit counts are known on the host; a CTA pair shape leaves some SMs to the kernels it runs beside
+        shared_unit_counts(c, T, &cap1, &cap2);
+        if (pair) { cap1 = std::min(2 * cap1, c->early_shared_sms); cap2 = std::min(2 * cap2, c->early_shared_sms); }
+    }
     p1.perm = perm; p1.top_k = g.top_k; p1.direct = direct ? 1 : 0; p1.n_tokens_pad = (T + 15) & ~15;
     p1.k_routed = H; p1.k_shared = H;
     p1.rows_per_slot = I; p1.cb_rows = swap ? 32 : 64;      // token-major: colblocks count steps of 64 weight rows
@@ -1026,29 +1036,31 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     p1.wide = tc_wide_mode(c, T) ? 1 : 0;
     p1.group = p1.wide ? 1 : 2;
     if (swap) p1.group = 1;
-    cudaError_t e = pair ? launch_gemm<0, true, false>(c, p1, m1, st)
-                         : (swap ? launch_gemm<0, false, true>(c, p1, m1, st) : launch_gemm<0, false, false>(c, p1, m1, st));
+    cudaError_t e = pair ? launch_gemm<0, true, false>(c, p1, m1, st, cap1)
+                         : (swap ? launch_gemm<0, false, true>(c, p1, m1, st, cap1)
+                                 : launch_gemm<0, false, false>(c, p1, m1, st, cap1));
     if (e != cudaSuccess) return e;
-    stage_mark(c, st, kEvGateUp);
+    if (!shared_only) stage_mark(c, st, kEvGateUp);
 
     GemmMaps& m2 = swap ? lm.m2t : lm.m2;
-    ok = make_b(m2.b_routed, c->ws.h, R, I, false);
+    ok = shared_only || make_b(m2.b_routed, c->ws.h, R, I, false);
     if (shared) ok = ok && make_b(m2.b_shared, c->ws.hs, T, Is, true);
     else copy_b(m2.b_shared, m2.b_routed);
+    if (shared_only) copy_b(m2.b_routed, m2.b_shared);
     if (!ok) return cudaErrorInvalidValue;
     GemmParams p2 = p1;
-    p2.units = c->ws.units2; p2.n_units = c->ws.plan_counts + 3; p2.counter = c->ws.plan_counts + 5;
-    p2.n_shared = c->ws.plan_counts + 7;
+    p2.units = shared_only ? c->ws.units2_sh : c->ws.units2;
+    p2.n_units = counts + 3; p2.counter = counts + 5; p2.n_shared = counts + 7;
     p2.direct = 0;
     p2.k_routed = I; p2.k_shared = Is;
     p2.rows_per_slot = H; p2.cb_rows = swap ? 64 : 128;
     p2.out_routed = y_perm; p2.out_shared = y_shared; p2.ld_routed = H; p2.ld_shared = H;
     p2.shared_dst_rows = shared_dst_rows;
     p2.idesc_fmt_routed = fmt_bf16; p2.idesc_fmt_shared = fmt_fp16;
-    e = pair ? launch_gemm<1, true, false>(c, p2, m2, st)
-             : (swap ? launch_gemm<1, false, true>(c, p2, m2, st) : launch_gemm<1, false, false>(c, p2, m2, st));
+    e = pair ? launch_gemm<1, true, false>(c, p2, m2, st, cap2)
+             : (swap ? launch_gemm<1, false, true>(c, p2, m2, st, cap2) : launch_gemm<1, false, false>(c, p2, m2, st, cap2));
     if (e != cudaSuccess) return e;
-    stage_mark(c, st, kEvDown);
+    if (!shared_only) stage_mark(c, st, kEvDown);
     c->launches += 2;
     return cudaGetLastError();
 }

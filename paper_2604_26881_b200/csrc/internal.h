@@ -80,6 +80,11 @@ struct Workspace {
     int32_t* plan_counts = nullptr;  // [8]: n_tiles, n_stiles, n_units1, n_units2
     Unit* units1 = nullptr;        // gate/up GEMM units (shared, then routed)
     Unit* units2 = nullptr;        // down GEMM units
+    // the same for the shared expert alone (one model), when it runs beside the router and the dispatch
+    Tile* stiles_sh = nullptr;
+    int32_t* plan_counts_sh = nullptr;  // [8]
+    Unit* units1_sh = nullptr;
+    Unit* units2_sh = nullptr;
     // activations
     bf16* x_perm = nullptr;        // [R,H]
     bf16* xs_perm = nullptr;       // [T,H] tokens grouped by model (M > 1 only)
@@ -127,6 +132,11 @@ struct moe_ctx {
     int pair_mode_enabled;        // allow the 2-CTA (cta_group::2) shape of the grouped GEMM for long tiles
     int token_major_enabled;      // one-CTA units take the tokens as the M operand of the MMA (up to 256 weight rows per tile)
     int wide_tiles_enabled;       // allow 512-row tiles (two accumulators per weight tile) in the 2-CTA shape
+    int early_shared_enabled;     // one model: run the shared expert on a second stream beside router and dispatch
+                                  // (1: batches of the token-major shape, 2: every batch)
+    int early_shared_sms;         // SMs the shared expert's CTA pairs may take while they run beside other kernels
+    cudaStream_t side;            // second stream of the layer pass
+    cudaEvent_t ev_fork, ev_join; // order between the caller's stream and the second one
     bool timing;                  // record an event after every stage (moe_layer_forward_timed)
     cudaEvent_t ev[8];
     char errbuf[256];
@@ -189,12 +199,16 @@ size_t plan_smem_ints(const moe_ctx* c, int G);
 
 // Builds the tile lists (and the unit lists of the tensor-core path) from expert_off.
 cudaError_t launch_plan(moe_ctx* c, const int32_t* expert_off, int T, int G, bool with_shared, cudaStream_t st);
+// unit lists of the shared expert alone (one model) and how many units they hold
+cudaError_t launch_plan_shared(moe_ctx* c, int T, cudaStream_t st);
+void shared_unit_counts(moe_ctx* c, int T, int* n_units1, int* n_units2);
 
 cudaError_t launch_experts_fma(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, int T, float* y_perm,
                                float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st);
 
 cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, const int32_t* perm, int T,
-                              float* y_perm, float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st);
+                              float* y_perm, float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st,
+                              bool shared_only = false);
 
 cudaError_t launch_combine(moe_ctx* c, const float* y_perm, const int32_t* inv_perm, const float* topk_w,
                            const float* y_shared, const float* shared_gate, const bf16* residual, int T, bf16* out,

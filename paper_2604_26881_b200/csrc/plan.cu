@@ -18,6 +18,48 @@ plan_kernel(const int32_t* __restrict__ expert_off, PlanArgs a)
     plan_body(expert_off, a, s_mem, s_warp);
 }
 
+// Tiles and unit lists of the shared expert alone, for one model: none of it depends on the routing, so these units
+// can run while the router and the dispatch are still at work (same order and encoding as in plan_body).
+__global__ void __launch_bounds__(256)
+plan_shared_kernel(PlanArgs a)
+{
+    pdl_wait();
+    pdl_launch_dependents();
+    const int tid = threadIdx.x, nth = blockDim.x;
+    const int n_stiles = (a.T + a.tile_rows - 1) / a.tile_rows;
+    for (int i = tid; i < n_stiles; i += nth) {
+        Tile t;
+        t.row0 = i * a.tile_rows;
+        t.nrows = min(a.tile_rows, a.T - t.row0);
+        t.slot = 0;
+        t.group = 0;
+        a.stiles[i] = t;
+    }
+    const int su1 = n_stiles * a.snblk1, su2 = n_stiles * a.snblk2;
+    const int tm = a.token_major;
+    const int wsh = a.shared_down_width;
+    const int sh_step = wsh / 64, sh_code = wsh == 256 ? 0 : (wsh == 128 ? 1 : 2);
+    for (int i = tid; i < su1; i += nth) {
+        Unit u;
+        u.colblock = (i / n_stiles) * (tm ? 4 : 1);
+        u.tile = ~(i % n_stiles);
+        a.units1[i] = u;
+    }
+    for (int i = tid; i < su2; i += nth) {
+        Unit u;
+        const int cb = i / n_stiles;
+        u.colblock = tm ? (cb * sh_step) | (sh_code << 24) : cb;
+        u.tile = ~(i % n_stiles);
+        a.units2[i] = u;
+    }
+    if (tid == 0) {
+        a.plan_counts[0] = 0; a.plan_counts[1] = n_stiles;
+        a.plan_counts[2] = su1; a.plan_counts[3] = su2;
+        a.plan_counts[4] = 0; a.plan_counts[5] = 0;     // work counters
+        a.plan_counts[6] = 0; a.plan_counts[7] = 0;     // nothing to deal out between routed units
+    }
+}
+
 }  // namespace
 
 PlanArgs make_plan_args(moe_ctx* c, int T, int G, bool with_shared)
@@ -66,6 +108,24 @@ cudaError_t launch_plan(moe_ctx* c, const int32_t* expert_off, int T, int G, boo
 {
     const PlanArgs a = make_plan_args(c, T, G, with_shared);
     launch_pdl(plan_kernel, dim3(1), dim3(512), plan_smem_ints(c, G) * sizeof(int32_t), st, expert_off, a);
+    c->launches += 1;
+    return cudaGetLastError();
+}
+
+void shared_unit_counts(moe_ctx* c, int T, int* n_units1, int* n_units2)
+{
+    const PlanArgs a = make_plan_args(c, T, 1, true);
+    const int n_stiles = (T + a.tile_rows - 1) / a.tile_rows;
+    *n_units1 = n_stiles * a.snblk1;
+    *n_units2 = n_stiles * a.snblk2;
+}
+
+cudaError_t launch_plan_shared(moe_ctx* c, int T, cudaStream_t st)
+{
+    PlanArgs a = make_plan_args(c, T, 1, true);
+    a.stiles = c->ws.stiles_sh; a.units1 = c->ws.units1_sh; a.units2 = c->ws.units2_sh;
+    a.plan_counts = c->ws.plan_counts_sh;
+    launch_pdl(plan_shared_kernel, dim3(1), dim3(256), 0, st, a);
     c->launches += 1;
     return cudaGetLastError();
 }

@@ -254,6 +254,33 @@ def test_wide_tiles_and_narrow_tiles_agree_bit_for_bit(qwen_weights, T):
         g.close()
 
 
+@pytest.mark.parametrize("T", [7, 64, 300, 1024, 4096])
+def test_shared_expert_on_second_stream_agrees_bit_for_bit(qwen_weights, T):
+    # one model: the shared expert's launches may run on the context's second stream beside the router and the
+    # dispatch.  The same units do the same arithmetic, so the output bits do not change, call after call (the
+    # buffers of one call are reused by the next one while two streams are in flight).
+    wl = W.scaled(W.WORKLOADS["prefill"], T=T)
+    x, tenant, mot = W.make_tokens(wl, seed=6)
+    x2, tenant2, _ = W.make_tokens(wl, seed=7)
+    g = GpuLayer(wl, [qwen_weights], wl.T, model_of_tenant=mot)
+    try:
+        B.moe_set_option(g.ctx, B.MOE_OPT_EARLY_SHARED, 0)
+        ref, ref2 = g.forward(x, tenant, wl.G), g.forward(x2, tenant2, wl.G)
+        for sms in (116, 32, 148):
+            B.moe_set_option(g.ctx, B.MOE_OPT_EARLY_SHARED, 2)
+            B.moe_set_option(g.ctx, B.MOE_OPT_EARLY_SHARED_SMS, sms)
+            xd, td, xd2, td2 = x.to(g.dev), tenant.to(g.dev), x2.to(g.dev), tenant2.to(g.dev)
+            outs = [torch.zeros_like(xd) for _ in range(6)]
+            for i, o in enumerate(outs):                 # back to back, no synchronisation in between
+                B.moe_layer_forward(g.ctx, 0, xd if i % 2 == 0 else xd2, td if i % 2 == 0 else td2, T, wl.G, o)
+            torch.cuda.synchronize()
+            assert B.moe_last_status(g.ctx)[0] == 0
+            for i, o in enumerate(outs):
+                assert torch.equal(o, ref if i % 2 == 0 else ref2), (sms, i)
+    finally:
+        g.close()
+
+
 def _sampled_check(g, wl, wts, x, tenant, mot, G, out, n_sample=32, layer_inputs=None):
     """Routing/dispatch of the last layer call in full, layer outputs on sampled tokens."""
     ws = B.moe_get_workspace(g.ctx)
