@@ -27,6 +27,7 @@ MOE_OPT_WIDE_TILES = 4
 MOE_OPT_TOKEN_MAJOR = 5
 MOE_OPT_EARLY_SHARED = 6
 MOE_OPT_EARLY_SHARED_SMS = 7
+MOE_OPT_ROUTE_LANES = 8
 MOE_PATH_AUTO, MOE_PATH_FMA, MOE_PATH_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["moe_create", "moe_destroy", "moe_set_expert_pool", "moe_set_model_weights", "moe_set_slot_table",

@@ -225,6 +225,7 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->tmaps = nullptr;
     c->rmaps = nullptr;
     c->route_path = MOE_PATH_AUTO;
+    c->route_lanes2 = 1;
     c->pair_mode_enabled = 1;
     c->wide_tiles_enabled = 1;
     c->token_major_enabled = 1;
@@ -367,6 +368,11 @@ int moe_set_option(moe_ctx* c, int option, int value)
     if (option == MOE_OPT_PAIR_MODE) {
         if (value < 0 || value > 2) return MOE_ERR_SHAPE;
         c->pair_mode_enabled = value;
+        return MOE_OK;
+    }
+    if (option == MOE_OPT_ROUTE_LANES) {
+        if (value < 1 || value > 2) return MOE_ERR_SHAPE;
+        c->route_lanes2 = value == 2 ? 1 : 0;
         return MOE_OK;
     }
     if (option == MOE_OPT_EARLY_SHARED) {

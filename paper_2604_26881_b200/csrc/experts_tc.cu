@@ -309,7 +309,11 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     if (PAIR) cluster_sync_all();          // the peer's barriers are initialised before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
-    pdl_wait();                            // set-up above overlaps the previous kernel; its results are read from here on
+    // Set-up above overlaps the previous kernel; its results are read from here on.  The down projection follows the
+    // gate/up launch, which had itself waited for the plan before it let this kernel start: the unit lists are
+    // complete, and the scheduler and the weight producer (static data) go ahead and fill the ring while the token
+    // producer and the epilogue wait for the activations.
+    if (!(MODE == 1 && (warp == 0 || warp == kSchedWarp))) pdl_wait();
     pdl_launch_dependents();
     const int n_units = *p.n_units;
     const int n_shared = *p.n_shared;

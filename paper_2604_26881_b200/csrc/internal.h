@@ -129,6 +129,7 @@ struct moe_ctx {
     faasmoe::TensorMaps* tmaps;   // TMA descriptors of the tensor-core path (host)
     void* rmaps;                  // TMA descriptors of the tensor-core router
     int route_path;
+    int route_lanes2;             // the tensor-core router issues its MMAs from two warps
     int pair_mode_enabled;        // allow the 2-CTA (cta_group::2) shape of the grouped GEMM for long tiles
     int token_major_enabled;      // one-CTA units take the tokens as the M operand of the MMA (up to 256 weight rows per tile)
     int wide_tiles_enabled;       // allow 512-row tiles (two accumulators per weight tile) in the 2-CTA shape

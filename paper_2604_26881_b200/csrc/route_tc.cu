@@ -23,7 +23,8 @@ constexpr int kRABytes = kRTokens * kRBK * 2;          // 16 KB of tokens per st
 constexpr int kRMaxN = 256;                            // router rows of all models, padded
 constexpr int kRTileBudget = 192 * 1024;               // shared memory for the pipeline stages
 constexpr int kRSmemBytes = kRTileBudget + kRABytes /* a short token tile is read as 128 rows */ + 1024 + 512;
-constexpr int kRThreads = 256;                         // warp 0: TMA (tokens), 1: MMA, 2..5: epilogue, 6 / 7: TMA (routers / gates)
+constexpr int kRThreads = 288;                         // warp 0: TMA (tokens), 1: MMA, 2..5: epilogue, 6 / 7: TMA (routers / gates),
+                                                       // 8: second MMA lane
 constexpr int kRMaxE = 64;                             // logits one thread keeps in registers
 
 struct RouteParams {
@@ -35,6 +36,8 @@ struct RouteParams {
     int gate_mma;                  // 1: the gate logit of model m is accumulator column gate_col + m*16
     int gate_col;                  // first gate column: right after the router columns when one MMA covers both
     int gate_merged;               // 1: router rows and gate rows are one N operand (n_models * (Epad + 16) <= 256)
+    int lanes2;                    // 1: two warps issue the MMAs, even and odd stages into accumulators of their own
+                                   // (TMEM columns 0.. and 256..) that the epilogue adds up
     int group;                     // stages handed back to the producer per commit (divides n_stages)
     int kb;                        // slices of 64 K elements per stage (1, 2 or 4): a wait, a fence and a commit per stage
                                    // cost the MMA lane as much as several of these narrow MMAs
@@ -88,7 +91,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kRStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        mbar_init(bar_tfull, 1);
+        mbar_init(bar_tfull, p.lanes2 ? 2 : 1);
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -106,7 +109,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
     pdl_wait();                     // set-up above overlaps the previous kernel; its results are read from here on
     pdl_launch_dependents();
 
-    if (warp == 0 || warp >= 6) {
+    if (warp == 0 || warp == 6 || warp == 7) {
         // three producer lanes (tokens / routers / gates) in three warps, so that the TMA instructions of one stage
         // are issued side by side (a tile load costs its issuing lane about 140 cycles, the barrier handshake about
         // 290; lanes of one warp would run their branches one after the other); the token lane also posts the
@@ -144,9 +147,13 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                     if (armed & (1u << s)) mbar_wait(bar_full + 8 * s, (armed_phase >> s) & 1u, &s_abort, p.status);
         }
         __syncwarp();
-    } else if (warp == 1) {
-        if (lane == 0) {
+    } else if (warp == 1 || warp == 8) {
+        // The MMAs of a stage cost their issuing lane more than the tensor pipe: with two lanes (in two warps) the
+        // stages alternate between them.
+        const int mine = warp == 1 ? 0 : 1;
+        if (lane == 0 && (mine == 0 || p.lanes2)) {
             uint32_t stage = 0, phase = 0;
+            const uint32_t tmem_acc = tmem_base + (uint32_t)mine * 256u;
             // a tcgen05.mma costs its issuing lane about 100 cycles whatever its width, a commit about 200: the gate
             // rows ride in the router's MMA when they fit, and stages go back to the producer in groups
             const int n_main = p.gate_merged ? N + p.n_models * 16 : N;
@@ -158,6 +165,10 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
             const bool two_mmas = p.gate_mma && !p.gate_merged;
             uint32_t acc = 0;                   // the first MMA overwrites the accumulators
             for (int ks = 0; ks < ksteps; ++ks) {
+                if (p.lanes2 && (ks & 1) != mine) {
+                    if (++stage == kRStages) { stage = 0; phase ^= 1; }
+                    continue;
+                }
                 if (!mbar_wait(bar_full + 8 * stage, phase, &s_abort, p.status)) { ok = false; break; }
                 tc_fence_after();
                 // (this lane is alone in its warp and pays for every instruction: descriptors from 32-bit words)
@@ -167,8 +178,8 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                     const uint32_t lo_g = lo_b + g_off;
 #pragma unroll
                     for (int kk = 0; kk < kRBK / 16; ++kk) {
-                        umma_bf16(tmem_base, smem_desc_pack(lo_a + 2 * kk), smem_desc_pack(lo_b + 2 * kk), idesc, acc);
-                        if (two_mmas) umma_bf16(tmem_base + p.gate_col, smem_desc_pack(lo_a + 2 * kk), smem_desc_pack(lo_g + 2 * kk), idesc_g, acc);
+                        umma_bf16(tmem_acc, smem_desc_pack(lo_a + 2 * kk), smem_desc_pack(lo_b + 2 * kk), idesc, acc);
+                        if (two_mmas) umma_bf16(tmem_acc + p.gate_col, smem_desc_pack(lo_a + 2 * kk), smem_desc_pack(lo_g + 2 * kk), idesc_g, acc);
                         acc = 1;
                     }
                     lo_a += a_step; lo_b += bg_step;
@@ -179,7 +190,7 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
             if (ok) umma_commit(bar_tfull);
         }
         __syncwarp();
-    } else if (warp < 6) {
+    } else {
         // ---- epilogue warps: thread <-> token (TMEM lane) ----
         const int quarter = warp & 3;
         const int t = t0 + quarter * 32 + lane;
@@ -213,6 +224,13 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                 gate = 1.f / (1.f + expf(-((a0 + a1) + (a2 + a3))));
             }
         }
+        // this token's router bias (-inf beyond the last expert) is fetched while the MMAs run
+        float zb[kRMaxE];
+        {
+            const float* rb = valid ? p.models[model].router_bias : nullptr;
+#pragma unroll
+            for (int e = 0; e < kRMaxE; ++e) zb[e] = e < p.E ? (rb ? __ldg(rb + e) : 0.f) : -INFINITY;
+        }
         const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_tfull, 0, &s_abort, p.status));
         if (ok) {
             tc_fence_after();
@@ -231,7 +249,15 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                         tmem_ld_wait();
                         if (m == model) {
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) z[c * 16 + j] = __uint_as_float(r[j]);
+                            for (int j = 0; j < 16; ++j) z[c * 16 + j] = __uint_as_float(r[j]) + zb[c * 16 + j];
+                        }
+                        if (p.lanes2) {                                   // the second lane's share of the sum over K
+                            tmem_ld16(taddr + 256 + m * p.Epad + c * 16, r);
+                            tmem_ld_wait();
+                            if (m == model) {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) z[c * 16 + j] += __uint_as_float(r[j]);
+                            }
                         }
                     }
                 }
@@ -241,19 +267,19 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                     uint32_t r[16];
                     tmem_ld16(taddr + p.gate_col + m * 16, r);
                     tmem_ld_wait();
-                    if (m == model && valid && p.models[m].shared_gate_w) gate = 1.f / (1.f + expf(-__uint_as_float(r[0])));
+                    float gl = __uint_as_float(r[0]);
+                    if (p.lanes2) {
+                        tmem_ld16(taddr + 256 + p.gate_col + m * 16, r);
+                        tmem_ld_wait();
+                        gl += __uint_as_float(r[0]);
+                    }
+                    if (m == model && valid && p.models[m].shared_gate_w) gate = 1.f / (1.f + expf(-gl));
                 }
             }
             if (valid) {
                 // Softmax is monotone, so the ranking is done on the logits themselves; the
                 // probabilities are exp2((z - zmax) * log2 e) / sum.  Four independent chains keep
                 // the one warp per scheduler busy.
-                const float* rb = p.models[model].router_bias;
-#pragma unroll
-                for (int e = 0; e < kRMaxE; ++e) {
-                    if (e < p.E) { if (rb) z[e] += rb[e]; }
-                    else z[e] = -INFINITY;
-                }
                 float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
                 for (int e = 0; e < kRMaxE; e += 4) {
@@ -394,9 +420,12 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     p.n_stages = kRTileBudget / p.stage_bytes;
     if (p.n_stages > kRMaxStages) p.n_stages = kRMaxStages;
     p.group = p.n_stages >= 8 ? 4 : (p.n_stages >= 4 ? 2 : 1);
-    p.n_stages -= p.n_stages % p.group;
     // the gate rows follow the router rows in shared memory (b_bytes has no padding: Epad is a multiple of 16)
     p.gate_merged = (p.gate_mma && M * (epad + 16) <= kRMaxN && p.b_bytes == M * epad * kRBK * 2) ? 1 : 0;
+    // two MMA lanes unless the gate rows need an accumulator region of their own; each lane hands back its own stages
+    p.lanes2 = ((!p.gate_mma || p.gate_merged) && H / (kRBK * p.kb) >= 2 && c->route_lanes2) ? 1 : 0;
+    if (p.lanes2) p.group = 1;
+    p.n_stages -= p.n_stages % p.group;
     p.gate_col = p.gate_merged ? M * epad : kRMaxN;
     launch_pdl(route_tc_kernel, dim3((T + kRTokens - 1) / kRTokens), dim3(kRThreads), kRSmemBytes, st, p, mp);
     c->launches += 1;
