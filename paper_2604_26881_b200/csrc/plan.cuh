@@ -153,12 +153,15 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
                     mine = list[total - r + tid];
                     const int rows = a.direct ? a.T : a.tiles[mine.tile].nrows;
                     cnt = rows <= 64 ? 2 : 1;
-                    s_split[tid] = cnt;
                 }
+                // position of each unit after the split: a prefix count of the units that become two (r <= 128: the
+                // first four warps hold them all)
+                const unsigned two = __ballot_sync(0xffffffffu, cnt == 2);
+                if (tid < 128 && (tid & 31) == 0) s_split[tid >> 5] = __popc(two);
                 __syncthreads();
                 if (tid < r) {
-                    int off = 0;
-                    for (int j = 0; j < tid; ++j) off += s_split[j];
+                    int off = tid + __popc(two & ((1u << (tid & 31)) - 1u));
+                    for (int w = 0; w < (tid >> 5); ++w) off += s_split[w];
                     Unit u = mine;
                     if (cnt == 2) {
                         u.colblock = mine.colblock | (1 << 24);
@@ -169,11 +172,7 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
                         list[total - r + off] = u;
                     }
                 }
-                if (tid == 0) {
-                    int extra = 0;
-                    for (int j = 0; j < r; ++j) extra += s_split[j] - 1;
-                    a.plan_counts[2 + l] = total + extra;
-                }
+                if (tid == 0) a.plan_counts[2 + l] = total + s_split[0] + s_split[1] + s_split[2] + s_split[3];
                 __syncthreads();
             }
         }
