@@ -41,6 +41,10 @@ def parse_args():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "fma", "tcgen05"])
     ap.add_argument("--pair", default="auto", choices=["auto", "never"])
+    ap.add_argument("--early-shared", default="auto", choices=["auto", "0", "1", "2"],
+                    help="shared expert on the context's second stream (auto: the library's default, batches of more than 64 tokens); "
+                         "the per-stage times and the roofline block always come from passes without it, where one "
+                         "grouped-GEMM launch holds the shared and the routed units")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -128,7 +132,7 @@ def algorithmic_work(wl, active_experts: int, T: int):
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
 # ncu captures summarised in profiles/grouped_gemm_decode_ncu.md and profiles/grouped_gemm_prefill_ncu.md; None where
 # no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"decode": 657.657600e6 + 3.586304e6, "prefill": 858.381312e6 + 84.442624e6}
+NCU_TRAFFIC_BYTES = {"decode": 657.659136e6 + 4.132608e6, "prefill": 860.452352e6 + 84.881920e6}
 
 
 def run_reference(args, wl, rank):
@@ -210,6 +214,8 @@ def run_stack(args, wl, rank, local_rank, world):
     layer.set_tables(model_of_tenant=mot)
     ctx = layer.ctx
     B.moe_set_option(ctx, B.MOE_OPT_PAIR_MODE, {"auto": 1, "never": 0}[args.pair])
+    if args.early_shared != "auto":
+        B.moe_set_option(ctx, B.MOE_OPT_EARLY_SHARED, int(args.early_shared))
     xd, td = x.to(dev), tenant.to(dev)
     xw = xd.clone()
     stream = torch.cuda.current_stream()
@@ -297,6 +303,8 @@ def main():
     ctx = layer.ctx
     B.moe_set_option(ctx, B.MOE_OPT_EXPERT_PATH, {"auto": 0, "fma": 1, "tcgen05": 2}[args.path])
     B.moe_set_option(ctx, B.MOE_OPT_PAIR_MODE, {"auto": 1, "never": 0}[args.pair])
+    if args.early_shared != "auto":
+        B.moe_set_option(ctx, B.MOE_OPT_EARLY_SHARED, int(args.early_shared))
     xd, td = x.to(dev), tenant.to(dev)
     out = torch.zeros_like(xd)
     stream = torch.cuda.current_stream()
@@ -377,7 +385,7 @@ def main():
                 "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": wl.name, "tokens_per_step_per_gpu": T, "hidden": wl.H, "experts": wl.E,
                            "inter": wl.I, "top_k": wl.k, "shared_inter": wl.Is, "G": wl.G, "tenants": wl.n_tenants,
-                           "models": wl.M, "expert_path": args.path,
+                           "models": wl.M, "expert_path": args.path, "early_shared": args.early_shared,
                            "l2": "expert weights (about 1 GB per pass) exceed the 126 MB L2; no flush",
                            "parallelism": f"replicas x{world}"},
                 "clocks": clocks, "gpu_launches": int(launches),

@@ -165,9 +165,10 @@ int layer_forward_impl(moe_ctx* c, int layer, const bf16* x, const int32_t* tena
     const bool shared = g.shared_inter > 0;
     // One model: the shared expert's work does not depend on the routing.  Its two launches go to a second stream, where
     // they run beside the router and the dispatch (HBM- or tensor-bound work beside latency-bound work); the combine
-    // waits for both streams.  Not while the stages are being timed one by one.
+    // waits for both streams.  By default only for batches of the 2-CTA shape: with fewer tokens the two event
+    // edges cost what the overlap gains.  Not while the stages are being timed one by one.
     const bool early = shared && g.n_models == 1 && use_tc(c) && !c->timing && c->side != nullptr &&
-                       (c->early_shared_enabled == 2 || (c->early_shared_enabled == 1 && tc_token_major(c, T)));
+                       (c->early_shared_enabled == 2 || (c->early_shared_enabled == 1 && tc_pair_mode(c, T)));
     if (early) {
         const int rc = tc_setup_layer(c, layer);
         if (rc != MOE_OK) return rc;
@@ -230,7 +231,7 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->wide_tiles_enabled = 1;
     c->token_major_enabled = 1;
     c->timing = false;
-    c->early_shared_enabled = 2;
+    c->early_shared_enabled = 1;
     c->early_shared_sms = 1 << 20;      // no limit
     c->side = nullptr; c->ev_fork = nullptr; c->ev_join = nullptr;
     for (auto& e : c->ev) e = nullptr;

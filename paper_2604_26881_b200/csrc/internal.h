@@ -134,7 +134,7 @@ struct moe_ctx {
     int token_major_enabled;      // one-CTA units take the tokens as the M operand of the MMA (up to 256 weight rows per tile)
     int wide_tiles_enabled;       // allow 512-row tiles (two accumulators per weight tile) in the 2-CTA shape
     int early_shared_enabled;     // one model: run the shared expert on a second stream beside router and dispatch
-                                  // (1: batches of the token-major shape, 2: every batch)
+                                  // (1: batches of the 2-CTA shape, 2: every batch)
     int early_shared_sms;         // SMs the shared expert's CTA pairs may take while they run beside other kernels
     cudaStream_t side;            // second stream of the layer pass
     cudaEvent_t ev_fork, ev_join; // order between the caller's stream and the second one

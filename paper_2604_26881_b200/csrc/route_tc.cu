@@ -244,19 +244,15 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
 #pragma unroll
                 for (int c = 0; c < kRMaxE / 16; ++c) {
                     if (c * 16 < p.Epad) {                                // warp-uniform
-                        uint32_t r[16];
+                        uint32_t r[16], r2[16];
                         tmem_ld16(taddr + m * p.Epad + c * 16, r);
+                        if (p.lanes2) tmem_ld16(taddr + 256 + m * p.Epad + c * 16, r2);   // the second lane's share of the sum over K
                         tmem_ld_wait();
                         if (m == model) {
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) z[c * 16 + j] = __uint_as_float(r[j]) + zb[c * 16 + j];
-                        }
-                        if (p.lanes2) {                                   // the second lane's share of the sum over K
-                            tmem_ld16(taddr + 256 + m * p.Epad + c * 16, r);
-                            tmem_ld_wait();
-                            if (m == model) {
-#pragma unroll
-                                for (int j = 0; j < 16; ++j) z[c * 16 + j] += __uint_as_float(r[j]);
+                            for (int j = 0; j < 16; ++j) {
+                                z[c * 16 + j] = __uint_as_float(r[j]) + zb[c * 16 + j];
+                                if (p.lanes2) z[c * 16 + j] += __uint_as_float(r2[j]);
                             }
                         }
                     }
