@@ -75,7 +75,9 @@ enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2,
        MOE_OPT_EARLY_SHARED = 6, /* one model with a shared expert, moe_layer_forward and the calls built on it: the
                                     shared expert's two launches go to a second stream of the context, beside the
                                     router and the dispatch; the combine waits for both.  1 (default): batches of
-                                    more than 64 tokens; 2: every batch; 0: never.  Results are bit-identical. */
+                                    more than 64 tokens; 2: every batch; 0: never.  Results are bit-identical.
+                                    With several models the second stream groups the tokens by model (the input
+                                    of the shared experts) beside the router and the dispatch, unless 0. */
        MOE_OPT_EARLY_SHARED_SMS = 7, /* SMs that the shared expert's CTA pairs may hold while they run beside other
                                        kernels (batches of more than 64 tokens; default: no limit) */
        MOE_OPT_ROUTE_LANES = 8 /* 2 (default): the tensor-core router issues its MMAs from two warps, even and odd K

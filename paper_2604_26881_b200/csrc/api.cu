@@ -133,14 +133,14 @@ bool use_tc(const moe_ctx* c)
 
 int experts_impl(moe_ctx* c, int layer, const bf16* x, const bf16* x_perm, const int32_t* perm,
                  const int32_t* expert_off, const int32_t* tenant_id, int T, int G, float* y_perm, float* y_shared,
-                 cudaStream_t st, bool plan_done = false)
+                 cudaStream_t st, bool plan_done = false, bool sort_done = false)
 {
     const moe_config& g = c->cfg;
     const bool with_shared = y_shared != nullptr && g.shared_inter > 0;
     const bf16* xs = x;
     const int32_t* dst_rows = nullptr;
     if (with_shared && g.n_models > 1) {
-        MOE_CUDA(c, launch_token_sort(c, x, tenant_id, T, st));
+        if (!sort_done) MOE_CUDA(c, launch_token_sort(c, x, tenant_id, T, st));
         xs = c->ws.xs_perm;
         dst_rows = c->ws.tok_perm;
     }
@@ -178,6 +178,15 @@ int layer_forward_impl(moe_ctx* c, int layer, const bf16* x, const int32_t* tena
         MOE_CUDA(c, launch_experts_tc(c, layer, x, nullptr, nullptr, T, nullptr, w.y_shared, nullptr, c->side, true));
         MOE_CUDA(c, cudaEventRecord(c->ev_join, c->side));
     }
+    // Several models: the shared experts read the tokens grouped by model.  That grouping (four small launches) depends
+    // on the tenant ids only and runs on the second stream beside the router and the dispatch; the plan waits for it.
+    const bool sort_early = shared && g.n_models > 1 && !c->timing && c->side != nullptr && c->early_shared_enabled != 0;
+    if (sort_early) {
+        MOE_CUDA(c, cudaEventRecord(c->ev_fork, st));
+        MOE_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+        MOE_CUDA(c, launch_token_sort(c, x, tenant_id, T, c->side));
+        MOE_CUDA(c, cudaEventRecord(c->ev_join, c->side));
+    }
     stage_mark(c, st, kEvBegin);
     MOE_CUDA(c, launch_route(c, layer, x, tenant_id, T, w.topk_idx, w.topk_w, shared ? w.shared_gate : nullptr,
                              w.tie_flag, st));
@@ -188,8 +197,9 @@ int layer_forward_impl(moe_ctx* c, int layer, const bf16* x, const int32_t* tena
     MOE_CUDA(c, launch_dispatch(c, x, w.topk_idx, tenant_id, T, G, w.perm, w.inv_perm, w.tenant_expert_count,
                                 w.expert_off, w.group_off, direct ? nullptr : w.x_perm, st, true, shared && !early, &plan_done));
     stage_mark(c, st, kEvDispatch);
+    if (sort_early) MOE_CUDA(c, cudaStreamWaitEvent(st, c->ev_join, 0));
     const int rc = experts_impl(c, layer, x, w.x_perm, w.perm, w.expert_off, tenant_id, T, G, w.y_perm,
-                                (shared && !early) ? w.y_shared : nullptr, st, plan_done);
+                                (shared && !early) ? w.y_shared : nullptr, st, plan_done, sort_early);
     if (rc != MOE_OK) return rc;
     if (early) MOE_CUDA(c, cudaStreamWaitEvent(st, c->ev_join, 0));
     MOE_CUDA(c, launch_combine(c, w.y_perm, w.inv_perm, w.topk_w, shared ? w.y_shared : nullptr,
@@ -264,7 +274,7 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     }
     if (rc == MOE_OK) rc = upload_tenant_tables(c);
     if (rc == MOE_OK) rc = alloc_workspace(c);
-    if (rc == MOE_OK && g.shared_inter > 0 && g.n_models == 1) {
+    if (rc == MOE_OK && g.shared_inter > 0) {
         e = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);

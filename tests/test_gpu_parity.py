@@ -281,6 +281,31 @@ def test_shared_expert_on_second_stream_agrees_bit_for_bit(qwen_weights, T):
         g.close()
 
 
+def test_token_grouping_on_second_stream_agrees_bit_for_bit():
+    # several models: the tokens are grouped by model (input of the shared experts) on the context's second stream
+    # while the router and the dispatch run; calls back to back reuse the grouping buffers
+    wl = W.MoEWorkload("small-pool", T=333, H=256, E=12, I=128, k=3, Is=256, M=3, n_tenants=5, G=5,
+                       zipf_bias=True, tenant_layout="uniform")
+    wts = W.make_weights(wl, seed=3, shuffle_slots=True)
+    x, tenant, mot = W.make_tokens(wl, seed=3)
+    x2, tenant2, _ = W.make_tokens(wl, seed=4)
+    g = GpuLayer(wl, [wts], wl.T, model_of_tenant=mot)
+    try:
+        B.moe_set_option(g.ctx, B.MOE_OPT_EARLY_SHARED, 0)
+        ref, ref2 = g.forward(x, tenant, wl.G), g.forward(x2, tenant2, wl.G)
+        B.moe_set_option(g.ctx, B.MOE_OPT_EARLY_SHARED, 1)
+        xd, td, xd2, td2 = x.to(g.dev), tenant.to(g.dev), x2.to(g.dev), tenant2.to(g.dev)
+        outs = [torch.zeros_like(xd) for _ in range(6)]
+        for i, o in enumerate(outs):
+            B.moe_layer_forward(g.ctx, 0, xd if i % 2 == 0 else xd2, td if i % 2 == 0 else td2, wl.T, wl.G, o)
+        torch.cuda.synchronize()
+        assert B.moe_last_status(g.ctx)[0] == 0
+        for i, o in enumerate(outs):
+            assert torch.equal(o, ref if i % 2 == 0 else ref2), i
+    finally:
+        g.close()
+
+
 def _sampled_check(g, wl, wts, x, tenant, mot, G, out, n_sample=32, layer_inputs=None):
     """Routing/dispatch of the last layer call in full, layer outputs on sampled tokens."""
     ws = B.moe_get_workspace(g.ctx)
