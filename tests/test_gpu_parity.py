@@ -57,6 +57,19 @@ def test_small_multi_model_pool(path, G):
     assert ref.dispatch.n_invocations <= 3 * -(-12 // G)
 
 
+@pytest.mark.parametrize("H", [128, 384, 640])
+@pytest.mark.parametrize("M", [1, 2])
+def test_router_stage_counts_of_the_two_mma_lanes(H, M):
+    # the tensor-core router splits its K stages between two MMA lanes (even / odd) with an accumulator each:
+    # hidden sizes that give one stage (one lane only), three and five stages (lanes with unequal shares), with the
+    # shared gate's rows riding in the same MMA, one and two models, a ragged last token tile
+    wl = W.MoEWorkload("router-lanes", T=300, H=H, E=12, I=128, k=3, Is=128, M=M, n_tenants=3, G=4,
+                       zipf_bias=True, tenant_layout="uniform")
+    wts = W.make_weights(wl, seed=31)
+    x, tenant, mot = W.make_tokens(wl, seed=31)
+    run_and_compare(wl, wts, x, tenant, mot, wl.G, B.MOE_PATH_AUTO)
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_decode_config(qwen_weights, path):
     wl = W.WORKLOADS["decode"]
