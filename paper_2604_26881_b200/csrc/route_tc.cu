@@ -38,6 +38,8 @@ struct RouteParams {
     int gate_merged;               // 1: router rows and gate rows are one N operand (n_models * (Epad + 16) <= 256)
     int lanes2;                    // 1: two warps issue the MMAs, even and odd stages into accumulators of their own
                                    // (TMEM columns 0.. and 256..) that the epilogue adds up
+    int per_model;                 // 1: blockIdx.y is a model; the CTA computes that model's logits only and writes the
+                                   // results of the tile's tokens that belong to it
     int group;                     // stages handed back to the producer per commit (divides n_stages)
     int kb;                        // slices of 64 K elements per stage (1, 2 or 4): a wait, a fence and a commit per stage
                                    // cost the MMA lane as much as several of these narrow MMAs
@@ -87,7 +89,9 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t0 = blockIdx.x * kRTokens;
     const int ksteps = p.H / (kRBK * p.kb);        // stages to go through
-    const int N = p.n_models * p.Epad;
+    const int m0 = p.per_model ? (int)blockIdx.y : 0;       // first model and number of models of this CTA
+    const int nm = p.per_model ? 1 : p.n_models;
+    const int N = nm * p.Epad;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kRStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
@@ -128,16 +132,16 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                 armed |= 1u << stage;
                 armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
                 if (role == 0) {
-                    mbar_expect_tx(full, p.kb * (p.a_bytes + N * kRBK * 2 + (p.gate_mma ? p.n_models * 16 * kRBK * 2 : 0)));
+                    mbar_expect_tx(full, p.kb * (p.a_bytes + N * kRBK * 2 + (p.gate_mma ? nm * 16 * kRBK * 2 : 0)));
                     for (int a = 0; a < p.kb; ++a) tma_load_2d_hint(sa + a * p.a_bytes, &maps.x, full, (ks * p.kb + a) * kRBK, t0, keep);
                 } else if (role == 1) {
                     for (int a = 0; a < p.kb; ++a)
-                        for (int m = 0; m < p.n_models; ++m)
-                            tma_load_2d_hint(sb + a * p.bg_bytes + m * p.Epad * kRBK * 2, &maps.r[m], full, (ks * p.kb + a) * kRBK, 0, keep);
+                        for (int m = 0; m < nm; ++m)
+                            tma_load_2d_hint(sb + a * p.bg_bytes + m * p.Epad * kRBK * 2, &maps.r[m0 + m], full, (ks * p.kb + a) * kRBK, 0, keep);
                 } else {
                     for (int a = 0; a < p.kb; ++a)
-                        for (int m = 0; m < p.n_models; ++m)
-                            tma_load_2d_hint(sb + a * p.bg_bytes + p.b_bytes + m * 16 * kRBK * 2, &maps.g[m], full, (ks * p.kb + a) * kRBK, 0,
+                        for (int m = 0; m < nm; ++m)
+                            tma_load_2d_hint(sb + a * p.bg_bytes + p.b_bytes + m * 16 * kRBK * 2, &maps.g[m0 + m], full, (ks * p.kb + a) * kRBK, 0,
                                              keep);
                 }
                 if (++stage == kRStages) { stage = 0; phase ^= 1; }
@@ -156,9 +160,9 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
             const uint32_t tmem_acc = tmem_base + (uint32_t)mine * 256u;
             // a tcgen05.mma costs its issuing lane about 100 cycles whatever its width, a commit about 200: the gate
             // rows ride in the router's MMA when they fit, and stages go back to the producer in groups
-            const int n_main = p.gate_merged ? N + p.n_models * 16 : N;
+            const int n_main = p.gate_merged ? N + nm * 16 : N;
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_main >> 3) << 17) | ((128u >> 4) << 24);
-            const uint32_t idesc_g = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_models * 16 >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t idesc_g = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(nm * 16 >> 3) << 17) | ((128u >> 4) << 24);
             bool ok = true;
             const uint32_t a_step = (uint32_t)p.a_bytes >> 4, bg_step = (uint32_t)p.bg_bytes >> 4;
             const uint32_t b_off = (uint32_t)(p.kb * p.a_bytes) >> 4, g_off = (uint32_t)p.b_bytes >> 4;
@@ -194,13 +198,14 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
         // ---- epilogue warps: thread <-> token (TMEM lane) ----
         const int quarter = warp & 3;
         const int t = t0 + quarter * 32 + lane;
-        const bool valid = t < p.T;
+        bool valid = t < p.T;
         bool bad = false;
         int model = 0;
         if (valid) {
             int u = p.tenant_id[t];
             if (u < 0 || u >= p.n_tenants) { bad = true; u = 0; }
             model = p.model_of_tenant[u];
+            if (p.per_model && model != m0) valid = false;      // another CTA of this tile has that model
         }
         // shared-expert gate, overlapped with the MMA pipeline: each thread walks its own token's row
         // (independent 16-byte loads, four accumulators), so no cross-lane traffic is needed
@@ -240,13 +245,14 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
             float z[kRMaxE];
 #pragma unroll
             for (int e = 0; e < kRMaxE; ++e) z[e] = -INFINITY;
-            for (int m = 0; m < p.n_models; ++m) {
+            for (int mi = 0; mi < nm; ++mi) {
+                const int m = m0 + mi;
 #pragma unroll
                 for (int c = 0; c < kRMaxE / 16; ++c) {
                     if (c * 16 < p.Epad) {                                // warp-uniform
                         uint32_t r[16], r2[16];
-                        tmem_ld16(taddr + m * p.Epad + c * 16, r);
-                        if (p.lanes2) tmem_ld16(taddr + 256 + m * p.Epad + c * 16, r2);   // the second lane's share of the sum over K
+                        tmem_ld16(taddr + mi * p.Epad + c * 16, r);
+                        if (p.lanes2) tmem_ld16(taddr + 256 + mi * p.Epad + c * 16, r2);   // the second lane's share of the sum over K
                         tmem_ld_wait();
                         if (m == model) {
 #pragma unroll
@@ -259,13 +265,14 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
                 }
             }
             if (p.gate_mma && p.shared_gate) {
-                for (int m = 0; m < p.n_models; ++m) {
+                for (int mi = 0; mi < nm; ++mi) {
+                    const int m = m0 + mi;
                     uint32_t r[16];
-                    tmem_ld16(taddr + p.gate_col + m * 16, r);
+                    tmem_ld16(taddr + p.gate_col + mi * 16, r);
                     tmem_ld_wait();
                     float gl = __uint_as_float(r[0]);
                     if (p.lanes2) {
-                        tmem_ld16(taddr + 256 + p.gate_col + m * 16, r);
+                        tmem_ld16(taddr + 256 + p.gate_col + mi * 16, r);
                         tmem_ld_wait();
                         gl += __uint_as_float(r[0]);
                     }
@@ -406,8 +413,12 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     p.topk_idx = topk_idx; p.topk_w = topk_w; p.shared_gate = shared_gate; p.tie_flag = tie_flag;
     p.status = c->ws.status;
     p.a_bytes = (a_rows * kRBK * 2 + 1023) & ~1023;
-    p.b_bytes = (M * epad * kRBK * 2 + 1023) & ~1023;
-    p.bg_bytes = p.b_bytes + (p.gate_mma ? ((M * 16 * kRBK * 2 + 1023) & ~1023) : 0);
+    // several models: a CTA per (token tile, model) computes that model's logits only (4x the CTAs for a quarter of
+    // the operand bytes and MMA columns each; a token needs the logits of its own model alone)
+    p.per_model = M > 1 ? 1 : 0;
+    const int Mc = p.per_model ? 1 : M;             // models per CTA
+    p.b_bytes = (Mc * epad * kRBK * 2 + 1023) & ~1023;
+    p.bg_bytes = p.b_bytes + (p.gate_mma ? ((Mc * 16 * kRBK * 2 + 1023) & ~1023) : 0);
     const int slice_bytes = p.a_bytes + p.bg_bytes;
     p.kb = 1;
     for (int kb = 4; kb > 1; kb >>= 1)
@@ -417,13 +428,13 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     if (p.n_stages > kRMaxStages) p.n_stages = kRMaxStages;
     p.group = p.n_stages >= 8 ? 4 : (p.n_stages >= 4 ? 2 : 1);
     // the gate rows follow the router rows in shared memory (b_bytes has no padding: Epad is a multiple of 16)
-    p.gate_merged = (p.gate_mma && M * (epad + 16) <= kRMaxN && p.b_bytes == M * epad * kRBK * 2) ? 1 : 0;
+    p.gate_merged = (p.gate_mma && Mc * (epad + 16) <= kRMaxN && p.b_bytes == Mc * epad * kRBK * 2) ? 1 : 0;
     // two MMA lanes unless the gate rows need an accumulator region of their own; each lane hands back its own stages
     p.lanes2 = ((!p.gate_mma || p.gate_merged) && H / (kRBK * p.kb) >= 2 && c->route_lanes2) ? 1 : 0;
     if (p.lanes2) p.group = 1;
     p.n_stages -= p.n_stages % p.group;
-    p.gate_col = p.gate_merged ? M * epad : kRMaxN;
-    launch_pdl(route_tc_kernel, dim3((T + kRTokens - 1) / kRTokens), dim3(kRThreads), kRSmemBytes, st, p, mp);
+    p.gate_col = p.gate_merged ? Mc * epad : kRMaxN;
+    launch_pdl(route_tc_kernel, dim3((T + kRTokens - 1) / kRTokens, p.per_model ? M : 1), dim3(kRThreads), kRSmemBytes, st, p, mp);
     c->launches += 1;
     return cudaGetLastError();
 }
