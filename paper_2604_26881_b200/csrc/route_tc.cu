@@ -1,10 +1,11 @@
 // Gating network on the tensor cores (paper Sec. 2.1: the gate scores every expert and selects
-// the top-k per token).  One CTA scores 128 tokens against the routers of all tenant models at
-// once: the tokens are the M operand of tcgen05.mma (one TMEM lane per token), the router rows of
-// every model the N operand (E rows per model, padded to a multiple of 16).  The epilogue is one
-// thread per token: it picks the columns of its tenant's model out of TMEM and does the fp32
-// softmax and the top-k in registers.  While the MMA pipeline runs, the epilogue warps compute the
-// shared expert's sigmoid gate with plain FMAs.
+// the top-k per token).  One CTA scores 128 tokens against the router of one tenant model: the
+// tokens are the M operand of tcgen05.mma (one TMEM lane per token), the router rows the N operand
+// (E rows, padded to a multiple of 16, followed by 16 rows for the shared expert's gate vector).
+// With several models the grid is (token tiles x models) and a CTA writes the results of those
+// tokens of its tile that belong to its model.  Two warps issue the MMAs, even and odd K stages
+// into an accumulator each.  The epilogue is one thread per token: it adds the two accumulators and
+// the router bias (fetched while the MMAs run) and does the fp32 softmax and the top-k in registers.
 #include <cstring>
 
 #include "internal.h"
