@@ -319,6 +319,40 @@ def test_token_grouping_on_second_stream_agrees_bit_for_bit():
         g.close()
 
 
+@pytest.mark.parametrize("seed", [2, 3])
+def test_random_configurations_agree_across_entry_points_and_paths(seed):
+    # 20 random layer shapes per seed (hidden size, experts, top-k, shared expert or none, one to four models, block
+    # size, 1 ... 4096 tokens): the fused entry point equals the four calls bit for bit, with the shared expert on the
+    # second stream or not, is reproducible, and stays within the tolerance of the CUDA-core expert path
+    import random
+    rng = random.Random(seed)
+    for it in range(20):
+        H = rng.choice([256, 512, 768, 1024, 2048]); E = rng.choice([4, 8, 12, 16, 33, 60, 64])
+        I = rng.choice([128, 256, 384]); k = rng.randint(1, min(6, E))
+        Is = rng.choice([0, 128, 256, 512]); M = rng.choice([1, 1, 2, 3, 4]); nt = rng.randint(M, M + 4)
+        G = rng.randint(1, E)
+        T = rng.choice([1, 2, 3, 17, 31, 64, 65, 100, 128, 129, 255, 300, 513, 700, 1025, 1500, 2600, 4096])
+        wl = W.MoEWorkload(f"random{it}", T=T, H=H, E=E, I=I, k=k, Is=Is, M=M, n_tenants=nt, G=G,
+                           zipf_bias=rng.random() < 0.5, tenant_layout=rng.choice(["uniform", "contiguous"]))
+        wts = W.make_weights(wl, seed=it, shuffle_slots=rng.random() < 0.5)
+        x, tenant, mot = W.make_tokens(wl, seed=it)
+        g = GpuLayer(wl, [wts], T, model_of_tenant=mot)
+        try:
+            o = g.four_calls(x, tenant, G)
+            f1, f2 = g.forward(x, tenant, G), g.forward(x, tenant, G)
+            B.moe_set_option(g.ctx, B.MOE_OPT_EARLY_SHARED, 2)
+            f3 = g.forward(x, tenant, G)
+            B.moe_set_option(g.ctx, B.MOE_OPT_EARLY_SHARED, 0)
+            f4 = g.forward(x, tenant, G)
+            assert B.moe_last_status(g.ctx)[0] == 0, wl
+            assert torch.equal(f1, o["out"]) and torch.equal(f1, f2) and torch.equal(f1, f3) and torch.equal(f1, f4), wl
+            B.moe_set_option(g.ctx, B.MOE_OPT_EXPERT_PATH, B.MOE_PATH_FMA)
+            fma = g.forward(x, tenant, G)
+            assert_close(f"{wl}: tensor-core vs CUDA-core experts", bf16_to_f64(f1), bf16_to_f64(fma))
+        finally:
+            g.close()
+
+
 def _sampled_check(g, wl, wts, x, tenant, mot, G, out, n_sample=32, layer_inputs=None):
     """Routing/dispatch of the last layer call in full, layer outputs on sampled tokens."""
     ws = B.moe_get_workspace(g.ctx)
