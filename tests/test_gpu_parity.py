@@ -319,6 +319,27 @@ def test_token_grouping_on_second_stream_agrees_bit_for_bit():
         g.close()
 
 
+@pytest.mark.parametrize("seed", [6, 7])
+def test_random_small_configurations_against_the_oracle(seed):
+    # 30 random small layer shapes per seed, every output of the four calls against the oracle element by element:
+    # hidden sizes with one to six K stages of the router (H = 128 ... 768; the experts run on the CUDA cores where
+    # H is not a multiple of 256), E = 3 ... 64, top-1 ... top-6, one to four models (a router CTA per model), with and
+    # without a shared expert, block sizes that do not divide E, 1 ... 400 tokens
+    import random
+    rng = random.Random(seed)
+    for it in range(30):
+        H = rng.choice([128, 256, 384, 512, 640, 768]); E = rng.choice([3, 8, 12, 16, 33, 60, 64])
+        I = rng.choice([128, 256]); k = rng.randint(1, min(6, E))
+        Is = rng.choice([0, 128, 256]); M = rng.choice([1, 2, 3, 4]); nt = rng.randint(M, M + 3)
+        G = rng.randint(1, E)
+        T = rng.choice([1, 5, 31, 64, 65, 130, 257, 400])
+        wl = W.MoEWorkload(f"random{it}", T=T, H=H, E=E, I=I, k=k, Is=Is, M=M, n_tenants=nt, G=G,
+                           zipf_bias=rng.random() < 0.5, tenant_layout=rng.choice(["uniform", "contiguous"]))
+        wts = W.make_weights(wl, seed=100 + it, shuffle_slots=rng.random() < 0.5)
+        x, tenant, mot = W.make_tokens(wl, seed=100 + it)
+        run_and_compare(wl, wts, x, tenant, mot, G, B.MOE_PATH_AUTO)
+
+
 @pytest.mark.parametrize("seed", [2, 3])
 def test_random_configurations_agree_across_entry_points_and_paths(seed):
     # 20 random layer shapes per seed (hidden size, experts, top-k, shared expert or none, one to four models, block
