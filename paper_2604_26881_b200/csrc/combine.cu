@@ -48,22 +48,45 @@ combine_kernel(const float* __restrict__ y_perm, const int32_t* __restrict__ inv
     const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (gid >= (long long)T * hv) return;
     const int t = (int)(gid / hv), v = (int)(gid - (long long)t * hv);
-    float acc[8], tmp[8];
+    float acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-    if (residual) unpack8(reinterpret_cast<const uint4*>(residual + (size_t)t * H)[v], acc);
-    for (int j = 0; j < k; ++j) {
-        const int r = inv_perm[(size_t)t * k + j];
-        const float w = topk_w[(size_t)t * k + j];
-        load8(y_perm + (size_t)r * H + 8 * v, tmp);
+    // All loads are issued before the first sum: positions and weights of the k rows, then the rows themselves (four
+    // at a time), the shared row and the residual.  With few tokens this kernel is a chain of memory latencies, and
+    // position -> row, once per j, made it k times as long.  The order of the sums stays residual, j = 0..k-1, shared.
+    int rj[kMaxTopK];
+    float wj[kMaxTopK];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, tmp[i], acc[i]);
+    for (int j = 0; j < kMaxTopK; ++j) {
+        rj[j] = j < k ? inv_perm[(size_t)t * k + j] : 0;
+        wj[j] = j < k ? topk_w[(size_t)t * k + j] : 0.f;
+    }
+    float sh[8];
+    float s = 0.f;
+    if (y_shared) {
+        s = shared_gate[t];
+        load8(y_shared + (size_t)t * H + 8 * v, sh);
+    }
+    if (residual) unpack8(reinterpret_cast<const uint4*>(residual + (size_t)t * H)[v], acc);
+#pragma unroll
+    for (int j0 = 0; j0 < kMaxTopK; j0 += 4) {
+        if (j0 < k) {
+            float rows[4][8];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj)
+                if (j0 + jj < k) load8(y_perm + (size_t)rj[j0 + jj] * H + 8 * v, rows[jj]);
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                if (j0 + jj < k) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc[i] = fmaf(wj[j0 + jj], rows[jj][i], acc[i]);
+                }
+            }
+        }
     }
     if (y_shared) {
-        const float s = shared_gate[t];
-        load8(y_shared + (size_t)t * H + 8 * v, tmp);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i] = fmaf(s, tmp[i], acc[i]);
+        for (int i = 0; i < 8; ++i) acc[i] = fmaf(s, sh[i], acc[i]);
     }
     reinterpret_cast<uint4*>(out + (size_t)t * H)[v] = pack8(acc);
 }
