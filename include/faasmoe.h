@@ -23,6 +23,9 @@
  *    Data-dependent errors (an id out of range inside a device buffer, a
  *    bounded device-side wait that ran out) set bits in a sticky device
  *    status word, never fault, and are read with moe_last_status().
+ *  - Activation and output buffers (x, x_perm, y_perm, y_shared, out, x_inout and the
+ *    debug buffers) must be 16-byte aligned: they are accessed with 16-byte vectors and
+ *    TMA tiles.  A misaligned pointer returns MOE_ERR_SHAPE and launches nothing.
  *  - Shapes: hidden, inter and shared_inter must be multiples of 128;
  *    1 <= top_k <= min(n_experts, 8); n_experts <= 256.
  *  - One context serves one device (the device current at moe_create) and
@@ -108,7 +111,10 @@ int moe_destroy(moe_ctx* ctx);
  * extracted from each MoE layer and packaged by layer and expert id).
  *   w_gate, w_up : bf16 [S, I, H]    w_down : bf16 [S, H, I]
  * Slot s holds one SwiGLU expert: y = W_down . (silu(W_gate . x) * (W_up . x)).
- * The buffers are used in place.  16-byte aligned.
+ * The buffers are used in place.  16-byte aligned.  Where the tcgen05 kernels serve the
+ * shape (hidden % 256 == 0), w_gate and w_up must be two distinct arrays whose addresses
+ * differ by less than 2^40 bytes (one TMA descriptor walks both, with their distance as a
+ * stride); otherwise MOE_ERR_UNSUPPORTED.  Two allocations of one process always qualify.
  */
 int moe_set_expert_pool(moe_ctx* ctx, int layer, const void* w_gate, const void* w_up, const void* w_down);
 
@@ -120,7 +126,12 @@ int moe_set_expert_pool(moe_ctx* ctx, int layer, const void* w_gate, const void*
  *   ws_gate/ws_up bf16 [I_s, H], ws_down bf16 [H, I_s], or all NULL if I_s = 0
  *                                      (Sec. 5: the always-active shared experts)
  *   rms_w         bf16 [H] or NULL     RMSNorm scale, needed by moe_stack_forward only
- * Used in place.
+ * Used in place; every pointer 16-byte aligned.  ws_gate and ws_up obey the same distance
+ * rule as w_gate and w_up of moe_set_expert_pool (MOE_ERR_UNSUPPORTED otherwise).
+ * Range: the shared expert's SwiGLU activations are kept in fp16 between its two
+ * projections (its 4x longer contraction needs the finer mantissa); an activation
+ * beyond +-65504 saturates there.  With weights and inputs of ordinary scale
+ * (|activation| of a few units) that range is never approached.
  */
 int moe_set_model_weights(moe_ctx* ctx, int layer, int model, const void* router_w, const float* router_bias,
                           const void* shared_gate_w, const void* ws_gate, const void* ws_up, const void* ws_down,
@@ -215,7 +226,7 @@ int moe_combine(moe_ctx* ctx, const float* y_perm, const int32_t* inv_perm, cons
  * [n_tenants] (DEVICE; an entry outside [0, M) counts as model 0), perm / inv_perm int32 [T*k], tenant_expert_count int32
  * [n_tenants*E] or NULL, expert_off int32 [M*E+1], group_off int32 [M*ceil(E/G)+1] or NULL.
  * status_out, if not NULL, is a device int32 that receives the MOE_DEV_* bits of this call
- * (it is cleared first).
+ * (it is cleared first, also when T = 0 and nothing else is launched).
  *
  * Limit: 10 + 2*n_tenants + 2*M + (ceil(T*k/256) + 1) * E*n_tenants words must fit in the
  * array; larger problems return MOE_ERR_UNSUPPORTED and launch nothing.

@@ -31,6 +31,16 @@ cudaError_t dev_alloc(T** p, size_t n)
 
 int div_up(int a, int b) { return (a + b - 1) / b; }
 
+// Activation and output buffers are read and written with 16-byte vector accesses (and as TMA tiles), so a pointer
+// that is not 16-byte aligned is refused on the host: a kernel given one would fault.
+template <typename... P>
+bool misaligned16(P... ptrs)
+{
+    uintptr_t bits = 0;
+    ((bits |= (uintptr_t)ptrs), ...);
+    return (bits & 15u) != 0;
+}
+
 int alloc_workspace(moe_ctx* c)
 {
     const moe_config& g = c->cfg;
@@ -111,6 +121,16 @@ int upload_tenant_tables(moe_ctx* c)
                            cudaMemcpyHostToDevice));
     MOE_CUDA(c, cudaMemcpy(c->d_bin_base, base.data(), sizeof(int32_t) * (g.n_models + 1), cudaMemcpyHostToDevice));
     return MOE_OK;
+}
+
+// The tensor-core gate/up kernel reads W_gate and W_up through ONE 3-D TMA map whose middle dimension steps from one
+// array to the other, so the distance between the two arrays becomes a stride of the map: it must be a non-zero
+// multiple of 16 bytes below 2^40.
+bool pair_distance_ok(const void* a, const void* b)
+{
+    const uintptr_t pa = (uintptr_t)a, pb = (uintptr_t)b;
+    const uintptr_t diff = pa < pb ? pb - pa : pa - pb;
+    return diff != 0 && (diff & 15) == 0 && diff < (1ull << 40);
 }
 
 int check_layer_ready(const moe_ctx* c, int layer, bool need_pool, bool need_shared)
@@ -315,6 +335,7 @@ int moe_set_expert_pool(moe_ctx* c, int layer, const void* w_gate, const void* w
     if (!c || !w_gate || !w_up || !w_down) return MOE_ERR_NULL;
     if (layer < 0 || layer >= c->cfg.n_layers) return MOE_ERR_SHAPE;
     if (((uintptr_t)w_gate | (uintptr_t)w_up | (uintptr_t)w_down) & 15) return MOE_ERR_SHAPE;
+    if (tc_supported(c) && !pair_distance_ok(w_gate, w_up)) return MOE_ERR_UNSUPPORTED;
     c->pools[layer] = PoolWeights{(const bf16*)w_gate, (const bf16*)w_up, (const bf16*)w_down};
     c->pool_set[layer] = 1;
     tc_destroy(c);     // descriptors are rebuilt lazily
@@ -335,6 +356,7 @@ int moe_set_model_weights(moe_ctx* c, int layer, int model, const void* router_w
     if (((uintptr_t)router_w | (uintptr_t)shared_gate_w | (uintptr_t)ws_gate | (uintptr_t)ws_up | (uintptr_t)ws_down |
          (uintptr_t)rms_w) & 15)
         return MOE_ERR_SHAPE;
+    if (any_shared && tc_supported(c) && !pair_distance_ok(ws_gate, ws_up)) return MOE_ERR_UNSUPPORTED;
     ModelWeights mw{(const bf16*)router_w, router_bias, (const bf16*)shared_gate_w, (const bf16*)ws_gate,
                     (const bf16*)ws_up, (const bf16*)ws_down, (const bf16*)rms_w};
     const size_t i = (size_t)layer * g.n_models + model;
@@ -419,6 +441,7 @@ int moe_route(moe_ctx* c, int layer, const void* x, const int32_t* tenant_id, in
 {
     if (!c || !x || !tenant_id || !topk_idx || !topk_w) return MOE_ERR_NULL;
     if (T < 0 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
+    if (misaligned16(x)) return MOE_ERR_SHAPE;
     const int rc = check_layer_ready(c, layer, false, false);
     if (rc != MOE_OK) return rc;
     if (T == 0) return MOE_OK;
@@ -434,6 +457,7 @@ int moe_dispatch(moe_ctx* c, const void* x, const int32_t* topk_idx, const int32
     if (!c || !topk_idx || !tenant_id || !perm || !inv_perm || !expert_off) return MOE_ERR_NULL;
     if (x_perm && !x) return MOE_ERR_NULL;
     if (T < 0 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
+    if (misaligned16(x, x_perm)) return MOE_ERR_SHAPE;
     if (G < 1 || G > c->cfg.n_experts) return MOE_ERR_G;
     if (T == 0) return MOE_OK;
     MOE_CUDA(c, launch_dispatch(c, (const bf16*)x, topk_idx, tenant_id, T, G, perm, inv_perm, tenant_expert_count,
@@ -446,7 +470,7 @@ int moe_experts(moe_ctx* c, int layer, const void* x, const void* x_perm, const 
 {
     if (!c || !x_perm || !expert_off || !y_perm) return MOE_ERR_NULL;
     if (y_shared && (!x || !tenant_id)) return MOE_ERR_NULL;
-    if (((uintptr_t)x_perm | (uintptr_t)x | (uintptr_t)y_perm | (uintptr_t)y_shared) & 15) return MOE_ERR_SHAPE;
+    if (misaligned16(x_perm, x, y_perm, y_shared)) return MOE_ERR_SHAPE;
     if (T < 0 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
     if (G < 1 || G > c->cfg.n_experts) return MOE_ERR_G;
     const int rc = check_layer_ready(c, layer, true, y_shared != nullptr);
@@ -463,6 +487,7 @@ int moe_combine(moe_ctx* c, const float* y_perm, const int32_t* inv_perm, const 
     if (!c || !y_perm || !inv_perm || !topk_w || !out) return MOE_ERR_NULL;
     if ((y_shared == nullptr) != (shared_gate == nullptr)) return MOE_ERR_NULL;
     if (T < 0 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
+    if (misaligned16(y_perm, y_shared, out)) return MOE_ERR_SHAPE;
     if (T == 0) return MOE_OK;
     MOE_CUDA(c, launch_combine(c, (const float*)y_perm, inv_perm, topk_w, (const float*)y_shared, shared_gate, nullptr,
                                T, (bf16*)out, (cudaStream_t)stream));
@@ -474,6 +499,7 @@ int moe_layer_forward(moe_ctx* c, int layer, const void* x, const int32_t* tenan
 {
     if (!c || !x || !tenant_id || !out) return MOE_ERR_NULL;
     if (T < 0 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
+    if (misaligned16(x, out)) return MOE_ERR_SHAPE;
     if (G < 1 || G > c->cfg.n_experts) return MOE_ERR_G;
     const int rc = check_layer_ready(c, layer, true, true);
     if (rc != MOE_OK) return rc;
@@ -507,6 +533,7 @@ int moe_layer_forward_timed(moe_ctx* c, int layer, const void* x, const int32_t*
 {
     if (!c || !x || !tenant_id || !out || !stage_ms_host) return MOE_ERR_NULL;
     if (T < 1 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
+    if (misaligned16(x, out)) return MOE_ERR_SHAPE;
     if (G < 1 || G > c->cfg.n_experts) return MOE_ERR_G;
     const int rc = check_layer_ready(c, layer, true, true);
     if (rc != MOE_OK) return rc;
@@ -527,6 +554,7 @@ int moe_stack_forward(moe_ctx* c, void* x_inout, const int32_t* tenant_id, int T
 {
     if (!c || !x_inout || !tenant_id) return MOE_ERR_NULL;
     if (T < 0 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
+    if (misaligned16(x_inout, dbg_layer_inputs, dbg_layer_outputs)) return MOE_ERR_SHAPE;
     if (G < 1 || G > c->cfg.n_experts) return MOE_ERR_G;
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         const int rc = check_layer_ready(c, l, true, true);

@@ -454,7 +454,6 @@ namespace {
 constexpr int kNoAllocWords = MOE_DISPATCH_NOALLOC_MAX_WORDS;
 static __device__ __align__(256) int32_t g_dispatch_scratch[kNoAllocWords];
 
-constexpr int kMaxDevices = 64;
 std::mutex g_scratch_mutex;
 int32_t* g_scratch_ptr[kMaxDevices] = {nullptr};
 
@@ -530,7 +529,11 @@ extern "C" int moe_dispatch_noalloc(const int32_t* topk_idx, const int32_t* tena
                     o_base = o_tim + M, o_binoff = o_base + M + 1, o_blk = o_binoff + nbins + 1,
                     total = o_blk + (long long)nblk * nbins;
     if (total > kNoAllocWords) return MOE_ERR_UNSUPPORTED;     // beyond the fixed scratch: see the header
-    if (T == 0) return MOE_OK;
+    if (T == 0) {
+        // nothing to dispatch; the caller's status word is still cleared, as for any other call
+        if (status_out && cudaMemsetAsync(status_out, 0, sizeof(int32_t), (cudaStream_t)stream) != cudaSuccess) return MOE_ERR_CUDA;
+        return MOE_OK;
+    }
     int32_t* s = nullptr;
     if (scratch_address(&s) != cudaSuccess) return MOE_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;

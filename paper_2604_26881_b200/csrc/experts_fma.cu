@@ -113,7 +113,7 @@ ffn_fma_kernel(const Tile* __restrict__ tiles, const int32_t* __restrict__ n_til
                     const int drow = dst_rows ? dst_rows[row] : row;
                     const size_t o = (size_t)drow * ld_out + c;
                     if (!SWIGLU) reinterpret_cast<float*>(out_raw)[o] = val;                       // y: fp32
-                    else if (SHARED) reinterpret_cast<__half*>(out_raw)[o] = __float2half_rn(val);  // hs: fp16
+                    else if (SHARED) reinterpret_cast<__half*>(out_raw)[o] = __float2half_rn(fminf(fmaxf(val, -65504.f), 65504.f));  // hs: fp16
                     else reinterpret_cast<bf16*>(out_raw)[o] = __float2bfloat16_rn(val);            // h: bf16
                 }
             }

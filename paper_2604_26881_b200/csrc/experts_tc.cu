@@ -190,6 +190,11 @@ __device__ __forceinline__ bool group_and(int id, bool v)
 }
 __device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 
+// The shared expert's SwiGLU activations are stored as fp16 (finer than bf16, but a range of only +-65504): a value
+// beyond that range saturates instead of becoming infinite.  Activations of that size do not occur with weights and
+// inputs of ordinary scale; every value inside the range is unchanged.
+__device__ __forceinline__ float clamp_fp16(float v) { return fminf(fmaxf(v, -65504.f), 65504.f); }
+
 struct UnitInfo {
     int a_row, amap;              // first weight row of the tile; -1: routed map, m: shared map of model m
     int b_row0, nrows, npad, ksteps, shared, cb, model;
@@ -567,7 +572,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                                     const float a = __uint_as_float(r[4 * j + 2 * t]), b = __uint_as_float(r[4 * j + 2 * t + 1]);
                                     const float g = gf ? a : b, up = gf ? b : a;
                                     const float v = __fdividef(g, 1.f + __expf(-g)) * up;
-                                    h2[t] = ui.shared ? __half_as_ushort(__float2half_rn(v)) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+                                    h2[t] = ui.shared ? __half_as_ushort(__float2half_rn(clamp_fp16(v))) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
                                 }
                                 o[j] = (uint32_t)h2[0] | ((uint32_t)h2[1] << 16);
                             }
@@ -659,7 +664,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                             const float own = __uint_as_float(even ? r[j] : r[j + 1]);
                             const float g = own_is_gate ? own : recv, up = own_is_gate ? recv : own;
                             const float v = __fdividef(g, 1.f + __expf(-g)) * up;
-                            const unsigned short o = ui.shared ? __half_as_ushort(__float2half_rn(v))
+                            const unsigned short o = ui.shared ? __half_as_ushort(__float2half_rn(clamp_fp16(v)))
                                                                : __bfloat16_as_ushort(__float2bfloat16_rn(v));
                             const uint32_t a = my_col + (uint32_t)(i * 16 + j + (even ? 0 : 1)) * 128u;
                             asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "h"(o) : "memory");
@@ -948,10 +953,13 @@ template <int MODE, bool PAIR, bool SWAP>
 cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, cudaStream_t st, int grid_cap)
 {
     auto kern = grouped_gemm_kernel<MODE, PAIR, SWAP>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        attr_set = true;
+    // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
+    static bool attr_set[kMaxDevices] = {false};
+    if (c->device < 0 || c->device >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!attr_set[c->device]) {
+        const cudaError_t ea = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (ea != cudaSuccess) return ea;
+        attr_set[c->device] = true;
     }
     if (!PAIR) {
         return launch_pdl(kern, dim3(std::max(1, std::min(c->sm_count, grid_cap))), dim3(kThreads), kSmemBytes, st, p, maps);

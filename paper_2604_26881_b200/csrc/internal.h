@@ -18,6 +18,7 @@ constexpr int kMaxExperts = 256;
 constexpr int kMaxBins = 8192;       // E * n_tenants
 constexpr int kTileRows = 128;       // rows (tokens) of one expert handled by one work unit
 constexpr int kDispatchChunk = 256;  // routed rows ranked by one block of the dispatch kernels
+constexpr int kMaxDevices = 64;      // per-device state of the library (kernel attributes, scratch addresses)
 
 // Per (layer, model) weight pointers, as the kernels see them.
 struct ModelWeights {

@@ -185,7 +185,7 @@ route_kernel(const bf16* __restrict__ x, const int32_t* __restrict__ tenant_id, 
 cudaError_t launch_route(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,
                          float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st)
 {
-    const bool tc = c->route_path != MOE_PATH_FMA && route_tc_supported(c) && ((uintptr_t)x & 15) == 0;
+    const bool tc = c->route_path != MOE_PATH_FMA && route_tc_supported(c);      // (x is 16-byte aligned: checked at the ABI)
     return tc ? launch_route_tc(c, layer, x, tenant_id, T, topk_idx, topk_w, shared_gate, tie_flag, st)
               : launch_route_fma(c, layer, x, tenant_id, T, topk_idx, topk_w, shared_gate, tie_flag, st);
 }

@@ -396,10 +396,13 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
         rm->gate_mma[layer] = gate_mma;
         rm->ready[layer] = 1;
     }
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(route_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes);
-        attr_set = true;
+    // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
+    static bool attr_set[kMaxDevices] = {false};
+    if (c->device < 0 || c->device >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!attr_set[c->device]) {
+        const cudaError_t ea = cudaFuncSetAttribute(route_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmemBytes);
+        if (ea != cudaSuccess) return ea;
+        attr_set[c->device] = true;
     }
     // token tile: only as many rows as the batch has (the MMA still reads 128 rows; the lanes of the
     // rows that were not loaded are never looked at)

@@ -19,12 +19,13 @@ from paper_2604_26881_b200 import workloads as W
 
 RTOL, ATOL = 2e-2, 2e-3
 W_RTOL = 1e-4          # router weights: fp32 softmax against fp64
-# Un-gated, un-weighted expert outputs (y_perm, y_shared) are intermediates of magnitude ~0.4-0.7
-# that the layer output scales by p ~ 0.1 or the gate ~ 0.5.  Their error is dominated by the bf16
-# rounding of the SwiGLU activations h: each of the I (or I_s) terms of a down-projection carries a
-# relative error of std 2^-9/sqrt(3), which sums to an absolute std of about 4e-4 (I = 1408) or
-# 8e-4 (I_s = 5632) whatever the size of the result.  6e-3 is seven of the larger sigmas.
-INTERMEDIATE_ATOL = 6e-3
+# Un-weighted outputs of the routed experts (y_perm) are intermediates of magnitude ~0.4 that the layer output
+# scales by p ~ 0.1-0.5.  Their error is dominated by the bf16 rounding of the SwiGLU activations h: each of the
+# I = 1408 terms of a down projection carries a relative error of std 2^-9/sqrt(3), which sums to an absolute std of
+# about 6e-4 whatever the size of the result (measured: rms 6.0e-4 at decode and prefill).  The largest excess over
+# rtol * |ref| measured over the 33.5 million elements of the full prefill is 3.1e-3 (5.2 sigma); the bound is 4e-3.
+# The shared expert keeps h in fp16 (rms error 1.5e-4, largest excess 6.6e-4) and is held to the output tolerance.
+Y_PERM_ATOL = 4e-3
 
 
 def bf16_to_f64(t: torch.Tensor) -> np.ndarray:
@@ -129,6 +130,27 @@ def check_routing(gpu_idx: np.ndarray, gpu_w: np.ndarray, ref, k: int):
     return gpu_idx.copy(), mask
 
 
+def check_tie_flag(gpu_flag: np.ndarray, probs: np.ndarray, oracle_flag: np.ndarray, k: int):
+    """The GPU's near-tie flag against the oracle's.
+
+    The flag says that two neighbouring ranks among ranks 1..k+1 differ by less than 1e-5 relative.  The GPU
+    decides that on fp32 probabilities, so a token whose smallest such gap lies within rounding of the threshold
+    may be flagged either way; everywhere else (smallest gap outside [0.5e-5, 2e-5], in the oracle's fp64
+    probabilities) the two flags must be equal.  Returns the number of tokens compared."""
+    T, E = probs.shape
+    srt = -np.sort(-probs, axis=1)[:, :min(k + 1, E)]
+    if srt.shape[1] < 2:
+        assert not gpu_flag.any() and not oracle_flag.any()
+        return T
+    gap = ((srt[:, :-1] - srt[:, 1:]) / srt[:, :-1]).min(axis=1)
+    decided = (gap < 0.5e-5) | (gap > 2e-5)
+    # the oracle's own flag agrees with this restatement wherever the gap is clear of the threshold
+    assert np.array_equal(oracle_flag[decided].astype(bool), gap[decided] < 1e-5)
+    bad = np.nonzero(decided & (gpu_flag.astype(bool) != oracle_flag.astype(bool)))[0]
+    assert bad.size == 0, f"tie_flag differs from the oracle on tokens {bad[:8]} (gaps {gap[bad[:8]]})"
+    return int(decided.sum())
+
+
 def oracle_layer(wl, wts: dict, x: torch.Tensor, tenant: torch.Tensor, mot: torch.Tensor, G: int,
                  gpu_idx=None, gpu_w=None):
     """Oracle result for a layer; with gpu_idx given, applies the near-tie protocol first."""
@@ -163,6 +185,7 @@ def compare_four_calls(o: dict, ref, wl, x: torch.Tensor):
     np.testing.assert_allclose(o["topk_w"].cpu().numpy(), ref.routing.topk_w, rtol=W_RTOL, atol=1e-9)
     if wl.Is:
         np.testing.assert_allclose(o["shared_gate"].cpu().numpy(), ref.routing.shared_gate, rtol=1e-5, atol=1e-7)
+    check_tie_flag(o["tie_flag"].cpu().numpy(), ref.routing.probs, ref.routing.tie_flag, k)
     d = ref.dispatch
     assert np.array_equal(o["perm"].cpu().numpy(), d.perm)
     assert np.array_equal(o["inv_perm"].cpu().numpy(), d.inv_perm)
@@ -175,7 +198,7 @@ def compare_four_calls(o: dict, ref, wl, x: torch.Tensor):
     xp = o["x_perm"].cpu().view(torch.int16).numpy()
     xs = x.view(torch.int16).numpy()
     assert np.array_equal(xp, xs[d.perm // k])
-    assert_close("y_perm", bf16_to_f64(o["y_perm"]), ref.y_perm, atol=INTERMEDIATE_ATOL)
+    assert_close("y_perm", bf16_to_f64(o["y_perm"]), ref.y_perm, atol=Y_PERM_ATOL)
     if wl.Is:
-        assert_close("y_shared", bf16_to_f64(o["y_shared"]), ref.y_shared, atol=INTERMEDIATE_ATOL)
+        assert_close("y_shared", bf16_to_f64(o["y_shared"]), ref.y_shared)
     assert_close("out", bf16_to_f64(o["out"]), ref.out)

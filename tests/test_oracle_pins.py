@@ -405,3 +405,38 @@ def test_rmsnorm_matches_numpy_and_zero_weights_make_block_identity():
     assert np.array_equal(x_next, c["x_u"])
     assert np.array_equal(xn_u, oracle.round_bf16(ref)) or np.max(np.abs(
         xn_u.astype(np.int32) - oracle.round_bf16(ref).astype(np.int32))) <= 1
+
+
+def _nearest_bf16_by_table(v):
+    """Round-to-nearest-even onto bf16 by searching the sorted table of all finite bf16 values."""
+    bits = np.arange(1 << 16, dtype=np.uint32)
+    with np.errstate(invalid="ignore"):
+        vals = (bits << 16).view(np.float32).astype(np.float64)
+    ok = np.isfinite(vals) & ~((bits == 0x8000))            # one zero
+    bits, vals = bits[ok], vals[ok]
+    order = np.argsort(vals, kind="stable")
+    bits, vals = bits[order], vals[order]
+    hi = np.clip(np.searchsorted(vals, v), 1, len(vals) - 1)
+    lo = hi - 1
+    dl, dh = np.abs(v - vals[lo]), np.abs(vals[hi] - v)
+    pick_hi = (dh < dl) | ((dh == dl) & ((bits[hi] & 1) == 0))
+    return np.where(pick_hi, bits[hi], bits[lo]).astype(np.uint16)
+
+
+def test_block_forward_residual_add_with_nonzero_layer_output():
+    # x_next = bf16(x + layer(xn)) with a layer output that is far from zero.  The sum is restated with numpy on the
+    # exact bf16 values of x and rounded by a table search over all bf16 values (no shared rounding code), so a wrong
+    # sign, a dropped summand or a scale on either term fails.
+    c = small_case(seed=33, Is=8)
+    g_u, _ = bf16(1.0 + 0.02 * np.random.default_rng(2).standard_normal(c["H"]))
+    wts = dict(c["wts"]); wts["rms_w"] = g_u
+    x_next, xn_u, res = oracle.block_forward(c["x_u"], c["tenant"], c["mot"], wts, k=2, G=1, eps=1e-6)
+    assert np.abs(res.out).max() > 1e-2                       # the layer really contributes
+    # the layer inside the block ran on the rounded normalised input
+    direct = _layer(dict(c, wts=wts), x_u=xn_u)
+    assert np.array_equal(direct.out, res.out)
+    total = c["x"] + res.out                                   # fp64, exact inputs
+    assert np.array_equal(x_next, _nearest_bf16_by_table(total))
+    # the classic mistakes give other bits
+    for wrong in (c["x"] - res.out, c["x"] + 2 * res.out, res.out, c["x"]):
+        assert not np.array_equal(_nearest_bf16_by_table(wrong), x_next)

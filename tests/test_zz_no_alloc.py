@@ -66,6 +66,15 @@ def test_noalloc_dispatch_matches_dispatch_on_two_calls_in_a_row():
     _run_both(seed=3, T=1500, k=4, E=60, M=3, n_tenants=7, G=60, dev=dev)
 
 
+def test_noalloc_dispatch_of_an_empty_batch_clears_the_status_word():
+    dev = torch.device("cuda:0")
+    z = torch.zeros(8, dtype=torch.int32, device=dev)
+    status = torch.full((1,), 99, dtype=torch.int32, device=dev)
+    B.moe_dispatch_noalloc(z, z, z, 0, 2, 8, 1, 1, 1, z, z, None, z, None, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+
+
 def test_noalloc_dispatch_rejects_what_does_not_fit():
     dev = torch.device("cuda:0")
     z = torch.zeros(8, dtype=torch.int32, device=dev)
