@@ -1,18 +1,27 @@
 #!/usr/bin/env python
 """Benchmark of the multi-tenant MoE layer hot path (route -> dispatch -> experts -> combine).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload decode|prefill|pool] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload decode|prefill|pool|stack] [--impl reference]
 
-One step is one pass of the whole layer over one batch of seeded synthetic tokens at the
-Qwen1.5-MoE layer shape.  With N > 1 (launched by torch.distributed.run) every rank runs an
-independent replica on its own batch (the layer has no exchange step), time is the maximum over
-ranks and the value is the aggregate tokens/s.  Prints one JSON line on rank 0.
+One step is one pass of the whole layer (for `stack`: of the 24 blocks) over one batch of seeded synthetic
+tokens at the Qwen1.5-MoE layer shape.  A timed block is exactly K steps between a barrier + device synchronise on
+both sides; blocks are repeated until at least --min-time seconds have been timed, and the MEDIAN block gives
+`ms_per_step` (the first, fastest and slowest blocks and the clocks sampled meanwhile are printed beside it), so a
+burst of a few milliseconds on a cold part cannot stand for the step time.
+
+Without --workload the headline line is the 32-token decode layer and the same JSON line carries the other
+workloads (prefill, pool, stack) under "workloads".  With N > 1 every rank runs an independent replica on its own
+batch (the layer has no exchange step), time is the maximum over ranks and the value the aggregate tokens/s;
+`--gpus N` starts its own ranks (one process per GPU) unless a launcher already did.  Rank 0 prints one JSON line.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import math
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -30,14 +39,19 @@ from paper_2604_26881_b200 import workloads as W
 
 METRIC = "MoE-layer tokens/s at Qwen1.5-MoE shape on 1 B200"
 UNIT = "tokens/s"
+DEFAULT_STEPS = {"decode": 1000, "prefill": 200, "pool": 100, "stack": 20}
+EXTRA_WORKLOADS = ("prefill", "pool", "stack")     # measured beside the headline when no --workload is given
 
 
-def parse_args():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill", "pool", "stack"])
+    ap.add_argument("--workload", default=None, choices=["decode", "prefill", "pool", "stack"],
+                    help="one workload only; default: decode as the headline and the others under 'workloads'")
+    ap.add_argument("--min-time", type=float, default=1.5,
+                    help="seconds of timed blocks per workload (each block is exactly --steps steps)")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "fma", "tcgen05"])
     ap.add_argument("--pair", default="auto", choices=["auto", "never"])
@@ -46,7 +60,24 @@ def parse_args():
                          "the per-stage times and the roofline block always come from passes without it, where one "
                          "grouped-GEMM launch holds the shared and the routed units")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    return ap.parse_args()
+    ap.add_argument("--dry", action="store_true",
+                    help="exercise the launch and reduction protocol without a GPU (gloo ranks, a sleep as the step)")
+    return ap.parse_args(argv)
+
+
+def _free_port() -> int:
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def spawn_ranks(n: int) -> int:
+    """Re-runs this command line as n ranks (one process per GPU) under torch.distributed.run."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def measured_peaks():
@@ -90,7 +121,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, smax, reasons = [], [], set()
+        sm, smax, power, reasons = [], [], [], set()
         try:
             with open(self.path) as f:
                 for line in f:
@@ -99,6 +130,7 @@ class ClockSampler:
                         continue
                     try:
                         sm.append(float(c[1])); smax.append(float(c[2]))
+                        power.append(float(c[3]))
                     except ValueError:
                         continue
                     for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
@@ -109,9 +141,64 @@ class ClockSampler:
         except Exception:
             pass
         if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
+            out.update(sm_mhz=statistics.median(sm), sm_min_mhz=min(sm), sm_max_mhz=max(smax), samples=len(sm))
+        if power:
+            out["power_w_median"] = statistics.median(power)
         out["reasons"] = sorted(reasons)
         return out
+
+
+def timed_blocks(step_fn, steps: int, min_time_s: float, world: int, sync, dev, make_events, max_blocks: int = 5000):
+    """Times blocks of exactly `steps` calls of step_fn, each between a barrier + synchronise on both sides, until
+    min_time_s seconds have been timed (every rank runs the same number of blocks: the slowest rank's first block
+    decides).  Returns per-block durations in ms, already reduced to the maximum over ranks."""
+    def one_block():
+        replicas.barrier(world, sync)
+        e0, e1 = make_events()
+        e0.record()
+        for _ in range(steps):
+            step_fn()
+        e1.record()
+        replicas.barrier(world, sync)
+        return e0.elapsed_time(e1)
+
+    blocks = [one_block()]
+    first = replicas.max_over_ranks([blocks[0]], world, dev)[0]
+    n_more = int(min(max_blocks, math.ceil(max(0.0, min_time_s * 1e3 - first) / max(first, 1e-3))))
+    for _ in range(n_more):
+        blocks.append(one_block())
+    return replicas.max_over_ranks(blocks, world, dev)
+
+
+def block_summary(blocks_ms, steps: int) -> dict:
+    return {"n": len(blocks_ms), "steps_per_block": steps, "median_ms": statistics.median(blocks_ms),
+            "first_ms": blocks_ms[0], "min_ms": min(blocks_ms), "max_ms": max(blocks_ms), "timed_s": sum(blocks_ms) * 1e-3}
+
+
+def kernel_source_digest() -> str:
+    """SHA-256 over the grouped-GEMM sources: a DRAM-traffic figure taken from a profile is only quoted while the
+    kernel it was measured on is still the one that runs."""
+    h = hashlib.sha256()
+    for name in ("experts_tc.cu", "tc_ptx.cuh", "plan.cuh"):
+        with open(os.path.join(ROOT, "paper_2604_26881_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, copied from the
+# ncu summaries under profiles/ together with the digest of the kernel sources they were captured on.  bench.py prints
+# the figure only while kernel_source_digest() still equals `digest`; otherwise `traffic` is null.
+NCU_TRAFFIC = {
+}
+
+
+def traffic_record(workload: str, path: str):
+    rec = NCU_TRAFFIC.get(workload)
+    if rec is None or path != "auto":
+        return None, None
+    if rec["digest"] != kernel_source_digest():
+        return None, f"{rec['source']} (stale: the kernel sources have changed since that capture)"
+    return rec["bytes"], rec["source"]
 
 
 def algorithmic_work(wl, active_experts: int, T: int):
@@ -129,30 +216,29 @@ def algorithmic_work(wl, active_experts: int, T: int):
     return dict(total_bytes=total_bytes, flops=flops, gateup_bytes=gateup_bytes, gateup_flops=gateup_flops)
 
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
-# ncu captures summarised in profiles/grouped_gemm_decode_ncu.md and profiles/grouped_gemm_prefill_ncu.md; None where
-# no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"decode": 657.659136e6 + 4.132608e6, "prefill": 860.452352e6 + 84.881920e6}
+def oracle_sample(wl, wts, x, tenant, mot):
+    """Inputs of the oracle's timed sample: the first 32 tokens of the batch."""
+    n = min(x.shape[0], 32)
+    xs, ts = x[:n].contiguous(), tenant[:n].contiguous()
+    return n, W.as_u16(xs), ts.numpy(), mot.numpy(), W.weights_as_numpy(wts)
 
 
-def run_reference(args, wl, rank):
+def run_reference(args, rank):
     """The oracle, as it stands, on the host cores: each step is a bounded sample of the workload."""
     import oracle
     if rank != 0:
         return
+    wl = W.WORKLOADS[args.workload or "decode"]
     steps = args.steps if args.steps is not None else 3
     warmup = args.warmup if args.warmup is not None else 1
     steps, warmup = min(steps, 10), min(warmup, 2)      # bounded: each pass is about a second of CPU work
     wts = W.make_weights(wl, seed=0)
     x, tenant, mot = W.make_tokens(wl, seed=0)
-    n = min(x.shape[0], 32)
-    xs, ts = x[:n].contiguous(), tenant[:n].contiguous()
-    wn = W.weights_as_numpy(wts)
-    xu = W.as_u16(xs)
+    n, xu, ts, mn, wn = oracle_sample(wl, wts, x, tenant, mot)
     times = []
     for i in range(warmup + steps):
         t0 = time.perf_counter()
-        oracle.layer_forward(xu, ts.numpy(), mot.numpy(), wn, k=wl.k, G=wl.G)
+        oracle.layer_forward(xu, ts, mn, wn, k=wl.k, G=wl.G)
         if i >= warmup:
             times.append(time.perf_counter() - t0)
     total = sum(times)
@@ -171,30 +257,157 @@ def run_reference(args, wl, rank):
 def cpu_baseline(wl, wts, x, tenant, mot):
     """The oracle timed on the host cores on a bounded sample of the same batch."""
     import oracle
-    n = min(x.shape[0], 32)
-    xs, ts = x[:n].contiguous(), tenant[:n].contiguous()
-    wn = W.weights_as_numpy(wts)
-    xu = W.as_u16(xs)
-    oracle.layer_forward(xu[:2], ts.numpy()[:2], mot.numpy(), wn, k=wl.k, G=wl.G)     # page in
+    n, xu, ts, mn, wn = oracle_sample(wl, wts, x, tenant, mot)
+    oracle.layer_forward(xu[:2], ts[:2], mn, wn, k=wl.k, G=wl.G)     # page in
     reps, t0 = 0, time.perf_counter()
     while reps < 3 or (time.perf_counter() - t0 < 10.0 and reps < 20):
-        oracle.layer_forward(xu, ts.numpy(), mot.numpy(), wn, k=wl.k, G=wl.G)
+        oracle.layer_forward(xu, ts, mn, wn, k=wl.k, G=wl.G)
         reps += 1
     dt = time.perf_counter() - t0
     return {"value": n * reps / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"first {n} tokens of the {wl.name} batch, {reps} passes, {dt:.1f} s"}
 
 
-def run_stack(args, wl, rank, local_rank, world):
+def apply_options(B, ctx, args):
+    B.moe_set_option(ctx, B.MOE_OPT_EXPERT_PATH, {"auto": 0, "fma": 1, "tcgen05": 2}[args.path])
+    B.moe_set_option(ctx, B.MOE_OPT_PAIR_MODE, {"auto": 1, "never": 0}[args.pair])
+    if args.early_shared != "auto":
+        B.moe_set_option(ctx, B.MOE_OPT_EARLY_SHARED, int(args.early_shared))
+
+
+def cuda_events():
+    return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+
+def dispatch_mode_report(B, ctx, step_fn, steps, world, dev):
+    """Invocations and step time under a shared orchestrator and under private (per-tenant) orchestrators: the same
+    work, the same results, batched across tenants or per tenant (a short timed block per mode)."""
+    out = {}
+    for name, mode in (("shared", B.MOE_DISPATCH_SHARED), ("private", B.MOE_DISPATCH_PRIVATE)):
+        B.moe_set_option(ctx, B.MOE_OPT_DISPATCH_MODE, mode)
+        for _ in range(3):
+            step_fn()
+        blocks = timed_blocks(step_fn, steps, 0.25, world, torch.cuda.synchronize, dev, cuda_events)
+        status, n_inv, _ = B.moe_last_status(ctx)
+        if status != 0:
+            raise SystemExit(f"device status {status} in dispatch mode {name}")
+        out[name] = {"invocations_last_layer": n_inv, "ms_per_step": statistics.median(blocks) / steps}
+    B.moe_set_option(ctx, B.MOE_OPT_DISPATCH_MODE, B.MOE_DISPATCH_SHARED)
+    return out
+
+
+def measure_layer(args, wl, rank, local_rank, world, dev, wts_cache, with_cpu_baseline):
+    """One single-layer workload (decode, prefill, pool): device-resident throughput, per-stage times, end to end
+    through the host-buffer entry point, roofline of the dominant kernel and of the whole path."""
+    from paper_2604_26881_b200 import binding as B
+    steps = args.steps if args.steps is not None else DEFAULT_STEPS[wl.name]
+    warmup = max(args.warmup if args.warmup is not None else 20, 3)
+    # every rank is an independent replica with its own batch (different seed), same weights recipe; the Qwen-shape
+    # decode and prefill layers share their expert weights (prefill adds the router bias)
+    key = (wl.H, wl.E, wl.I, wl.Is, wl.M)
+    if key not in wts_cache:
+        wts_cache[key] = W.make_weights(W.scaled(wl, zipf_bias=True), seed=0)
+    wts = dict(wts_cache[key])
+    if not wl.zipf_bias:
+        wts["router_bias"] = None
+    x, tenant, mot = W.make_tokens(wl, seed=replicas.rank_seed(0, rank))
+    T = x.shape[0]
+    layer = B.MoELayer(H=wl.H, E=wl.E, I=wl.I, k=wl.k, Is=wl.Is, M=wl.M, n_tenants=wl.n_tenants, max_tokens=T,
+                       device=str(dev))
+    try:
+        layer.set_layer_weights(0, wts)
+        layer.set_tables(slot_table=wts["slot_table"], model_of_tenant=mot)
+        ctx = layer.ctx
+        apply_options(B, ctx, args)
+        xd, td = x.to(dev), tenant.to(dev)
+        out = torch.zeros_like(xd)
+        stream = torch.cuda.current_stream()
+
+        # ---- device-resident throughput -----------------------------------------------------------
+        for _ in range(warmup):
+            B.moe_layer_forward(ctx, 0, xd, td, T, wl.G, out, stream)
+        torch.cuda.synchronize()
+        status, n_inv, active = B.moe_last_status(ctx)
+        if status != 0:
+            raise SystemExit(f"device status {status} after warm-up")
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        l0 = B.moe_launch_count(ctx)
+        blocks = timed_blocks(lambda: B.moe_layer_forward(ctx, 0, xd, td, T, wl.G, out, stream), steps, args.min_time,
+                              world, torch.cuda.synchronize, dev, cuda_events)
+        clocks = sampler.stop()
+        launches = (B.moe_launch_count(ctx) - l0) // len(blocks)
+
+        # ---- per-stage durations (CUDA events on the launching stream, between the kernels) ---------
+        stage_ms = B.moe_stage_times(ctx, xd, td, T, wl.G, out, reps=max(10, min(steps, 100)))
+
+        # ---- end to end through the host-buffer entry point ---------------------------------------
+        xh, th = x.contiguous().pin_memory(), tenant.contiguous().pin_memory()
+        oh = torch.zeros_like(xh).pin_memory()
+        e2e_steps = max(10, min(steps, 200))
+        for _ in range(3):
+            B.moe_layer_forward_host(ctx, 0, xh, th, T, wl.G, oh, stream)
+        e2e_blocks = timed_blocks(lambda: B.moe_layer_forward_host(ctx, 0, xh, th, T, wl.G, oh, stream), e2e_steps,
+                                  min(args.min_time, 0.5), world, torch.cuda.synchronize, dev, cuda_events)
+        modes = None
+        if wl.n_tenants > 1:
+            modes = dispatch_mode_report(B, ctx, lambda: B.moe_layer_forward(ctx, 0, xd, td, T, wl.G, out, stream),
+                                         max(10, steps // 10), world, dev)
+    finally:
+        layer.close()
+
+    if rank != 0:
+        return None
+    peaks = measured_peaks()
+    work = algorithmic_work(wl, active, T)
+    bs = block_summary(blocks, steps)
+    ms_step = bs["median_ms"] / steps
+    e2e_ms_step = statistics.median(e2e_blocks) / e2e_steps
+    t_hbm = work["total_bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_tc = work["flops"] / (peaks["bf16_tflops"] * 1e12)
+    bound = "hbm" if t_hbm >= t_tc else "tensor"
+    gu_ms = stage_ms.get("experts_gateup")            # dominant kernel: the gate/up grouped GEMM of moe_experts
+    if bound == "hbm":
+        achieved = work["gateup_bytes"] / (gu_ms * 1e-3) / 1e9 if gu_ms else None
+        peak, runit = peaks["hbm_gbs"], "GB/s"
+    else:
+        achieved = work["gateup_flops"] / (gu_ms * 1e-3) / 1e12 if gu_ms else None
+        peak, runit = peaks["bf16_tflops"], "TFLOP/s"
+    traffic, traffic_source = traffic_record(wl.name, args.path)
+    roofline = {"bound": bound, "kernel": "moe_experts gate/up grouped GEMM", "achieved": achieved, "peak": peak,
+                "unit": runit, "frac": (achieved / peak) if achieved else None,
+                "traffic": traffic, "traffic_source": traffic_source,
+                "algorithmic": work["gateup_bytes"] if bound == "hbm" else work["gateup_flops"],
+                "peak_source": peaks["source"],
+                "path": {"roofline_ms": 1e3 * max(t_hbm, t_tc), "measured_ms": ms_step,
+                         "frac": 1e3 * max(t_hbm, t_tc) / ms_step, "algorithmic_bytes": work["total_bytes"],
+                         "flops": work["flops"], "active_experts": active},
+                "stage_ms": stage_ms}
+    line = {"metric": METRIC, "value": world * T / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "tokens_per_step_per_gpu": T, "hidden": wl.H, "experts": wl.E,
+                       "inter": wl.I, "top_k": wl.k, "shared_inter": wl.Is, "G": wl.G, "tenants": wl.n_tenants,
+                       "models": wl.M, "expert_path": args.path, "early_shared": args.early_shared,
+                       "l2": "expert weights (about 1 GB per pass) exceed the 126 MB L2; no flush",
+                       "parallelism": f"replicas x{world}"},
+            "blocks": bs, "clocks": clocks, "gpu_launches": int(launches) * len(blocks),
+            "gpu_launches_per_block": int(launches),
+            "e2e": {"value": world * T / (e2e_ms_step * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": int(T * wl.H * 2 + T * 4), "d2h_bytes_per_step": int(T * wl.H * 2),
+                    "ms_per_step": e2e_ms_step},
+            "roofline": roofline}
+    if modes:
+        line["dispatch_modes"] = modes
+    if with_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl, wts, x, tenant, mot)
+    return line
+
+
+def measure_stack(args, wl, rank, local_rank, world, dev):
     """The 24-block configuration: RMSNorm -> MoE layer (+shared expert) -> residual, 26.6 GB of weights resident."""
     from paper_2604_26881_b200 import binding as B
-    import torch.distributed as dist
-    dev = torch.device(f"cuda:{local_rank}")
-    torch.cuda.set_device(dev)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
-    steps = args.steps if args.steps is not None else 30
+    steps = args.steps if args.steps is not None else DEFAULT_STEPS["stack"]
     warmup = max(args.warmup if args.warmup is not None else 3, 3)
     x, tenant, mot = W.make_tokens(wl, seed=replicas.rank_seed(0, rank))
     T = x.shape[0]
@@ -204,80 +417,138 @@ def run_stack(args, wl, rank, local_rank, world):
         return (torch.randn(*shape, generator=gen, device=dev, dtype=torch.float32) * std).to(torch.bfloat16)
     layer = B.MoELayer(H=wl.H, E=wl.E, I=wl.I, k=wl.k, Is=wl.Is, M=1, n_tenants=wl.n_tenants, max_tokens=T,
                        n_layers=wl.n_layers, device=str(dev))
-    S = wl.n_slots
-    for l in range(wl.n_layers):
-        layer.set_layer_weights(l, {
-            "router_w": rnd(1, wl.E, wl.H), "router_bias": None, "pool_gate": rnd(S, wl.I, wl.H),
-            "pool_up": rnd(S, wl.I, wl.H), "pool_down": rnd(S, wl.H, wl.I), "shared_gate_w": rnd(1, wl.H),
-            "ws_gate": rnd(1, wl.Is, wl.H), "ws_up": rnd(1, wl.Is, wl.H), "ws_down": rnd(1, wl.H, wl.Is),
-            "rms_w": (1.0 + torch.randn(wl.H, generator=gen, device=dev) * 0.02).to(torch.bfloat16)})
-    layer.set_tables(model_of_tenant=mot)
-    ctx = layer.ctx
-    B.moe_set_option(ctx, B.MOE_OPT_PAIR_MODE, {"auto": 1, "never": 0}[args.pair])
-    if args.early_shared != "auto":
-        B.moe_set_option(ctx, B.MOE_OPT_EARLY_SHARED, int(args.early_shared))
-    xd, td = x.to(dev), tenant.to(dev)
-    xw = xd.clone()
-    stream = torch.cuda.current_stream()
-    for _ in range(warmup):
+    try:
+        S = wl.n_slots
+        for l in range(wl.n_layers):
+            layer.set_layer_weights(l, {
+                "router_w": rnd(1, wl.E, wl.H), "router_bias": None, "pool_gate": rnd(S, wl.I, wl.H),
+                "pool_up": rnd(S, wl.I, wl.H), "pool_down": rnd(S, wl.H, wl.I), "shared_gate_w": rnd(1, wl.H),
+                "ws_gate": rnd(1, wl.Is, wl.H), "ws_up": rnd(1, wl.Is, wl.H), "ws_down": rnd(1, wl.H, wl.Is),
+                "rms_w": (1.0 + torch.randn(wl.H, generator=gen, device=dev) * 0.02).to(torch.bfloat16)})
+        layer.set_tables(model_of_tenant=mot)
+        ctx = layer.ctx
+        apply_options(B, ctx, args)
+        xd, td = x.to(dev), tenant.to(dev)
+        xw = xd.clone()
+        stream = torch.cuda.current_stream()
+
+        def step():
+            xw.copy_(xd)
+            B.moe_stack_forward(ctx, xw, td, T, wl.G, None, None, stream)
+        for _ in range(warmup):
+            step()
+        torch.cuda.synchronize()
+        if B.moe_last_status(ctx)[0] != 0:
+            raise SystemExit("device status set after warm-up")
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        l0 = B.moe_launch_count(ctx)
+        blocks = timed_blocks(step, steps, args.min_time, world, torch.cuda.synchronize, dev, cuda_events)
+        clocks = sampler.stop()
+        launches = (B.moe_launch_count(ctx) - l0) // len(blocks)
+        # Realised active experts and stage times per block: one more pass keeps every block's normalised input, then
+        # each block's layer is run alone on it (same kernels, same inputs) with events between its stages.
+        dbg_in = torch.zeros((wl.n_layers, T, wl.H), dtype=torch.bfloat16, device=dev)
         xw.copy_(xd)
-        B.moe_stack_forward(ctx, xw, td, T, wl.G, None, None, stream)
-    torch.cuda.synchronize()
-    if B.moe_last_status(ctx)[0] != 0:
-        raise SystemExit("device status set after warm-up")
-    sampler = ClockSampler(local_rank)
-    replicas.barrier(world, torch.cuda.synchronize)
-    sampler.start()
-    l0 = B.moe_launch_count(ctx)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record(stream)
-    for _ in range(steps):
-        xw.copy_(xd)
-        B.moe_stack_forward(ctx, xw, td, T, wl.G, None, None, stream)
-    ev1.record(stream)
-    replicas.barrier(world, torch.cuda.synchronize)
-    clocks = sampler.stop()
-    launches = B.moe_launch_count(ctx) - l0
-    ms_total = replicas.max_over_ranks([ev0.elapsed_time(ev1)], world, dev)[0]
+        B.moe_stack_forward(ctx, xw, td, T, wl.G, dbg_in, None, stream)
+        torch.cuda.synchronize()
+        out = torch.zeros_like(xd)
+        active_per_block, stage_ms = [], {}
+        for l in range(wl.n_layers):
+            st = B.moe_stage_times(ctx, dbg_in[l], td, T, wl.G, out, reps=5, layer=l)
+            for k_, v in st.items():
+                stage_ms[k_] = stage_ms.get(k_, 0.0) + v
+            active_per_block.append(B.moe_last_status(ctx)[2])
+        modes = dispatch_mode_report(B, ctx, step, max(3, steps // 4), world, dev)
+    finally:
+        layer.close()
+    if rank != 0:
+        return None
+    peaks = measured_peaks()
+    expert_bytes = 3 * wl.H * wl.I * 2
+    fixed_bytes = 3 * wl.H * wl.Is * 2 + (wl.E + 1) * wl.H * 2 + wl.H * 2 + 4 * T * wl.H
+    total_bytes = sum(a * expert_bytes + fixed_bytes for a in active_per_block)
+    flops = wl.n_layers * T * (wl.k * 6 * wl.H * wl.I + 6 * wl.H * wl.Is + 2 * wl.H * wl.E)
+    t_hbm, t_tc = total_bytes / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)
+    bs = block_summary(blocks, steps)
+    ms_step = bs["median_ms"] / steps
+    stage_ms["rmsnorm_and_gaps"] = ms_step - sum(stage_ms.values())
+    resident_bytes = wl.n_layers * (wl.E * expert_bytes + 3 * wl.H * wl.Is * 2 + (wl.E + 1) * wl.H * 2 + wl.H * 2)
+    return {"metric": METRIC, "value": world * T / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "blocks": wl.n_layers, "tokens_per_step_per_gpu": T, "tenants": wl.n_tenants,
+                       "G": wl.G, "weights_gb": resident_bytes / 1e9,
+                       "l2": "26.6 GB of weights per pass exceed the 126 MB L2; no flush",
+                       "parallelism": f"replicas x{world}"},
+            "blocks": bs, "clocks": clocks, "gpu_launches": int(launches) * len(blocks),
+            "gpu_launches_per_block": int(launches), "dispatch_modes": modes,
+            "roofline": {"bound": "hbm" if t_hbm >= t_tc else "tensor", "kernel": "whole stack",
+                         "achieved": total_bytes / (ms_step * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": 1e3 * max(t_hbm, t_tc) / ms_step, "traffic": None, "traffic_source": None,
+                         "algorithmic": total_bytes, "peak_source": peaks["source"],
+                         "active_experts_per_block": active_per_block,
+                         "path": {"roofline_ms": 1e3 * max(t_hbm, t_tc), "measured_ms": ms_step,
+                                  "frac": 1e3 * max(t_hbm, t_tc) / ms_step, "algorithmic_bytes": total_bytes,
+                                  "flops": flops},
+                         "stage_ms": stage_ms,
+                         "stage_note": "stage times: every block's layer run alone on its own input (merged launches); "
+                                       "rmsnorm_and_gaps = step time minus their sum"}}
+
+
+def run_dry(args, rank, world):
+    """The launch and reduction protocol without a GPU: gloo ranks, a short sleep as the step.  What the ranks do is
+    what the GPU run does around its kernels: one batch per rank, blocks of exactly K steps between barriers, the
+    maximum over ranks per block, the median block, one JSON line from rank 0."""
+    import torch.distributed as dist
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("gloo")
+    wl = W.WORKLOADS[args.workload or "decode"]
+    steps = args.steps if args.steps is not None else 5
+    x, _, _ = W.make_tokens(W.scaled(wl, T=min(wl.T or 64, 64), H=128), seed=replicas.rank_seed(0, rank))
+    T = x.shape[0]
+
+    class HostEvent:
+        def record(self):
+            self.t = time.perf_counter()
+
+        def elapsed_time(self, other):
+            return 1e3 * (other.t - self.t)
+
+    step_s = 1e-3 * (rank + 1)                      # the last rank is the slow one
+    blocks = timed_blocks(lambda: time.sleep(step_s), steps, min(args.min_time, 0.05), world, None, None,
+                          lambda: (HostEvent(), HostEvent()))
+    checksum = replicas.sum_over_ranks(float(x.to(torch.float64).sum()), world)
     if rank == 0:
-        peaks = measured_peaks()
-        layer_bytes = wl.E * 3 * wl.H * wl.I * 2 + 3 * wl.H * wl.Is * 2 + (wl.E + 1) * wl.H * 2 + wl.H * 2
-        total_bytes = wl.n_layers * (layer_bytes + 4 * T * wl.H)          # upper bound: all experts active
-        flops = wl.n_layers * T * (wl.k * 6 * wl.H * wl.I + 6 * wl.H * wl.Is + 2 * wl.H * wl.E)
-        t_hbm, t_tc = total_bytes / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)
-        ms_step = ms_total / steps
-        line = {"metric": METRIC, "value": world * T * steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
-                "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": wl.name, "blocks": wl.n_layers, "tokens_per_step_per_gpu": T, "tenants": wl.n_tenants,
-                           "G": wl.G, "weights_gb": wl.n_layers * layer_bytes / 1e9,
-                           "l2": "26.6 GB of weights per pass exceed the 126 MB L2; no flush",
-                           "parallelism": f"replicas x{world}"},
-                "clocks": clocks, "gpu_launches": int(launches),
-                "roofline": {"bound": "hbm" if t_hbm >= t_tc else "tensor", "kernel": "whole stack",
-                             "achieved": total_bytes / (ms_step * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                             "frac": 1e3 * max(t_hbm, t_tc) / ms_step, "traffic": None, "peak_source": peaks["source"],
-                             "note": "bytes assume every expert of every block is active"}}
-        print(json.dumps(line), flush=True)
-    layer.close()
+        bs = block_summary(blocks, steps)
+        ms_step = bs["median_ms"] / steps
+        print(json.dumps({"metric": METRIC, "value": world * T / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+                          "steps": steps, "warmup": 0, "ms_per_step": ms_step, "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "none", "data": "synthetic", "dry": True,
+                          "config": {"workload": wl.name, "tokens_per_step_per_gpu": T, "parallelism": f"replicas x{world}"},
+                          "blocks": bs, "batch_checksum": checksum, "gpu_launches": 0}), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
 def main():
     args = parse_args()
+    # `--gpus N` without a launcher: start the N ranks here (one process per GPU); the reference arm runs on rank 0 alone
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        sys.exit(spawn_ranks(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    wl = W.WORKLOADS[args.workload]
 
     if args.impl == "reference":
-        run_reference(args, wl, rank)
+        run_reference(args, rank)
+        return
+    if args.dry:
+        run_dry(args, rank, world)
         return
 
-    from paper_2604_26881_b200 import binding as B
     import torch.distributed as dist
-
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     dev = torch.device(f"cuda:{local_rank}")
@@ -286,116 +557,25 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
 
-    if wl.n_layers > 1:
-        run_stack(args, wl, rank, local_rank, world)
-        return
-    steps = args.steps if args.steps is not None else {"decode": 3000, "prefill": 200, "pool": 200}[args.workload]
-    warmup = max(args.warmup if args.warmup is not None else 20, 3)
-
-    # every rank is an independent replica with its own batch (different seed), same weights recipe
-    wts = W.make_weights(wl, seed=0)
-    x, tenant, mot = W.make_tokens(wl, seed=replicas.rank_seed(0, rank))
-    T = x.shape[0]
-    layer = B.MoELayer(H=wl.H, E=wl.E, I=wl.I, k=wl.k, Is=wl.Is, M=wl.M, n_tenants=wl.n_tenants, max_tokens=T,
-                       device=str(dev))
-    layer.set_layer_weights(0, wts)
-    layer.set_tables(slot_table=wts["slot_table"], model_of_tenant=mot)
-    ctx = layer.ctx
-    B.moe_set_option(ctx, B.MOE_OPT_EXPERT_PATH, {"auto": 0, "fma": 1, "tcgen05": 2}[args.path])
-    B.moe_set_option(ctx, B.MOE_OPT_PAIR_MODE, {"auto": 1, "never": 0}[args.pair])
-    if args.early_shared != "auto":
-        B.moe_set_option(ctx, B.MOE_OPT_EARLY_SHARED, int(args.early_shared))
-    xd, td = x.to(dev), tenant.to(dev)
-    out = torch.zeros_like(xd)
-    stream = torch.cuda.current_stream()
-
-    def barrier():
-        replicas.barrier(world, torch.cuda.synchronize)
-
-    # ---- device-resident throughput -----------------------------------------------------------
-    for _ in range(warmup):
-        B.moe_layer_forward(ctx, 0, xd, td, T, wl.G, out, stream)
-    torch.cuda.synchronize()
-    status, n_inv, active = B.moe_last_status(ctx)
-    if status != 0:
-        raise SystemExit(f"device status {status} after warm-up")
-    sampler = ClockSampler(local_rank)
-    barrier()
-    sampler.start()
-    l0 = B.moe_launch_count(ctx)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record(stream)
-    for _ in range(steps):
-        B.moe_layer_forward(ctx, 0, xd, td, T, wl.G, out, stream)
-    ev1.record(stream)
-    barrier()
-    clocks = sampler.stop()
-    launches = B.moe_launch_count(ctx) - l0
-    ms_total = ev0.elapsed_time(ev1)
-
-    # ---- per-stage durations (CUDA events on the launching stream, between the kernels) ---------
-    stage_ms = B.moe_stage_times(ctx, xd, td, T, wl.G, out, reps=max(10, min(steps, 100)))
-
-    # ---- end to end through the host-buffer entry point ---------------------------------------
-    xh, th = x.contiguous().pin_memory(), tenant.contiguous().pin_memory()
-    oh = torch.zeros_like(xh).pin_memory()
-    e2e_steps = max(10, min(steps, 500))
-    for _ in range(3):
-        B.moe_layer_forward_host(ctx, 0, xh, th, T, wl.G, oh, stream)
-    barrier()
-    t0 = time.perf_counter()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(e2e_steps):
-        B.moe_layer_forward_host(ctx, 0, xh, th, T, wl.G, oh, stream)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0))
-    barrier()
-
-    ms_total, e2e_ms = replicas.max_over_ranks([ms_total, e2e_ms], world, dev)
-
-    if rank == 0:
-        peaks = measured_peaks()
-        work = algorithmic_work(wl, active, T)
-        ms_step = ms_total / steps
-        value = world * T * steps / (ms_total * 1e-3)
-        t_hbm = work["total_bytes"] / (peaks["hbm_gbs"] * 1e9)
-        t_tc = work["flops"] / (peaks["bf16_tflops"] * 1e12)
-        bound = "hbm" if t_hbm >= t_tc else "tensor"
-        # dominant kernel: the gate/up grouped GEMM of moe_experts
-        gu_ms = stage_ms.get("experts_gateup")
-        if bound == "hbm":
-            achieved = work["gateup_bytes"] / (gu_ms * 1e-3) / 1e9 if gu_ms else None
-            peak, runit = peaks["hbm_gbs"], "GB/s"
+    names = [args.workload] if args.workload else ["decode"] + list(EXTRA_WORKLOADS)
+    wts_cache, lines = {}, {}
+    for i, name in enumerate(names):
+        wl = W.WORKLOADS[name]
+        if wl.n_layers > 1:
+            if torch.cuda.mem_get_info()[0] < 32e9:
+                lines[name] = {"skipped": "needs about 30 GB of free device memory"}
+                continue
+            lines[name] = measure_stack(args, wl, rank, local_rank, world, dev)
         else:
-            achieved = work["gateup_flops"] / (gu_ms * 1e-3) / 1e12 if gu_ms else None
-            peak, runit = peaks["bf16_tflops"], "TFLOP/s"
-        roofline = {"bound": bound, "kernel": "moe_experts gate/up grouped GEMM", "achieved": achieved, "peak": peak,
-                    "unit": runit, "frac": (achieved / peak) if achieved else None,
-                    "traffic": NCU_TRAFFIC_BYTES.get(wl.name) if args.path == "auto" else None,
-                    "algorithmic": work["gateup_bytes"] if bound == "hbm" else work["gateup_flops"],
-                    "peak_source": peaks["source"],
-                    "path": {"roofline_ms": 1e3 * max(t_hbm, t_tc), "measured_ms": ms_step,
-                             "frac": 1e3 * max(t_hbm, t_tc) / ms_step, "algorithmic_bytes": work["total_bytes"],
-                             "flops": work["flops"], "active_experts": active},
-                    "stage_ms": stage_ms}
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-                "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": wl.name, "tokens_per_step_per_gpu": T, "hidden": wl.H, "experts": wl.E,
-                           "inter": wl.I, "top_k": wl.k, "shared_inter": wl.Is, "G": wl.G, "tenants": wl.n_tenants,
-                           "models": wl.M, "expert_path": args.path, "early_shared": args.early_shared,
-                           "l2": "expert weights (about 1 GB per pass) exceed the 126 MB L2; no flush",
-                           "parallelism": f"replicas x{world}"},
-                "clocks": clocks, "gpu_launches": int(launches),
-                "e2e": {"value": world * T * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
-                        "h2d_bytes_per_step": int(T * wl.H * 2 + T * 4), "d2h_bytes_per_step": int(T * wl.H * 2)},
-                "roofline": roofline}
-        if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(wl, wts, x, tenant, mot)
+            lines[name] = measure_layer(args, wl, rank, local_rank, world, dev, wts_cache,
+                                        with_cpu_baseline=(i == 0 and not args.no_cpu_baseline and world == 1))
+        torch.cuda.empty_cache()
+    if rank == 0:
+        line = lines[names[0]]
+        if len(names) > 1:
+            # the other workloads ride in the same line: the fields the headline has, without the CPU baseline
+            line["workloads"] = {n: lines[n] for n in names[1:]}
         print(json.dumps(line), flush=True)
-    layer.close()
     if world > 1:
         dist.destroy_process_group()
 

@@ -66,6 +66,7 @@ enum {
  * (experts: hidden % 256 == 0; router: n_experts <= 64 and n_models * ceil16(n_experts) <= 256),
  * FMA forces the CUDA-core kernels, TCGEN05 fails with MOE_ERR_UNSUPPORTED if not possible. */
 enum { MOE_PATH_AUTO = 0, MOE_PATH_FMA = 1, MOE_PATH_TCGEN05 = 2 };
+enum { MOE_DISPATCH_SHARED = 0, MOE_DISPATCH_PRIVATE = 1 };
 enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2,
        MOE_OPT_PAIR_MODE = 3, /* 1 (default): batches of more than 64 tokens use the 2-CTA tcgen05 shape; 0: never;
                                  2: every batch */
@@ -83,6 +84,22 @@ enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2,
                                     of the shared experts) beside the router and the dispatch, unless 0. */
        MOE_OPT_EARLY_SHARED_SMS = 7, /* SMs that the shared expert's CTA pairs may hold while they run beside other
                                        kernels (batches of more than 64 tokens; default: no limit) */
+       MOE_OPT_DISPATCH_MODE = 9, /* orchestrator placement (Sec. 4.2, strategies FaaSMoE-Shared and FaaSMoE-Private;
+                                     Sec. 5 on orchestrator placement).  MOE_DISPATCH_SHARED (default): one orchestrator
+                                     batches across tenants -- all rows that reach an expert block form one invocation
+                                     and the rows of an expert are tiled whoever owns them.  MOE_DISPATCH_PRIVATE: every
+                                     tenant's orchestrator batches only its own tokens -- an invocation is a (tenant,
+                                     block) pair with rows, and no tile of expert work spans two tenants (more, smaller
+                                     tiles; an expert's weights are fetched once per tenant that uses it).  The
+                                     permutation, the offset tables and every output bit are the same in both modes
+                                     (rows are ordered (model, expert, tenant, token) either way); what changes is the
+                                     invocation count reported by moe_last_status and the cost of moe_experts.
+                                     In private mode moe_experts takes the (expert, tenant) boundaries from the last
+                                     moe_dispatch on the same context. */
+       MOE_OPT_BACKGROUND_LANES = 10, /* 2-CTA shape: 1 (default): expert tiles of at most 64 rows are run by a second,
+                                         small pipeline of every CTA pair (its own stage ring, MMA lane and accumulator)
+                                         beside the pair's long tiles; 0: one pipeline runs all tiles in turn.  Results
+                                         are bit-identical. */
        MOE_OPT_ROUTE_LANES = 8 /* 2 (default): the tensor-core router issues its MMAs from two warps, even and odd K
                                   stages into two accumulators that the epilogue adds; 1: one warp, one accumulator
                                   (another summation order over K: logits differ in the last bits) */ };
@@ -272,9 +289,16 @@ int moe_get_workspace(moe_ctx* ctx, int32_t** topk_idx, float** topk_w, float** 
                       int32_t** perm, int32_t** inv_perm, int32_t** expert_off, int32_t** group_off);
 
 /* Synchronises the device, returns the device status word in *status_host and clears it.
- * Also reports, if not NULL, stats_host[0] = non-empty expert blocks (invocations) and
- * stats_host[1] = active routed experts of the last dispatch. */
+ * Also reports, if not NULL, stats_host[0] = invocations of the last dispatch (shared
+ * orchestrator: non-empty expert blocks; private orchestrators: (tenant, block) pairs with
+ * rows -- see MOE_OPT_DISPATCH_MODE) and stats_host[1] = its active routed experts. */
 int moe_last_status(moe_ctx* ctx, int32_t* status_host, int32_t* stats_host);
+
+/* Synchronises the device and reports how the last moe_experts / moe_layer_forward call on this context cut the
+ * expert work (Sec. 4.1: requests are batched per block; Sec. 4.2: per tenant too under private orchestrators):
+ * plan_host[0] = tiles of routed rows, plan_host[1] = tiles of shared-expert tokens, plan_host[2] = most rows a
+ * tile holds at batch size T.  plan_host is a host pointer to 3 ints. */
+int moe_last_plan(moe_ctx* ctx, int T, int32_t* plan_host);
 
 /* Number of kernels this library has launched on this context since creation. */
 int64_t moe_launch_count(moe_ctx* ctx);

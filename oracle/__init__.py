@@ -44,7 +44,7 @@ def _load():
         _lib = ctypes.CDLL(_LIB)
         _lib.oracle_num_threads.restype = ctypes.c_int
         for name in ("oracle_route", "oracle_dispatch", "oracle_experts", "oracle_shared_expert",
-                     "oracle_combine", "oracle_rmsnorm"):
+                     "oracle_combine", "oracle_rmsnorm", "oracle_invocations"):
             getattr(_lib, name).restype = ctypes.c_int
         _lib.oracle_round_bf16.restype = None
     return _lib
@@ -130,6 +130,35 @@ def dispatch(topk_idx, tenant_id, model_of_tenant, *, n_models, E, G):
     if rc != 0:
         raise ValueError(f"oracle_dispatch failed: {rc}")
     return Dispatch(perm, inv, cnt, eoff, goff, int(ninv.value))
+
+
+SHARED, PRIVATE = 0, 1
+
+
+@dataclass
+class Invocations:
+    n_invocations: int
+    tenant_invocations: np.ndarray   # [n_tenants] i32
+    token_fanout: np.ndarray         # [T] i32
+    n_row_batches: int
+
+
+def invocations(topk_idx, tenant_id, model_of_tenant, *, n_models, E, G, mode, batch_rows=128):
+    """Invocations of expert blocks under a shared orchestrator (mode SHARED: rows of all tenants to a block travel
+    together) or private ones (mode PRIVATE: every tenant batches only its own tokens) -- Sec. 4.2, Sec. 5."""
+    lib = _load()
+    topk_idx = _c(topk_idx, np.int32); tenant_id = _c(tenant_id, np.int32)
+    model_of_tenant = _c(model_of_tenant, np.int32)
+    T, k = topk_idx.shape
+    n_tenants = len(model_of_tenant)
+    ninv, nbatch = ctypes.c_int32(0), ctypes.c_int32(0)
+    per_tenant = np.empty((n_tenants,), np.int32)
+    fan = np.empty((T,), np.int32)
+    rc = lib.oracle_invocations(_p(topk_idx), _p(tenant_id), T, E, k, n_models, n_tenants, _p(model_of_tenant), G, mode,
+                                batch_rows, ctypes.byref(ninv), _p(per_tenant), _p(fan), ctypes.byref(nbatch))
+    if rc != 0:
+        raise ValueError(f"oracle_invocations failed: {rc}")
+    return Invocations(int(ninv.value), per_tenant, fan, int(nbatch.value))
 
 
 def experts(x, tenant_id, topk_idx, perm, model_of_tenant, pool_gate, pool_up, pool_down, slot_table, *, n_models):

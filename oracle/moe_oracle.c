@@ -58,8 +58,8 @@ static double dot_bf16(const uint16_t* a, const uint16_t* b, int n)
 }
 
 /*
- * Gating network (Sec. 2.1: "gating network ... selects top-k experts";
- * Sec. 3: gating modules live in the orchestrator).
+ * Gating network (Sec. 2.1: a gate picks the k best experts of every token;
+ * Sec. 3: the gating modules live in the orchestrator).
  *
  *   z[t,e] = sum_h x[t,h] * W_r[m][e,h] + b[m][e]      m = model_of_tenant[tenant_id[t]]
  *   p[t,:] = softmax_e(z[t,:])
@@ -140,9 +140,9 @@ int oracle_route(const uint16_t* x, const int32_t* tenant_id, int T, int H, int 
 }
 
 /*
- * Micro-batched routing requests (Sec. 3: "constructs micro-batched routing
- * requests"; Sec. 4.1: all tokens routed to the same expert block are
- * consolidated into one batched invocation; blocks are packaged by layer and
+ * Routing requests, batched per expert block (Sec. 3: the orchestrator groups
+ * the routed tokens into one request per block; Sec. 4.1: whatever goes to the
+ * same block travels in one invocation; blocks are packaged by layer and
  * expert id, G experts per block).
  *
  * A routed row is (t, j) with flat id t*k + j.  Rows are ordered by the key
@@ -217,8 +217,92 @@ int oracle_dispatch(const int32_t* topk_idx, const int32_t* tenant_id, int T, in
 }
 
 /*
- * One SwiGLU expert on one token (Sec. 3: an expert block "performs stateless
- * computation on assigned tokens"; Sec. 5: experts are small MLPs):
+ * Invocation accounting of the two orchestrator placements (Sec. 4.2,
+ * deployment strategies FaaSMoE-Shared and FaaSMoE-Private; Sec. 4.3.1 on
+ * batching across tenants and fan-out; Sec. 5 on orchestrator placement).
+ *
+ *   mode 0, shared orchestrator: one orchestrator serves every tenant, so all
+ *     rows that reach a block travel in ONE invocation whoever owns them:
+ *     invocations = blocks (m, b) that received at least one row.
+ *   mode 1, private orchestrators: every tenant has an orchestrator of its own
+ *     that batches only its own tokens: invocations = pairs (tenant u, block b
+ *     of u's model) with at least one row of u.
+ *
+ * Outputs (any may be NULL):
+ *   *n_invocations        as above
+ *   tenant_invocations[u] blocks that rows of tenant u reach (private: the
+ *                         invocations u's orchestrator issues, they sum to
+ *                         *n_invocations; shared: how many of the shared
+ *                         invocations carry rows of u)
+ *   token_fanout[t]       distinct blocks among the k experts of token t (the
+ *                         invocations one token takes part in; same in both modes)
+ *   *n_row_batches        row batches when the rows that ONE invocation sends to
+ *                         ONE expert are cut into pieces of at most batch_rows
+ *                         rows: shared sum over (m,e) of ceil(cnt/batch_rows),
+ *                         private sum over (u,e)
+ * Returns 0, -1 on bad ids, -2 on bad G / mode / batch_rows.
+ */
+int oracle_invocations(const int32_t* topk_idx, const int32_t* tenant_id, int T, int E, int k,
+                       int n_models, int n_tenants, const int32_t* model_of_tenant, int G, int mode,
+                       int batch_rows, int32_t* n_invocations, int32_t* tenant_invocations,
+                       int32_t* token_fanout, int32_t* n_row_batches)
+{
+    if (G < 1 || G > E || mode < 0 || mode > 1 || batch_rows < 1) return -2;
+    const int B = (E + G - 1) / G;
+    /* rows[u][e]: rows of tenant u routed to expert e */
+    int32_t* rows = (int32_t*)calloc((size_t)n_tenants * E, sizeof(int32_t));
+    for (int t = 0; t < T; ++t) {
+        const int u = tenant_id[t];
+        if (u < 0 || u >= n_tenants || model_of_tenant[u] < 0 || model_of_tenant[u] >= n_models) { free(rows); return -1; }
+        int fan = 0;
+        for (int j = 0; j < k; ++j) {
+            const int e = topk_idx[(size_t)t * k + j];
+            if (e < 0 || e >= E) { free(rows); return -1; }
+            rows[(size_t)u * E + e] += 1;
+            int seen = 0;                       /* was this block already counted for the token? */
+            for (int j2 = 0; j2 < j; ++j2) if (topk_idx[(size_t)t * k + j2] / G == e / G) seen = 1;
+            if (!seen) ++fan;
+        }
+        if (token_fanout) token_fanout[t] = fan;
+    }
+    int ninv = 0, nbatch = 0;
+    if (tenant_invocations) memset(tenant_invocations, 0, sizeof(int32_t) * (size_t)n_tenants);
+    /* blocks reached per tenant */
+    for (int u = 0; u < n_tenants; ++u) {
+        for (int b = 0; b < B; ++b) {
+            int any = 0;
+            for (int e = b * G; e < E && e < (b + 1) * G; ++e) if (rows[(size_t)u * E + e] > 0) any = 1;
+            if (any) {
+                if (tenant_invocations) tenant_invocations[u] += 1;
+                if (mode == 1) ++ninv;
+            }
+        }
+        if (mode == 1)
+            for (int e = 0; e < E; ++e) nbatch += (rows[(size_t)u * E + e] + batch_rows - 1) / batch_rows;
+    }
+    if (mode == 0) {
+        for (int m = 0; m < n_models; ++m) {
+            for (int b = 0; b < B; ++b) {
+                int any = 0;
+                for (int e = b * G; e < E && e < (b + 1) * G; ++e) {
+                    int cnt = 0;
+                    for (int u = 0; u < n_tenants; ++u) if (model_of_tenant[u] == m) cnt += rows[(size_t)u * E + e];
+                    if (cnt > 0) any = 1;
+                    nbatch += (cnt + batch_rows - 1) / batch_rows;
+                }
+                if (any) ++ninv;
+            }
+        }
+    }
+    free(rows);
+    if (n_invocations) *n_invocations = ninv;
+    if (n_row_batches) *n_row_batches = nbatch;
+    return 0;
+}
+
+/*
+ * One SwiGLU expert on one token (Sec. 3: an expert block keeps no state and
+ * computes on the tokens it was sent; Sec. 5: experts are small MLPs):
  *   y = W_d . ( silu(W_g . x) * (W_u . x) )
  * W_g, W_u [I,H]; W_d [H,I]; all bf16 row-major.  scratch holds I doubles.
  */

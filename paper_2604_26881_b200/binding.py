@@ -28,12 +28,15 @@ MOE_OPT_TOKEN_MAJOR = 5
 MOE_OPT_EARLY_SHARED = 6
 MOE_OPT_EARLY_SHARED_SMS = 7
 MOE_OPT_ROUTE_LANES = 8
+MOE_OPT_DISPATCH_MODE = 9
+MOE_OPT_BACKGROUND_LANES = 10
+MOE_DISPATCH_SHARED, MOE_DISPATCH_PRIVATE = 0, 1
 MOE_PATH_AUTO, MOE_PATH_FMA, MOE_PATH_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["moe_create", "moe_destroy", "moe_set_expert_pool", "moe_set_model_weights", "moe_set_slot_table",
            "moe_set_tenant_models", "moe_set_option", "moe_route", "moe_dispatch", "moe_experts", "moe_combine",
            "moe_layer_forward", "moe_layer_forward_host", "moe_layer_forward_timed", "moe_stack_forward",
-           "moe_get_workspace", "moe_last_status", "moe_launch_count", "moe_strerror", "moe_dispatch_noalloc"]
+           "moe_get_workspace", "moe_last_status", "moe_last_plan", "moe_launch_count", "moe_strerror", "moe_dispatch_noalloc"]
 MOE_DISPATCH_NOALLOC_MAX_WORDS = 1 << 18
 
 STAGES = ["route", "dispatch", "plan", "experts_gateup", "experts_down", "combine"]
@@ -88,6 +91,7 @@ def load_library(path: str | None = None):
         lib.moe_dispatch_noalloc.argtypes = [c_void_p] * 3 + [c_int] * 6 + [c_void_p] * 7
         lib.moe_get_workspace.argtypes = [c_void_p] + [POINTER(c_void_p)] * 8
         lib.moe_last_status.argtypes = [c_void_p, POINTER(c_int32), POINTER(c_int32)]
+        lib.moe_last_plan.argtypes = [c_void_p, c_int, POINTER(c_int32)]
         _lib = lib
     return _lib
 
@@ -247,6 +251,13 @@ def moe_last_status(ctx):
     stats = (c_int32 * 2)()
     _check("moe_last_status", load_library().moe_last_status(ctx, byref(st), stats))
     return int(st.value), int(stats[0]), int(stats[1])
+
+
+def moe_last_plan(ctx, T):
+    """(routed tiles, shared-expert tiles, rows per tile) of the last expert call; synchronises the device."""
+    plan = (c_int32 * 3)()
+    _check("moe_last_plan", load_library().moe_last_plan(ctx, T, plan))
+    return int(plan[0]), int(plan[1]), int(plan[2])
 
 
 def moe_launch_count(ctx) -> int:

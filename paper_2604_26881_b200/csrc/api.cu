@@ -1,9 +1,11 @@
 // C-ABI entry points: argument validation, context and workspace management, call sequencing.
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <new>
 
 #include "internal.h"
+#include "plan.cuh"
 
 using namespace faasmoe;
 
@@ -50,7 +52,8 @@ int alloc_workspace(moe_ctx* c)
     c->nbins = g.n_experts * g.n_tenants;
     c->nblk_rows = div_up((int)R, kDispatchChunk);
     c->nblk_tok = div_up((int)T, kDispatchChunk);
-    c->max_tiles = div_up((int)R, kTileRows) + (int)ME;
+    // (+ one ragged tile per expert; per (tenant, expert) bin when private orchestrators keep the tenants' rows apart)
+    c->max_tiles = div_up((int)R, kTileRows) + std::max((int)ME, c->nbins);
     c->max_stiles = div_up((int)T, kTileRows) + g.n_models;
     const int nblk1 = g.inter / 64, nblk2 = div_up(g.hidden, 128), snblk1 = g.shared_inter / 64;
     // (+256: the token-major plan splits up to half a round of units in two; its shared units are up to 4x narrower)
@@ -65,10 +68,10 @@ int alloc_workspace(moe_ctx* c)
     A(&w.block_cnt, (size_t)c->nblk_rows * c->nbins); A(&w.bin_off, (size_t)c->nbins + 1);
     A(&w.tok_block_cnt, (size_t)c->nblk_tok * g.n_models); A(&w.model_tok_off, (size_t)g.n_models + 1);
     A(&w.tok_perm, T); A(&w.tok_inv, T);
-    A(&w.tiles, (size_t)c->max_tiles); A(&w.stiles, (size_t)c->max_stiles); A(&w.plan_counts, 8);
+    A(&w.tiles, (size_t)c->max_tiles); A(&w.tile_cidx, (size_t)c->max_tiles); A(&w.stiles, (size_t)c->max_stiles); A(&w.plan_counts, 16);
     A(&w.units1, (size_t)c->max_units1); A(&w.units2, (size_t)c->max_units2);
     if (Is > 0 && g.n_models == 1) {
-        A(&w.stiles_sh, (size_t)c->max_stiles); A(&w.plan_counts_sh, 8);
+        A(&w.stiles_sh, (size_t)c->max_stiles); A(&w.plan_counts_sh, 16);
         A(&w.units1_sh, (size_t)c->max_stiles * snblk1); A(&w.units2_sh, (size_t)4 * c->max_stiles * nblk2);
     }
     // activations: one extra tile of rows so that a whole-tile load never leaves the buffer
@@ -90,8 +93,8 @@ int alloc_workspace(moe_ctx* c)
     cudaMemset(w.status, 0, sizeof(int32_t));
     cudaMemset(w.stats, 0, 4 * sizeof(int32_t));
     cudaMemset(w.dispatch_done, 0, sizeof(int32_t));
-    cudaMemset(w.plan_counts, 0, 8 * sizeof(int32_t));
-    if (w.plan_counts_sh) cudaMemset(w.plan_counts_sh, 0, 8 * sizeof(int32_t));
+    cudaMemset(w.plan_counts, 0, 16 * sizeof(int32_t));
+    if (w.plan_counts_sh) cudaMemset(w.plan_counts_sh, 0, 16 * sizeof(int32_t));
     return MOE_OK;
 }
 
@@ -100,7 +103,7 @@ void free_workspace(moe_ctx* c)
     Workspace& w = c->ws;
     void* ptrs[] = {w.topk_idx, w.topk_w, w.shared_gate, w.tie_flag, w.perm, w.inv_perm, w.tenant_expert_count,
                     w.expert_off, w.group_off, w.block_cnt, w.bin_off, w.tok_block_cnt, w.model_tok_off, w.tok_perm,
-                    w.tok_inv, w.tiles, w.stiles, w.plan_counts, w.units1, w.units2, w.stiles_sh, w.plan_counts_sh, w.units1_sh,
+                    w.tok_inv, w.tiles, w.tile_cidx, w.stiles, w.plan_counts, w.units1, w.units2, w.stiles_sh, w.plan_counts_sh, w.units1_sh,
                     w.units2_sh, w.x_perm, w.xs_perm, w.h, w.hs,
                     w.y_perm, w.y_shared, w.xn, w.x_stage, w.tenant_stage, w.out_stage, w.status, w.stats, w.dispatch_done};
     for (void* p : ptrs) if (p) cudaFree(p);
@@ -260,6 +263,8 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->pair_mode_enabled = 1;
     c->wide_tiles_enabled = 1;
     c->token_major_enabled = 1;
+    c->dispatch_private = 0;
+    c->background_enabled = 0;
     c->timing = false;
     c->early_shared_enabled = 1;
     c->early_shared_sms = 1 << 20;      // no limit
@@ -425,6 +430,15 @@ int moe_set_option(moe_ctx* c, int option, int value)
     if (option == MOE_OPT_WIDE_TILES) {
         if (value < 0 || value > 2) return MOE_ERR_SHAPE;
         c->wide_tiles_enabled = value;
+        return MOE_OK;
+    }
+    if (option == MOE_OPT_BACKGROUND_LANES) {
+        c->background_enabled = value ? 1 : 0;
+        return MOE_OK;
+    }
+    if (option == MOE_OPT_DISPATCH_MODE) {
+        if (value != MOE_DISPATCH_SHARED && value != MOE_DISPATCH_PRIVATE) return MOE_ERR_SHAPE;
+        c->dispatch_private = value == MOE_DISPATCH_PRIVATE ? 1 : 0;
         return MOE_OK;
     }
     if (option == MOE_OPT_ROUTE_PATH) {
@@ -600,6 +614,16 @@ int moe_last_status(moe_ctx* c, int32_t* status_host, int32_t* stats_host)
     MOE_CUDA(c, cudaMemcpy(status_host, c->ws.status, sizeof(int32_t), cudaMemcpyDeviceToHost));
     if (stats_host) MOE_CUDA(c, cudaMemcpy(stats_host, c->ws.stats, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost));
     MOE_CUDA(c, cudaMemset(c->ws.status, 0, sizeof(int32_t)));
+    return MOE_OK;
+}
+
+int moe_last_plan(moe_ctx* c, int T, int32_t* plan_host)
+{
+    if (!c || !plan_host) return MOE_ERR_NULL;
+    if (T < 1 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
+    MOE_CUDA(c, cudaDeviceSynchronize());
+    MOE_CUDA(c, cudaMemcpy(plan_host, c->ws.plan_counts, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    plan_host[2] = make_plan_args(c, T, 1, false).tile_rows;
     return MOE_OK;
 }
 

@@ -1,8 +1,10 @@
-// Micro-batched routing requests: per-(tenant, expert) histogram, prefix scan, stable ranks,
-// token permute into expert segments (paper Sec. 3: the orchestrator "constructs micro-batched
-// routing requests"; Sec. 4.1: all tokens routed to the same expert block become one batched
-// invocation).  Rows are ordered by (model, expert, tenant, token); the order is produced
-// without order-dependent atomics so that the permutation is reproducible bit for bit.
+// Routing requests batched per expert block: per-(tenant, expert) histogram, prefix scan, stable ranks,
+// token permute into expert segments (paper Sec. 3: the orchestrator groups the routed tokens into one
+// request per block; Sec. 4.1: whatever goes to the same block travels in one invocation).  Rows are
+// ordered by (model, expert, tenant, token); the order is produced without order-dependent atomics so
+// that the permutation is reproducible bit for bit.  The invocation statistics follow the orchestrator
+// placement (Sec. 4.2, Sec. 5): a shared orchestrator sends one invocation per non-empty block, private
+// orchestrators one per (tenant, block) pair that has rows.
 #include <cstring>
 #include <mutex>
 
@@ -37,7 +39,7 @@ __device__ void scan_and_tables(int32_t* s_tot, int32_t* s_part /* [33] */, int3
                                 int nbins, int R, int E, int M, int G, int n_tenants, const BinMap& bm,
                                 int32_t* __restrict__ bin_off /* may be null */,
                                 int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
-                                int32_t* __restrict__ group_off, int32_t* __restrict__ stats)
+                                int32_t* __restrict__ group_off, int32_t* __restrict__ stats, int private_mode)
 {
     const int tid = threadIdx.x, nth = blockDim.x;
     if (tid < 2) s_count[tid] = 0;
@@ -74,9 +76,25 @@ __device__ void scan_and_tables(int32_t* s_tot, int32_t* s_part /* [33] */, int3
             const int m = i / B, b = i - m * B;
             const int e0 = b * G, e1 = min(E, e0 + G);
             v = expert_off[m * E + e0];
-            if (expert_off[m * E + e1] > v) atomicAdd(&s_count[0], 1);
+            if (!private_mode && expert_off[m * E + e1] > v) atomicAdd(&s_count[0], 1);
         }
         if (group_off) group_off[i] = v;
+    }
+    if (private_mode) {
+        // private orchestrators (Sec. 4.2): every tenant batches its own tokens, so an invocation is a pair
+        // (tenant, block of its model) with at least one row
+        for (int i = tid; i < n_tenants * B; i += nth) {
+            const int u = i / B, b = i - u * B;
+            const int m = bm.model_of_tenant[u];
+            const int tim = bm.tenants_in_model[m], ul = bm.tenant_local[u];
+            bool any = false;
+            for (int e = b * G; e < min(E, (b + 1) * G); ++e) {
+                const int bin = bm.bin_base[m] + e * tim + ul;
+                const int end = bin + 1 < nbins ? s_tot[bin + 1] : R;
+                any = any || end > s_tot[bin];
+            }
+            if (any) atomicAdd(&s_count[0], 1);
+        }
     }
     for (int i = tid; i < M * E; i += nth)
         if (expert_off[i + 1] > expert_off[i]) atomicAdd(&s_count[1], 1);
@@ -97,7 +115,7 @@ dispatch_count_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
                       int32_t* __restrict__ bin_off, int32_t* __restrict__ inv_perm,
                       int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
                       int32_t* __restrict__ group_off, int32_t* __restrict__ stats, int32_t* __restrict__ status,
-                      int32_t* __restrict__ done_counter, int do_plan, PlanArgs pa)
+                      int32_t* __restrict__ done_counter, int do_plan, PlanArgs pa, int private_mode)
 {
     extern __shared__ int32_t s_tot[];       // [nbins] counts of this block; in the last block: totals, then offsets,
                                              // followed by the plan's scratch
@@ -160,7 +178,7 @@ dispatch_count_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
     }
     __syncthreads();
     scan_and_tables(s_tot, s_part, s_count, nbins, R, E, M, G, n_tenants, bm, bin_off, tenant_expert_count,
-                    expert_off, group_off, stats);
+                    expert_off, group_off, stats, private_mode);
     if (do_plan) {
         __syncthreads();
         plan_body(expert_off, pa, s_tot + nbins, s_part);
@@ -207,7 +225,7 @@ dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
                       int32_t* __restrict__ inv_perm, int32_t* __restrict__ tenant_expert_count,
                       int32_t* __restrict__ expert_off, int32_t* __restrict__ group_off, int32_t* __restrict__ stats,
                       int32_t* __restrict__ status, const bf16* __restrict__ x, bf16* __restrict__ x_perm, int H,
-                      int do_plan, int plan_ints, PlanArgs pa)
+                      int do_plan, int plan_ints, PlanArgs pa, int32_t* __restrict__ bin_off, int private_mode)
 {
     extern __shared__ int32_t s_tot[];       // [nbins], then the plan's scratch, then the bin of every row (u16)
     __shared__ int32_t s_part[33];
@@ -224,8 +242,8 @@ dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
         atomicAdd(&s_tot[bin], 1);
     }
     __syncthreads();
-    scan_and_tables(s_tot, s_part, s_count, nbins, R, E, M, G, n_tenants, bm, nullptr, tenant_expert_count,
-                    expert_off, group_off, stats);
+    scan_and_tables(s_tot, s_part, s_count, nbins, R, E, M, G, n_tenants, bm, bin_off, tenant_expert_count,
+                    expert_off, group_off, stats, private_mode);
     __syncthreads();
     if (tid < 32) {                           // s_tot now holds the next free position of every bin
         const int lane = tid;
@@ -385,7 +403,7 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
         launch_pdl(dispatch_small_kernel, dim3(1), dim3(threads), smem_small, st,
             topk_idx, tenant_id, R, k, bm, nbins, g.n_experts, g.n_models, G, g.n_tenants, perm, inv_perm,
             tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, x, gather_inside ? x_perm : nullptr,
-            g.hidden, do_plan ? 1 : 0, (int)plan_ints, pa);
+            g.hidden, do_plan ? 1 : 0, (int)plan_ints, pa, c->ws.bin_off, c->dispatch_private);
         if (plan_done) *plan_done = do_plan;
         c->launches += 1;
         if (x_perm && !gather_inside) {
@@ -405,7 +423,7 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
     launch_pdl(dispatch_count_kernel, dim3(nblk), dim3(kCountThreads), smem_count, st,
         topk_idx, tenant_id, nblk, nbins, R, k, g.n_experts, g.n_models, G, g.n_tenants, bm, c->ws.block_cnt, c->ws.bin_off,
         inv_perm, tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, c->ws.dispatch_done,
-        do_plan ? 1 : 0, pa);
+        do_plan ? 1 : 0, pa, c->dispatch_private);
     if (plan_done) *plan_done = do_plan;
     if (x_perm)
         launch_pdl(dispatch_place_kernel<true>, dim3((R * 32 + 255) / 256), dim3(256), 0, st, R, k, nbins, c->ws.block_cnt, c->ws.bin_off, perm,
@@ -552,7 +570,7 @@ extern "C" int moe_dispatch_noalloc(const int32_t* topk_idx, const int32_t* tena
     dispatch_count_kernel<<<nblk, kCountThreads, smem, st>>>(topk_idx, tenant_id, nblk, nbins, R, k, E, M, G, n_tenants, bm,
                                                              s + o_blk, s + o_binoff, inv_perm, tenant_expert_count,
                                                              expert_off, group_off, s + o_stats, status, s + o_stats + 2, 0,
-                                                             PlanArgs());
+                                                             PlanArgs(), 0);
     dispatch_place_kernel<false><<<(R + 255) / 256, 256, 0, st>>>(R, k, nbins, s + o_blk, s + o_binoff, perm, inv_perm,
                                                                   nullptr, nullptr, 0);
     return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;

@@ -46,8 +46,19 @@ constexpr int kBBytes = kBRows * kBK * 2;      // 16 KB
 constexpr int kRingBytes = kMaxStages * (kABytes + kBBytes);
 constexpr int kWideStages = kRingBytes / (kABytes + 2 * kBBytes);
 constexpr int kQueue = 4;                      // depth of the unit queue of the dynamic scheduler
-constexpr int kNumBars = 2 * kMaxStages + 4 + 2 * kQueue + 1;
-constexpr int kBarBytes = 256;                 // >= 8 * kNumBars, keeps the staging area 128-byte aligned
+// The background pipeline of the pair shape (see the kernel): a ring, a unit queue and an accumulator of its own.
+constexpr int kBgStages = 3;
+constexpr int kBgRows = kShortRows / 2;        // token rows one CTA of the pair loads per stage (at most)
+constexpr int kBgStageBytes = kABytes + kBgRows * kBK * 2;      // 20 KB: 128 weight rows + 32 token rows
+constexpr int kBgRingBytes = kBgStages * kBgStageBytes;         // 60 KB
+constexpr int kBgQueue = 2;
+constexpr int kBgAccRows = kAccRowsBg;         // token rows per accumulator of a wide tile when the background pipeline runs
+constexpr int kBgStageBytesMain = kABytes + 2 * (kBgAccRows / 2) * kBK * 2;    // 44 KB: weights + two token tiles of 112 rows
+constexpr int kBgMainStages = (kRingBytes - kBgRingBytes) / kBgStageBytesMain;  // 3
+static_assert(kBgMainStages * kBgStageBytesMain + kBgRingBytes <= kRingBytes, "the two rings share the 192 KB");
+static_assert(kBgStageBytesMain % 1024 == 0 && kBgStageBytes % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+constexpr int kNumBars = 2 * kMaxStages + 4 + 2 * kQueue + 1 + 2 * kBgStages + 2 + 2 * kBgQueue;
+constexpr int kBarBytes = 512;                 // >= 8 * kNumBars, keeps the staging area 128-byte aligned
 // Output staging of the epilogue: results go to shared memory and leave as bulk copies of one row each,
 // so that the epilogue warps never wait on the global store path (which the operand loads saturate).
 // Each group of four epilogue warps owns a quarter of it.
@@ -60,6 +71,11 @@ constexpr int kEpiWarps = 4 * kEpiGroups;      // four warps per TMEM lane quart
 constexpr int kSchedWarp = 2 + kEpiWarps;      // warp 0: TMA (weights), warp 1: MMA + TMEM, warps 2..17: epilogue, warp 18: scheduler,
 constexpr int kTokWarp = kSchedWarp + 1;       // warp 19: TMA (tokens)
 constexpr int kThreads = 32 * (kTokWarp + 1);
+// background pipeline (pair shape only): warp 20 = its TMA producer (and, in the leader CTA, its scheduler), warp 21 =
+// its MMA lane, warps 22..25 = its epilogue (one warp per TMEM lane quarter)
+constexpr int kBgProdWarp = kTokWarp + 1, kBgMmaWarp = kTokWarp + 2, kBgEpiWarp0 = kTokWarp + 3;
+constexpr int kThreadsBg = 32 * (kBgEpiWarp0 + 4);
+constexpr uint32_t kBgTmemCol = 2 * kBgAccRows;     // its accumulator: TMEM columns 448 .. 511
 constexpr int kClaimAhead = 8;                 // the next unit is claimed this many K steps before the current one is loaded
 constexpr uint32_t kTmemCols = 512;            // 2 accumulator buffers x 256 columns
 
@@ -68,7 +84,9 @@ struct GemmParams {
     const int32_t* n_units;
     const int32_t* n_shared;      // shared-expert units at the head of the list that are to be spread evenly over the
                                   // launch (0: take the list in order)
-    int32_t* counter;             // work counter of the dynamic scheduler (zeroed by the plan kernel)
+    const int32_t* n_short;       // units at the tail of the list that the background lanes may take (0: none)
+    unsigned long long* counter;  // work counter of the dynamic scheduler (zeroed by the plan kernel): units taken from
+                                  // the front of the list in the low word, from its tail in the high word
     const Tile* tiles;
     const Tile* stiles;
     const int32_t* perm;          // direct mode: routed row -> flat (token, j) id
@@ -211,7 +229,7 @@ struct __align__(16) QEntry {
     int colblock, shared, pad0, pad1;
 };
 
-template <int MODE, bool PAIR, bool SWAP>
+template <int MODE, bool PAIR, bool SWAP, bool BG>
 __device__ __forceinline__ UnitInfo unit_info(const GemmParams& p, const QEntry& e, uint32_t rank)
 {
     UnitInfo ui;
@@ -228,8 +246,9 @@ __device__ __forceinline__ UnitInfo unit_info(const GemmParams& p, const QEntry&
     ui.npad1 = 0;
     if (ui.direct) { ui.npad = p.n_tokens_pad; }
     else if (PAIR) {
-        // up to 512 rows: the first 256 go to one accumulator, the rest to the other
-        const int n0 = e.nrows < 256 ? e.nrows : 256;
+        // wide tiles: the first kAcc rows go to one accumulator, the rest to the other
+        constexpr int kAcc = BG ? kBgAccRows : 256;
+        const int n0 = e.nrows < kAcc ? e.nrows : kAcc;
         ui.npad = (n0 + 31) & ~31;
         ui.npad1 = (e.nrows - n0 + 31) & ~31;
     }
@@ -237,7 +256,8 @@ __device__ __forceinline__ UnitInfo unit_info(const GemmParams& p, const QEntry&
     const int k_len = ui.shared ? p.k_shared : p.k_routed;
     // pair shape with 48 KB stages: a unit of at most 128 tokens puts two K slices into a stage (2 x 16 KB of weights
     // and 2 x at most 8 KB of tokens per CTA), which halves the waits and commits of its MMA lane -- all a short unit costs
-    if (PAIR && p.wide && ui.npad1 == 0 && ui.npad <= 128 && (k_len / kBK) % 2 == 0) ui.kb = 2;
+    // (with the background pipeline the stages are 44 KB: two K slices fit up to 96 tokens)
+    if (PAIR && p.wide && ui.npad1 == 0 && ui.npad <= (BG ? 96 : 128) && (k_len / kBK) % 2 == 0) ui.kb = 2;
     ui.ksteps = k_len / (kBK * ui.kb);
     return ui;
 }
@@ -251,31 +271,249 @@ __device__ __forceinline__ QEntry read_entry(const QEntry* q)
     return e;
 }
 
+// The background pipeline of the pair shape: producer (+ scheduler in the leader CTA), MMA lane and epilogue warps for
+// the short tiles (at most kShortRows tokens) at the tail of the unit list.  One K slice per stage (128 weight rows and
+// at most 32 token rows per CTA), a ring of kBgStages stages, one accumulator of 64 TMEM columns.
+template <int MODE>
+__device__ __forceinline__ void bg_roles(const GemmParams& p, const GemmMaps& maps, int warp, int lane, uint32_t rank,
+                                         uint32_t ring, uint32_t b_full, uint32_t b_empty, uint32_t b_tfull,
+                                         uint32_t b_tempty, uint32_t b_qfull, uint32_t b_qempty, QEntry* queue,
+                                         uint32_t tmem_base, int n_units, int n_short, int* s_abort)
+{
+    const bool leader = rank == 0;
+    const uint32_t qempty_leader = map_to_cta(b_qempty, 0);
+    const int ksteps = p.k_routed / kBK;
+    if (warp == kBgProdWarp) {
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, q = 0, qphase = 0, armed = 0, armed_phase = 0;
+            const uint64_t pol_w = l2_evict_first(), pol_x = l2_evict_last();
+            const uint32_t peer_queue = map_to_cta(smem_u32(queue), 1), peer_qfull = map_to_cta(b_qfull, 1);
+            bool ok = true;
+            while (ok) {
+                QEntry e;
+                if (leader) {
+                    // scheduler: a free queue slot, then a unit from the tail of the list (while short units are left
+                    // there and the two ends have not met)
+                    if (!mbar_wait_cluster(b_qempty + 8 * q, qphase ^ 1, s_abort, p.status)) { ok = false; break; }
+                    int ix = -1;
+                    for (;;) {
+                        const unsigned long long w = *reinterpret_cast<volatile unsigned long long*>(p.counter);
+                        const uint32_t f = (uint32_t)w, b = (uint32_t)(w >> 32);
+                        if ((int)b >= n_short || (unsigned long long)f + b >= (unsigned long long)n_units) break;
+                        if (atomicCAS(p.counter, w, w + (1ull << 32)) == w) { ix = n_units - 1 - (int)b; break; }
+                    }
+                    e.u = -1; e.tile_slot = 0; e.b_row0 = 0; e.nrows = 0; e.colblock = 0; e.shared = 0; e.pad0 = 0; e.pad1 = 0;
+                    if (ix >= 0) {
+                        const Unit un = p.units[ix];
+                        const Tile t = p.tiles[un.tile];
+                        e.u = ix; e.tile_slot = t.slot; e.b_row0 = t.row0; e.nrows = t.nrows; e.colblock = un.colblock & 0xffffff;
+                    }
+                    *reinterpret_cast<int4*>(&queue[q]) = make_int4(e.u, e.tile_slot, e.b_row0, e.nrows);
+                    *reinterpret_cast<int2*>(&queue[q].colblock) = make_int2(e.colblock, 0);
+                    queue[q].pad0 = 0;
+                    mbar_arrive(b_qfull + 8 * q);
+                    const uint32_t dst = peer_queue + (uint32_t)sizeof(QEntry) * q;
+                    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(e.u), "r"(e.tile_slot),
+                                 "r"(e.b_row0), "r"(e.nrows) : "memory");
+                    asm volatile("st.shared::cluster.v2.b32 [%0], {%1, %2};" ::"r"(dst + 16), "r"(e.colblock), "r"(0) : "memory");
+                    asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(dst + 24), "r"(0) : "memory");
+                    mbar_arrive_cluster(peer_qfull + 8 * q);
+                } else {
+                    if (!mbar_wait_cluster(b_qfull + 8 * q, qphase, s_abort, p.status)) { ok = false; break; }
+                    e = read_entry(&queue[q]);
+                    mbar_arrive_cluster(qempty_leader + 8 * q);
+                }
+                if (++q == kBgQueue) { q = 0; qphase ^= 1; }
+                if (e.u < 0) break;
+                // this CTA's half of the unit: 128 weight rows, half of the (padded) token rows
+                const int npad = (e.nrows + 31) & ~31;
+                const int my_rows = npad >> 1;                                        // 16 or 32
+                const int cb = 2 * e.colblock + (int)rank;
+                const int a_row = e.tile_slot * p.rows_per_slot + cb * p.cb_rows;
+                const int my_row0 = e.b_row0 + (int)rank * my_rows;
+                const CUtensorMap* ma = &maps.a_routed[0];
+                const CUtensorMap* mb = maps.b_routed + (my_rows == 32 ? 2 : 3);     // boxes of 32 / 16 rows
+                for (int ks = 0; ks < ksteps; ++ks) {
+                    if (!mbar_wait(b_empty + 8 * stage, phase ^ 1, s_abort, p.status)) { ok = false; break; }
+                    const uint32_t sa = ring + stage * kBgStageBytes;
+                    const uint32_t full = b_full + 8 * stage;
+                    if (leader) mbar_expect_tx(full, 2u * (uint32_t)(kABytes + my_rows * kBK * 2));
+                    armed |= 1u << stage;
+                    armed_phase = (armed_phase & ~(1u << stage)) | (phase << stage);
+                    if (MODE == 0) tma_load_3d_pair(sa, ma, full, ks * kBK, 0, a_row, pol_w);
+                    else tma_load_2d_pair(sa, ma, full, ks * kBK, a_row, pol_w);
+                    tma_load_2d_pair(sa + kABytes, mb, full, ks * kBK, my_row0, pol_x);
+                    if (++stage == kBgStages) { stage = 0; phase ^= 1; }
+                }
+            }
+            if (!ok && leader) {
+                // gave up: let the copies already in flight land before the block exits
+                for (int s2 = 0; s2 < kBgStages; ++s2)
+                    if (armed & (1u << s2)) mbar_wait(b_full + 8 * s2, (armed_phase >> s2) & 1u, s_abort, p.status);
+            }
+        }
+        __syncwarp();
+    } else if (warp == kBgMmaWarp) {
+        if (lane == 0 && leader) {
+            uint32_t stage = 0, phase = 0, q = 0, qphase = 0, tphase = 0;
+            const uint32_t d = tmem_base + kBgTmemCol;
+            bool ok = true;
+            while (ok) {
+                if (!mbar_wait(b_qfull + 8 * q, qphase, s_abort, p.status)) { ok = false; break; }
+                const QEntry e = read_entry(&queue[q]);
+                mbar_arrive(b_qempty + 8 * q);
+                if (++q == kBgQueue) { q = 0; qphase ^= 1; }
+                if (e.u < 0) break;
+                const int npad = (e.nrows + 31) & ~31;
+                const uint32_t idesc = (1u << 4) | p.idesc_fmt_routed | ((256u >> 4) << 24) | ((uint32_t)(npad >> 3) << 17);
+                if (!mbar_wait_cluster(b_tempty, tphase ^ 1, s_abort, p.status)) { ok = false; break; }
+                tc_fence_after();
+                uint32_t acc = 0;
+                for (int ks = 0; ks < ksteps; ++ks) {
+                    if (!mbar_wait(b_full + 8 * stage, phase, s_abort, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t lo_m = smem_desc_lo(ring + stage * kBgStageBytes), lo_n = lo_m + (kABytes >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < kBK / 16; ++kk) {
+                        umma_bf16_pair(d, smem_desc_pack(lo_m + 2 * kk), smem_desc_pack(lo_n + 2 * kk), idesc, acc);
+                        acc = 1;
+                    }
+                    umma_commit_pair(b_empty + 8 * stage);
+                    if (++stage == kBgStages) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                umma_commit_pair(b_tfull);
+                tphase ^= 1;
+            }
+        }
+        __syncwarp();
+    } else {
+        // epilogue: one warp per TMEM lane quarter; results go straight to global memory (a few KB per unit)
+        const int quarter = warp & 3;
+        const uint32_t d = tmem_base + ((uint32_t)(quarter * 32) << 16) + kBgTmemCol;
+        const uint32_t tempty_leader = map_to_cta(b_tempty, 0);
+        uint32_t q = 0, qphase = 0, tphase = 0;
+        bool ok = true;
+        while (ok) {
+            ok = __all_sync(0xffffffffu, mbar_wait_cluster(b_qfull + 8 * q, qphase, s_abort, p.status));
+            if (!ok) break;
+            const QEntry e = read_entry(&queue[q]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(qempty_leader + 8 * q);
+            if (++q == kBgQueue) { q = 0; qphase ^= 1; }
+            if (e.u < 0) break;
+            ok = __all_sync(0xffffffffu, mbar_wait(b_tfull, tphase, s_abort, p.status));
+            if (!ok) break;
+            tphase ^= 1;
+            tc_fence_after();
+            const int cb = 2 * e.colblock + (int)rank;
+            const int nchunk = ((e.nrows + 31) & ~31) >> 4;                 // 16-token chunks: 2 or 4
+            if (MODE == 0) {
+                // lanes 2i / 2i+1 hold the gate / up row (or up / gate) of intermediate index cb*64 + quarter*16 + i
+                const bool even = (lane & 1) == 0;
+                const bool own_is_gate = even == ((p.gate_first_routed & 1u) != 0);
+                uint32_t o[16];                                             // 8 outputs of 16 bits per chunk
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if (c < nchunk) {
+                        uint32_t r[16];
+                        tmem_ld16(d + c * 16, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4) {
+                            unsigned short h2[2];
+#pragma unroll
+                            for (int t = 0; t < 2; ++t) {
+                                // the even lane finishes token c*16 + j + 2t, the odd lane the one after it
+                                const float send = __uint_as_float(even ? r[j + 2 * t + 1] : r[j + 2 * t]);
+                                const float recv = __shfl_xor_sync(0xffffffffu, send, 1);
+                                const float own = __uint_as_float(even ? r[j + 2 * t] : r[j + 2 * t + 1]);
+                                const float g = own_is_gate ? own : recv, up = own_is_gate ? recv : own;
+                                h2[t] = __bfloat16_as_ushort(__float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * up));
+                            }
+                            o[c * 4 + (j >> 2)] = (uint32_t)h2[0] | ((uint32_t)h2[1] << 16);
+                        }
+                    }
+                }
+                // the accumulator is free as soon as it has been read
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(tempty_leader);
+                unsigned short* out16 = reinterpret_cast<unsigned short*>(p.out_routed) + cb * 64 + quarter * 16 + (lane >> 1);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                    for (int jj = 0; jj < 8; ++jj) {
+                        const int n = c * 16 + 2 * jj + (even ? 0 : 1);
+                        if (c < nchunk && n < e.nrows)
+                            out16[(size_t)(e.b_row0 + n) * p.ld_routed] = (unsigned short)(o[c * 4 + (jj >> 1)] >> ((jj & 1) * 16));
+                    }
+                }
+            } else {
+                // this thread's TMEM lane is output feature cb*128 + quarter*32 + lane; a chunk holds 16 tokens
+                float* outp = reinterpret_cast<float*>(p.out_routed) + cb * 128 + quarter * 32 + lane;
+                for (int c = 0; c < nchunk; ++c) {
+                    uint32_t r[16];
+                    tmem_ld16(d + c * 16, r);
+                    tmem_ld_wait();
+                    if (c == nchunk - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(tempty_leader);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int n = c * 16 + j;
+                        if (n < e.nrows) outp[(size_t)(e.b_row0 + n) * p.ld_routed] = __uint_as_float(r[j]);
+                    }
+                }
+            }
+        }
+    }
+}
+
 // MODE 0: gate/up + SwiGLU (output bf16 for routed units, fp16 for shared units)
 // MODE 1: down projection (output fp32)
 // SWAP (one CTA per unit only): the tokens are the M operand (one TMEM lane per token, up to 128) and up to 256
 // weight rows the N operand.  One MMA then covers twice the weight bytes of the other orientation, which is what
 // counts for short tiles: an MMA costs its issuing lane about 100 cycles however narrow it is, so with weights as M
 // a tile of a few tokens is bound by MMA issue, not by the weight stream.
-template <int MODE, bool PAIR, bool SWAP>
-__global__ void __launch_bounds__(kThreads, 1)
+// BG (pair shape only): a second, small pipeline beside the main one.  A short tile (at most kShortRows tokens) costs the
+// main MMA lane about as many issue slots as a tile of hundreds of tokens, while it hardly loads the tensor pipe; and
+// while a CTA pair works through it, its share of the HBM stream is all it uses.  So the short tiles sit at the tail of
+// the unit list, and every CTA pair has a background TMA lane, MMA lane, 60 KB stage ring and 64-column accumulator
+// that take units from that tail while the main lanes take units from the front: the short tiles' weights stream in
+// behind the tensor-bound tiles.  Whichever side reaches the other's end of the list first stops there (one packed
+// counter orders all claims), so the main lanes finish whatever short tiles are left.  Every output element is still
+// accumulated over K in the same order by one lane: results do not depend on which pipeline ran a unit.
+template <int MODE, bool PAIR, bool SWAP, bool BG>
+__global__ void __launch_bounds__(BG ? kThreadsBg : kThreads, 1)
 grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
 {
     static_assert(!(PAIR && SWAP), "the token-major shape is a one-CTA shape");
+    static_assert(PAIR || !BG, "the background pipeline belongs to the pair shape");
+    constexpr int kAcc = BG ? kBgAccRows : 256;                               // token rows (TMEM columns) per accumulator
+    constexpr uint32_t kAccBytes = (uint32_t)(kAcc / 2) * kBK * 2;            // pair shape: token tile of one CTA per accumulator
     constexpr uint32_t kWBytes = SWAP ? 2 * kABytes : kABytes;               // weight tile of one stage
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
     const uint32_t bars = smem_base + kRingBytes;                              // 8-byte barriers after the tiles
     const uint32_t bar_full = bars, bar_empty = bars + 8 * kMaxStages;
     const uint32_t bar_tfull = bars + 16 * kMaxStages, bar_tempty = bar_tfull + 16;
-    const uint32_t n_stages = ((PAIR && p.wide) || SWAP) ? kWideStages : kMaxStages;
-    const uint32_t stage_bytes = kRingBytes / n_stages;
+    const uint32_t n_stages = BG ? kBgMainStages : (((PAIR && p.wide) || SWAP) ? kWideStages : kMaxStages);
+    const uint32_t stage_bytes = BG ? kBgStageBytesMain : kRingBytes / n_stages;
     // Stages are handed back to the producer in groups: a tcgen05.commit costs the issuing lane about as much
     // as two MMAs, so with four MMAs per stage one commit per stage would starve the tensor pipe.
     const uint32_t group = (uint32_t)p.group;                                  // 1 or 2: masks and shifts below, a
     const uint32_t gmask = group - 1, gshift = group >> 1;                     // division per K step would be felt
     const uint32_t bar_qfull = bar_tempty + 16, bar_qempty = bar_qfull + 8 * kQueue;
     const uint32_t bar_sched = bar_qempty + 8 * kQueue;
+    // background pipeline: stage barriers, accumulator barriers, unit queue; its ring follows the main one
+    const uint32_t bg_full = bar_sched + 8, bg_empty = bg_full + 8 * kBgStages;
+    const uint32_t bg_tfull = bg_empty + 8 * kBgStages, bg_tempty = bg_tfull + 8;
+    const uint32_t bg_qfull = bg_tempty + 8, bg_qempty = bg_qfull + 8 * kBgQueue;
+    const uint32_t bg_ring = smem_base + kBgMainStages * kBgStageBytesMain;
+    __shared__ QEntry s_bg_queue[kBgQueue];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ QEntry s_queue[kQueue];
@@ -294,6 +532,14 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
             mbar_init(bar_qempty + 8 * q, 3 + kEpiWarps + (PAIR ? 2 + kEpiWarps : 0));
         }
         mbar_init(bar_sched, 1);
+        if (BG) {
+            for (int s2 = 0; s2 < kBgStages; ++s2) { mbar_init(bg_full + 8 * s2, 1); mbar_init(bg_empty + 8 * s2, 1); }
+            mbar_init(bg_tfull, 1);
+            mbar_init(bg_tempty, 2 * 4);                  // the four background epilogue warps of both CTAs
+            // unit queue: filled by the leader's background producer (which is the scheduler); drained by the leader's
+            // MMA lane and epilogue warps and by the peer's producer and epilogue warps
+            for (int q2 = 0; q2 < kBgQueue; ++q2) { mbar_init(bg_qfull + 8 * q2, 1); mbar_init(bg_qempty + 8 * q2, 1 + 4 + 1 + 4); }
+        }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -322,6 +568,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     pdl_launch_dependents();
     const int n_units = *p.n_units;
     const int n_shared = *p.n_shared;
+    const int n_short = BG ? *p.n_short : 0;
 
     // Units are pulled from a global counter by one scheduler lane per CTA (pair: per CTA pair, the leader's),
     // decoded, and handed to the other roles through a small queue in shared memory; in pair mode the scheduler
@@ -349,7 +596,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 if (leader) mbar_arrive(bar_qempty + 8 * q); else mbar_arrive_cluster(qempty_leader + 8 * q);
                 if (++q == kQueue) { q = 0; qphase ^= 1; }
                 if (e.u < 0) break;
-                const UnitInfo ui = unit_info<MODE, PAIR, SWAP>(p, e, rank);
+                const UnitInfo ui = unit_info<MODE, PAIR, SWAP, BG>(p, e, rank);
                 const int claim_ks = ui.ksteps > kClaimAhead ? ui.ksteps - kClaimAhead : 0;
                 // L2 policy of the weight tiles: a routed expert with at most 128 rows is read by one tile only, so its
                 // weights stream through (evict-first) and leave the cache to what is read again -- the shared expert's
@@ -363,7 +610,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 const int my_rows = PAIR ? (ui.npad >> 1) : ui.npad;          // token rows this CTA loads
                 const int my_row0 = brow0 + (PAIR ? (int)rank * my_rows : 0);
                 const int my_rows1 = ui.npad1 >> 1;                           // same for the second accumulator
-                const int my_row1 = brow0 + 256 + (int)rank * my_rows1;
+                const int my_row1 = brow0 + kAcc + (int)rank * my_rows1;
                 for (int ks = 0; ks < ui.ksteps; ++ks) {
                     if (wrole && leader && ks == claim_ks) mbar_arrive(bar_sched);      // time to claim the next unit
                     if ((stage & gmask) == 0 &&
@@ -397,7 +644,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                             // pair shape: the two accumulators' tiles, or the K slices of a short unit (behind its two weight
                             // slices); token-major shape: the K slices of the stage
                             const int rows = (by_acc && acc) ? my_rows1 : my_rows, r0 = (by_acc && acc) ? my_row1 : my_row0;
-                            const uint32_t dst = by_acc ? sb + acc * kBBytes
+                            const uint32_t dst = by_acc ? sb + acc * kAccBytes
                                                         : (PAIR ? sa + ui.kb * kABytes : sb) + acc * my_rows * kBK * 2;
                             const int kx = (by_acc ? ks : ks * ui.kb + acc) * kBK;
                             int j = 0;
@@ -433,7 +680,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 mbar_arrive(bar_qempty + 8 * q);
                 if (++q == kQueue) { q = 0; qphase ^= 1; }
                 if (e.u < 0) break;
-                const UnitInfo ui = unit_info<MODE, PAIR, SWAP>(p, e, rank);
+                const UnitInfo ui = unit_info<MODE, PAIR, SWAP, BG>(p, e, rank);
                 const uint32_t fmt = ui.shared ? p.idesc_fmt_shared : p.idesc_fmt_routed;
                 const uint32_t idesc_m = (1u << 4) | fmt | (((PAIR ? 256u : 128u) >> 4) << 24);
                 const uint32_t idesc = idesc_m | ((uint32_t)((SWAP ? ui.width : ui.npad) >> 3) << 17);
@@ -442,9 +689,9 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 // a wide unit takes both accumulator buffers, in the order the epilogue drains them
                 if (!(PAIR ? mbar_wait_cluster(bar_tempty + 8 * buf, bphase ^ 1, &s_abort, p.status)
                            : mbar_wait(bar_tempty + 8 * buf, bphase ^ 1, &s_abort, p.status))) { ok = false; break; }
-                const uint32_t d = tmem_base + buf * 256;
+                const uint32_t d = tmem_base + buf * kAcc;
                 const uint32_t buf1 = buf ^ 1u, bphase1 = buf ? (bphase ^ 1u) : bphase;
-                const uint32_t d1 = tmem_base + buf1 * 256;
+                const uint32_t d1 = tmem_base + buf1 * kAcc;
                 tc_fence_after();
                 // This lane is alone in its warp: every instruction of the loop below is paid in full, so whatever
                 // does not change inside a unit is worked out here, and the descriptors are put together from two
@@ -478,7 +725,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                             if (!mbar_wait_cluster(bar_tempty + 8 * buf1, bphase1 ^ 1, &s_abort, p.status)) { ok = false; break; }
                             tc_fence_after();
                         }
-                        const uint32_t lo_m1 = lo + m_off, lo_n1 = lo + n_off + (kBBytes >> 4);
+                        const uint32_t lo_m1 = lo + m_off, lo_n1 = lo + n_off + (kAccBytes >> 4);
 #pragma unroll
                         for (int kk = 0; kk < kBK / 16; ++kk) {
                             umma_bf16_pair(d1, smem_desc_pack(lo_m1 + 2 * kk), smem_desc_pack(lo_n1 + 2 * kk), idesc1, acc1);
@@ -525,16 +772,16 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
             }
             if (++q == kQueue) { q = 0; qphase ^= 1; }
             if (e.u < 0) break;
-            const UnitInfo ui = unit_info<MODE, PAIR, SWAP>(p, e, rank);
+            const UnitInfo ui = unit_info<MODE, PAIR, SWAP, BG>(p, e, rank);
             const int ld = ui.shared ? p.ld_shared : p.ld_routed;
             const int n_acc = (PAIR && ui.npad1 > 0) ? 2 : 1;
             for (int hh = 0; hh < n_acc && ok; ++hh) {
                 // rows of this accumulator: a wide unit keeps rows 256.. in its second one
-                const int row0 = ui.b_row0 + hh * 256;
-                const int nrows = hh ? ui.nrows - 256 : (n_acc == 2 ? 256 : ui.nrows);
+                const int row0 = ui.b_row0 + hh * kAcc;
+                const int nrows = hh ? ui.nrows - kAcc : (n_acc == 2 ? kAcc : ui.nrows);
                 const int npad = hh ? ui.npad1 : ui.npad;
                 ok = mbar_wait(bar_tfull + 8 * buf, bphase, &s_abort, p.status);
-                const uint32_t d = tmem_base + lane_addr + buf * 256;
+                const uint32_t d = tmem_base + lane_addr + buf * kAcc;
                 if (SWAP) {
                     // Token-major accumulator: this thread's TMEM lane is token `gtid` of the tile, the columns are the
                     // unit's weight rows (256, 128 or 64); each group takes a quarter of them.  Every thread stages and
@@ -743,7 +990,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
             }
         }
         bulk_wait_read<0>();       // staged rows are read before the block's shared memory goes away
-    } else {
+    } else if (warp == kSchedWarp) {
         // ---------------- scheduler (one lane of the leader CTA) ----------------
         if (lane == 0 && leader) {
             uint32_t q = 0, qphase = 0, sphase = 0;
@@ -759,20 +1006,26 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 first = false;
                 if (!(PAIR ? mbar_wait_cluster(bar_qempty + 8 * q, qphase ^ 1, &s_abort, p.status)
                            : mbar_wait(bar_qempty + 8 * q, qphase ^ 1, &s_abort, p.status))) break;
-                int u = atomicAdd(p.counter, 1);
+                // one packed counter orders the claims of both ends of the list: a claim is good while fewer than n_units
+                // units have been taken in all
+                const unsigned long long old = atomicAdd(p.counter, 1ull);
+                int u = (int)(uint32_t)old;
+                const bool good = (unsigned long long)(uint32_t)old + (old >> 32) < (unsigned long long)n_units;
                 int4 e0 = make_int4(-1, 0, 0, 0);
                 int2 e1 = make_int2(0, 0);
                 int e0w = 0;                  // token-major shape: weight rows of the unit
-                if (u < n_units) {
+                if (good) {
                     // The list holds the shared expert's units first.  They are fed from L2 (every token tile of the
                     // model reads the same weights) while the routed units stream theirs from HBM, so the two kinds are
                     // dealt out alternately, in proportion: HBM then stays busy for the whole launch.
                     // The last sixth of the launch is kept for routed units: the shared ones are full-length, and a
                     // long unit handed out at the very end is what the other CTAs then wait for.
+                    // (the short units at the tail of the list are taken in list order)
                     int ix = u;
-                    if (n_shared > 0) {
-                        const int routed = n_units - n_shared;
-                        const int cut = n_units - min(routed, n_units / 6);
+                    const int n_main = n_units - n_short;
+                    if (n_shared > 0 && u < n_main) {
+                        const int routed = n_main - n_shared;
+                        const int cut = n_main - min(routed, n_main / 6);
                         const int uc = min(u, cut), uc1 = min(u + 1, cut);
                         const int a = (int)((long long)uc * n_shared / cut), b = (int)((long long)uc1 * n_shared / cut);
                         ix = b > a ? a : n_shared + (u - a);
@@ -802,6 +1055,9 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
             }
         }
         __syncwarp();
+    } else if (BG) {
+        bg_roles<MODE>(p, maps, warp, lane, rank, bg_ring, bg_full, bg_empty, bg_tfull, bg_tempty, bg_qfull, bg_qempty,
+                       s_bg_queue, tmem_base, n_units, n_short, &s_abort);
     }
 
     tc_fence_before();
@@ -853,7 +1109,7 @@ struct LayerMaps {
 
 struct TensorMaps {
     std::vector<LayerMaps> layers;
-    int max_clusters = -1;              // co-resident 2-CTA clusters of the pair kernels
+    int max_clusters[2] = {-1, -1};     // co-resident 2-CTA clusters of the pair kernels (without / with background lanes)
 };
 
 bool tc_supported(const moe_ctx* c)
@@ -881,6 +1137,13 @@ bool tc_pair_mode(const moe_ctx* c, int T)
 bool tc_wide_mode(const moe_ctx* c, int T)
 {
     return tc_pair_mode(c, T) && c->wide_tiles_enabled != 0;
+}
+
+// Pair shape: the short tiles (at most kShortRows rows) are run by a second, small pipeline of the same CTAs beside
+// the long ones.
+bool tc_background_mode(const moe_ctx* c, int T)
+{
+    return tc_wide_mode(c, T) && c->background_enabled != 0;
 }
 
 // One-CTA units with the tokens as the M operand: every batch that does not take the pair shape.
@@ -949,10 +1212,11 @@ int tc_setup_layer(moe_ctx* c, int layer)
 
 namespace {
 
-template <int MODE, bool PAIR, bool SWAP>
+template <int MODE, bool PAIR, bool SWAP, bool BG>
 cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, cudaStream_t st, int grid_cap)
 {
-    auto kern = grouped_gemm_kernel<MODE, PAIR, SWAP>;
+    auto kern = grouped_gemm_kernel<MODE, PAIR, SWAP, BG>;
+    constexpr int kThr = BG ? kThreadsBg : kThreads;
     // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
     static bool attr_set[kMaxDevices] = {false};
     if (c->device < 0 || c->device >= kMaxDevices) return cudaErrorInvalidDevice;
@@ -962,11 +1226,11 @@ cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, c
         attr_set[c->device] = true;
     }
     if (!PAIR) {
-        return launch_pdl(kern, dim3(std::max(1, std::min(c->sm_count, grid_cap))), dim3(kThreads), kSmemBytes, st, p, maps);
+        return launch_pdl(kern, dim3(std::max(1, std::min(c->sm_count, grid_cap))), dim3(kThr), kSmemBytes, st, p, maps);
     }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(kThr);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
@@ -976,15 +1240,16 @@ cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, c
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (c->tmaps->max_clusters < 0) {
+    int& max_clusters = c->tmaps->max_clusters[BG ? 1 : 0];
+    if (max_clusters < 0) {
         // a persistent kernel must not launch more clusters than can be resident at once
         cfg.gridDim = dim3((unsigned)(c->sm_count & ~1));
         int n = 0;
         if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) n = 1;
         if (n > c->sm_count / 2) n = c->sm_count / 2;
-        c->tmaps->max_clusters = n;
+        max_clusters = n;
     }
-    cfg.gridDim = dim3((unsigned)(2 * std::max(1, std::min(c->tmaps->max_clusters, grid_cap / 2))));
+    cfg.gridDim = dim3((unsigned)(2 * std::max(1, std::min(max_clusters, grid_cap / 2))));
     return cudaLaunchKernelEx(&cfg, kern, p, maps);
 }
 
@@ -1028,7 +1293,8 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     // the shared expert alone runs from unit lists of its own (it may be in flight beside the routed launches)
     int32_t* counts = shared_only ? c->ws.plan_counts_sh : c->ws.plan_counts;
     p1.units = shared_only ? c->ws.units1_sh : c->ws.units1;
-    p1.n_units = counts + 2; p1.counter = counts + 4; p1.n_shared = counts + 6;
+    p1.n_units = counts + 2; p1.counter = reinterpret_cast<unsigned long long*>(counts + 10); p1.n_shared = counts + 6;
+    p1.n_short = counts + 8;
     p1.tiles = c->ws.tiles; p1.stiles = shared_only ? c->ws.stiles_sh : c->ws.stiles;
     int cap1 = c->sm_count, cap2 = c->sm_count;
     if (shared_only) {
@@ -1048,9 +1314,11 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     p1.wide = tc_wide_mode(c, T) ? 1 : 0;
     p1.group = p1.wide ? 1 : 2;
     if (swap) p1.group = 1;
-    cudaError_t e = pair ? launch_gemm<0, true, false>(c, p1, m1, st, cap1)
-                         : (swap ? launch_gemm<0, false, true>(c, p1, m1, st, cap1)
-                                 : launch_gemm<0, false, false>(c, p1, m1, st, cap1));
+    const bool bg = pair && tc_background_mode(c, T);
+    cudaError_t e = pair ? (bg ? launch_gemm<0, true, false, true>(c, p1, m1, st, cap1)
+                               : launch_gemm<0, true, false, false>(c, p1, m1, st, cap1))
+                         : (swap ? launch_gemm<0, false, true, false>(c, p1, m1, st, cap1)
+                                 : launch_gemm<0, false, false, false>(c, p1, m1, st, cap1));
     if (e != cudaSuccess) return e;
     if (!shared_only) stage_mark(c, st, kEvGateUp);
 
@@ -1062,15 +1330,17 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     if (!ok) return cudaErrorInvalidValue;
     GemmParams p2 = p1;
     p2.units = shared_only ? c->ws.units2_sh : c->ws.units2;
-    p2.n_units = counts + 3; p2.counter = counts + 5; p2.n_shared = counts + 7;
+    p2.n_units = counts + 3; p2.counter = reinterpret_cast<unsigned long long*>(counts + 12); p2.n_shared = counts + 7;
+    p2.n_short = counts + 9;
     p2.direct = 0;
     p2.k_routed = I; p2.k_shared = Is;
     p2.rows_per_slot = H; p2.cb_rows = swap ? 64 : 128;
     p2.out_routed = y_perm; p2.out_shared = y_shared; p2.ld_routed = H; p2.ld_shared = H;
     p2.shared_dst_rows = shared_dst_rows;
     p2.idesc_fmt_routed = fmt_bf16; p2.idesc_fmt_shared = fmt_fp16;
-    e = pair ? launch_gemm<1, true, false>(c, p2, m2, st, cap2)
-             : (swap ? launch_gemm<1, false, true>(c, p2, m2, st, cap2) : launch_gemm<1, false, false>(c, p2, m2, st, cap2));
+    e = pair ? (bg ? launch_gemm<1, true, false, true>(c, p2, m2, st, cap2) : launch_gemm<1, true, false, false>(c, p2, m2, st, cap2))
+             : (swap ? launch_gemm<1, false, true, false>(c, p2, m2, st, cap2)
+                     : launch_gemm<1, false, false, false>(c, p2, m2, st, cap2));
     if (e != cudaSuccess) return e;
     if (!shared_only) stage_mark(c, st, kEvDown);
     c->launches += 2;

@@ -18,6 +18,8 @@ constexpr int kMaxExperts = 256;
 constexpr int kMaxBins = 8192;       // E * n_tenants
 constexpr int kTileRows = 128;       // rows (tokens) of one expert handled by one work unit
 constexpr int kDispatchChunk = 256;  // routed rows ranked by one block of the dispatch kernels
+constexpr int kAccRowsBg = 224;      // pair shape with background lanes: token rows per accumulator of a wide tile (two per tile)
+constexpr int kShortRows = 64;       // pair shape: tiles of at most this many rows may be run by the background lanes
 constexpr int kMaxDevices = 64;      // per-device state of the library (kernel attributes, scratch addresses)
 
 // Per (layer, model) weight pointers, as the kernels see them.
@@ -78,12 +80,14 @@ struct Workspace {
     // plan
     Tile* tiles = nullptr;         // routed tiles
     Tile* stiles = nullptr;        // shared-expert tiles
-    int32_t* plan_counts = nullptr;  // [8]: n_tiles, n_stiles, n_units1, n_units2
+    int32_t* tile_cidx = nullptr;  // [tiles] index of a routed tile inside its class (long / short)
+    int32_t* plan_counts = nullptr;  // [16]: n_tiles, n_stiles, n_units1, n_units2, -, -, shared units to spread (2),
+                                     //       short units (2), work counters of the two launches (2 words each)
     Unit* units1 = nullptr;        // gate/up GEMM units (shared, then routed)
     Unit* units2 = nullptr;        // down GEMM units
     // the same for the shared expert alone (one model), when it runs beside the router and the dispatch
     Tile* stiles_sh = nullptr;
-    int32_t* plan_counts_sh = nullptr;  // [8]
+    int32_t* plan_counts_sh = nullptr;  // [16]
     Unit* units1_sh = nullptr;
     Unit* units2_sh = nullptr;
     // activations
@@ -134,6 +138,9 @@ struct moe_ctx {
     int pair_mode_enabled;        // allow the 2-CTA (cta_group::2) shape of the grouped GEMM for long tiles
     int token_major_enabled;      // one-CTA units take the tokens as the M operand of the MMA (up to 256 weight rows per tile)
     int wide_tiles_enabled;       // allow 512-row tiles (two accumulators per weight tile) in the 2-CTA shape
+    int background_enabled;       // pair shape: short tiles are run by a second set of lanes beside the long ones
+    int dispatch_private;         // 0: shared orchestrator (one request per expert block), 1: private orchestrators
+                                  // (one request per tenant and block): invocation statistics and tile formation
     int early_shared_enabled;     // one model: run the shared expert on a second stream beside router and dispatch
                                   // (1: batches of the 2-CTA shape, 2: every batch)
     int early_shared_sms;         // SMs the shared expert's CTA pairs may take while they run beside other kernels
@@ -224,7 +231,8 @@ int tc_setup_layer(moe_ctx* c, int layer);
 void tc_destroy(moe_ctx* c);
 bool tc_supported(const moe_ctx* c);
 bool tc_pair_mode(const moe_ctx* c, int T);      // long tiles: two CTAs share a token tile
-bool tc_wide_mode(const moe_ctx* c, int T);      // pair shape with tiles of up to 512 rows
+bool tc_wide_mode(const moe_ctx* c, int T);      // pair shape with tiles of up to 2 * kAccRows rows
+bool tc_background_mode(const moe_ctx* c, int T);   // pair shape with background lanes for the short tiles
 bool tc_token_major(const moe_ctx* c, int T);    // one-CTA shape with the tokens as the M operand
 
 // Few tokens of one model: the routed gate/up units read the tokens in place, no permuted copy is needed.

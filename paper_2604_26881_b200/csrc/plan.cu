@@ -57,6 +57,8 @@ plan_shared_kernel(PlanArgs a)
         a.plan_counts[2] = su1; a.plan_counts[3] = su2;
         a.plan_counts[4] = 0; a.plan_counts[5] = 0;     // work counters
         a.plan_counts[6] = 0; a.plan_counts[7] = 0;     // nothing to deal out between routed units
+        a.plan_counts[8] = 0; a.plan_counts[9] = 0;     // no short units
+        a.plan_counts[10] = 0; a.plan_counts[11] = 0; a.plan_counts[12] = 0; a.plan_counts[13] = 0;
     }
 }
 
@@ -73,7 +75,7 @@ PlanArgs make_plan_args(moe_ctx* c, int T, int G, bool with_shared)
     PlanArgs a;
     a.slot_table = c->d_slot;
     a.M = g.n_models; a.E = g.n_experts; a.G = G; a.T = T;
-    a.tile_rows = pair ? (tc_wide_mode(c, T) ? 512 : 256) : kTileRows;
+    a.tile_rows = pair ? (tc_wide_mode(c, T) ? (tc_background_mode(c, T) ? 2 * kAccRowsBg : 512) : 256) : kTileRows;
     a.model_tok_off = g.n_models > 1 ? c->ws.model_tok_off : nullptr;
     a.with_shared = with_shared ? 1 : 0;
     a.nblk1 = g.inter / div1; a.nblk2 = g.hidden / div2;
@@ -91,6 +93,11 @@ PlanArgs make_plan_args(moe_ctx* c, int T, int G, bool with_shared)
     a.direct = tc_direct_mode(c, T) ? 1 : 0;
     a.interleave_down = (a.token_major && g.shared_inter > 0 &&
                          (long long)a.shared_down_width * g.shared_inter == 256ll * g.inter) ? 1 : 0;
+    // pair shape: tiles of at most kShortRows rows are kept apart for the background lanes of the grouped GEMM
+    a.short_rows = (pair && tc_background_mode(c, T)) ? kShortRows : 0;
+    a.tile_cidx = a.short_rows ? c->ws.tile_cidx : nullptr;
+    a.private_mode = c->dispatch_private;
+    a.bin_off = c->ws.bin_off; a.bin_base = c->d_bin_base; a.tenants_in_model = c->d_tenants_in_model;
     a.tiles = c->ws.tiles; a.stiles = c->ws.stiles;
     a.units1 = tc ? c->ws.units1 : nullptr; a.units2 = tc ? c->ws.units2 : nullptr;
     a.plan_counts = c->ws.plan_counts;
@@ -101,7 +108,7 @@ size_t plan_smem_ints(const moe_ctx* c, int G)
 {
     const moe_config& g = c->cfg;
     const int B = (g.n_experts + G - 1) / G;
-    return (size_t)g.n_models * g.n_experts + (size_t)g.n_models * B + 1;
+    return 2 * ((size_t)g.n_models * g.n_experts + (size_t)g.n_models * B + 1);
 }
 
 cudaError_t launch_plan(moe_ctx* c, const int32_t* expert_off, int T, int G, bool with_shared, cudaStream_t st)

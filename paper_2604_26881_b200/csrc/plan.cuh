@@ -20,6 +20,12 @@ struct PlanArgs {
     int split_ok[2];                  // token-major: K / 64 of the routed units is even (gate/up, down)
     int direct;                       // the routed gate/up units read all T tokens in place
     int interleave_down;              // the shared units of the down projection are as long as the routed ones
+    int short_rows;                   // tiles of at most this many rows are "short" (0: none)
+    int32_t* tile_cidx;               // [tiles] index of a tile inside its class (long / short); null when short_rows == 0
+    int private_mode;                 // 1: tiles never span two tenants (private orchestrators batch per tenant)
+    const int32_t* bin_off;           //    offsets of the (model, expert, tenant) bins, [nbins + 1]
+    const int32_t* bin_base;          //    first bin of each model
+    const int32_t* tenants_in_model;
     Tile* tiles;
     Tile* stiles;
     Unit* units1;                     // null: no unit lists (CUDA-core path)
@@ -28,42 +34,70 @@ struct PlanArgs {
 };
 
 // Whole block.  expert_off [M*E+1] may live in shared or global memory (already visible to the block).
-// s_mem: M*E + M*B + 1 ints of shared memory; s_warp: 33 ints.
+// s_mem: 2*M*E + 2*(M*B + 1) ints of shared memory; s_warp: 33 ints.
 __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanArgs& a, int32_t* s_mem, int32_t* s_warp)
 {
     const int ME = a.M * a.E;
     const int B = (a.E + a.G - 1) / a.G;
     const int NG = a.M * B;
-    int32_t* s_tile_base = s_mem;            // [ME]   tiles before expert i
-    int32_t* s_group_tile0 = s_mem + ME;     // [NG+1] first tile of each expert block
+    int32_t* s_tile_base = s_mem;               // [ME]   tiles before expert i
+    int32_t* s_short_base = s_mem + ME;         // [ME]   short tiles before expert i
+    int32_t* s_group_long0 = s_mem + 2 * ME;    // [NG+1] long tiles before each expert block
+    int32_t* s_group_short0 = s_group_long0 + NG + 1;   // [NG+1] short tiles before each expert block
     const int tid = threadIdx.x, nth = blockDim.x;
 
+    // Shared orchestrator (Sec. 4.2): the rows of an expert form one segment whoever owns them, cut into tiles.
+    // Private orchestrators: every tenant's rows of an expert are a request of their own, so the segments are the
+    // (expert, tenant) bins and no tile spans two tenants.  Row order, and with it every result, is the same.
+    // A tile of at most short_rows rows is "short": its units form the tail of the unit lists, from where the
+    // background lanes of the pair-shaped grouped GEMM take them (short_rows = 0: no such class).
     for (int i = tid; i < ME; i += nth) {
-        const int cnt = expert_off[i + 1] - expert_off[i];
-        s_tile_base[i] = (cnt + a.tile_rows - 1) / a.tile_rows;
+        const int m = i / a.E, e = i - m * a.E;
+        const int tim = a.private_mode ? a.tenants_in_model[m] : 1;
+        const int b0 = a.private_mode ? a.bin_base[m] + e * tim : 0;
+        int ntile = 0, nshort = 0;
+        for (int ul = 0; ul < tim; ++ul) {
+            const int cnt = a.private_mode ? a.bin_off[b0 + ul + 1] - a.bin_off[b0 + ul] : expert_off[i + 1] - expert_off[i];
+            ntile += (cnt + a.tile_rows - 1) / a.tile_rows;
+            const int rem = cnt % a.tile_rows;          // only the last tile of a segment is ragged
+            if (rem > 0 && rem <= a.short_rows) ++nshort;
+        }
+        s_tile_base[i] = ntile;
+        s_short_base[i] = nshort;
     }
     __syncthreads();
     const int n_tiles = block_scan_exclusive(s_tile_base, ME, s_warp);
+    const int n_short_tiles = block_scan_exclusive(s_short_base, ME, s_warp);
+    const int n_long_tiles = n_tiles - n_short_tiles;
     for (int i = tid; i < ME; i += nth) {
         const int m = i / a.E, e = i - m * a.E;
-        const int row_begin = expert_off[i], row_end = expert_off[i + 1];
-        int tix = s_tile_base[i];
-        for (int r = row_begin; r < row_end; r += a.tile_rows, ++tix) {
-            Tile t;
-            t.row0 = r;
-            t.nrows = min(a.tile_rows, row_end - r);
-            t.slot = a.slot_table[i];
-            t.group = m * B + e / a.G;
-            a.tiles[tix] = t;
+        const int tim = a.private_mode ? a.tenants_in_model[m] : 1;
+        const int b0 = a.private_mode ? a.bin_base[m] + e * tim : 0;
+        int tix = s_tile_base[i], six = s_short_base[i];
+        int lix = tix - six;
+        for (int ul = 0; ul < tim; ++ul) {
+            const int row_begin = a.private_mode ? a.bin_off[b0 + ul] : expert_off[i];
+            const int row_end = a.private_mode ? a.bin_off[b0 + ul + 1] : expert_off[i + 1];
+            for (int r = row_begin; r < row_end; r += a.tile_rows, ++tix) {
+                Tile t;
+                t.row0 = r;
+                t.nrows = min(a.tile_rows, row_end - r);
+                t.slot = a.slot_table[i];
+                t.group = m * B + e / a.G;
+                a.tiles[tix] = t;
+                if (a.tile_cidx) a.tile_cidx[tix] = (t.nrows <= a.short_rows) ? six++ : lix++;   // index inside its class
+            }
         }
     }
     for (int gidx = tid; gidx <= NG; gidx += nth) {
-        int v = n_tiles;
+        int vt = n_tiles, vs = n_short_tiles;
         if (gidx < NG) {
             const int m = gidx / B, b = gidx - m * B;
-            v = s_tile_base[m * a.E + b * a.G];
+            vt = s_tile_base[m * a.E + b * a.G];
+            vs = s_short_base[m * a.E + b * a.G];
         }
-        s_group_tile0[gidx] = v;
+        s_group_long0[gidx] = vt - vs;
+        s_group_short0[gidx] = vs;
     }
     __syncthreads();
 
@@ -106,17 +140,20 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
             u.tile = ~(i % n_stiles);
             a.units2[i] = u;
         }
+        // routed units: the long tiles first, then the short ones; inside each class ordered by (expert block,
+        // weight-row block, tile), so that all experts of a block advance through the same weight-row block together
         const int nmax = n_tiles * max(a.nblk1, a.nblk2);
         for (int i = tid; i < nmax; i += nth) {
             const int tile = i % n_tiles, cb = i / n_tiles;
-            // expert block of the tile: last block whose first tile is <= tile
-            int lo = 0, hi = NG;
-            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (s_group_tile0[mid] <= tile) lo = mid; else hi = mid; }
-            // empty blocks share their first tile with the next one: step to the last of them
-            const int t0 = s_group_tile0[lo], nt = s_group_tile0[lo + 1] - t0;
+            const Tile t = a.tiles[tile];
+            const bool is_short = t.nrows <= a.short_rows;
+            const int ci = a.tile_cidx ? a.tile_cidx[tile] : tile;
+            const int32_t* g0 = is_short ? s_group_short0 : s_group_long0;
+            const int c0 = g0[t.group], nc = g0[t.group + 1] - c0;      // first tile of the block in this class, tiles
+            const int base = is_short ? n_long_tiles : 0;
             Unit u; u.colblock = cb * (tm ? 4 : 1); u.tile = tile;
-            if (cb < a.nblk1) a.units1[su1 + t0 * a.nblk1 + cb * nt + (tile - t0)] = u;
-            if (cb < a.nblk2) a.units2[su2 + t0 * a.nblk2 + cb * nt + (tile - t0)] = u;
+            if (cb < a.nblk1) a.units1[su1 + (base + c0) * a.nblk1 + cb * nc + (ci - c0)] = u;
+            if (cb < a.nblk2) a.units2[su2 + (base + c0) * a.nblk2 + cb * nc + (ci - c0)] = u;
         }
         if (tid == 0) {
             a.plan_counts[2] = su1 + n_tiles * a.nblk1;
@@ -127,6 +164,8 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
             const bool reread = n_stiles > a.M;
             a.plan_counts[6] = reread ? su1 : 0;
             a.plan_counts[7] = (reread && a.interleave_down) ? su2 : 0;
+            a.plan_counts[8] = n_short_tiles * a.nblk1;     // units at the tail of the lists that the background lanes may take
+            a.plan_counts[9] = n_short_tiles * a.nblk2;
         }
         if (a.token_major) {
             // U equally long units on S CTAs take ceil(U / S) rounds; when the last round is less than half full, its
@@ -180,8 +219,9 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
     if (tid == 0) {
         a.plan_counts[0] = n_tiles;
         a.plan_counts[1] = n_stiles;
-        a.plan_counts[4] = 0;           // work counters of the two grouped GEMM launches
-        a.plan_counts[5] = 0;
+        a.plan_counts[4] = 0; a.plan_counts[5] = 0;           // work counters of the two grouped GEMM launches:
+        a.plan_counts[10] = 0; a.plan_counts[11] = 0; a.plan_counts[12] = 0; a.plan_counts[13] = 0;         //   two words each (units taken from the front of the
+                                                              //   list, units taken from its tail)
     }
 }
 

@@ -486,6 +486,56 @@ def test_stack_full_size_teacher_forced():
         g.close()
 
 
+def _modes_case(name):
+    if name == "small-pool":
+        wl = W.MoEWorkload("small-pool", T=333, H=256, E=12, I=128, k=3, Is=256, M=3, n_tenants=5, G=5,
+                           zipf_bias=True, tenant_layout="uniform")
+        return wl, W.make_weights(wl, seed=3, shuffle_slots=True), 3
+    if name == "decode":
+        wl = W.WORKLOADS["decode"]
+        return wl, dict(W.make_weights(W.WORKLOADS["prefill"], seed=0), router_bias=None), 0
+    wl = W.scaled(W.WORKLOADS["prefill"], T=1500, n_tenants=6, tenant_layout="uniform")
+    return wl, W.make_weights(W.WORKLOADS["prefill"], seed=0), 12
+
+
+@pytest.mark.parametrize("case", ["small-pool", "decode", "prefill-6-tenants"])
+def test_shared_and_private_orchestrator_modes(case):
+    # Orchestrator placement: with private orchestrators every tenant's rows of an expert are a request of their own.
+    # Invocation counts and the number of row tiles follow the oracle's accounting in both modes; the permutation,
+    # the tables and every output bit are the same in both (the row order does not change), and equal the oracle.
+    wl, wts, seed = _modes_case(case)
+    x, tenant, mot = W.make_tokens(wl, seed=seed)
+    T = x.shape[0]
+    g = GpuLayer(wl, [wts], T, model_of_tenant=mot)
+    try:
+        res = {}
+        for mode in (B.MOE_DISPATCH_SHARED, B.MOE_DISPATCH_PRIVATE):
+            B.moe_set_option(g.ctx, B.MOE_OPT_DISPATCH_MODE, mode)
+            o = g.four_calls(x, tenant, wl.G)
+            n_tiles, n_stiles, tile_rows = B.moe_last_plan(g.ctx, T)
+            f = g.forward(x, tenant, wl.G)
+            st = B.moe_last_status(g.ctx)
+            assert st[0] == 0 and st[1] == o["n_invocations"] and torch.equal(f, o["out"])
+            assert B.moe_last_plan(g.ctx, T)[0] == n_tiles
+            acc = oracle.invocations(o["topk_idx"].cpu().numpy(), tenant.numpy(), mot.numpy(), n_models=wl.M, E=wl.E,
+                                     G=wl.G, mode=mode, batch_rows=tile_rows)
+            assert o["n_invocations"] == acc.n_invocations, (mode, o["n_invocations"], acc.n_invocations)
+            assert n_tiles == acc.n_row_batches, (mode, n_tiles, acc.n_row_batches, tile_rows)
+            res[mode] = (o, acc)
+        o_s, a_s = res[B.MOE_DISPATCH_SHARED]
+        o_p, a_p = res[B.MOE_DISPATCH_PRIVATE]
+        for key in ("topk_idx", "perm", "inv_perm", "tenant_expert_count", "expert_off", "group_off", "y_perm",
+                    "y_shared", "out"):
+            if o_s[key] is not None:
+                assert torch.equal(o_s[key], o_p[key]), key
+        assert a_p.n_invocations > a_s.n_invocations and a_p.n_row_batches > a_s.n_row_batches
+        ref = oracle_layer(wl, wts, x, tenant, mot, wl.G, o_p["topk_idx"].cpu().numpy(), o_p["topk_w"].cpu().numpy())
+        o_p["n_invocations"] = o_s["n_invocations"]        # (the oracle's dispatch counts the shared placement)
+        compare_four_calls(o_p, ref, wl, x)
+    finally:
+        g.close()
+
+
 def test_host_entry_point_matches_device_entry_point():
     wl = W.WORKLOADS["tiny"]
     wts = W.make_weights(wl, seed=0)

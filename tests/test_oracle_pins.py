@@ -440,3 +440,73 @@ def test_block_forward_residual_add_with_nonzero_layer_output():
     # the classic mistakes give other bits
     for wrong in (c["x"] - res.out, c["x"] + 2 * res.out, res.out, c["x"]):
         assert not np.array_equal(_nearest_bf16_by_table(wrong), x_next)
+
+
+# ----------------------------------------------------------------------------- orchestrator placement (Sec. 4.2, Sec. 5)
+
+def _brute_invocations(idx, tenant, mot, E, G, mode, batch_rows):
+    """Python sets over (tenant, model, block, expert) of every routed row."""
+    rows = [(int(tenant[t]), int(mot[tenant[t]]), int(e) // G, int(e)) for t in range(idx.shape[0]) for e in idx[t]]
+    if mode == oracle.SHARED:
+        inv = {(m, b) for (_, m, b, _) in rows}
+        segs = {}
+        for (_, m, _, e) in rows:
+            segs[(m, e)] = segs.get((m, e), 0) + 1
+    else:
+        inv = {(u, b) for (u, _, b, _) in rows}
+        segs = {}
+        for (u, _, _, e) in rows:
+            segs[(u, e)] = segs.get((u, e), 0) + 1
+    per_tenant = [len({b for (u2, _, b, _) in rows if u2 == u}) for u in range(len(mot))]
+    fan = [len({int(e) // G for e in idx[t]}) for t in range(idx.shape[0])]
+    batches = sum(-(-c // batch_rows) for c in segs.values())
+    return len(inv), per_tenant, fan, batches
+
+
+def test_invocations_match_brute_force_for_both_orchestrator_placements():
+    rng = np.random.default_rng(40)
+    for trial in range(60):
+        E = int(rng.integers(2, 13)); k = int(rng.integers(1, min(E, 4) + 1)); M = int(rng.integers(1, 4))
+        nt = int(rng.integers(M, M + 4)); T = int(rng.integers(1, 40)); G = int(rng.integers(1, E + 1))
+        br = int(rng.integers(1, 6))
+        idx = np.stack([rng.permutation(E)[:k] for _ in range(T)]).astype(np.int32)
+        tenant = rng.integers(0, nt, T).astype(np.int32)
+        mot = (np.arange(nt) % M).astype(np.int32)
+        for mode in (oracle.SHARED, oracle.PRIVATE):
+            r = oracle.invocations(idx, tenant, mot, n_models=M, E=E, G=G, mode=mode, batch_rows=br)
+            n, per_tenant, fan, batches = _brute_invocations(idx, tenant, mot, E, G, mode, br)
+            assert r.n_invocations == n and r.n_row_batches == batches
+            assert r.tenant_invocations.tolist() == per_tenant and r.token_fanout.tolist() == fan
+        sh = oracle.invocations(idx, tenant, mot, n_models=M, E=E, G=G, mode=oracle.SHARED, batch_rows=br)
+        pr = oracle.invocations(idx, tenant, mot, n_models=M, E=E, G=G, mode=oracle.PRIVATE, batch_rows=br)
+        # the shared count is what the dispatch reports; private orchestrators can only add invocations, never more
+        # than one per tenant and shared invocation; and they are the sum of what each tenant issues
+        d = oracle.dispatch(idx, tenant, mot, n_models=M, E=E, G=G)
+        assert sh.n_invocations == d.n_invocations
+        assert sh.n_invocations <= pr.n_invocations <= sh.n_invocations * nt
+        assert pr.n_invocations == int(pr.tenant_invocations.sum())
+        assert pr.n_row_batches >= sh.n_row_batches
+        # a token takes part in between 1 and min(k, blocks) invocations
+        assert fan and min(pr.token_fanout) >= 1 and max(pr.token_fanout) <= min(k, -(-E // G))
+
+
+def test_private_placement_with_one_tenant_equals_shared_placement():
+    rng = np.random.default_rng(41)
+    E, k, T = 10, 3, 50
+    idx = np.stack([rng.permutation(E)[:k] for _ in range(T)]).astype(np.int32)
+    tenant = np.zeros(T, np.int32); mot = np.zeros(1, np.int32)
+    for G in (1, 3, 10):
+        a = oracle.invocations(idx, tenant, mot, n_models=1, E=E, G=G, mode=oracle.SHARED, batch_rows=4)
+        b = oracle.invocations(idx, tenant, mot, n_models=1, E=E, G=G, mode=oracle.PRIVATE, batch_rows=4)
+        assert a.n_invocations == b.n_invocations and a.n_row_batches == b.n_row_batches
+        assert np.array_equal(a.token_fanout, b.token_fanout)
+        assert np.array_equal(a.tenant_invocations, b.tenant_invocations)
+    # one block holding every expert: one shared invocation per model, one private invocation per tenant with tokens
+    tenant = rng.integers(0, 5, T).astype(np.int32); mot = (np.arange(5) % 2).astype(np.int32)
+    a = oracle.invocations(idx, tenant, mot, n_models=2, E=E, G=E, mode=oracle.SHARED)
+    b = oracle.invocations(idx, tenant, mot, n_models=2, E=E, G=E, mode=oracle.PRIVATE)
+    assert a.n_invocations == len(set(mot[tenant])) and b.n_invocations == len(set(tenant.tolist()))
+    assert (a.token_fanout == 1).all()
+    # G = 1: a token reaches k blocks
+    c = oracle.invocations(idx, tenant, mot, n_models=2, E=E, G=1, mode=oracle.PRIVATE)
+    assert (c.token_fanout == k).all()
