@@ -264,7 +264,7 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->wide_tiles_enabled = 1;
     c->token_major_enabled = 1;
     c->dispatch_private = 0;
-    c->background_enabled = 0;
+    c->background_enabled = 1;
     c->timing = false;
     c->early_shared_enabled = 1;
     c->early_shared_sms = 1 << 20;      // no limit
@@ -433,7 +433,8 @@ int moe_set_option(moe_ctx* c, int option, int value)
         return MOE_OK;
     }
     if (option == MOE_OPT_BACKGROUND_LANES) {
-        c->background_enabled = value ? 1 : 0;
+        if (value < 0 || value > 2) return MOE_ERR_SHAPE;
+        c->background_enabled = value;
         return MOE_OK;
     }
     if (option == MOE_OPT_DISPATCH_MODE) {

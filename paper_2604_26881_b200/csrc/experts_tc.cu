@@ -37,6 +37,7 @@ namespace {
 using namespace tc;
 
 constexpr int kMaxStages = 6;
+constexpr int kBarBytesDecl = 512;
 constexpr int kBK = 64;                        // K elements per stage = one 128-byte swizzle row
 constexpr int kABytes = 128 * kBK * 2;         // 128 weight rows: 16 KB
 constexpr int kBRows = 128;                    // token rows one CTA loads per accumulator and stage (pair: half of them)
@@ -47,18 +48,22 @@ constexpr int kRingBytes = kMaxStages * (kABytes + kBBytes);
 constexpr int kWideStages = kRingBytes / (kABytes + 2 * kBBytes);
 constexpr int kQueue = 4;                      // depth of the unit queue of the dynamic scheduler
 // The background pipeline of the pair shape (see the kernel): a ring, a unit queue and an accumulator of its own.
-constexpr int kBgStages = 3;
+constexpr int kBgStages = 4;
 constexpr int kBgRows = kShortRows / 2;        // token rows one CTA of the pair loads per stage (at most)
 constexpr int kBgStageBytes = kABytes + kBgRows * kBK * 2;      // 20 KB: 128 weight rows + 32 token rows
 constexpr int kBgRingBytes = kBgStages * kBgStageBytes;         // 60 KB
 constexpr int kBgQueue = 2;
 constexpr int kBgAccRows = kAccRowsBg;         // token rows per accumulator of a wide tile when the background pipeline runs
 constexpr int kBgStageBytesMain = kABytes + 2 * (kBgAccRows / 2) * kBK * 2;    // 44 KB: weights + two token tiles of 112 rows
-constexpr int kBgMainStages = (kRingBytes - kBgRingBytes) / kBgStageBytesMain;  // 3
-static_assert(kBgMainStages * kBgStageBytesMain + kBgRingBytes <= kRingBytes, "the two rings share the 192 KB");
+constexpr int kBgMainStages = 3;               // (4 main + 2 background stages measured no better: the background lanes, bound
+                                               // by the latency of their few stages in flight, then become the long pole)
+// the two rings take 212 KB: with the background pipeline the epilogue writes its results straight to global memory
+// and the 32 KB output staging area goes to the rings
+constexpr int kBgRingsBytes = kBgMainStages * kBgStageBytesMain + kBgRingBytes;
+
 static_assert(kBgStageBytesMain % 1024 == 0 && kBgStageBytes % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 constexpr int kNumBars = 2 * kMaxStages + 4 + 2 * kQueue + 1 + 2 * kBgStages + 2 + 2 * kBgQueue;
-constexpr int kBarBytes = 512;                 // >= 8 * kNumBars, keeps the staging area 128-byte aligned
+constexpr int kBarBytes = kBarBytesDecl;       // >= 8 * kNumBars, keeps the staging area 128-byte aligned
 // Output staging of the epilogue: results go to shared memory and leave as bulk copies of one row each,
 // so that the epilogue warps never wait on the global store path (which the operand loads saturate).
 // Each group of four epilogue warps owns a quarter of it.
@@ -67,6 +72,7 @@ constexpr int kEpiGroups = 4;                  // groups of four epilogue warps 
 constexpr int kOutGroupBytes = kOutStageBytes / kEpiGroups;
 constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + kBarBytes + kOutStageBytes;
 static_assert(8 * kNumBars <= kBarBytes, "barrier area too small");
+static_assert(kBgRingsBytes <= kRingBytes + kOutStageBytes, "the two rings must fit the shared memory of the CTA");
 constexpr int kEpiWarps = 4 * kEpiGroups;      // four warps per TMEM lane quarter, taking the 16-column chunks in turn
 constexpr int kSchedWarp = 2 + kEpiWarps;      // warp 0: TMA (weights), warp 1: MMA + TMEM, warps 2..17: epilogue, warp 18: scheduler,
 constexpr int kTokWarp = kSchedWarp + 1;       // warp 19: TMA (tokens)
@@ -115,8 +121,8 @@ constexpr int kTcMaxModels = 8;
 struct GemmMaps {
     CUtensorMap a_routed[3];               // gate/up: 3-D (K, {gate,up}, S*I); down: 2-D (K, S*H); [1], [2]: boxes of a half
     CUtensorMap a_shared[kTcMaxModels][3]; //   and a quarter of the weight rows (token-major shape); same for the shared experts
-    CUtensorMap b_routed[4];               // activations of the routed units, boxes of 128 / 64 / 32 / 16 rows
-    CUtensorMap b_shared[4];
+    CUtensorMap b_routed[5];               // activations of the routed units, boxes of 128 / 64 / 32 / 16 rows, and of
+    CUtensorMap b_shared[5];               //   kBgAccRows / 2 rows (one CTA's share of a full accumulator of the background shape)
 };
 
 __device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z,
@@ -497,7 +503,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     constexpr uint32_t kWBytes = SWAP ? 2 * kABytes : kABytes;               // weight tile of one stage
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
-    const uint32_t bars = smem_base + kRingBytes;                              // 8-byte barriers after the tiles
+    const uint32_t bars = smem_base + (BG ? kBgRingsBytes : kRingBytes);       // 8-byte barriers after the tiles
     const uint32_t bar_full = bars, bar_empty = bars + 8 * kMaxStages;
     const uint32_t bar_tfull = bars + 16 * kMaxStages, bar_tempty = bar_tfull + 16;
     const uint32_t n_stages = BG ? kBgMainStages : (((PAIR && p.wide) || SWAP) ? kWideStages : kMaxStages);
@@ -648,6 +654,12 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                                                         : (PAIR ? sa + ui.kb * kABytes : sb) + acc * my_rows * kBK * 2;
                             const int kx = (by_acc ? ks : ks * ui.kb + acc) * kBK;
                             int j = 0;
+                            if (BG && rows == kBgAccRows / 2) {
+                                // a full accumulator of the background shape: one box (a load costs its issuing lane about
+                                // 140 cycles; three boxes per accumulator and stage would make this lane the bottleneck)
+                                tma_load_2d_pair(dst, mb + 4, full, kx, r0, pol_x);
+                                j = rows;
+                            }
 #pragma unroll
                             for (int bx = 0; bx < 4; ++bx) {
                                 const int n = 128 >> bx;
@@ -885,6 +897,82 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+                } else if (BG && MODE == 0) {
+                    // (background shape: no staging area) every thread writes its own results; the accumulator is
+                    // released as soon as its last chunk is in registers
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t gf = ui.shared ? (p.gate_first_shared >> ui.model) & 1u : p.gate_first_routed & 1u;
+                    const bool even = (lane & 1) == 0;
+                    const bool own_is_gate = even == (gf != 0);
+                    // lanes 2i / 2i+1 hold the gate / up row (or up / gate) of intermediate index cb*64 + quarter*16 + i
+                    unsigned short* out16 = reinterpret_cast<unsigned short*>(ui.shared ? p.out_shared : p.out_routed) +
+                                            ui.cb * 64 + quarter * 16 + (lane >> 1);
+                    bool released = false;
+                    for (int c0 = half * 16; c0 < npad; c0 += 16 * kEpiGroups) {
+                        uint32_t r[16];
+                        tmem_ld16(d + c0, r);
+                        tmem_ld_wait();
+                        if (c0 + 16 * kEpiGroups >= npad) {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * buf);
+                            released = true;
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; j += 2) {
+                            // the even lane finishes token c0+j, the odd lane token c0+j+1
+                            const float send = __uint_as_float(even ? r[j + 1] : r[j]);
+                            const float recv = __shfl_xor_sync(0xffffffffu, send, 1);
+                            const float own = __uint_as_float(even ? r[j] : r[j + 1]);
+                            const float g = own_is_gate ? own : recv, up = own_is_gate ? recv : own;
+                            const float v = __fdividef(g, 1.f + __expf(-g)) * up;
+                            const unsigned short o = ui.shared ? __half_as_ushort(__float2half_rn(clamp_fp16(v)))
+                                                               : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+                            const int n = c0 + j + (even ? 0 : 1);
+                            if (n < nrows) out16[(size_t)(row0 + n) * ld] = o;
+                        }
+                    }
+                    if (!released) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * buf);
+                    }
+                } else if (BG) {
+                    // fp32 results: this thread's TMEM lane is output feature cb*128 + quarter*32 + lane, so the lanes
+                    // of a warp write 128 contiguous bytes per token
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const bool remap = ui.shared && p.shared_dst_rows != nullptr;
+                    float* outp = reinterpret_cast<float*>(ui.shared ? p.out_shared : p.out_routed) + ui.cb * 128 + quarter * 32 + lane;
+                    bool released = false;
+                    for (int c0 = half * 16; c0 < npad; c0 += 16 * kEpiGroups) {
+                        uint32_t r[16];
+                        tmem_ld16(d + c0, r);
+                        tmem_ld_wait();
+                        if (c0 + 16 * kEpiGroups >= npad) {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * buf);
+                            released = true;
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int n = c0 + j;
+                            if (n < nrows) {
+                                int row = row0 + n;
+                                if (remap) row = p.shared_dst_rows[row];
+                                outp[(size_t)row * ld] = __uint_as_float(r[j]);
+                            }
+                        }
+                    }
+                    if (!released) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * buf);
+                    }
                 } else if (MODE == 0) {
                     // The group's staging area holds its 4 chunks of 16 tokens as rows of 64 outputs (128 bytes).
                     // Its previous contents must have left (every thread waits for the rows it sent itself), and the
@@ -1143,7 +1231,11 @@ bool tc_wide_mode(const moe_ctx* c, int T)
 // the long ones.
 bool tc_background_mode(const moe_ctx* c, int T)
 {
-    return tc_wide_mode(c, T) && c->background_enabled != 0;
+    // measured: it pays where long, tensor-bound tiles dominate and the short tiles can hide behind them (4096-token
+    // prefill: step -3 %); where nearly every tile is short the launch is bound by HBM and the background lanes, with
+    // their shallow ring, stream worse than the main ones (240-expert pool +10 %, 1126 tokens +4 %)
+    if (!tc_wide_mode(c, T) || c->background_enabled == 0) return false;
+    return c->background_enabled == 2 || (c->cfg.n_models == 1 && T >= 2048);
 }
 
 // One-CTA units with the tokens as the M operand: every batch that does not take the pair shape.
@@ -1276,9 +1368,9 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     auto make_b = [](CUtensorMap* m, const void* base, uint64_t rows, uint64_t k, bool fp16) {
         bool good = true;
         for (int bx = 0; bx < 4; ++bx) good = good && make_map(m + bx, base, rows, k, 128u >> bx, fp16);
-        return good;
+        return good && make_map(m + 4, base, rows, k, kBgAccRows / 2, fp16);
     };
-    auto copy_b = [](CUtensorMap* dst, const CUtensorMap* src) { for (int bx = 0; bx < 4; ++bx) dst[bx] = src[bx]; };
+    auto copy_b = [](CUtensorMap* dst, const CUtensorMap* src) { for (int bx = 0; bx < 5; ++bx) dst[bx] = src[bx]; };
     if (!direct && !shared_only) ok = make_b(m1.b_routed, x_perm, R, H, false);
     if (shared || direct) {
         ok = ok && make_b(m1.b_shared, x_or_xs, T, H, false);
@@ -1314,7 +1406,8 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     p1.wide = tc_wide_mode(c, T) ? 1 : 0;
     p1.group = p1.wide ? 1 : 2;
     if (swap) p1.group = 1;
-    const bool bg = pair && tc_background_mode(c, T);
+    // (the shared expert alone has no short tiles: its launches keep the shape without the background pipeline)
+    const bool bg = pair && tc_background_mode(c, T) && !shared_only;
     cudaError_t e = pair ? (bg ? launch_gemm<0, true, false, true>(c, p1, m1, st, cap1)
                                : launch_gemm<0, true, false, false>(c, p1, m1, st, cap1))
                          : (swap ? launch_gemm<0, false, true, false>(c, p1, m1, st, cap1)

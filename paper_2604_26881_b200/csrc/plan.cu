@@ -121,7 +121,8 @@ cudaError_t launch_plan(moe_ctx* c, const int32_t* expert_off, int T, int G, boo
 
 void shared_unit_counts(moe_ctx* c, int T, int* n_units1, int* n_units2)
 {
-    const PlanArgs a = make_plan_args(c, T, 1, true);
+    PlanArgs a = make_plan_args(c, T, 1, true);
+    if (tc_background_mode(c, T)) a.tile_rows = 512;
     const int n_stiles = (T + a.tile_rows - 1) / a.tile_rows;
     *n_units1 = n_stiles * a.snblk1;
     *n_units2 = n_stiles * a.snblk2;
@@ -130,6 +131,7 @@ void shared_unit_counts(moe_ctx* c, int T, int* n_units1, int* n_units2)
 cudaError_t launch_plan_shared(moe_ctx* c, int T, cudaStream_t st)
 {
     PlanArgs a = make_plan_args(c, T, 1, true);
+    if (tc_background_mode(c, T)) a.tile_rows = 512;      // launched in the shape without the background pipeline
     a.stiles = c->ws.stiles_sh; a.units1 = c->ws.units1_sh; a.units2 = c->ws.units2_sh;
     a.plan_counts = c->ws.plan_counts_sh;
     launch_pdl(plan_shared_kernel, dim3(1), dim3(256), 0, st, a);

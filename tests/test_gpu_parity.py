@@ -297,6 +297,36 @@ def test_wide_tiles_and_narrow_tiles_agree_bit_for_bit(qwen_weights, T):
         g.close()
 
 
+@pytest.mark.parametrize("T", [200, 1500, 4096])
+def test_background_lanes_agree_bit_for_bit(qwen_weights, T):
+    # the 2-CTA shape may run the short tiles (at most 64 rows) in a second pipeline beside the long ones; which
+    # pipeline runs a unit, and in what order, depends on timing, the result does not: every output element is summed
+    # over K in the same order by one lane.  Several tenants and the private orchestrator mode give many short tiles;
+    # calls back to back reuse the work counters.
+    wl = W.scaled(W.WORKLOADS["prefill"], T=T, n_tenants=5, tenant_layout="uniform")
+    x, tenant, mot = W.make_tokens(wl, seed=9)
+    g = GpuLayer(wl, [qwen_weights], wl.T, model_of_tenant=mot)
+    try:
+        for mode in (B.MOE_DISPATCH_SHARED, B.MOE_DISPATCH_PRIVATE):
+            B.moe_set_option(g.ctx, B.MOE_OPT_DISPATCH_MODE, mode)
+            for early in (0, 2):
+                B.moe_set_option(g.ctx, B.MOE_OPT_EARLY_SHARED, early)
+                B.moe_set_option(g.ctx, B.MOE_OPT_BACKGROUND_LANES, 0)
+                ref = g.forward(x, tenant, wl.G)
+                B.moe_set_option(g.ctx, B.MOE_OPT_BACKGROUND_LANES, 2)
+                outs = [g.forward(x, tenant, wl.G) for _ in range(4)]
+                assert B.moe_last_status(g.ctx)[0] == 0
+                for o in outs:
+                    assert torch.equal(o, ref), (mode, early)
+        # and against the oracle through the four calls, background lanes on
+        o = g.four_calls(x, tenant, wl.G)
+        ref = oracle_layer(wl, qwen_weights, x, tenant, mot, wl.G, o["topk_idx"].cpu().numpy(), o["topk_w"].cpu().numpy())
+        o["n_invocations"] = ref.dispatch.n_invocations      # (private mode counts per tenant: checked elsewhere)
+        compare_four_calls(o, ref, wl, x)
+    finally:
+        g.close()
+
+
 @pytest.mark.parametrize("T", [7, 64, 300, 1024, 4096])
 def test_shared_expert_on_second_stream_agrees_bit_for_bit(qwen_weights, T):
     # one model: the shared expert's launches may run on the context's second stream beside the router and the
