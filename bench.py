@@ -59,6 +59,8 @@ def parse_args(argv=None):
                     help="shared expert on the context's second stream (auto: the library's default, batches of more than 64 tokens); "
                          "the per-stage times and the roofline block always come from passes without it, where one "
                          "grouped-GEMM launch holds the shared and the routed units")
+    ap.add_argument("--background", default="auto", choices=["auto", "0", "1", "2"],
+                    help="background lanes of the 2-CTA grouped GEMM for short tiles (auto: the library's default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dry", action="store_true",
                     help="exercise the launch and reduction protocol without a GPU (gloo ranks, a sleep as the step)")
@@ -273,6 +275,8 @@ def apply_options(B, ctx, args):
     B.moe_set_option(ctx, B.MOE_OPT_PAIR_MODE, {"auto": 1, "never": 0}[args.pair])
     if args.early_shared != "auto":
         B.moe_set_option(ctx, B.MOE_OPT_EARLY_SHARED, int(args.early_shared))
+    if args.background != "auto":
+        B.moe_set_option(ctx, B.MOE_OPT_BACKGROUND_LANES, int(args.background))
 
 
 def cuda_events():

@@ -164,6 +164,26 @@ int moe_set_slot_table(moe_ctx* ctx, const int32_t* slot);
  * Default: u % M.  Copied; synchronises the device. */
 int moe_set_tenant_models(moe_ctx* ctx, const int32_t* model_of_tenant);
 
+/*
+ * Load-aware formation of expert blocks (Sec. 5, on expert granularity: blocks that follow expert popularity are the
+ * paper's outlook; the rule here is greedy).  For every model the E experts are put into B = ceil(E/G) blocks of at
+ * most G experts so that the blocks' loads are even: experts in order of (load descending, id ascending), each into
+ * the block with the smallest load so far among those with fewer than G experts (ties: lowest block id).
+ * Host function, no GPU work: load is a host array [M, E] (for instance the per-expert row counts of earlier
+ * batches, summed from tenant_expert_count), block_of_expert a host array [M, E] that receives ids in [0, B).
+ */
+int moe_form_blocks(const int64_t* load, int n_models, int n_experts, int G, int32_t* block_of_expert);
+
+/*
+ * Makes the context use blocks given by a table instead of blocks of G consecutive experts: block_of_expert is a host
+ * array [M, E] of ids in [0, n_blocks) (copied; synchronises the device); NULL restores the ranges.  While a table is
+ * set the G argument of the calls is only validated; a block is a set of experts, so group_off (M*n_blocks + 1
+ * entries) holds the running sum of the rows the blocks receive, in block order, and the invocation statistics count
+ * the table's blocks.  The permutation and every output bit stay the same (Sec. 3: block size and composition do not
+ * affect routing or results); the table orders the expert work and defines what one invocation carries.
+ */
+int moe_set_block_table(moe_ctx* ctx, const int32_t* block_of_expert, int n_blocks);
+
 int moe_set_option(moe_ctx* ctx, int option, int value);
 
 /*

@@ -44,7 +44,8 @@ def _load():
         _lib = ctypes.CDLL(_LIB)
         _lib.oracle_num_threads.restype = ctypes.c_int
         for name in ("oracle_route", "oracle_dispatch", "oracle_experts", "oracle_shared_expert",
-                     "oracle_combine", "oracle_rmsnorm", "oracle_invocations"):
+                     "oracle_combine", "oracle_rmsnorm", "oracle_invocations", "oracle_form_blocks",
+                     "oracle_invocations_table"):
             getattr(_lib, name).restype = ctypes.c_int
         _lib.oracle_round_bf16.restype = None
     return _lib
@@ -159,6 +160,46 @@ def invocations(topk_idx, tenant_id, model_of_tenant, *, n_models, E, G, mode, b
     if rc != 0:
         raise ValueError(f"oracle_invocations failed: {rc}")
     return Invocations(int(ninv.value), per_tenant, fan, int(nbatch.value))
+
+
+def form_blocks(load, *, G):
+    """Load-aware expert blocks (Sec. 5): experts in order of (load descending, id ascending), each to the least
+    loaded block that still has room.  load [M,E] -> block_of_expert [M,E] int32 with ids in [0, ceil(E/G))."""
+    lib = _load()
+    load = np.ascontiguousarray(load, dtype=np.int64)
+    M, E = load.shape
+    out = np.empty((M, E), np.int32)
+    rc = lib.oracle_form_blocks(_p(load), M, E, G, _p(out))
+    if rc != 0:
+        raise ValueError(f"oracle_form_blocks failed: {rc}")
+    return out
+
+
+@dataclass
+class TableInvocations:
+    n_invocations: int
+    tenant_invocations: np.ndarray   # [n_tenants] i32
+    token_fanout: np.ndarray         # [T] i32
+    block_rows: np.ndarray           # [M, n_blocks] i32
+
+
+def invocations_table(topk_idx, tenant_id, model_of_tenant, block_of_expert, *, n_blocks, mode):
+    """Invocation accounting when the blocks are given by a table [M,E] instead of ranges of G experts."""
+    lib = _load()
+    topk_idx = _c(topk_idx, np.int32); tenant_id = _c(tenant_id, np.int32)
+    model_of_tenant = _c(model_of_tenant, np.int32); block_of_expert = _c(block_of_expert, np.int32)
+    T, k = topk_idx.shape
+    M, E = block_of_expert.shape
+    n_tenants = len(model_of_tenant)
+    ninv = ctypes.c_int32(0)
+    per_tenant = np.empty((n_tenants,), np.int32); fan = np.empty((T,), np.int32)
+    rows = np.empty((M, n_blocks), np.int32)
+    rc = lib.oracle_invocations_table(_p(topk_idx), _p(tenant_id), T, E, k, M, n_tenants, _p(model_of_tenant),
+                                      _p(block_of_expert), n_blocks, mode, ctypes.byref(ninv), _p(per_tenant), _p(fan),
+                                      _p(rows))
+    if rc != 0:
+        raise ValueError(f"oracle_invocations_table failed: {rc}")
+    return TableInvocations(int(ninv.value), per_tenant, fan, rows)
 
 
 def experts(x, tenant_id, topk_idx, perm, model_of_tenant, pool_gate, pool_up, pool_down, slot_table, *, n_models):

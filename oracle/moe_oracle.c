@@ -217,6 +217,103 @@ int oracle_dispatch(const int32_t* topk_idx, const int32_t* tenant_id, int T, in
 }
 
 /*
+ * Load-aware formation of expert blocks (Sec. 5, on expert granularity: the
+ * paper leaves blocks that take expert popularity into account as future
+ * work; the reading taken here is the greedy rule below).
+ *
+ * For every model, its E experts are put into B = ceil(E/G) blocks of at most
+ * G experts each so that the blocks' loads are even: experts are taken in the
+ * order (load descending, expert id ascending) and each goes to the block that
+ * has the smallest load so far among the blocks with fewer than G experts
+ * (ties: the lowest block id).
+ *
+ * load [M,E] (rows routed to every expert, any non-negative weights);
+ * block_of_expert [M,E] receives block ids in [0, B).  Returns 0, -2 on bad G.
+ */
+int oracle_form_blocks(const int64_t* load, int n_models, int E, int G, int32_t* block_of_expert)
+{
+    if (G < 1 || G > E) return -2;
+    const int B = (E + G - 1) / G;
+    int* order = (int*)malloc(sizeof(int) * (size_t)E);
+    int64_t* bload = (int64_t*)malloc(sizeof(int64_t) * (size_t)B);
+    int* bsize = (int*)malloc(sizeof(int) * (size_t)B);
+    for (int m = 0; m < n_models; ++m) {
+        const int64_t* l = load + (size_t)m * E;
+        for (int e = 0; e < E; ++e) order[e] = e;
+        /* insertion sort by (load descending, id ascending) */
+        for (int i = 1; i < E; ++i) {
+            const int v = order[i];
+            int j = i - 1;
+            while (j >= 0 && (l[order[j]] < l[v] || (l[order[j]] == l[v] && order[j] > v))) { order[j + 1] = order[j]; --j; }
+            order[j + 1] = v;
+        }
+        for (int b = 0; b < B; ++b) { bload[b] = 0; bsize[b] = 0; }
+        for (int i = 0; i < E; ++i) {
+            const int e = order[i];
+            int best = -1;
+            for (int b = 0; b < B; ++b)
+                if (bsize[b] < G && (best < 0 || bload[b] < bload[best])) best = b;
+            block_of_expert[(size_t)m * E + e] = best;
+            bload[best] += l[e];
+            bsize[best] += 1;
+        }
+    }
+    free(order); free(bload); free(bsize);
+    return 0;
+}
+
+/*
+ * Invocation accounting for blocks given by a table (block_of_expert [M,E],
+ * ids in [0, n_blocks)) instead of ranges of G consecutive experts; same
+ * meaning of mode and of the outputs as oracle_invocations below.  block_rows
+ * [M, n_blocks] (or NULL) receives the rows every block gets.
+ */
+int oracle_invocations_table(const int32_t* topk_idx, const int32_t* tenant_id, int T, int E, int k,
+                             int n_models, int n_tenants, const int32_t* model_of_tenant,
+                             const int32_t* block_of_expert, int n_blocks, int mode,
+                             int32_t* n_invocations, int32_t* tenant_invocations, int32_t* token_fanout,
+                             int32_t* block_rows)
+{
+    if (mode < 0 || mode > 1 || n_blocks < 1) return -2;
+    for (int i = 0; i < n_models * E; ++i) if (block_of_expert[i] < 0 || block_of_expert[i] >= n_blocks) return -1;
+    /* reached[u][b]: tenant u has a row in block b of its model */
+    unsigned char* reached = (unsigned char*)calloc((size_t)n_tenants * n_blocks, 1);
+    unsigned char* any = (unsigned char*)calloc((size_t)n_models * n_blocks, 1);
+    if (block_rows) memset(block_rows, 0, sizeof(int32_t) * (size_t)n_models * n_blocks);
+    for (int t = 0; t < T; ++t) {
+        const int u = tenant_id[t];
+        if (u < 0 || u >= n_tenants || model_of_tenant[u] < 0 || model_of_tenant[u] >= n_models) { free(reached); free(any); return -1; }
+        const int m = model_of_tenant[u];
+        int fan = 0;
+        for (int j = 0; j < k; ++j) {
+            const int e = topk_idx[(size_t)t * k + j];
+            if (e < 0 || e >= E) { free(reached); free(any); return -1; }
+            const int b = block_of_expert[(size_t)m * E + e];
+            reached[(size_t)u * n_blocks + b] = 1;
+            any[(size_t)m * n_blocks + b] = 1;
+            if (block_rows) block_rows[(size_t)m * n_blocks + b] += 1;
+            int seen = 0;
+            for (int j2 = 0; j2 < j; ++j2)
+                if (block_of_expert[(size_t)m * E + topk_idx[(size_t)t * k + j2]] == b) seen = 1;
+            if (!seen) ++fan;
+        }
+        if (token_fanout) token_fanout[t] = fan;
+    }
+    int ninv = 0;
+    for (int u = 0; u < n_tenants; ++u) {
+        int c = 0;
+        for (int b = 0; b < n_blocks; ++b) c += reached[(size_t)u * n_blocks + b];
+        if (tenant_invocations) tenant_invocations[u] = c;
+        if (mode == 1) ninv += c;
+    }
+    if (mode == 0)
+        for (int i = 0; i < n_models * n_blocks; ++i) ninv += any[i];
+    free(reached); free(any);
+    if (n_invocations) *n_invocations = ninv;
+    return 0;
+}
+
+/*
  * Invocation accounting of the two orchestrator placements (Sec. 4.2,
  * deployment strategies FaaSMoE-Shared and FaaSMoE-Private; Sec. 4.3.1 on
  * batching across tenants and fan-out; Sec. 5 on orchestrator placement).

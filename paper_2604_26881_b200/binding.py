@@ -34,7 +34,7 @@ MOE_DISPATCH_SHARED, MOE_DISPATCH_PRIVATE = 0, 1
 MOE_PATH_AUTO, MOE_PATH_FMA, MOE_PATH_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["moe_create", "moe_destroy", "moe_set_expert_pool", "moe_set_model_weights", "moe_set_slot_table",
-           "moe_set_tenant_models", "moe_set_option", "moe_route", "moe_dispatch", "moe_experts", "moe_combine",
+           "moe_set_tenant_models", "moe_set_option", "moe_form_blocks", "moe_set_block_table", "moe_route", "moe_dispatch", "moe_experts", "moe_combine",
            "moe_layer_forward", "moe_layer_forward_host", "moe_layer_forward_timed", "moe_stack_forward",
            "moe_get_workspace", "moe_last_status", "moe_last_plan", "moe_launch_count", "moe_strerror", "moe_dispatch_noalloc"]
 MOE_DISPATCH_NOALLOC_MAX_WORDS = 1 << 18
@@ -78,6 +78,8 @@ def load_library(path: str | None = None):
         lib.moe_set_slot_table.argtypes = [c_void_p, c_void_p]
         lib.moe_set_tenant_models.argtypes = [c_void_p, c_void_p]
         lib.moe_set_option.argtypes = [c_void_p, c_int, c_int]
+        lib.moe_form_blocks.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p]
+        lib.moe_set_block_table.argtypes = [c_void_p, c_void_p, c_int]
         lib.moe_route.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int] + [c_void_p] * 5
         lib.moe_dispatch.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int] + [c_void_p] * 7
         lib.moe_experts.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int,
@@ -152,6 +154,24 @@ def moe_set_slot_table(ctx, slot_host):
 def moe_set_tenant_models(ctx, model_of_tenant_host):
     assert model_of_tenant_host.dtype == torch.int32 and not model_of_tenant_host.is_cuda
     _check("moe_set_tenant_models", load_library().moe_set_tenant_models(ctx, _ptr(model_of_tenant_host)))
+
+
+def moe_form_blocks(load, G):
+    """Load-aware expert blocks from a host tensor load [M, E] (int64): returns block_of_expert [M, E] int32."""
+    load = load.to(torch.int64).contiguous().cpu()
+    M, E = load.shape
+    out = torch.empty((M, E), dtype=torch.int32)
+    _check("moe_form_blocks", load_library().moe_form_blocks(c_void_p(load.data_ptr()), M, E, G, c_void_p(out.data_ptr())))
+    return out
+
+
+def moe_set_block_table(ctx, block_of_expert, n_blocks=0):
+    """block_of_expert: host int32 tensor [M, E] with ids in [0, n_blocks), or None for blocks of G consecutive experts."""
+    if block_of_expert is None:
+        _check("moe_set_block_table", load_library().moe_set_block_table(ctx, None, 0))
+        return
+    t = block_of_expert.to(torch.int32).contiguous().cpu()
+    _check("moe_set_block_table", load_library().moe_set_block_table(ctx, c_void_p(t.data_ptr()), n_blocks))
 
 
 def moe_set_option(ctx, option, value):

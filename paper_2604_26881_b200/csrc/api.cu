@@ -273,6 +273,7 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->errbuf[0] = 0;
     c->d_models = nullptr; c->d_slot = nullptr; c->d_model_of_tenant = nullptr; c->d_tenant_local = nullptr;
     c->d_bin_base = nullptr; c->d_tenants_in_model = nullptr;
+    c->d_block_table = nullptr; c->table_blocks = 0;
     int rc = MOE_OK;
     cudaError_t e = cudaGetDevice(&c->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
@@ -329,7 +330,7 @@ int moe_destroy(moe_ctx* c)
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     if (c->side) cudaStreamDestroy(c->side);
     void* ptrs[] = {c->d_models, c->d_slot, c->d_model_of_tenant, c->d_tenant_local, c->d_bin_base,
-                    c->d_tenants_in_model};
+                    c->d_tenants_in_model, c->d_block_table};
     for (void* p : ptrs) if (p) cudaFree(p);
     delete c;
     return MOE_OK;
@@ -392,6 +393,52 @@ int moe_set_tenant_models(moe_ctx* c, const int32_t* model_of_tenant)
     c->h_model_of_tenant.assign(model_of_tenant, model_of_tenant + c->cfg.n_tenants);
     MOE_CUDA(c, cudaDeviceSynchronize());
     return upload_tenant_tables(c);
+}
+
+int moe_form_blocks(const int64_t* load, int n_models, int n_experts, int G, int32_t* block_of_expert)
+{
+    if (!load || !block_of_expert) return MOE_ERR_NULL;
+    if (n_models < 1 || n_experts < 1) return MOE_ERR_SHAPE;
+    if (G < 1 || G > n_experts) return MOE_ERR_G;
+    const int E = n_experts, B = (E + G - 1) / G;
+    std::vector<int> order(E), members(B);
+    std::vector<int64_t> weight(B);
+    for (int m = 0; m < n_models; ++m) {
+        const int64_t* l = load + (size_t)m * E;
+        for (int e = 0; e < E; ++e) order[e] = e;
+        // heaviest expert first; equal loads in id order
+        std::stable_sort(order.begin(), order.end(), [&](int x, int y) { return l[x] > l[y]; });
+        std::fill(members.begin(), members.end(), 0);
+        std::fill(weight.begin(), weight.end(), (int64_t)0);
+        for (int e : order) {
+            int best = -1;
+            for (int b = 0; b < B; ++b)
+                if (members[b] < G && (best < 0 || weight[b] < weight[best])) best = b;
+            block_of_expert[(size_t)m * E + e] = best;
+            weight[best] += l[e];
+            members[best] += 1;
+        }
+    }
+    return MOE_OK;
+}
+
+int moe_set_block_table(moe_ctx* c, const int32_t* block_of_expert, int n_blocks)
+{
+    if (!c) return MOE_ERR_NULL;
+    const size_t ME = (size_t)c->cfg.n_models * c->cfg.n_experts;
+    MOE_CUDA(c, cudaDeviceSynchronize());
+    if (!block_of_expert) {               // back to blocks of G consecutive experts
+        if (c->d_block_table) cudaFree(c->d_block_table);
+        c->d_block_table = nullptr;
+        c->table_blocks = 0;
+        return MOE_OK;
+    }
+    if (n_blocks < 1 || n_blocks > c->cfg.n_experts) return MOE_ERR_SHAPE;
+    for (size_t i = 0; i < ME; ++i) if (block_of_expert[i] < 0 || block_of_expert[i] >= n_blocks) return MOE_ERR_SHAPE;
+    if (!c->d_block_table) MOE_CUDA(c, dev_alloc(&c->d_block_table, ME));
+    MOE_CUDA(c, cudaMemcpy(c->d_block_table, block_of_expert, ME * sizeof(int32_t), cudaMemcpyHostToDevice));
+    c->table_blocks = n_blocks;
+    return MOE_OK;
 }
 
 int moe_set_option(moe_ctx* c, int option, int value)

@@ -39,7 +39,8 @@ __device__ void scan_and_tables(int32_t* s_tot, int32_t* s_part /* [33] */, int3
                                 int nbins, int R, int E, int M, int G, int n_tenants, const BinMap& bm,
                                 int32_t* __restrict__ bin_off /* may be null */,
                                 int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
-                                int32_t* __restrict__ group_off, int32_t* __restrict__ stats, int private_mode)
+                                int32_t* __restrict__ group_off, int32_t* __restrict__ stats, int private_mode,
+                                const int32_t* __restrict__ block_table = nullptr, int table_blocks = 0)
 {
     const int tid = threadIdx.x, nth = blockDim.x;
     if (tid < 2) s_count[tid] = 0;
@@ -68,6 +69,46 @@ __device__ void scan_and_tables(int32_t* s_tot, int32_t* s_part /* [33] */, int3
         expert_off[i] = v;
     }
     __syncthreads();
+    if (block_table) {
+        // Blocks given by a table (load-aware formation, Sec. 5) are sets of experts, not ranges of rows: group_off
+        // then holds the running sum of the rows every block receives, in block order.  Sizes are small (M * B blocks,
+        // E experts each): plain loops.
+        const int B = table_blocks;
+        for (int i = tid; i < M * B; i += nth) {
+            const int m = i / B, b = i - m * B;
+            int rows = 0;
+            for (int e = 0; e < E; ++e)
+                if (block_table[m * E + e] == b) rows += expert_off[m * E + e + 1] - expert_off[m * E + e];
+            if (rows > 0 && !private_mode) atomicAdd(&s_count[0], 1);
+            if (group_off) group_off[i + 1] = rows;
+        }
+        __syncthreads();
+        if (tid == 0 && group_off) {
+            int run = 0;
+            group_off[0] = 0;
+            for (int i = 1; i <= M * B; ++i) { run += group_off[i]; group_off[i] = run; }
+        }
+        if (private_mode) {
+            for (int i = tid; i < n_tenants * B; i += nth) {
+                const int u = i / B, b = i - u * B;
+                const int m = bm.model_of_tenant[u];
+                const int tim = bm.tenants_in_model[m], ul = bm.tenant_local[u];
+                bool any = false;
+                for (int e = 0; e < E; ++e) {
+                    if (block_table[m * E + e] != b) continue;
+                    const int bin = bm.bin_base[m] + e * tim + ul;
+                    const int end = bin + 1 < nbins ? s_tot[bin + 1] : R;
+                    any = any || end > s_tot[bin];
+                }
+                if (any) atomicAdd(&s_count[0], 1);
+            }
+        }
+        for (int i = tid; i < M * E; i += nth)
+            if (expert_off[i + 1] > expert_off[i]) atomicAdd(&s_count[1], 1);
+        __syncthreads();
+        if (tid < 2) stats[tid] = s_count[tid];
+        return;
+    }
     // expert blocks of G experts; invocation statistics
     const int B = (E + G - 1) / G;
     for (int i = tid; i <= M * B; i += nth) {
@@ -115,7 +156,8 @@ dispatch_count_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
                       int32_t* __restrict__ bin_off, int32_t* __restrict__ inv_perm,
                       int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
                       int32_t* __restrict__ group_off, int32_t* __restrict__ stats, int32_t* __restrict__ status,
-                      int32_t* __restrict__ done_counter, int do_plan, PlanArgs pa, int private_mode)
+                      int32_t* __restrict__ done_counter, int do_plan, PlanArgs pa, int private_mode,
+                      const int32_t* __restrict__ block_table, int table_blocks)
 {
     extern __shared__ int32_t s_tot[];       // [nbins] counts of this block; in the last block: totals, then offsets,
                                              // followed by the plan's scratch
@@ -178,7 +220,7 @@ dispatch_count_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
     }
     __syncthreads();
     scan_and_tables(s_tot, s_part, s_count, nbins, R, E, M, G, n_tenants, bm, bin_off, tenant_expert_count,
-                    expert_off, group_off, stats, private_mode);
+                    expert_off, group_off, stats, private_mode, block_table, table_blocks);
     if (do_plan) {
         __syncthreads();
         plan_body(expert_off, pa, s_tot + nbins, s_part);
@@ -225,7 +267,8 @@ dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
                       int32_t* __restrict__ inv_perm, int32_t* __restrict__ tenant_expert_count,
                       int32_t* __restrict__ expert_off, int32_t* __restrict__ group_off, int32_t* __restrict__ stats,
                       int32_t* __restrict__ status, const bf16* __restrict__ x, bf16* __restrict__ x_perm, int H,
-                      int do_plan, int plan_ints, PlanArgs pa, int32_t* __restrict__ bin_off, int private_mode)
+                      int do_plan, int plan_ints, PlanArgs pa, int32_t* __restrict__ bin_off, int private_mode,
+                      const int32_t* __restrict__ block_table, int table_blocks)
 {
     extern __shared__ int32_t s_tot[];       // [nbins], then the plan's scratch, then the bin of every row (u16)
     __shared__ int32_t s_part[33];
@@ -243,7 +286,7 @@ dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __res
     }
     __syncthreads();
     scan_and_tables(s_tot, s_part, s_count, nbins, R, E, M, G, n_tenants, bm, bin_off, tenant_expert_count,
-                    expert_off, group_off, stats, private_mode);
+                    expert_off, group_off, stats, private_mode, block_table, table_blocks);
     __syncthreads();
     if (tid < 32) {                           // s_tot now holds the next free position of every bin
         const int lane = tid;
@@ -403,7 +446,7 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
         launch_pdl(dispatch_small_kernel, dim3(1), dim3(threads), smem_small, st,
             topk_idx, tenant_id, R, k, bm, nbins, g.n_experts, g.n_models, G, g.n_tenants, perm, inv_perm,
             tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, x, gather_inside ? x_perm : nullptr,
-            g.hidden, do_plan ? 1 : 0, (int)plan_ints, pa, c->ws.bin_off, c->dispatch_private);
+            g.hidden, do_plan ? 1 : 0, (int)plan_ints, pa, c->ws.bin_off, c->dispatch_private, c->d_block_table, c->table_blocks);
         if (plan_done) *plan_done = do_plan;
         c->launches += 1;
         if (x_perm && !gather_inside) {
@@ -423,7 +466,7 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
     launch_pdl(dispatch_count_kernel, dim3(nblk), dim3(kCountThreads), smem_count, st,
         topk_idx, tenant_id, nblk, nbins, R, k, g.n_experts, g.n_models, G, g.n_tenants, bm, c->ws.block_cnt, c->ws.bin_off,
         inv_perm, tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, c->ws.dispatch_done,
-        do_plan ? 1 : 0, pa, c->dispatch_private);
+        do_plan ? 1 : 0, pa, c->dispatch_private, c->d_block_table, c->table_blocks);
     if (plan_done) *plan_done = do_plan;
     if (x_perm)
         launch_pdl(dispatch_place_kernel<true>, dim3((R * 32 + 255) / 256), dim3(256), 0, st, R, k, nbins, c->ws.block_cnt, c->ws.bin_off, perm,
@@ -570,7 +613,7 @@ extern "C" int moe_dispatch_noalloc(const int32_t* topk_idx, const int32_t* tena
     dispatch_count_kernel<<<nblk, kCountThreads, smem, st>>>(topk_idx, tenant_id, nblk, nbins, R, k, E, M, G, n_tenants, bm,
                                                              s + o_blk, s + o_binoff, inv_perm, tenant_expert_count,
                                                              expert_off, group_off, s + o_stats, status, s + o_stats + 2, 0,
-                                                             PlanArgs(), 0);
+                                                             PlanArgs(), 0, nullptr, 0);
     dispatch_place_kernel<false><<<(R + 255) / 256, 256, 0, st>>>(R, k, nbins, s + o_blk, s + o_binoff, perm, inv_perm,
                                                                   nullptr, nullptr, 0);
     return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;

@@ -128,6 +128,8 @@ struct moe_ctx {
     int32_t* d_slot;              // [M*E]
     int32_t* d_model_of_tenant;   // [Nt]
     int32_t* d_tenant_local;      // [Nt] index of the tenant among the tenants of its model
+    int32_t* d_block_table;       // [M*E] block of every expert (load-aware formation), null: blocks of G consecutive experts
+    int table_blocks;             // blocks per model of that table
     int32_t* d_bin_base;          // [M+1] first bin of each model (bins = (model, expert, tenant of model))
     int32_t* d_tenants_in_model;  // [M]
     faasmoe::Workspace ws;

@@ -95,7 +95,8 @@ PlanArgs make_plan_args(moe_ctx* c, int T, int G, bool with_shared)
                          (long long)a.shared_down_width * g.shared_inter == 256ll * g.inter) ? 1 : 0;
     // pair shape: tiles of at most kShortRows rows are kept apart for the background lanes of the grouped GEMM
     a.short_rows = (pair && tc_background_mode(c, T)) ? kShortRows : 0;
-    a.tile_cidx = a.short_rows ? c->ws.tile_cidx : nullptr;
+    a.tile_cidx = c->ws.tile_cidx;
+    a.block_table = c->d_block_table; a.table_blocks = c->table_blocks;
     a.private_mode = c->dispatch_private;
     a.bin_off = c->ws.bin_off; a.bin_base = c->d_bin_base; a.tenants_in_model = c->d_tenants_in_model;
     a.tiles = c->ws.tiles; a.stiles = c->ws.stiles;
@@ -107,7 +108,7 @@ PlanArgs make_plan_args(moe_ctx* c, int T, int G, bool with_shared)
 size_t plan_smem_ints(const moe_ctx* c, int G)
 {
     const moe_config& g = c->cfg;
-    const int B = (g.n_experts + G - 1) / G;
+    const int B = c->d_block_table ? c->table_blocks : (g.n_experts + G - 1) / G;
     return 2 * ((size_t)g.n_models * g.n_experts + (size_t)g.n_models * B + 1);
 }
 

@@ -20,8 +20,10 @@ struct PlanArgs {
     int split_ok[2];                  // token-major: K / 64 of the routed units is even (gate/up, down)
     int direct;                       // the routed gate/up units read all T tokens in place
     int interleave_down;              // the shared units of the down projection are as long as the routed ones
+    const int32_t* block_table;       // null: block of expert e = e / G; else [M*E] block ids in [0, table_blocks)
+    int table_blocks;
     int short_rows;                   // tiles of at most this many rows are "short" (0: none)
-    int32_t* tile_cidx;               // [tiles] index of a tile inside its class (long / short); null when short_rows == 0
+    int32_t* tile_cidx;               // [tiles] rank of a tile among the tiles of its block and class (long / short)
     int private_mode;                 // 1: tiles never span two tenants (private orchestrators batch per tenant)
     const int32_t* bin_off;           //    offsets of the (model, expert, tenant) bins, [nbins + 1]
     const int32_t* bin_base;          //    first bin of each model
@@ -38,8 +40,11 @@ struct PlanArgs {
 __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanArgs& a, int32_t* s_mem, int32_t* s_warp)
 {
     const int ME = a.M * a.E;
-    const int B = (a.E + a.G - 1) / a.G;
+    const int B = a.block_table ? a.table_blocks : (a.E + a.G - 1) / a.G;
     const int NG = a.M * B;
+    // block of expert i = (m, e): consecutive experts (Sec. 3: packaged by expert id) or, with a table, any set of
+    // experts of the model (load-aware formation, Sec. 5)
+    auto block_of = [&](int m, int e) { return m * B + (a.block_table ? a.block_table[m * a.E + e] : e / a.G); };
     int32_t* s_tile_base = s_mem;               // [ME]   tiles before expert i
     int32_t* s_short_base = s_mem + ME;         // [ME]   short tiles before expert i
     int32_t* s_group_long0 = s_mem + 2 * ME;    // [NG+1] long tiles before each expert block
@@ -69,12 +74,38 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
     const int n_tiles = block_scan_exclusive(s_tile_base, ME, s_warp);
     const int n_short_tiles = block_scan_exclusive(s_short_base, ME, s_warp);
     const int n_long_tiles = n_tiles - n_short_tiles;
+    // per block: its long and its short tiles, then the first tile of every block inside each class
+    for (int gidx = tid; gidx < NG; gidx += nth) {
+        const int m = gidx / B;
+        int nt = 0, ns = 0;
+        for (int e = 0; e < a.E; ++e) {
+            if (block_of(m, e) != gidx) continue;
+            const int i = m * a.E + e;
+            nt += (i + 1 < ME ? s_tile_base[i + 1] : n_tiles) - s_tile_base[i];
+            ns += (i + 1 < ME ? s_short_base[i + 1] : n_short_tiles) - s_short_base[i];
+        }
+        s_group_long0[gidx] = nt - ns;
+        s_group_short0[gidx] = ns;
+    }
+    if (tid == 0) { s_group_long0[NG] = 0; s_group_short0[NG] = 0; }
+    __syncthreads();
+    block_scan_exclusive(s_group_long0, NG + 1, s_warp);
+    block_scan_exclusive(s_group_short0, NG + 1, s_warp);
     for (int i = tid; i < ME; i += nth) {
         const int m = i / a.E, e = i - m * a.E;
         const int tim = a.private_mode ? a.tenants_in_model[m] : 1;
         const int b0 = a.private_mode ? a.bin_base[m] + e * tim : 0;
-        int tix = s_tile_base[i], six = s_short_base[i];
-        int lix = tix - six;
+        const int g = block_of(m, e);
+        // tiles of the same block and class that belong to earlier experts
+        int lix = 0, six = 0;
+        for (int e2 = 0; e2 < e; ++e2) {
+            if (block_of(m, e2) != g) continue;
+            const int j = m * a.E + e2;
+            const int nt = s_tile_base[j + 1] - s_tile_base[j], ns = s_short_base[j + 1] - s_short_base[j];
+            lix += nt - ns;
+            six += ns;
+        }
+        int tix = s_tile_base[i];
         for (int ul = 0; ul < tim; ++ul) {
             const int row_begin = a.private_mode ? a.bin_off[b0 + ul] : expert_off[i];
             const int row_end = a.private_mode ? a.bin_off[b0 + ul + 1] : expert_off[i + 1];
@@ -83,21 +114,11 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
                 t.row0 = r;
                 t.nrows = min(a.tile_rows, row_end - r);
                 t.slot = a.slot_table[i];
-                t.group = m * B + e / a.G;
+                t.group = g;
                 a.tiles[tix] = t;
-                if (a.tile_cidx) a.tile_cidx[tix] = (t.nrows <= a.short_rows) ? six++ : lix++;   // index inside its class
+                if (a.tile_cidx) a.tile_cidx[tix] = (t.nrows <= a.short_rows) ? six++ : lix++;   // rank inside (block, class)
             }
         }
-    }
-    for (int gidx = tid; gidx <= NG; gidx += nth) {
-        int vt = n_tiles, vs = n_short_tiles;
-        if (gidx < NG) {
-            const int m = gidx / B, b = gidx - m * B;
-            vt = s_tile_base[m * a.E + b * a.G];
-            vs = s_short_base[m * a.E + b * a.G];
-        }
-        s_group_long0[gidx] = vt - vs;
-        s_group_short0[gidx] = vs;
     }
     __syncthreads();
 
@@ -147,13 +168,13 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
             const int tile = i % n_tiles, cb = i / n_tiles;
             const Tile t = a.tiles[tile];
             const bool is_short = t.nrows <= a.short_rows;
-            const int ci = a.tile_cidx ? a.tile_cidx[tile] : tile;
+            const int ci = a.tile_cidx[tile];                           // rank of the tile inside (block, class)
             const int32_t* g0 = is_short ? s_group_short0 : s_group_long0;
-            const int c0 = g0[t.group], nc = g0[t.group + 1] - c0;      // first tile of the block in this class, tiles
+            const int c0 = g0[t.group], nc = g0[t.group + 1] - c0;      // tiles of earlier blocks in this class, tiles of this block
             const int base = is_short ? n_long_tiles : 0;
             Unit u; u.colblock = cb * (tm ? 4 : 1); u.tile = tile;
-            if (cb < a.nblk1) a.units1[su1 + (base + c0) * a.nblk1 + cb * nc + (ci - c0)] = u;
-            if (cb < a.nblk2) a.units2[su2 + (base + c0) * a.nblk2 + cb * nc + (ci - c0)] = u;
+            if (cb < a.nblk1) a.units1[su1 + (base + c0) * a.nblk1 + cb * nc + ci] = u;
+            if (cb < a.nblk2) a.units2[su2 + (base + c0) * a.nblk2 + cb * nc + ci] = u;
         }
         if (tid == 0) {
             a.plan_counts[2] = su1 + n_tiles * a.nblk1;

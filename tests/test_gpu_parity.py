@@ -566,6 +566,53 @@ def test_shared_and_private_orchestrator_modes(case):
         g.close()
 
 
+@pytest.mark.parametrize("case", ["small-pool", "decode", "prefill-6-tenants"])
+def test_load_aware_block_table(case):
+    # Blocks formed from the observed expert loads (greedy, heaviest expert first) instead of ranges of G consecutive
+    # experts: the library's host routine equals the oracle's bit for bit; with the table set, the permutation and
+    # every output bit are unchanged, the invocation counts and the rows per block follow the oracle's table
+    # accounting in both orchestrator modes, and the blocks are more even than the ranges.
+    wl, wts, seed = _modes_case(case)
+    x, tenant, mot = W.make_tokens(wl, seed=seed)
+    T, G, E, M = x.shape[0], max(wl.G, 4), wl.E, wl.M
+    Bn = -(-E // G)
+    g = GpuLayer(wl, [wts], T, model_of_tenant=mot)
+    try:
+        base = g.four_calls(x, tenant, G)
+        idx = base["topk_idx"].cpu().numpy()
+        cnt = base["tenant_expert_count"].cpu().numpy().astype(np.int64)           # [n_tenants, E]
+        load = np.zeros((M, E), np.int64)
+        for u in range(wl.n_tenants):
+            load[int(mot[u])] += cnt[u]
+        table = B.moe_form_blocks(torch.from_numpy(load), G)
+        ref_table = oracle.form_blocks(load, G=G)
+        assert np.array_equal(table.numpy(), ref_table)
+        B.moe_set_block_table(g.ctx, table, Bn)
+        for mode in (B.MOE_DISPATCH_SHARED, B.MOE_DISPATCH_PRIVATE):
+            B.moe_set_option(g.ctx, B.MOE_OPT_DISPATCH_MODE, mode)
+            o = g.four_calls(x, tenant, G)
+            f = g.forward(x, tenant, G)
+            assert o["status"] == 0 and torch.equal(f, base["out"])
+            for key in ("topk_idx", "perm", "inv_perm", "tenant_expert_count", "expert_off", "y_perm", "y_shared", "out"):
+                if base[key] is not None:
+                    assert torch.equal(o[key], base[key]), key
+            acc = oracle.invocations_table(idx, tenant.numpy(), mot.numpy(), ref_table, n_blocks=Bn, mode=mode)
+            assert o["n_invocations"] == acc.n_invocations
+            goff = o["group_off"].cpu().numpy()
+            assert np.array_equal(np.diff(goff), acc.block_rows.reshape(-1)) and goff[0] == 0 and goff[-1] == T * wl.k
+        rows_table = acc.block_rows.max(axis=1)
+        rows_ranges = np.stack([load[:, b * G:(b + 1) * G].sum(axis=1) for b in range(Bn)], axis=1).max(axis=1)
+        assert (rows_table <= rows_ranges).all()
+        # back to ranges
+        B.moe_set_block_table(g.ctx, None)
+        B.moe_set_option(g.ctx, B.MOE_OPT_DISPATCH_MODE, B.MOE_DISPATCH_SHARED)
+        again = g.four_calls(x, tenant, G)
+        assert torch.equal(again["group_off"], base["group_off"]) and again["n_invocations"] == base["n_invocations"]
+        assert torch.equal(again["out"], base["out"])
+    finally:
+        g.close()
+
+
 def test_host_entry_point_matches_device_entry_point():
     wl = W.WORKLOADS["tiny"]
     wts = W.make_weights(wl, seed=0)

@@ -510,3 +510,86 @@ def test_private_placement_with_one_tenant_equals_shared_placement():
     # G = 1: a token reaches k blocks
     c = oracle.invocations(idx, tenant, mot, n_models=2, E=E, G=1, mode=oracle.PRIVATE)
     assert (c.token_fanout == k).all()
+
+
+# ----------------------------------------------------------------------------- load-aware block formation (Sec. 5)
+
+def _best_makespan(load, G):
+    """Smallest possible largest block load over ALL assignments with at most G experts per block (tiny E only)."""
+    import itertools
+    E = len(load); B = -(-E // G)
+    best = None
+    for assign in itertools.product(range(B), repeat=E):
+        sizes = [assign.count(b) for b in range(B)]
+        if max(sizes) > G:
+            continue
+        ms = max(sum(load[e] for e in range(E) if assign[e] == b) for b in range(B))
+        best = ms if best is None or ms < best else best
+    return best
+
+
+def test_form_blocks_hand_worked_example_and_structure():
+    # loads 10 9 8 7 1 1, blocks of 2: 10 -> b0, 9 -> b1, 8 -> b2, 7 -> lightest with room = b2 (8), 1 -> b1 (9),
+    # 1 -> b0 (10): worked by hand from the rule
+    blk = oracle.form_blocks(np.array([[10, 9, 8, 7, 1, 1]]), G=2)
+    assert blk.tolist() == [[0, 1, 2, 2, 1, 0]]
+    # equal loads: ties go to the lower expert id and the lower block id, so the experts are dealt round robin
+    assert oracle.form_blocks(np.full((1, 6), 5), G=2).tolist() == [[0, 1, 2, 0, 1, 2]]
+    # G = 1: every expert its own block; G = E: one block
+    l = np.array([[3, 9, 1, 4]])
+    assert sorted(oracle.form_blocks(l, G=1)[0].tolist()) == [0, 1, 2, 3]
+    assert oracle.form_blocks(l, G=4).tolist() == [[0, 0, 0, 0]]
+    # models are independent
+    two = oracle.form_blocks(np.array([[10, 9, 8, 7, 1, 1], [1, 1, 7, 8, 9, 10]]), G=2)
+    # (second model: 10 -> b0, 9 -> b1, 8 -> b2, 7 -> b2, then expert 0 before expert 1: 1 -> b1 (9), 1 -> b0 (10))
+    assert two[0].tolist() == [0, 1, 2, 2, 1, 0] and two[1].tolist() == [1, 0, 2, 2, 1, 0]
+
+
+def test_form_blocks_is_a_partition_with_capacity_and_close_to_the_best_assignment():
+    rng = np.random.default_rng(50)
+    for trial in range(150):
+        E = int(rng.integers(2, 8)); G = int(rng.integers(1, E + 1)); B = -(-E // G)
+        load = rng.integers(0, 30, E)
+        if trial % 2:
+            load = (30 / np.arange(1, E + 1) ** 1.1).astype(np.int64)[rng.permutation(E)]      # Zipf-like skew
+        blk = oracle.form_blocks(load[None], G=G)[0]
+        assert blk.min() >= 0 and blk.max() < B
+        assert np.bincount(blk, minlength=B).max() <= G
+        ms = max(int(load[blk == b].sum()) for b in range(B))
+        best = _best_makespan(load.tolist(), G)
+        assert best <= ms <= best * 4 / 3 + 1e-9, (load, G, blk, ms, best)
+        # never worse than the blocks of G consecutive experts on their best day: the heaviest expert bounds both
+        assert ms >= load.max()
+    # on a Zipf-skewed load the greedy blocks are more even than blocks of consecutive experts
+    load = (4096 * 4 / np.arange(1, 61) ** 1.1)
+    load = (load / load.sum() * 16384).astype(np.int64)[np.random.default_rng(1).permutation(60)]
+    blk = oracle.form_blocks(load[None], G=4)[0]
+    greedy = max(int(load[blk == b].sum()) for b in range(15))
+    ranges = max(int(load[b * 4:(b + 1) * 4].sum()) for b in range(15))
+    assert greedy <= ranges and greedy == max(int(load.max()), greedy)
+
+
+def test_invocations_table_equals_range_accounting_for_range_tables_and_brute_force_otherwise():
+    rng = np.random.default_rng(51)
+    for trial in range(40):
+        E = int(rng.integers(2, 13)); k = int(rng.integers(1, min(E, 4) + 1)); M = int(rng.integers(1, 4))
+        nt = int(rng.integers(M, M + 4)); T = int(rng.integers(1, 40)); G = int(rng.integers(1, E + 1)); B = -(-E // G)
+        idx = np.stack([rng.permutation(E)[:k] for _ in range(T)]).astype(np.int32)
+        tenant = rng.integers(0, nt, T).astype(np.int32)
+        mot = (np.arange(nt) % M).astype(np.int32)
+        ranges = np.tile((np.arange(E) // G).astype(np.int32), (M, 1))
+        table = np.stack([rng.permutation(np.arange(E) % B) for _ in range(M)]).astype(np.int32)
+        for mode in (oracle.SHARED, oracle.PRIVATE):
+            a = oracle.invocations(idx, tenant, mot, n_models=M, E=E, G=G, mode=mode)
+            b = oracle.invocations_table(idx, tenant, mot, ranges, n_blocks=B, mode=mode)
+            assert a.n_invocations == b.n_invocations and np.array_equal(a.token_fanout, b.token_fanout)
+            assert np.array_equal(a.tenant_invocations, b.tenant_invocations)
+            c = oracle.invocations_table(idx, tenant, mot, table, n_blocks=B, mode=mode)
+            rows = [(int(tenant[t]), int(mot[tenant[t]]), int(table[mot[tenant[t]], e])) for t in range(T) for e in idx[t]]
+            want = len({(m, bb) for (_, m, bb) in rows}) if mode == oracle.SHARED else len({(u, bb) for (u, _, bb) in rows})
+            assert c.n_invocations == want
+            assert c.block_rows.sum() == T * k
+            for m in range(M):
+                for bb in range(B):
+                    assert c.block_rows[m, bb] == sum(1 for (_, m2, b2) in rows if m2 == m and b2 == bb)
+            assert c.token_fanout.tolist() == [len({int(table[mot[tenant[t]], e]) for e in idx[t]}) for t in range(T)]
