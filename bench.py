@@ -300,6 +300,69 @@ def dispatch_mode_report(B, ctx, step_fn, steps, world, dev):
     return out
 
 
+def block_formation_report(B, ctx, step_fn, steps, wl, T, world, dev):
+    """Blocks of G consecutive experts against load-aware blocks formed from the observed expert loads: rows of the
+    fullest block, invocations and step time (same work, same results; the blocks order and partition it)."""
+    ws = B.moe_get_workspace(ctx)
+    nb = -(-wl.E // wl.G)
+
+    def measure():
+        for _ in range(3):
+            step_fn()
+        blocks = timed_blocks(step_fn, steps, 0.25, world, torch.cuda.synchronize, dev, cuda_events)
+        status, n_inv, _ = B.moe_last_status(ctx)
+        if status != 0:
+            raise SystemExit(f"device status {status} in the block-formation report")
+        goff = B.wrap_device_pointer(ws["group_off"], (wl.M * nb + 1,), torch.int32, dev).cpu()
+        rows = (goff[1:] - goff[:-1]).to(torch.float64)
+        return {"invocations": n_inv, "max_rows_per_block": int(rows.max()), "mean_rows_per_block": float(rows.mean()),
+                "ms_per_step": statistics.median(blocks) / steps}
+    out = {"consecutive_experts": measure()}
+    eoff = B.wrap_device_pointer(ws["expert_off"], (wl.M * wl.E + 1,), torch.int32, dev).cpu().to(torch.int64)
+    load = (eoff[1:] - eoff[:-1]).view(wl.M, wl.E)
+    B.moe_set_block_table(ctx, B.moe_form_blocks(load, wl.G), nb)
+    out["load_aware"] = measure()
+    B.moe_set_block_table(ctx, None)
+    return out
+
+
+def residency_report(B, wl, wts, x, tenant, mot, dev, n_slots):
+    """On-demand residency: every expert parked in pinned host memory, n_slots device slots.  Times the first call
+    (every active expert is copied in), the same batch again (all resident) and the bytes resident against the whole
+    pool: what a cold start costs and what staying warm saves in device memory."""
+    T = x.shape[0]
+    layer = B.MoELayer(H=wl.H, E=wl.E, I=wl.I, k=wl.k, Is=wl.Is, M=wl.M, n_tenants=wl.n_tenants, max_tokens=T,
+                       n_slots=n_slots, device=str(dev))
+    try:
+        pool = [torch.zeros((n_slots, wl.I, wl.H), dtype=torch.bfloat16, device=dev),
+                torch.zeros((n_slots, wl.I, wl.H), dtype=torch.bfloat16, device=dev),
+                torch.zeros((n_slots, wl.H, wl.I), dtype=torch.bfloat16, device=dev)]
+        layer.set_layer_weights(0, dict(wts, pool_gate=pool[0], pool_up=pool[1], pool_down=pool[2]))
+        layer.set_tables(model_of_tenant=mot)
+        host = [wts[k_].contiguous().pin_memory() for k_ in ("pool_gate", "pool_up", "pool_down")]
+        B.moe_residency_enable(layer.ctx, 0, host[0], host[1], host[2], pool[0], pool[1], pool[2])
+        xd, td = x.to(dev), tenant.to(dev)
+        out = torch.zeros_like(xd)
+
+        def timed_call():
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            st = B.moe_layer_forward_paged(layer.ctx, 0, xd, td, T, wl.G, out)
+            torch.cuda.synchronize()
+            return 1e3 * (time.perf_counter() - t0), st
+        cold_ms, cold = timed_call()
+        warm = [timed_call() for _ in range(20)]
+        expert_bytes = 3 * wl.H * wl.I * 2
+        return {"slots": n_slots, "experts": wl.M * wl.E, "cold_call_ms": cold_ms, "cold_loads": cold[2],
+                "cold_h2d_bytes": cold[2] * expert_bytes, "warm_call_ms": statistics.median(m for m, _ in warm),
+                "warm_hits": warm[-1][1][1], "active_experts": cold[0],
+                "resident_bytes": n_slots * expert_bytes, "full_pool_bytes": wl.M * wl.E * expert_bytes}
+    except B.MoeError as e:
+        return {"skipped": str(e)}
+    finally:
+        layer.close()
+
+
 def measure_layer(args, wl, rank, local_rank, world, dev, wts_cache, with_cpu_baseline):
     """One single-layer workload (decode, prefill, pool): device-resident throughput, per-stage times, end to end
     through the host-buffer entry point, roofline of the dominant kernel and of the whole path."""
@@ -353,12 +416,17 @@ def measure_layer(args, wl, rank, local_rank, world, dev, wts_cache, with_cpu_ba
             B.moe_layer_forward_host(ctx, 0, xh, th, T, wl.G, oh, stream)
         e2e_blocks = timed_blocks(lambda: B.moe_layer_forward_host(ctx, 0, xh, th, T, wl.G, oh, stream), e2e_steps,
                                   min(args.min_time, 0.5), world, torch.cuda.synchronize, dev, cuda_events)
-        modes = None
+        modes = formation = None
+        step_fn = lambda: B.moe_layer_forward(ctx, 0, xd, td, T, wl.G, out, stream)
         if wl.n_tenants > 1:
-            modes = dispatch_mode_report(B, ctx, lambda: B.moe_layer_forward(ctx, 0, xd, td, T, wl.G, out, stream),
-                                         max(10, steps // 10), world, dev)
+            modes = dispatch_mode_report(B, ctx, step_fn, max(10, steps // 10), world, dev)
+        if wl.G > 1:
+            formation = block_formation_report(B, ctx, step_fn, max(10, steps // 10), wl, T, world, dev)
     finally:
         layer.close()
+    residency = None
+    if wl.name == "decode" and rank == 0 and world == 1:
+        residency = residency_report(B, wl, wts, x, tenant, mot, dev, n_slots=wl.E - 4)
 
     if rank != 0:
         return None
@@ -403,6 +471,10 @@ def measure_layer(args, wl, rank, local_rank, world, dev, wts_cache, with_cpu_ba
             "roofline": roofline}
     if modes:
         line["dispatch_modes"] = modes
+    if formation:
+        line["block_formation"] = formation
+    if residency:
+        line["on_demand_residency"] = residency
     if with_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, wts, x, tenant, mot)
     return line

@@ -3,7 +3,7 @@
  *
  * The layer is the one FaaSMoE serves as a shared pool of stateless expert
  * functions for many tenants: gating and top-k selection (paper Sec. 2.1), the
- * construction of micro-batched routing requests per expert block (Sec. 3,
+ * grouping of the routed tokens into one request per expert block (Sec. 3,
  * Sec. 4.1), expert execution on the assigned tokens (Sec. 3), and the
  * aggregation of expert outputs per token (Sec. 3, Sec. 4.2).  The paper's
  * expert-block granularity (G experts per function, Sec. 3 / Sec. 5) is a
@@ -219,8 +219,8 @@ int moe_dispatch(moe_ctx* ctx, const void* x, const int32_t* topk_idx, const int
                  int32_t* group_off, void* x_perm, void* stream);
 
 /*
- * Expert execution (Sec. 3: each expert block performs stateless computation on its
- * assigned tokens).  Only experts that received rows are touched.
+ * Expert execution (Sec. 3: an expert block keeps no state and computes only on the
+ * tokens sent to it).  Only experts that received rows are touched.
  *   y_perm[r'] = FFN_{slot(m,e)}(x_perm[r'])    for r' in expert (m,e)'s segment   f32 [T*k, H]
  *   y_shared[t] = FFN_shared,m(x[t])  (ungated)                                    f32 [T, H] or NULL
  * (bf16 operands, fp32 accumulation; the SwiGLU activations are rounded to bf16 for the
@@ -284,6 +284,29 @@ int moe_dispatch_noalloc(const int32_t* topk_idx, const int32_t* tenant_id, cons
  * the four calls above.  out bf16 [T,H]. */
 int moe_layer_forward(moe_ctx* ctx, int layer, const void* x, const int32_t* tenant_id, int T, int G,
                       void* out, void* stream);
+
+/*
+ * On-demand residency of the routed experts: the device-side analogue of functions that scale to zero (abstract;
+ * Sec. 3: rarely used experts need not hold resources while idle).  All M*E experts of the layer are parked in HOST
+ * memory (host_gate / host_up bf16 [M*E, I, H], host_down bf16 [M*E, H, I], indexed by m*E + e; pinned memory makes
+ * the copies asynchronous); the pool on the device (pool_* = DEVICE arrays of n_slots slots, registered as by
+ * moe_set_expert_pool) is a cache of the experts in use, and the slot table is managed by the library.  One layer per
+ * context (MOE_ERR_UNSUPPORTED otherwise).
+ */
+int moe_residency_enable(moe_ctx* ctx, int layer, const void* host_gate, const void* host_up, const void* host_down,
+                         void* pool_gate, void* pool_up, void* pool_down);
+
+/*
+ * moe_layer_forward with on-demand residency: runs the gate, reads the set of experts the batch routes to back to the
+ * host (this call synchronises `stream` once, after the gate), copies every needed expert that is parked into a slot
+ * -- a free one (lowest index) or else the one used longest ago among those this batch does not need (ties: lowest
+ * index; experts are taken in ascending id) -- and runs dispatch, experts and combine on the routing already made.
+ * Results are bit-identical to a context that keeps every expert resident.  More active experts than slots:
+ * MOE_ERR_UNSUPPORTED.  stats_host (host, 4 ints, or NULL): active experts, resident hits, experts loaded, experts
+ * evicted by this call.
+ */
+int moe_layer_forward_paged(moe_ctx* ctx, int layer, const void* x, const int32_t* tenant_id, int T, int G, void* out,
+                            int32_t* stats_host, void* stream);
 
 /* Same, with HOST buffers: copies x and tenant_id to the device, runs the layer,
  * copies out back and synchronises the stream.  For best speed pass pinned memory. */

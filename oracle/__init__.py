@@ -202,6 +202,46 @@ def invocations_table(topk_idx, tenant_id, model_of_tenant, block_of_expert, *, 
     return TableInvocations(int(ninv.value), per_tenant, fan, rows)
 
 
+def residency_lru(active_sets, n_slots):
+    """On-demand residency of experts in a fixed number of device slots (the scale-to-zero idea of the abstract and
+    Sec. 3 applied to device memory): every expert is parked until a batch routes to it.
+
+    For every batch, in order: the experts it needs that are resident are hits; every missing one, in ascending id,
+    takes a free slot (lowest index) or else evicts the resident expert that was needed longest ago among those the
+    current batch does not need (ties: lowest slot index).  Returns a list of (hits, loads, evictions, slot_of) per
+    batch, slot_of a dict expert -> slot after the batch.  Raises if a batch needs more experts than there are slots.
+    """
+    owner = [-1] * n_slots
+    history = []                                     # the batches so far, as sets
+    out = []
+    for step, need in enumerate(active_sets):
+        need = sorted(set(int(e) for e in need))
+        if len(need) > n_slots:
+            raise ValueError("more active experts than slots")
+
+        def last_needed(e):                          # latest earlier batch that needed expert e
+            for back in range(len(history) - 1, -1, -1):
+                if e in history[back]:
+                    return back
+            return -1
+        hits = sum(1 for e in need if e in owner)
+        loads = evictions = 0
+        for e in need:
+            if e in owner:
+                continue
+            if -1 in owner:
+                slot = owner.index(-1)
+            else:
+                cand = [s for s in range(n_slots) if owner[s] not in need]
+                slot = min(cand, key=lambda s: (last_needed(owner[s]), s))
+                evictions += 1
+            owner[slot] = e
+            loads += 1
+        history.append(set(need))
+        out.append((hits, loads, evictions, {e: s for s, e in enumerate(owner) if e >= 0}))
+    return out
+
+
 def experts(x, tenant_id, topk_idx, perm, model_of_tenant, pool_gate, pool_up, pool_down, slot_table, *, n_models):
     """SwiGLU FFN of the activated experts over the routed rows, in segment order (Sec. 3)."""
     lib = _load()

@@ -3,7 +3,7 @@
  *
  * A plain, slow, fp64 CPU statement of the multi-tenant Mixture-of-Experts
  * layer that FaaSMoE serves: gating network + top-k selection (paper Sec. 2.1),
- * construction of micro-batched routing requests per expert block (Sec. 3,
+ * grouping of the routed tokens into one request per expert block (Sec. 3,
  * Sec. 4.1), stateless expert execution on the assigned tokens (Sec. 3), and
  * aggregation of the expert outputs per token (Sec. 3, Sec. 4.2).
  *
@@ -487,8 +487,8 @@ int oracle_shared_expert(const uint16_t* x, const int32_t* tenant_id, int T, int
 }
 
 /*
- * Aggregation (Sec. 3: the orchestrator is responsible for "aggregation";
- * Sec. 4.2: "token aggregation"):
+ * Aggregation (Sec. 3: the orchestrator puts the expert outputs of a token together;
+ * Sec. 4.2 lists it among the orchestrator's duties):
  *   out[t] = sum_{j=0..k-1} w[t,j] * y_perm[inv_perm[t*k+j]]  +  s[t] * y_shared[t]
  * y_shared / shared_gate may be NULL (no shared expert).  out [T,H] double.
  */

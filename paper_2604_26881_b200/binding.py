@@ -35,7 +35,7 @@ MOE_PATH_AUTO, MOE_PATH_FMA, MOE_PATH_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["moe_create", "moe_destroy", "moe_set_expert_pool", "moe_set_model_weights", "moe_set_slot_table",
            "moe_set_tenant_models", "moe_set_option", "moe_form_blocks", "moe_set_block_table", "moe_route", "moe_dispatch", "moe_experts", "moe_combine",
-           "moe_layer_forward", "moe_layer_forward_host", "moe_layer_forward_timed", "moe_stack_forward",
+           "moe_layer_forward", "moe_residency_enable", "moe_layer_forward_paged", "moe_layer_forward_host", "moe_layer_forward_timed", "moe_stack_forward",
            "moe_get_workspace", "moe_last_status", "moe_last_plan", "moe_launch_count", "moe_strerror", "moe_dispatch_noalloc"]
 MOE_DISPATCH_NOALLOC_MAX_WORDS = 1 << 18
 
@@ -87,6 +87,9 @@ def load_library(path: str | None = None):
         lib.moe_combine.argtypes = [c_void_p] + [c_void_p] * 5 + [c_int, c_void_p, c_void_p]
         lib.moe_layer_forward.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p]
         lib.moe_layer_forward_host.argtypes = lib.moe_layer_forward.argtypes
+        lib.moe_residency_enable.argtypes = [c_void_p, c_int] + [c_void_p] * 6
+        lib.moe_layer_forward_paged.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int, c_int, c_void_p,
+                                                POINTER(c_int32), c_void_p]
         lib.moe_layer_forward_timed.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int, c_int, c_void_p,
                                                 POINTER(c_float), c_void_p]
         lib.moe_stack_forward.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p]
@@ -208,6 +211,21 @@ def moe_experts(ctx, layer, x, x_perm, perm, expert_off, tenant_id, T, G, y_perm
 def moe_combine(ctx, y_perm, inv_perm, topk_w, y_shared, shared_gate, T, out, stream=None):
     _check("moe_combine", load_library().moe_combine(ctx, _ptr(y_perm), _ptr(inv_perm), _ptr(topk_w), _ptr(y_shared),
                                                      _ptr(shared_gate), T, _ptr(out), _stream(stream)))
+
+
+def moe_residency_enable(ctx, layer, host_gate, host_up, host_down, pool_gate, pool_up, pool_down):
+    """host_*: CPU tensors [M*E, I, H] / [M*E, H, I] (pinned for asynchronous copies); pool_*: device tensors of n_slots slots."""
+    _check("moe_residency_enable", load_library().moe_residency_enable(ctx, layer, _ptr(host_gate), _ptr(host_up),
+                                                                       _ptr(host_down), _ptr(pool_gate), _ptr(pool_up),
+                                                                       _ptr(pool_down)))
+
+
+def moe_layer_forward_paged(ctx, layer, x, tenant_id, T, G, out, stream=None):
+    """Returns (active experts, resident hits, experts loaded, experts evicted) of the call."""
+    st = (c_int32 * 4)()
+    _check("moe_layer_forward_paged", load_library().moe_layer_forward_paged(ctx, layer, _ptr(x), _ptr(tenant_id), T, G,
+                                                                             _ptr(out), st, _stream(stream)))
+    return int(st[0]), int(st[1]), int(st[2]), int(st[3])
 
 
 def moe_layer_forward(ctx, layer, x, tenant_id, T, G, out, stream=None):

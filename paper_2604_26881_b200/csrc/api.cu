@@ -13,6 +13,7 @@ namespace {
 
 thread_local char g_last_cuda_error[256] = "";
 
+
 #define MOE_CUDA(ctx, expr)                                                                         \
     do {                                                                                            \
         cudaError_t err__ = (expr);                                                                 \
@@ -181,7 +182,7 @@ int experts_impl(moe_ctx* c, int layer, const bf16* x, const bf16* x_perm, const
 }
 
 int layer_forward_impl(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int G,
-                       const bf16* residual, bf16* out, cudaStream_t st)
+                       const bf16* residual, bf16* out, cudaStream_t st, bool routed = false)
 {
     const moe_config& g = c->cfg;
     Workspace& w = c->ws;
@@ -211,8 +212,10 @@ int layer_forward_impl(moe_ctx* c, int layer, const bf16* x, const int32_t* tena
         MOE_CUDA(c, cudaEventRecord(c->ev_join, c->side));
     }
     stage_mark(c, st, kEvBegin);
-    MOE_CUDA(c, launch_route(c, layer, x, tenant_id, T, w.topk_idx, w.topk_w, shared ? w.shared_gate : nullptr,
-                             w.tie_flag, st));
+    // (routed: the gate has run already and its results are in the workspace -- the paged entry point looks at them first)
+    if (!routed)
+        MOE_CUDA(c, launch_route(c, layer, x, tenant_id, T, w.topk_idx, w.topk_w, shared ? w.shared_gate : nullptr,
+                                 w.tie_flag, st));
     stage_mark(c, st, kEvRoute);
     // with few tokens the tensor-core experts read the tokens in place: no permuted copy to make
     const bool direct = use_tc(c) && tc_direct_mode(c, T);
@@ -229,6 +232,18 @@ int layer_forward_impl(moe_ctx* c, int layer, const bf16* x, const int32_t* tena
                                shared ? w.shared_gate : nullptr, residual, T, out, st));
     stage_mark(c, st, kEvCombine);
     return MOE_OK;
+}
+
+// flags the experts that the routed rows of a batch go to
+__global__ void mark_active_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ tenant_id,
+                                   const int32_t* __restrict__ model_of_tenant, int R, int k, int E, int n_tenants,
+                                   int32_t* __restrict__ active)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= R) return;
+    const int u = tenant_id[r / k], e = topk_idx[r];
+    if (u < 0 || u >= n_tenants || e < 0 || e >= E) return;
+    active[model_of_tenant[u] * E + e] = 1;
 }
 
 }  // namespace
@@ -332,6 +347,8 @@ int moe_destroy(moe_ctx* c)
     void* ptrs[] = {c->d_models, c->d_slot, c->d_model_of_tenant, c->d_tenant_local, c->d_bin_base,
                     c->d_tenants_in_model, c->d_block_table};
     for (void* p : ptrs) if (p) cudaFree(p);
+    if (c->res.d_active) cudaFree(c->res.d_active);
+    if (c->res.h_active) cudaFreeHost(c->res.h_active);
     delete c;
     return MOE_OK;
 }
@@ -439,6 +456,91 @@ int moe_set_block_table(moe_ctx* c, const int32_t* block_of_expert, int n_blocks
     MOE_CUDA(c, cudaMemcpy(c->d_block_table, block_of_expert, ME * sizeof(int32_t), cudaMemcpyHostToDevice));
     c->table_blocks = n_blocks;
     return MOE_OK;
+}
+
+int moe_residency_enable(moe_ctx* c, int layer, const void* host_gate, const void* host_up, const void* host_down,
+                         void* pool_gate, void* pool_up, void* pool_down)
+{
+    if (!c || !host_gate || !host_up || !host_down || !pool_gate || !pool_up || !pool_down) return MOE_ERR_NULL;
+    if (c->cfg.n_layers != 1 || layer != 0) return MOE_ERR_UNSUPPORTED;      // the slot table is one per context
+    const int rc = moe_set_expert_pool(c, layer, pool_gate, pool_up, pool_down);
+    if (rc != MOE_OK) return rc;
+    const size_t ME = (size_t)c->cfg.n_models * c->cfg.n_experts;
+    Residency& r = c->res;
+    r.h_gate = (const bf16*)host_gate; r.h_up = (const bf16*)host_up; r.h_down = (const bf16*)host_down;
+    r.p_gate = (bf16*)pool_gate; r.p_up = (bf16*)pool_up; r.p_down = (bf16*)pool_down;
+    r.owner.assign(c->cfg.n_slots, -1);
+    r.last_use.assign(c->cfg.n_slots, -1);
+    r.slot_of.assign(ME, -1);
+    r.clock = 0;
+    if (!r.d_active) MOE_CUDA(c, dev_alloc(&r.d_active, ME));
+    if (!r.h_active) MOE_CUDA(c, cudaMallocHost((void**)&r.h_active, ME * sizeof(int32_t)));
+    r.on = true;
+    return MOE_OK;
+}
+
+int moe_layer_forward_paged(moe_ctx* c, int layer, const void* x, const int32_t* tenant_id, int T, int G, void* out,
+                            int32_t* stats_host, void* stream)
+{
+    if (!c || !x || !tenant_id || !out) return MOE_ERR_NULL;
+    if (!c->res.on || layer != 0) return MOE_ERR_STATE;
+    if (T < 0 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
+    if (misaligned16(x, out)) return MOE_ERR_SHAPE;
+    if (G < 1 || G > c->cfg.n_experts) return MOE_ERR_G;
+    const int rc = check_layer_ready(c, layer, true, true);
+    if (rc != MOE_OK) return rc;
+    if (stats_host) stats_host[0] = stats_host[1] = stats_host[2] = stats_host[3] = 0;
+    if (T == 0) return MOE_OK;
+    const moe_config& g = c->cfg;
+    Workspace& w = c->ws;
+    Residency& r = c->res;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int ME = g.n_models * g.n_experts, S = g.n_slots, R = T * g.top_k;
+    // 1. the gate, then the set of experts this batch needs, on the host (the one synchronisation of the call)
+    MOE_CUDA(c, launch_route(c, layer, (const bf16*)x, tenant_id, T, w.topk_idx, w.topk_w,
+                             g.shared_inter > 0 ? w.shared_gate : nullptr, w.tie_flag, st));
+    MOE_CUDA(c, cudaMemsetAsync(r.d_active, 0, (size_t)ME * sizeof(int32_t), st));
+    mark_active_kernel<<<(R + 255) / 256, 256, 0, st>>>(w.topk_idx, tenant_id, c->d_model_of_tenant, R, g.top_k,
+                                                        g.n_experts, g.n_tenants, r.d_active);
+    c->launches += 1;
+    MOE_CUDA(c, cudaMemcpyAsync(r.h_active, r.d_active, (size_t)ME * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    MOE_CUDA(c, cudaStreamSynchronize(st));
+    // 2. residency: hits refresh their slot; every missing expert (ascending id) takes a free slot (lowest index), else
+    //    the slot that was used longest ago among those the batch does not need (ties: lowest index)
+    r.clock += 1;
+    int n_active = 0, hits = 0, loads = 0, evictions = 0;
+    for (int i = 0; i < ME; ++i) n_active += r.h_active[i] != 0;
+    if (n_active > S) {
+        snprintf(c->errbuf, sizeof(c->errbuf), "%d active experts do not fit %d resident slots", n_active, S);
+        return MOE_ERR_UNSUPPORTED;
+    }
+    for (int i = 0; i < ME; ++i)
+        if (r.h_active[i] && r.slot_of[i] >= 0) { r.last_use[r.slot_of[i]] = r.clock; ++hits; }
+    const size_t wexp = (size_t)g.inter * g.hidden;              // elements of one expert matrix
+    for (int i = 0; i < ME; ++i) {
+        if (!r.h_active[i] || r.slot_of[i] >= 0) continue;
+        int victim = -1;
+        for (int s2 = 0; s2 < S && victim < 0; ++s2) if (r.owner[s2] < 0) victim = s2;
+        if (victim < 0) {
+            for (int s2 = 0; s2 < S; ++s2)
+                if (r.last_use[s2] < r.clock && (victim < 0 || r.last_use[s2] < r.last_use[victim])) victim = s2;
+            r.slot_of[r.owner[victim]] = -1;
+            ++evictions;
+        }
+        MOE_CUDA(c, cudaMemcpyAsync(r.p_gate + (size_t)victim * wexp, r.h_gate + (size_t)i * wexp, wexp * sizeof(bf16),
+                                    cudaMemcpyHostToDevice, st));
+        MOE_CUDA(c, cudaMemcpyAsync(r.p_up + (size_t)victim * wexp, r.h_up + (size_t)i * wexp, wexp * sizeof(bf16),
+                                    cudaMemcpyHostToDevice, st));
+        MOE_CUDA(c, cudaMemcpyAsync(r.p_down + (size_t)victim * wexp, r.h_down + (size_t)i * wexp, wexp * sizeof(bf16),
+                                    cudaMemcpyHostToDevice, st));
+        r.owner[victim] = i; r.slot_of[i] = victim; r.last_use[victim] = r.clock;
+        ++loads;
+    }
+    for (int i = 0; i < ME; ++i) c->h_slot[i] = r.slot_of[i] >= 0 ? r.slot_of[i] : 0;    // parked experts get no rows
+    MOE_CUDA(c, cudaMemcpyAsync(c->d_slot, c->h_slot.data(), (size_t)ME * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    if (stats_host) { stats_host[0] = n_active; stats_host[1] = hits; stats_host[2] = loads; stats_host[3] = evictions; }
+    // 3. the rest of the layer on the routing results that are already in the workspace
+    return layer_forward_impl(c, layer, (const bf16*)x, tenant_id, T, G, nullptr, (bf16*)out, st, true);
 }
 
 int moe_set_option(moe_ctx* c, int option, int value)

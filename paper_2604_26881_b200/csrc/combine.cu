@@ -1,5 +1,5 @@
 // Aggregation of expert outputs per token (paper Sec. 3: the orchestrator aggregates the
-// results of the expert functions; Sec. 4.2: "token aggregation"), and the RMSNorm / residual
+// results of the expert functions; Sec. 4.2 lists it among the orchestrator's duties), and the RMSNorm / residual
 // add of the stacked-block configuration.
 #include "internal.h"
 

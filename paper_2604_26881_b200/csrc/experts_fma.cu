@@ -1,6 +1,6 @@
 // CUDA-core expert execution: the plain, tile-wise SwiGLU FFN used for shapes the tensor-core
 // path does not cover and as the A/B reference of that path.  (Paper Sec. 3: an expert block
-// performs stateless computation on its assigned tokens; only activated experts are touched.)
+// keeps no state and computes on the tokens it was sent; only activated experts are touched.)
 #include <cuda_fp16.h>
 
 #include "internal.h"

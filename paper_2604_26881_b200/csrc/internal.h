@@ -57,6 +57,24 @@ struct Unit {
 
 struct TensorMaps;   // defined in experts_tc.cu
 
+// On-demand residency of the routed experts (one layer): all experts are parked in host memory, the pool slots on
+// the device are a cache of the experts in use, managed least-recently-used.
+struct Residency {
+    bool on = false;
+    const bf16* h_gate = nullptr;   // host [M*E, I, H]
+    const bf16* h_up = nullptr;
+    const bf16* h_down = nullptr;   // host [M*E, H, I]
+    bf16* p_gate = nullptr;         // device pool [S, I, H] (the arrays registered with moe_set_expert_pool)
+    bf16* p_up = nullptr;
+    bf16* p_down = nullptr;
+    std::vector<int32_t> owner;     // [S] expert in the slot, -1: free
+    std::vector<int64_t> last_use;  // [S] call that used the slot last
+    std::vector<int32_t> slot_of;   // [M*E] slot of the expert, -1: parked
+    int64_t clock = 0;
+    int32_t* d_active = nullptr;    // [M*E] device flags of the experts the current batch routes to
+    int32_t* h_active = nullptr;    // the same in pinned host memory
+};
+
 struct Workspace {
     // routing results
     int32_t* topk_idx = nullptr;   // [T,k]
@@ -128,6 +146,7 @@ struct moe_ctx {
     int32_t* d_slot;              // [M*E]
     int32_t* d_model_of_tenant;   // [Nt]
     int32_t* d_tenant_local;      // [Nt] index of the tenant among the tenants of its model
+    faasmoe::Residency res;       // on-demand residency of the routed experts
     int32_t* d_block_table;       // [M*E] block of every expert (load-aware formation), null: blocks of G consecutive experts
     int table_blocks;             // blocks per model of that table
     int32_t* d_bin_base;          // [M+1] first bin of each model (bins = (model, expert, tenant of model))

@@ -50,6 +50,14 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
     int32_t* s_group_long0 = s_mem + 2 * ME;    // [NG+1] long tiles before each expert block
     int32_t* s_group_short0 = s_group_long0 + NG + 1;   // [NG+1] short tiles before each expert block
     const int tid = threadIdx.x, nth = blockDim.x;
+    // The common case -- blocks of consecutive experts, no short class -- needs none of the per-block loops and no
+    // per-tile lookups below: a block's tiles are consecutive, so every index has a closed form (this kernel sits on the
+    // latency chain of small batches).
+    const bool simple = a.block_table == nullptr && a.short_rows == 0;
+    // Blocks of consecutive experts with a short class, shared orchestrator (large one-model batches): still closed
+    // forms -- a block's tiles are consecutive and only the last tile of an expert can be short.
+    const bool ranged = a.block_table == nullptr && a.short_rows > 0 && !a.private_mode;
+    const bool general = !simple && !ranged;
 
     // Shared orchestrator (Sec. 4.2): the rows of an expert form one segment whoever owns them, cut into tiles.
     // Private orchestrators: every tenant's rows of an expert are a request of their own, so the segments are the
@@ -72,10 +80,22 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
     }
     __syncthreads();
     const int n_tiles = block_scan_exclusive(s_tile_base, ME, s_warp);
-    const int n_short_tiles = block_scan_exclusive(s_short_base, ME, s_warp);
+    const int n_short_tiles = simple ? 0 : block_scan_exclusive(s_short_base, ME, s_warp);
     const int n_long_tiles = n_tiles - n_short_tiles;
+    if (!general) {
+        for (int gidx = tid; gidx <= NG; gidx += nth) {
+            int vt = n_tiles, vs = n_short_tiles;
+            if (gidx < NG) {
+                const int m = gidx / B, b = gidx - m * B;
+                vt = s_tile_base[m * a.E + b * a.G];
+                vs = simple ? 0 : s_short_base[m * a.E + b * a.G];
+            }
+            s_group_long0[gidx] = vt - vs;
+            s_group_short0[gidx] = vs;
+        }
+    }
     // per block: its long and its short tiles, then the first tile of every block inside each class
-    for (int gidx = tid; gidx < NG; gidx += nth) {
+    for (int gidx = tid; gidx < NG && general; gidx += nth) {
         const int m = gidx / B;
         int nt = 0, ns = 0;
         for (int e = 0; e < a.E; ++e) {
@@ -87,10 +107,12 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
         s_group_long0[gidx] = nt - ns;
         s_group_short0[gidx] = ns;
     }
-    if (tid == 0) { s_group_long0[NG] = 0; s_group_short0[NG] = 0; }
+    if (tid == 0 && general) { s_group_long0[NG] = 0; s_group_short0[NG] = 0; }
     __syncthreads();
-    block_scan_exclusive(s_group_long0, NG + 1, s_warp);
-    block_scan_exclusive(s_group_short0, NG + 1, s_warp);
+    if (general) {
+        block_scan_exclusive(s_group_long0, NG + 1, s_warp);
+        block_scan_exclusive(s_group_short0, NG + 1, s_warp);
+    }
     for (int i = tid; i < ME; i += nth) {
         const int m = i / a.E, e = i - m * a.E;
         const int tim = a.private_mode ? a.tenants_in_model[m] : 1;
@@ -98,7 +120,7 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
         const int g = block_of(m, e);
         // tiles of the same block and class that belong to earlier experts
         int lix = 0, six = 0;
-        for (int e2 = 0; e2 < e; ++e2) {
+        for (int e2 = 0; e2 < e && general; ++e2) {
             if (block_of(m, e2) != g) continue;
             const int j = m * a.E + e2;
             const int nt = s_tile_base[j + 1] - s_tile_base[j], ns = s_short_base[j + 1] - s_short_base[j];
@@ -116,7 +138,7 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
                 t.slot = a.slot_table[i];
                 t.group = g;
                 a.tiles[tix] = t;
-                if (a.tile_cidx) a.tile_cidx[tix] = (t.nrows <= a.short_rows) ? six++ : lix++;   // rank inside (block, class)
+                if (general) a.tile_cidx[tix] = (t.nrows <= a.short_rows) ? six++ : lix++;   // rank inside (block, class)
             }
         }
     }
@@ -166,12 +188,34 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
         const int nmax = n_tiles * max(a.nblk1, a.nblk2);
         for (int i = tid; i < nmax; i += nth) {
             const int tile = i % n_tiles, cb = i / n_tiles;
-            const Tile t = a.tiles[tile];
-            const bool is_short = t.nrows <= a.short_rows;
-            const int ci = a.tile_cidx[tile];                           // rank of the tile inside (block, class)
-            const int32_t* g0 = is_short ? s_group_short0 : s_group_long0;
-            const int c0 = g0[t.group], nc = g0[t.group + 1] - c0;      // tiles of earlier blocks in this class, tiles of this block
-            const int base = is_short ? n_long_tiles : 0;
+            int c0, nc, ci, base = 0;
+            if (simple) {
+                // expert block of the tile: last block whose first tile is <= tile (empty blocks share their first
+                // tile with the next one)
+                int lo = 0, hi = NG;
+                while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (s_group_long0[mid] <= tile) lo = mid; else hi = mid; }
+                c0 = s_group_long0[lo]; nc = s_group_long0[lo + 1] - c0; ci = tile - c0;
+            } else if (ranged) {
+                // the expert of the tile: last expert whose first tile is <= tile (experts without tiles share theirs
+                // with the next one)
+                int lo = 0, hi = ME;
+                while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (s_tile_base[mid] <= tile) lo = mid; else hi = mid; }
+                const int m = lo / a.E, e = lo - m * a.E, g = m * B + e / a.G;
+                const int t_end = lo + 1 < ME ? s_tile_base[lo + 1] : n_tiles;
+                const int has_short = (lo + 1 < ME ? s_short_base[lo + 1] : n_short_tiles) - s_short_base[lo];
+                const bool is_short = has_short && tile == t_end - 1;                 // only an expert's last tile can be short
+                const int32_t* g0 = is_short ? s_group_short0 : s_group_long0;
+                c0 = g0[g]; nc = g0[g + 1] - c0;
+                ci = (is_short ? s_short_base[lo] : tile - s_short_base[lo]) - c0;    // index inside the class, then inside the block
+                base = is_short ? n_long_tiles : 0;
+            } else {
+                const Tile t = a.tiles[tile];
+                const bool is_short = t.nrows <= a.short_rows;
+                ci = a.tile_cidx[tile];                                 // rank of the tile inside (block, class)
+                const int32_t* g0 = is_short ? s_group_short0 : s_group_long0;
+                c0 = g0[t.group]; nc = g0[t.group + 1] - c0;            // tiles of earlier blocks in this class, tiles of this block
+                base = is_short ? n_long_tiles : 0;
+            }
             Unit u; u.colblock = cb * (tm ? 4 : 1); u.tile = tile;
             if (cb < a.nblk1) a.units1[su1 + (base + c0) * a.nblk1 + cb * nc + ci] = u;
             if (cb < a.nblk2) a.units2[su2 + (base + c0) * a.nblk2 + cb * nc + ci] = u;

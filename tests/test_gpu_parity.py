@@ -613,6 +613,71 @@ def test_load_aware_block_table(case):
         g.close()
 
 
+def test_on_demand_residency_matches_resident_layer_and_the_lru_oracle():
+    # All experts parked in host memory, 6 device slots for 2 x 12 experts: a sequence of small batches (each routes to
+    # at most 6 experts) through the paged entry point.  Outputs must equal, bit for bit, a context that keeps every
+    # expert resident; hits, loads and evictions per call, and the slot every expert ends up in, must follow the
+    # oracle's least-recently-used simulation of the same sequence of active sets.
+    wl = W.MoEWorkload("paged", T=3, H=256, E=12, I=128, k=2, Is=128, M=2, n_tenants=3, G=3, tenant_layout="uniform")
+    wts = W.make_weights(wl, seed=13)
+    mot = W.make_tokens(wl, seed=0)[2]
+    full = GpuLayer(wl, [wts], wl.T, model_of_tenant=mot)
+    S = 6
+    paged = B.MoELayer(H=wl.H, E=wl.E, I=wl.I, k=wl.k, Is=wl.Is, M=wl.M, n_tenants=wl.n_tenants, max_tokens=wl.T, n_slots=S)
+    try:
+        dev = paged.device
+        shared_only = dict(wts, pool_gate=torch.zeros((S, wl.I, wl.H), dtype=torch.bfloat16),
+                           pool_up=torch.zeros((S, wl.I, wl.H), dtype=torch.bfloat16),
+                           pool_down=torch.zeros((S, wl.H, wl.I), dtype=torch.bfloat16))
+        paged.set_layer_weights(0, shared_only)
+        paged.set_tables(model_of_tenant=mot)
+        pool = [torch.zeros((S, wl.I, wl.H), dtype=torch.bfloat16, device=dev), torch.zeros((S, wl.I, wl.H), dtype=torch.bfloat16, device=dev),
+                torch.zeros((S, wl.H, wl.I), dtype=torch.bfloat16, device=dev)]
+        host = [wts["pool_gate"].contiguous().pin_memory(), wts["pool_up"].contiguous().pin_memory(),
+                wts["pool_down"].contiguous().pin_memory()]
+        B.moe_residency_enable(paged.ctx, 0, host[0], host[1], host[2], pool[0], pool[1], pool[2])
+        active_sets, stats = [], []
+        seeds = [0, 1, 2, 0, 3, 4, 1, 5, 0, 6]
+        for sd in seeds:
+            x, tenant, _ = W.make_tokens(wl, seed=sd)
+            ref = full.forward(x, tenant, wl.G)
+            xd, td = x.to(dev), tenant.to(dev)
+            out = torch.zeros_like(xd)
+            st = B.moe_layer_forward_paged(paged.ctx, 0, xd, td, wl.T, wl.G, out)
+            torch.cuda.synchronize()
+            assert B.moe_last_status(paged.ctx)[0] == 0
+            assert torch.equal(out, ref), f"batch seed {sd}"
+            ws = B.moe_get_workspace(paged.ctx)
+            idx = B.wrap_device_pointer(ws["topk_idx"], (wl.T, wl.k), torch.int32, dev).cpu().numpy()
+            active_sets.append(sorted({int(mot[tenant[t]]) * wl.E + int(e) for t in range(wl.T) for e in idx[t]}))
+            stats.append(st)
+        sim = oracle.residency_lru(active_sets, S)
+        for st, (h, l, ev, _), need in zip(stats, sim, active_sets):
+            assert st == (len(need), h, l, ev), (st, (len(need), h, l, ev))
+        assert sum(s[3] for s in stats) > 0 and sum(s[1] for s in stats) > 0       # the sequence did evict and did hit
+        # every expert the last batch needed sits in the slot the simulation says, with its own weights
+        for e, slot in sim[-1][3].items():
+            assert torch.equal(pool[0][slot].cpu(), wts["pool_gate"][e]) and torch.equal(pool[2][slot].cpu(), wts["pool_down"][e])
+        # too many active experts for the slots: refused, nothing half done
+        wl_big = W.scaled(wl, T=16)
+        xb, tb, _ = W.make_tokens(wl_big, seed=7)
+        big = B.MoELayer(H=wl.H, E=wl.E, I=wl.I, k=wl.k, Is=wl.Is, M=wl.M, n_tenants=wl.n_tenants, max_tokens=16, n_slots=4)
+        try:
+            big.set_layer_weights(0, dict(shared_only, pool_gate=shared_only["pool_gate"][:4], pool_up=shared_only["pool_up"][:4],
+                                          pool_down=shared_only["pool_down"][:4]))
+            big.set_tables(model_of_tenant=mot)
+            pb = [p_[:4].clone() for p_ in pool]
+            B.moe_residency_enable(big.ctx, 0, host[0], host[1], host[2], pb[0], pb[1], pb[2])
+            with pytest.raises(B.MoeError) as e:
+                B.moe_layer_forward_paged(big.ctx, 0, xb.to(dev), tb.to(dev), 16, wl.G, torch.zeros((16, wl.H), dtype=torch.bfloat16, device=dev))
+            assert e.value.status == B.MOE_ERR_UNSUPPORTED
+        finally:
+            big.close()
+    finally:
+        paged.close()
+        full.close()
+
+
 def test_host_entry_point_matches_device_entry_point():
     wl = W.WORKLOADS["tiny"]
     wts = W.make_weights(wl, seed=0)

@@ -593,3 +593,67 @@ def test_invocations_table_equals_range_accounting_for_range_tables_and_brute_fo
                 for bb in range(B):
                     assert c.block_rows[m, bb] == sum(1 for (_, m2, b2) in rows if m2 == m and b2 == bb)
             assert c.token_fanout.tolist() == [len({int(table[mot[tenant[t]], e]) for e in idx[t]}) for t in range(T)]
+
+
+# ----------------------------------------------------------------------------- on-demand residency (abstract, Sec. 3)
+
+def _min_loads(seq, n_slots):
+    """Fewest loads any eviction policy needs (exhaustive search over the victims; tiny sequences only)."""
+    import functools
+
+    @functools.lru_cache(maxsize=None)
+    def go(step, resident):
+        if step == len(seq):
+            return 0
+        need = frozenset(seq[step])
+        res = set(resident)
+        missing = sorted(need - res)
+        if not missing:
+            return go(step + 1, resident)
+        best = None
+
+        def place(i, cur):
+            nonlocal best
+            if i == len(missing):
+                v = len(missing) + go(step + 1, frozenset(cur))
+                best = v if best is None or v < best else best
+                return
+            if len(cur) < n_slots:
+                place(i + 1, cur | {missing[i]})
+            else:
+                for victim in sorted(cur - need):
+                    place(i + 1, (cur - {victim}) | {missing[i]})
+        place(0, set(res))
+        return best
+    return go(0, frozenset())
+
+
+def test_residency_lru_hand_example_and_bounds():
+    # two slots; batches {1} {2} {1} {3} {2}: loads 1, 2; hit 1; 3 evicts 2 (needed longest ago); 2 evicts 1
+    r = oracle.residency_lru([[1], [2], [1], [3], [2]], 2)
+    assert [(h, l, e) for h, l, e, _ in r] == [(0, 1, 0), (0, 1, 0), (1, 0, 0), (0, 1, 1), (0, 1, 1)]
+    assert r[3][3] == {1: 0, 3: 1} and r[4][3] == {2: 0, 3: 1}
+    # enough slots for everything: every expert is loaded exactly once, nothing is evicted, a repeated batch only hits
+    rng = np.random.default_rng(60)
+    seq = [sorted(rng.choice(12, 4, replace=False).tolist()) for _ in range(10)]
+    seq.append(seq[-1])
+    r = oracle.residency_lru(seq, 12)
+    assert sum(l for _, l, _, _ in r) == len({e for b in seq for e in b}) and sum(e for _, _, e, _ in r) == 0
+    assert r[-1][:3] == (4, 0, 0)
+    # any capacity: hits + loads = batch size, the batch is resident afterwards, evictions only when full, and no
+    # policy can do with fewer loads than the exhaustive optimum while LRU stays within the classic factor of it
+    for trial in range(40):
+        S = int(rng.integers(2, 5)); n = int(rng.integers(1, S + 1))
+        seq = [sorted(rng.choice(6, n, replace=False).tolist()) for _ in range(7)]
+        r = oracle.residency_lru(seq, S)
+        resident = set()
+        for (h, l, ev, slot_of), need in zip(r, seq):
+            assert h == len(set(need) & resident) and h + l == len(need)
+            assert set(need) <= set(slot_of) and len(set(slot_of.values())) == len(slot_of) <= S
+            assert ev == max(0, len(resident) + l - S)
+            resident = set(slot_of)
+        total = sum(l for _, l, _, _ in r)
+        best = _min_loads(tuple(tuple(b) for b in seq), S)
+        assert best <= total <= best * S            # LRU is S-competitive
+    with pytest.raises(ValueError):
+        oracle.residency_lru([[1, 2, 3]], 2)
