@@ -313,6 +313,20 @@ int moe_layer_forward_paged(moe_ctx* ctx, int layer, const void* x, const int32_
 int moe_layer_forward_host(moe_ctx* ctx, int layer, const void* x_host, const int32_t* tenant_id_host, int T, int G,
                            void* out_host, void* stream);
 
+/*
+ * The host-buffer call as a pipeline: submit enqueues the copy of x_host / tenant_id_host to the device (on a copy
+ * stream of the context), the layer (on `stream`, after the copy) and the copy of the result to out_host (on a second
+ * copy stream, after the layer), and returns a ticket without waiting; wait blocks until out_host of that ticket is
+ * complete.  Two submissions may be in flight: the third submit first waits for the first one's outputs (its staging
+ * buffers are reused).  The inputs of one call then travel while the previous call computes and the call before that
+ * returns its outputs, so a stream of calls runs at the slowest of the three instead of their sum.  x_host,
+ * tenant_id_host and out_host must be pinned and stay valid until the ticket has been waited for.  Results are those of
+ * moe_layer_forward_host.
+ */
+int moe_layer_forward_host_submit(moe_ctx* ctx, int layer, const void* x_host, const int32_t* tenant_id_host, int T, int G,
+                                  void* out_host, void* stream, int64_t* ticket);
+int moe_layer_forward_host_wait(moe_ctx* ctx, int64_t ticket);
+
 /* moe_layer_forward with a CUDA event recorded on `stream` after every stage; synchronises the
  * stream and writes the stage durations in milliseconds to stage_ms_host (host, 6 floats):
  * route, dispatch, plan, experts gate/up, experts down, combine. */

@@ -35,7 +35,7 @@ MOE_PATH_AUTO, MOE_PATH_FMA, MOE_PATH_TCGEN05 = 0, 1, 2
 
 EXPORTS = ["moe_create", "moe_destroy", "moe_set_expert_pool", "moe_set_model_weights", "moe_set_slot_table",
            "moe_set_tenant_models", "moe_set_option", "moe_form_blocks", "moe_set_block_table", "moe_route", "moe_dispatch", "moe_experts", "moe_combine",
-           "moe_layer_forward", "moe_residency_enable", "moe_layer_forward_paged", "moe_layer_forward_host", "moe_layer_forward_timed", "moe_stack_forward",
+           "moe_layer_forward", "moe_residency_enable", "moe_layer_forward_paged", "moe_layer_forward_host", "moe_layer_forward_host_submit", "moe_layer_forward_host_wait", "moe_layer_forward_timed", "moe_stack_forward",
            "moe_get_workspace", "moe_last_status", "moe_last_plan", "moe_launch_count", "moe_strerror", "moe_dispatch_noalloc"]
 MOE_DISPATCH_NOALLOC_MAX_WORDS = 1 << 18
 
@@ -87,6 +87,8 @@ def load_library(path: str | None = None):
         lib.moe_combine.argtypes = [c_void_p] + [c_void_p] * 5 + [c_int, c_void_p, c_void_p]
         lib.moe_layer_forward.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p]
         lib.moe_layer_forward_host.argtypes = lib.moe_layer_forward.argtypes
+        lib.moe_layer_forward_host_submit.argtypes = lib.moe_layer_forward.argtypes + [POINTER(c_int64)]
+        lib.moe_layer_forward_host_wait.argtypes = [c_void_p, c_int64]
         lib.moe_residency_enable.argtypes = [c_void_p, c_int] + [c_void_p] * 6
         lib.moe_layer_forward_paged.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_int, c_int, c_void_p,
                                                 POINTER(c_int32), c_void_p]
@@ -211,6 +213,19 @@ def moe_experts(ctx, layer, x, x_perm, perm, expert_off, tenant_id, T, G, y_perm
 def moe_combine(ctx, y_perm, inv_perm, topk_w, y_shared, shared_gate, T, out, stream=None):
     _check("moe_combine", load_library().moe_combine(ctx, _ptr(y_perm), _ptr(inv_perm), _ptr(topk_w), _ptr(y_shared),
                                                      _ptr(shared_gate), T, _ptr(out), _stream(stream)))
+
+
+def moe_layer_forward_host_submit(ctx, layer, x_host, tenant_id_host, T, G, out_host, stream=None) -> int:
+    """Enqueues H2D, the layer and D2H without waiting; returns the ticket to wait for (pinned host tensors)."""
+    ticket = c_int64(-1)
+    _check("moe_layer_forward_host_submit",
+           load_library().moe_layer_forward_host_submit(ctx, layer, _ptr(x_host), _ptr(tenant_id_host), T, G, _ptr(out_host),
+                                                        _stream(stream), byref(ticket)))
+    return int(ticket.value)
+
+
+def moe_layer_forward_host_wait(ctx, ticket: int):
+    _check("moe_layer_forward_host_wait", load_library().moe_layer_forward_host_wait(ctx, ticket))
 
 
 def moe_residency_enable(ctx, layer, host_gate, host_up, host_down, pool_gate, pool_up, pool_down):

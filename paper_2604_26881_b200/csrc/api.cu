@@ -86,6 +86,7 @@ int alloc_workspace(moe_ctx* c)
     }
     A(&w.xn, (T + kTileRows) * H);
     A(&w.x_stage, (T + kTileRows) * H); A(&w.tenant_stage, T); A(&w.out_stage, T * H);
+    A(&w.x_stage2, (T + kTileRows) * H); A(&w.tenant_stage2, T); A(&w.out_stage2, T * H);
     A(&w.status, 1); A(&w.stats, 4); A(&w.dispatch_done, 1);
     if (e != cudaSuccess) {
         snprintf(c->errbuf, sizeof(c->errbuf), "workspace allocation: %s", cudaGetErrorString(e));
@@ -106,7 +107,8 @@ void free_workspace(moe_ctx* c)
                     w.expert_off, w.group_off, w.block_cnt, w.bin_off, w.tok_block_cnt, w.model_tok_off, w.tok_perm,
                     w.tok_inv, w.tiles, w.tile_cidx, w.stiles, w.plan_counts, w.units1, w.units2, w.stiles_sh, w.plan_counts_sh, w.units1_sh,
                     w.units2_sh, w.x_perm, w.xs_perm, w.h, w.hs,
-                    w.y_perm, w.y_shared, w.xn, w.x_stage, w.tenant_stage, w.out_stage, w.status, w.stats, w.dispatch_done};
+                    w.y_perm, w.y_shared, w.xn, w.x_stage, w.tenant_stage, w.out_stage, w.x_stage2, w.tenant_stage2, w.out_stage2,
+                    w.status, w.stats, w.dispatch_done};
     for (void* p : ptrs) if (p) cudaFree(p);
     w = Workspace();
 }
@@ -284,6 +286,8 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->early_shared_enabled = 1;
     c->early_shared_sms = 1 << 20;      // no limit
     c->side = nullptr; c->ev_fork = nullptr; c->ev_join = nullptr;
+    c->copy_in = nullptr; c->copy_out = nullptr; c->submitted = 0; c->waited[0] = c->waited[1] = -1;
+    for (int i = 0; i < 2; ++i) { c->ev_in[i] = nullptr; c->ev_done[i] = nullptr; c->ev_out[i] = nullptr; }
     for (auto& e : c->ev) e = nullptr;
     c->errbuf[0] = 0;
     c->d_models = nullptr; c->d_slot = nullptr; c->d_model_of_tenant = nullptr; c->d_tenant_local = nullptr;
@@ -324,6 +328,19 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
             rc = MOE_ERR_CUDA;
         }
     }
+    if (rc == MOE_OK) {
+        e = cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking);
+        for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+            e = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_done[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_out[i], cudaEventDisableTiming);
+        }
+        if (e != cudaSuccess) {
+            snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "moe_create: %s", cudaGetErrorString(e));
+            rc = MOE_ERR_CUDA;
+        }
+    }
     if (rc != MOE_OK) {
         if (c->errbuf[0]) snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "%s", c->errbuf);
         moe_destroy(c);
@@ -344,6 +361,13 @@ int moe_destroy(moe_ctx* c)
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     if (c->side) cudaStreamDestroy(c->side);
+    for (int i = 0; i < 2; ++i) {
+        if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
+        if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
+        if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
+    }
+    if (c->copy_in) cudaStreamDestroy(c->copy_in);
+    if (c->copy_out) cudaStreamDestroy(c->copy_out);
     void* ptrs[] = {c->d_models, c->d_slot, c->d_model_of_tenant, c->d_tenant_local, c->d_bin_base,
                     c->d_tenants_in_model, c->d_block_table};
     for (void* p : ptrs) if (p) cudaFree(p);
@@ -689,6 +713,57 @@ int moe_layer_forward_host(moe_ctx* c, int layer, const void* x_host, const int3
     if (rc2 != MOE_OK) return rc2;
     MOE_CUDA(c, cudaMemcpyAsync(out_host, c->ws.out_stage, xbytes, cudaMemcpyDeviceToHost, st));
     MOE_CUDA(c, cudaStreamSynchronize(st));
+    return MOE_OK;
+}
+
+int moe_layer_forward_host_submit(moe_ctx* c, int layer, const void* x_host, const int32_t* tenant_id_host, int T, int G,
+                                  void* out_host, void* stream, int64_t* ticket)
+{
+    if (!c || !x_host || !tenant_id_host || !out_host || !ticket) return MOE_ERR_NULL;
+    if (T < 0 || T > c->cfg.max_tokens) return MOE_ERR_SHAPE;
+    if (G < 1 || G > c->cfg.n_experts) return MOE_ERR_G;
+    const int rc = check_layer_ready(c, layer, true, true);
+    if (rc != MOE_OK) return rc;
+    const int64_t n = c->submitted;
+    const int slot = (int)(n & 1);
+    // the slot's previous user (two submissions ago) must have delivered its outputs before its buffers are reused
+    if (n >= 2 && c->waited[slot] < n - 2) {
+        MOE_CUDA(c, cudaEventSynchronize(c->ev_out[slot]));
+        c->waited[slot] = n - 2;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    bf16* xs = slot ? c->ws.x_stage2 : c->ws.x_stage;
+    int32_t* ts = slot ? c->ws.tenant_stage2 : c->ws.tenant_stage;
+    bf16* os = slot ? c->ws.out_stage2 : c->ws.out_stage;
+    const size_t xbytes = (size_t)T * c->cfg.hidden * sizeof(bf16);
+    if (T > 0) {
+        // inputs on the copy-in stream (beside the layer pass of the submission before), the layer on the caller's
+        // stream, outputs on the copy-out stream (beside the next layer pass)
+        MOE_CUDA(c, cudaMemcpyAsync(xs, x_host, xbytes, cudaMemcpyHostToDevice, c->copy_in));
+        MOE_CUDA(c, cudaMemcpyAsync(ts, tenant_id_host, (size_t)T * sizeof(int32_t), cudaMemcpyHostToDevice, c->copy_in));
+        MOE_CUDA(c, cudaEventRecord(c->ev_in[slot], c->copy_in));
+        MOE_CUDA(c, cudaStreamWaitEvent(st, c->ev_in[slot], 0));
+        const int rc2 = layer_forward_impl(c, layer, xs, ts, T, G, nullptr, os, st);
+        if (rc2 != MOE_OK) return rc2;
+        MOE_CUDA(c, cudaEventRecord(c->ev_done[slot], st));
+        MOE_CUDA(c, cudaStreamWaitEvent(c->copy_out, c->ev_done[slot], 0));
+        MOE_CUDA(c, cudaMemcpyAsync(out_host, os, xbytes, cudaMemcpyDeviceToHost, c->copy_out));
+    }
+    MOE_CUDA(c, cudaEventRecord(c->ev_out[slot], c->copy_out));
+    *ticket = n;
+    c->submitted = n + 1;
+    return MOE_OK;
+}
+
+int moe_layer_forward_host_wait(moe_ctx* c, int64_t ticket)
+{
+    if (!c) return MOE_ERR_NULL;
+    if (ticket < 0 || ticket >= c->submitted) return MOE_ERR_SHAPE;
+    const int slot = (int)(ticket & 1);
+    if (c->waited[slot] >= ticket) return MOE_OK;                   // already known to be complete
+    if (ticket + 2 < c->submitted) return MOE_OK;                   // its slot has been reused: that submit waited for it
+    MOE_CUDA(c, cudaEventSynchronize(c->ev_out[slot]));
+    c->waited[slot] = ticket;
     return MOE_OK;
 }
 

@@ -122,6 +122,10 @@ struct Workspace {
     bf16* x_stage = nullptr;       // [T,H]
     int32_t* tenant_stage = nullptr;  // [T]
     bf16* out_stage = nullptr;     // [T,H]
+    // second set of staging buffers: the pipelined host entry point keeps two submissions in flight
+    bf16* x_stage2 = nullptr;
+    int32_t* tenant_stage2 = nullptr;
+    bf16* out_stage2 = nullptr;
     // status
     int32_t* status = nullptr;     // [1] sticky status bits
     int32_t* stats = nullptr;      // [4]
@@ -165,6 +169,10 @@ struct moe_ctx {
     int early_shared_enabled;     // one model: run the shared expert on a second stream beside router and dispatch
                                   // (1: batches of the 2-CTA shape, 2: every batch)
     int early_shared_sms;         // SMs the shared expert's CTA pairs may take while they run beside other kernels
+    cudaStream_t copy_in, copy_out;   // streams of the pipelined host entry point (H2D of the next call, D2H of the last)
+    cudaEvent_t ev_in[2], ev_done[2], ev_out[2];   // per staging slot: inputs landed, layer done, outputs landed
+    int64_t submitted;            // submissions so far (ticket of the next one)
+    int64_t waited[2];            // last ticket of each slot whose outputs are known to have landed
     cudaStream_t side;            // second stream of the layer pass
     cudaEvent_t ev_fork, ev_join; // order between the caller's stream and the second one
     bool timing;                  // record an event after every stage (moe_layer_forward_timed)

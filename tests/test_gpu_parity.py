@@ -689,6 +689,34 @@ def test_host_entry_point_matches_device_entry_point():
         g.close()
 
 
+def test_pipelined_host_calls_match_single_calls():
+    # submit / wait with two calls in flight: inputs of a call travel while the previous one computes; every ticket's
+    # output must be what the one-call-at-a-time entry point gives for the same batch, whatever the waiting order
+    wl = W.MoEWorkload("pipe", T=300, H=256, E=12, I=128, k=3, Is=256, M=2, n_tenants=3, G=4, zipf_bias=True,
+                       tenant_layout="uniform")
+    wts = W.make_weights(wl, seed=17)
+    mot = W.make_tokens(wl, seed=0)[2]
+    g = GpuLayer(wl, [wts], wl.T, model_of_tenant=mot)
+    try:
+        batches = [W.make_tokens(wl, seed=s_)[:2] for s_ in range(7)]
+        want = [g.forward_host(x, t, wl.G) for x, t in batches]
+        xs = [x.contiguous().pin_memory() for x, _ in batches]
+        ts = [t.contiguous().pin_memory() for _, t in batches]
+        outs = [torch.zeros_like(x).pin_memory() for x in xs]
+        tickets = [B.moe_layer_forward_host_submit(g.ctx, 0, xs[i], ts[i], wl.T, wl.G, outs[i]) for i in range(7)]
+        assert tickets == list(range(tickets[0], tickets[0] + 7))
+        for i in (6, 0, 3, 5, 1, 2, 4):                  # any order; earlier tickets are complete once a later one is
+            B.moe_layer_forward_host_wait(g.ctx, tickets[i])
+            assert torch.equal(outs[i], want[i]), i
+        assert B.moe_last_status(g.ctx)[0] == 0
+        # and the single-call entry point still works afterwards
+        assert torch.equal(g.forward_host(*batches[2], wl.G), want[2])
+        with pytest.raises(B.MoeError):
+            B.moe_layer_forward_host_wait(g.ctx, tickets[-1] + 1)
+    finally:
+        g.close()
+
+
 def test_edge_cases_and_errors():
     wl = W.MoEWorkload("edge", T=5, H=256, E=8, I=128, k=2, Is=128, M=1, n_tenants=3)
     wts = W.make_weights(wl, seed=9)
