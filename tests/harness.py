@@ -57,21 +57,33 @@ class GpuLayer:
         R = T * k
         Bn = -(-E // G)
         xd, td = x.to(dev), tenant.to(dev)
+        # every caller-owned output sits in front of a guard zone of a known pattern: a kernel that writes past the
+        # end of a buffer it was given is caught after the calls (a checked build by other means)
+        guards = []
+
+        def buf(shape, dtype, fill):
+            n = int(np.prod(shape))
+            pad = 64
+            flat = torch.full((n + pad,), fill, dtype=dtype, device=dev)
+            pattern = torch.arange(pad, device=dev).to(dtype) if dtype != torch.bfloat16 else torch.full((pad,), 1.5, dtype=dtype, device=dev)
+            flat[n:] = pattern
+            guards.append((flat, n, pattern.clone()))
+            return flat[:n].view(*shape)
         o = {
-            "topk_idx": torch.full((T, k), -7, dtype=torch.int32, device=dev),
-            "topk_w": torch.zeros((T, k), dtype=torch.float32, device=dev),
-            "shared_gate": torch.zeros((T,), dtype=torch.float32, device=dev),
-            "tie_flag": torch.zeros((T,), dtype=torch.uint8, device=dev),
-            "perm": torch.full((R,), -7, dtype=torch.int32, device=dev),
-            "inv_perm": torch.full((R,), -7, dtype=torch.int32, device=dev),
-            "tenant_expert_count": torch.full((wl.n_tenants, E), -7, dtype=torch.int32, device=dev),
-            "expert_off": torch.full((M * E + 1,), -7, dtype=torch.int32, device=dev),
-            "group_off": torch.full((M * Bn + 1,), -7, dtype=torch.int32, device=dev),
+            "topk_idx": buf((T, k), torch.int32, -7),
+            "topk_w": buf((T, k), torch.float32, 0),
+            "shared_gate": buf((T,), torch.float32, 0),
+            "tie_flag": buf((T,), torch.uint8, 0),
+            "perm": buf((R,), torch.int32, -7),
+            "inv_perm": buf((R,), torch.int32, -7),
+            "tenant_expert_count": buf((wl.n_tenants, E), torch.int32, -7),
+            "expert_off": buf((M * E + 1,), torch.int32, -7),
+            "group_off": buf((M * Bn + 1,), torch.int32, -7),
             # one spare tile of rows: the tensor-core path reads whole row tiles
             "x_perm": torch.zeros((R + 128, H), dtype=torch.bfloat16, device=dev),
-            "y_perm": torch.zeros((R, H), dtype=torch.float32, device=dev),
-            "y_shared": torch.zeros((T, H), dtype=torch.float32, device=dev) if wl.Is else None,
-            "out": torch.zeros((T, H), dtype=torch.bfloat16, device=dev),
+            "y_perm": buf((R, H), torch.float32, 0),
+            "y_shared": buf((T, H), torch.float32, 0) if wl.Is else None,
+            "out": buf((T, H), torch.bfloat16, 0),
         }
         B.moe_route(self.ctx, layer, xd, td, T, o["topk_idx"], o["topk_w"], o["shared_gate"] if wl.Is else None,
                     o["tie_flag"])
@@ -82,6 +94,9 @@ class GpuLayer:
                       o["shared_gate"] if wl.Is else None, T, o["out"])
         torch.cuda.synchronize()
         o["status"], o["n_invocations"], o["active_experts"] = B.moe_last_status(self.ctx)
+        for flat, n, pattern in guards:
+            assert torch.equal(flat[n:], pattern), "a kernel wrote past the end of a caller-owned buffer"
+        assert torch.count_nonzero(o["x_perm"][R:]) == 0, "rows were written past the end of x_perm"
         o["x_perm"] = o["x_perm"][:R]
         return o
 
