@@ -95,7 +95,8 @@ enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2,
                                      (rows are ordered (model, expert, tenant, token) either way); what changes is the
                                      invocation count reported by moe_last_status and the cost of moe_experts.
                                      In private mode moe_experts takes the (expert, tenant) boundaries from the last
-                                     moe_dispatch on the same context. */
+                                     moe_dispatch that the same context ran in private mode: set the mode before the
+                                     dispatch, not between dispatch and experts. */
        MOE_OPT_BACKGROUND_LANES = 10, /* 2-CTA shape: expert tiles of at most 64 rows are run by a second, small pipeline
                                          of every CTA pair (its own stage ring, TMA lane, MMA lane and accumulator)
                                          beside the pair's long tiles, so that the short tiles' weights stream in behind

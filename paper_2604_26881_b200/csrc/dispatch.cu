@@ -261,7 +261,7 @@ dispatch_place_kernel(int R, int k, int nbins, const int32_t* __restrict__ block
 // walks the rows in order), and the gather of the rows.  Same results as the multi-block kernels.
 constexpr int kSmallRows = 2048;   // above this the serial ranking pass of one warp costs more than the extra launches
 
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(1024, 1)
 dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ tenant_id, int R, int k,
                       BinMap bm, int nbins, int E, int M, int G, int n_tenants, int32_t* __restrict__ perm,
                       int32_t* __restrict__ inv_perm, int32_t* __restrict__ tenant_expert_count,
@@ -446,7 +446,8 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
         launch_pdl(dispatch_small_kernel, dim3(1), dim3(threads), smem_small, st,
             topk_idx, tenant_id, R, k, bm, nbins, g.n_experts, g.n_models, G, g.n_tenants, perm, inv_perm,
             tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, x, gather_inside ? x_perm : nullptr,
-            g.hidden, do_plan ? 1 : 0, (int)plan_ints, pa, c->ws.bin_off, c->dispatch_private, c->d_block_table, c->table_blocks);
+            g.hidden, do_plan ? 1 : 0, (int)plan_ints, pa, c->dispatch_private ? c->ws.bin_off : nullptr, c->dispatch_private,
+            c->d_block_table, c->table_blocks);
         if (plan_done) *plan_done = do_plan;
         c->launches += 1;
         if (x_perm && !gather_inside) {

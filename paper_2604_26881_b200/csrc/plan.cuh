@@ -108,8 +108,8 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
         s_group_short0[gidx] = ns;
     }
     if (tid == 0 && general) { s_group_long0[NG] = 0; s_group_short0[NG] = 0; }
-    __syncthreads();
     if (general) {
+        __syncthreads();
         block_scan_exclusive(s_group_long0, NG + 1, s_warp);
         block_scan_exclusive(s_group_short0, NG + 1, s_warp);
     }
