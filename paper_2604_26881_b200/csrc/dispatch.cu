@@ -234,10 +234,18 @@ template <bool GATHER>
 __global__ void __launch_bounds__(256)
 dispatch_place_kernel(int R, int k, int nbins, const int32_t* __restrict__ block_cnt, const int32_t* __restrict__ bin_off,
                       int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, const bf16* __restrict__ x,
-                      bf16* __restrict__ x_perm, int H)
+                      bf16* __restrict__ x_perm, int H, const int32_t* __restrict__ expert_off, int do_plan, PlanArgs pa)
 {
     pdl_wait();
     pdl_launch_dependents();
+    if (do_plan && blockIdx.x == gridDim.x - 1) {
+        // one extra block builds the expert work plan (it needs the offset tables of the counting kernel only) while
+        // the other blocks place and copy the rows: the plan is off the tail of the counting kernel's last block
+        extern __shared__ int32_t s_plan[];
+        __shared__ int32_t s_part[33];
+        plan_body(expert_off, pa, s_plan, s_part);
+        return;
+    }
     const int gtid = blockIdx.x * blockDim.x + threadIdx.x;
     const int r = GATHER ? gtid >> 5 : gtid;
     if (r >= R) return;
@@ -461,20 +469,25 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
     memset(&pa, 0, sizeof(pa));
     size_t plan_ints = 0;
     if (do_plan) { pa = make_plan_args(c, T, G, plan_shared); plan_ints = plan_smem_ints(c, G); }
-    const size_t smem_count = smem + plan_ints * sizeof(int32_t);
+    // the plan rides in an extra block of the placing kernel when its scratch fits the default shared memory
+    const bool plan_in_place = do_plan && plan_ints * sizeof(int32_t) <= 40 * 1024;
+    const bool plan_in_count = do_plan && !plan_in_place;
+    const size_t smem_count = smem + (plan_in_count ? plan_ints : 0) * sizeof(int32_t);
     if (smem_count > 48 * 1024)
         cudaFuncSetAttribute(dispatch_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_count);
+    const size_t smem_place = plan_in_place ? plan_ints * sizeof(int32_t) : 0;
     launch_pdl(dispatch_count_kernel, dim3(nblk), dim3(kCountThreads), smem_count, st,
         topk_idx, tenant_id, nblk, nbins, R, k, g.n_experts, g.n_models, G, g.n_tenants, bm, c->ws.block_cnt, c->ws.bin_off,
         inv_perm, tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, c->ws.dispatch_done,
-        do_plan ? 1 : 0, pa, c->dispatch_private, c->d_block_table, c->table_blocks);
+        plan_in_count ? 1 : 0, pa, c->dispatch_private, c->d_block_table, c->table_blocks);
     if (plan_done) *plan_done = do_plan;
+    const unsigned extra = plan_in_place ? 1u : 0u;
     if (x_perm)
-        launch_pdl(dispatch_place_kernel<true>, dim3((R * 32 + 255) / 256), dim3(256), 0, st, R, k, nbins, c->ws.block_cnt, c->ws.bin_off, perm,
-                                                                          inv_perm, x, x_perm, g.hidden);
+        launch_pdl(dispatch_place_kernel<true>, dim3((R * 32 + 255) / 256 + extra), dim3(256), smem_place, st, R, k, nbins,
+                   c->ws.block_cnt, c->ws.bin_off, perm, inv_perm, x, x_perm, g.hidden, expert_off, plan_in_place ? 1 : 0, pa);
     else
-        launch_pdl(dispatch_place_kernel<false>, dim3((R + 255) / 256), dim3(256), 0, st, R, k, nbins, c->ws.block_cnt, c->ws.bin_off, perm,
-                                                                      inv_perm, nullptr, nullptr, g.hidden);
+        launch_pdl(dispatch_place_kernel<false>, dim3((R + 255) / 256 + extra), dim3(256), smem_place, st, R, k, nbins,
+                   c->ws.block_cnt, c->ws.bin_off, perm, inv_perm, nullptr, nullptr, g.hidden, expert_off, plan_in_place ? 1 : 0, pa);
     c->launches += 2;
     return cudaGetLastError();
 }
@@ -616,6 +629,6 @@ extern "C" int moe_dispatch_noalloc(const int32_t* topk_idx, const int32_t* tena
                                                              expert_off, group_off, s + o_stats, status, s + o_stats + 2, 0,
                                                              PlanArgs(), 0, nullptr, 0);
     dispatch_place_kernel<false><<<(R + 255) / 256, 256, 0, st>>>(R, k, nbins, s + o_blk, s + o_binoff, perm, inv_perm,
-                                                                  nullptr, nullptr, 0);
+                                                                  nullptr, nullptr, 0, nullptr, 0, PlanArgs());
     return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
