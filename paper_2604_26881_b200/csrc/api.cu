@@ -57,9 +57,10 @@ int alloc_workspace(moe_ctx* c)
     c->max_tiles = div_up((int)R, kTileRows) + std::max((int)ME, c->nbins);
     c->max_stiles = div_up((int)T, kTileRows) + g.n_models;
     const int nblk1 = g.inter / 64, nblk2 = div_up(g.hidden, 128), snblk1 = g.shared_inter / 64;
-    // (+256: the token-major plan splits up to half a round of units in two; its shared units are up to 4x narrower)
-    c->max_units1 = c->max_tiles * nblk1 + c->max_stiles * snblk1 + 256;
-    c->max_units2 = (c->max_tiles + 4 * c->max_stiles) * nblk2 + 256;
+    // (+512: the token-major plan splits up to 128 units of the last round in two or four; its shared units are up to
+    // 4x narrower)
+    c->max_units1 = c->max_tiles * nblk1 + c->max_stiles * snblk1 + 512;
+    c->max_units2 = (c->max_tiles + 4 * c->max_stiles) * nblk2 + 512;
 
     cudaError_t e = cudaSuccess;
     auto A = [&](auto** p, size_t n) { if (e == cudaSuccess) e = dev_alloc(p, n); };

@@ -90,6 +90,7 @@ PlanArgs make_plan_args(moe_ctx* c, int T, int G, bool with_shared)
         a.snblk2 = g.hidden / a.shared_down_width;
     }
     a.split_ok[0] = (g.hidden / 64) % 2 == 0; a.split_ok[1] = (g.inter / 64) % 2 == 0;
+    a.split4_ok[0] = (g.hidden / 64) % 4 == 0; a.split4_ok[1] = (g.inter / 64) % 4 == 0;
     a.direct = tc_direct_mode(c, T) ? 1 : 0;
     a.interleave_down = (a.token_major && g.shared_inter > 0 &&
                          (long long)a.shared_down_width * g.shared_inter == 256ll * g.inter) ? 1 : 0;

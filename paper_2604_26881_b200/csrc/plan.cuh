@@ -18,6 +18,7 @@ struct PlanArgs {
     int n_ctas;                       // CTAs of the grouped GEMM launches
     int shared_down_width;            // token-major: weight rows of a shared-expert unit of the down projection
     int split_ok[2];                  // token-major: K / 64 of the routed units is even (gate/up, down)
+    int split4_ok[2];                 //              ... is divisible by 4
     int direct;                       // the routed gate/up units read all T tokens in place
     int interleave_down;              // the shared units of the down projection are as long as the routed ones
     const int32_t* block_table;       // null: block of expert e = e / G; else [M*E] block ids in [0, table_blocks)
@@ -233,17 +234,25 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
             a.plan_counts[9] = n_short_tiles * a.nblk2;
         }
         if (a.token_major) {
-            // U equally long units on S CTAs take ceil(U / S) rounds; when the last round is less than half full, its
-            // units (the tail of the list: routed ones) are split into two units of half the weight rows each, where
-            // the tile has at most 64 rows, so that round costs half.
-            __shared__ int s_split[128];
-            int r2[2];
+            // U equally long units on S CTAs take ceil(U / S) rounds.  The units of the last, partly filled round (the
+            // tail of the list: routed ones) are split into units of half the weight rows each (tiles of at most 64
+            // rows; narrower units pack more K slices into a stage and stream as fast per byte) whenever the pieces
+            // fill fewer (shorter) rounds than the round they replace: 627 units on 148 CTAs = 4 full rounds + 35
+            // units; as 70 halves these cost half a round.
+            __shared__ int s_split[4];
+            int r2[2], f2[2];
             for (int l = 0; l < 2; ++l) {
                 const int routed = n_tiles * (l ? a.nblk2 : a.nblk1);
                 const int total = (l ? su2 : su1) + routed;
                 int r = total % a.n_ctas;
-                if (2 * r > a.n_ctas || r > routed || r > 128 || !a.split_ok[l]) r = 0;
-                r2[l] = r;
+                // pieces per unit when every tile is as small as the batch (direct mode); otherwise halves at most
+                // (quarters -- possible where every tile has at most 32 rows and K / 64 is divisible by 4 -- were measured
+                // slower than halves at the 32-token decode layer, 110.4 against 107.6 us for gate/up: their eight stages
+                // per unit do not cover the fill of the pipeline; the code below would take them with f = 4)
+                const int f = 2;
+                const int rounds_f = (f * r + a.n_ctas - 1) / a.n_ctas;          // rounds of 1/f length the pieces take
+                if (rounds_f >= f || r > routed || r > 128 || !a.split_ok[l]) r = 0;
+                r2[l] = r; f2[l] = f;
             }
             for (int l = 0; l < 2; ++l) {
                 const int r = r2[l];
@@ -256,24 +265,28 @@ __device__ __forceinline__ void plan_body(const int32_t* expert_off, const PlanA
                 if (tid < r) {
                     mine = list[total - r + tid];
                     const int rows = a.direct ? a.T : a.tiles[mine.tile].nrows;
-                    cnt = rows <= 64 ? 2 : 1;
+                    cnt = (f2[l] == 4 && rows <= 32) ? 4 : (rows <= 64 ? 2 : 1);
                 }
-                // position of each unit after the split: a prefix count of the units that become two (r <= 128: the
+                // position of each unit after the split: the running sum of the extra pieces before it (r <= 128: the
                 // first four warps hold them all)
-                const unsigned two = __ballot_sync(0xffffffffu, cnt == 2);
-                if (tid < 128 && (tid & 31) == 0) s_split[tid >> 5] = __popc(two);
+                const int extra = cnt > 0 ? cnt - 1 : 0;
+                int incl = extra;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                    if ((tid & 31) >= o) incl += v;
+                }
+                if (tid < 128 && (tid & 31) == 31) s_split[tid >> 5] = incl;
                 __syncthreads();
                 if (tid < r) {
-                    int off = tid + __popc(two & ((1u << (tid & 31)) - 1u));
+                    int off = tid + incl - extra;
                     for (int w = 0; w < (tid >> 5); ++w) off += s_split[w];
-                    Unit u = mine;
-                    if (cnt == 2) {
-                        u.colblock = mine.colblock | (1 << 24);
-                        list[total - r + off] = u;
-                        u.colblock = (mine.colblock + 2) | (1 << 24);
-                        list[total - r + off + 1] = u;
-                    } else {
-                        list[total - r + off] = u;
+                    // pieces of 256 / cnt weight rows: colblocks count steps of 64 rows, the width code sits in the top byte
+                    const int step = 4 / cnt, code = cnt == 4 ? 2 : (cnt == 2 ? 1 : 0);
+                    for (int q = 0; q < cnt; ++q) {
+                        Unit u = mine;
+                        u.colblock = (mine.colblock + q * step) | (code << 24);
+                        list[total - r + off + q] = u;
                     }
                 }
                 if (tid == 0) a.plan_counts[2 + l] = total + s_split[0] + s_split[1] + s_split[2] + s_split[3];
