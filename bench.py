@@ -191,9 +191,9 @@ def kernel_source_digest() -> str:
 # ncu summaries under profiles/ together with the digest of the kernel sources they were captured on.  bench.py prints
 # the figure only while kernel_source_digest() still equals `digest`; otherwise `traffic` is null.
 NCU_TRAFFIC = {
-    "decode": {"bytes": 657.665792e6 + 4.441856e6, "digest": "d575108f2ff192dc",
+    "decode": {"bytes": 657.663232e6 + 4.260608e6, "digest": "5f36453cecdfe1c6",
                "source": "profiles/grouped_gemm_decode_ncu.md (gate/up launch, dram__bytes_read.sum + dram__bytes_write.sum)"},
-    "prefill": {"bytes": 920.745472e6 + 86.632448e6, "digest": "d575108f2ff192dc",
+    "prefill": {"bytes": 935.033600e6 + 84.373760e6, "digest": "5f36453cecdfe1c6",
                 "source": "profiles/grouped_gemm_prefill_ncu.md (merged gate/up launch, dram__bytes_read.sum + dram__bytes_write.sum)"},
 }
 
