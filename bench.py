@@ -481,6 +481,13 @@ def measure_layer(args, wl, rank, local_rank, world, dev, wts_cache, with_cpu_ba
                          "frac": 1e3 * max(t_hbm, t_tc) / ms_step, "algorithmic_bytes": work["total_bytes"],
                          "flops": work["flops"], "active_experts": active},
                 "stage_ms": stage_ms}
+    if bound == "tensor":
+        # the step is timed in long blocks, where the part has settled under its power cap: the same fractions
+        # against the GEMM throughput the library reaches in that state, beside the ones against its burst
+        sus = peaks["bf16_tflops_sustained"]
+        roofline["peak_sustained"] = sus
+        roofline["frac_of_sustained"] = (achieved / sus) if achieved else None
+        roofline["path"]["frac_of_sustained"] = 1e3 * max(t_hbm, work["flops"] / (sus * 1e12)) / ms_step
     line = {"metric": METRIC, "value": world * T / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
             "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",

@@ -105,7 +105,12 @@ enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2,
                                          in turn).  Results are bit-identical. */
        MOE_OPT_ROUTE_LANES = 8 /* 2 (default): the tensor-core router issues its MMAs from two warps, even and odd K
                                   stages into two accumulators that the epilogue adds; 1: one warp, one accumulator
-                                  (another summation order over K: logits differ in the last bits) */ };
+                                  (another summation order over K: logits differ in the last bits) */,
+       MOE_OPT_FUSED_DISPATCH = 11 /* moe_layer_forward and the calls built on it, batches of at most 128 tokens of one
+                                      model with the tensor-core router: 1 (default): the router's one CTA goes on to
+                                      batch the routed rows per expert block (Sec. 3, Sec. 4.1) and to lay out the
+                                      experts' work, in the same launch; 0: the dispatch is a launch of its own, as
+                                      in moe_dispatch.  Results are bit-identical. */ };
 
 typedef struct {
     int32_t hidden;        /* H */

@@ -215,16 +215,19 @@ int layer_forward_impl(moe_ctx* c, int layer, const bf16* x, const int32_t* tena
         MOE_CUDA(c, cudaEventRecord(c->ev_join, c->side));
     }
     stage_mark(c, st, kEvBegin);
-    // (routed: the gate has run already and its results are in the workspace -- the paged entry point looks at them first)
-    if (!routed)
-        MOE_CUDA(c, launch_route(c, layer, x, tenant_id, T, w.topk_idx, w.topk_w, shared ? w.shared_gate : nullptr,
-                                 w.tie_flag, st));
-    stage_mark(c, st, kEvRoute);
     // with few tokens the tensor-core experts read the tokens in place: no permuted copy to make
     const bool direct = use_tc(c) && tc_direct_mode(c, T);
-    bool plan_done = false;
-    MOE_CUDA(c, launch_dispatch(c, x, w.topk_idx, tenant_id, T, G, w.perm, w.inv_perm, w.tenant_expert_count,
-                                w.expert_off, w.group_off, direct ? nullptr : w.x_perm, st, true, shared && !early, &plan_done));
+    bool plan_done = false, dispatched = false;
+    // (routed: the gate has run already and its results are in the workspace -- the paged entry point looks at them first)
+    if (!routed)
+        MOE_CUDA(c, launch_route_dispatch(c, layer, x, tenant_id, T, G, w.topk_idx, w.topk_w, shared ? w.shared_gate : nullptr,
+                                          w.tie_flag, w.perm, w.inv_perm, w.tenant_expert_count, w.expert_off, w.group_off,
+                                          direct ? nullptr : w.x_perm, st, shared && !early, &dispatched, &plan_done));
+    stage_mark(c, st, kEvRoute);
+    // (a batch that one CTA routes has been dispatched by that CTA)
+    if (!dispatched)
+        MOE_CUDA(c, launch_dispatch(c, x, w.topk_idx, tenant_id, T, G, w.perm, w.inv_perm, w.tenant_expert_count,
+                                    w.expert_off, w.group_off, direct ? nullptr : w.x_perm, st, true, shared && !early, &plan_done));
     stage_mark(c, st, kEvDispatch);
     if (sort_early) MOE_CUDA(c, cudaStreamWaitEvent(st, c->ev_join, 0));
     const int rc = experts_impl(c, layer, x, w.x_perm, w.perm, w.expert_off, tenant_id, T, G, w.y_perm,
@@ -283,6 +286,7 @@ int moe_create(const moe_config* cfg, moe_ctx** out)
     c->token_major_enabled = 1;
     c->dispatch_private = 0;
     c->background_enabled = 1;
+    c->fused_dispatch_enabled = 1;
     c->timing = false;
     c->early_shared_enabled = 1;
     c->early_shared_sms = 1 << 20;      // no limit
@@ -609,6 +613,10 @@ int moe_set_option(moe_ctx* c, int option, int value)
     if (option == MOE_OPT_BACKGROUND_LANES) {
         if (value < 0 || value > 2) return MOE_ERR_SHAPE;
         c->background_enabled = value;
+        return MOE_OK;
+    }
+    if (option == MOE_OPT_FUSED_DISPATCH) {
+        c->fused_dispatch_enabled = value ? 1 : 0;
         return MOE_OK;
     }
     if (option == MOE_OPT_DISPATCH_MODE) {

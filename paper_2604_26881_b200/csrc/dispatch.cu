@@ -9,139 +9,13 @@
 #include <mutex>
 
 #include "internal.h"
+#include "dispatch_small.cuh"
 #include "plan.cuh"
 #include "scan.cuh"
 
 namespace faasmoe {
 
 namespace {
-
-// bin of a routed row: bins are laid out (model, expert, tenant-of-that-model)
-struct BinMap {
-    const int32_t* model_of_tenant;
-    const int32_t* tenant_local;
-    const int32_t* bin_base;          // [M+1]
-    const int32_t* tenants_in_model;  // [M]
-    int n_tenants, E;
-};
-
-__device__ __forceinline__ int row_bin(const BinMap& bm, int tenant, int expert, int32_t* status)
-{
-    if (tenant < 0 || tenant >= bm.n_tenants) { atomicOr(status, MOE_DEV_BAD_TENANT); tenant = 0; }
-    if (expert < 0 || expert >= bm.E) { atomicOr(status, MOE_DEV_BAD_EXPERT); expert = 0; }
-    const int m = bm.model_of_tenant[tenant];
-    return bm.bin_base[m] + expert * bm.tenants_in_model[m] + bm.tenant_local[tenant];
-}
-
-// Block-wide: exclusive scan of the per-bin totals in s_tot (in key order), then the offset tables
-// the caller sees and the invocation statistics.  s_tot holds the offsets afterwards.
-__device__ void scan_and_tables(int32_t* s_tot, int32_t* s_part /* [33] */, int32_t* s_count /* [2] */,
-                                int nbins, int R, int E, int M, int G, int n_tenants, const BinMap& bm,
-                                int32_t* __restrict__ bin_off /* may be null */,
-                                int32_t* __restrict__ tenant_expert_count, int32_t* __restrict__ expert_off,
-                                int32_t* __restrict__ group_off, int32_t* __restrict__ stats, int private_mode,
-                                const int32_t* __restrict__ block_table = nullptr, int table_blocks = 0)
-{
-    const int tid = threadIdx.x, nth = blockDim.x;
-    if (tid < 2) s_count[tid] = 0;
-    if (tenant_expert_count) {
-        for (int i = tid; i < n_tenants * E; i += nth) {
-            const int u = i / E, e = i - u * E;
-            const int m = bm.model_of_tenant[u];
-            tenant_expert_count[i] = s_tot[bm.bin_base[m] + e * bm.tenants_in_model[m] + bm.tenant_local[u]];
-        }
-    }
-    __syncthreads();
-    block_scan_exclusive(s_tot, nbins, s_part);
-    if (bin_off) {
-        for (int b = tid; b < nbins; b += nth) bin_off[b] = s_tot[b];
-        if (tid == 0) bin_off[nbins] = R;
-    }
-    // expert_off[m*E + e] = offset of the first bin of (m, e); a model without tenants owns
-    // no bins, so its experts start where the next model's bins start
-    for (int i = tid; i <= M * E; i += nth) {
-        int v = R;
-        if (i < M * E) {
-            const int m = i / E, e = i - m * E;
-            const int first = bm.bin_base[m] + e * bm.tenants_in_model[m];
-            v = (first < nbins) ? s_tot[first] : R;
-        }
-        expert_off[i] = v;
-    }
-    __syncthreads();
-    if (block_table) {
-        // Blocks given by a table (load-aware formation, Sec. 5) are sets of experts, not ranges of rows: group_off
-        // then holds the running sum of the rows every block receives, in block order.  Sizes are small (M * B blocks,
-        // E experts each): plain loops.
-        const int B = table_blocks;
-        for (int i = tid; i < M * B; i += nth) {
-            const int m = i / B, b = i - m * B;
-            int rows = 0;
-            for (int e = 0; e < E; ++e)
-                if (block_table[m * E + e] == b) rows += expert_off[m * E + e + 1] - expert_off[m * E + e];
-            if (rows > 0 && !private_mode) atomicAdd(&s_count[0], 1);
-            if (group_off) group_off[i + 1] = rows;
-        }
-        __syncthreads();
-        if (tid == 0 && group_off) {
-            int run = 0;
-            group_off[0] = 0;
-            for (int i = 1; i <= M * B; ++i) { run += group_off[i]; group_off[i] = run; }
-        }
-        if (private_mode) {
-            for (int i = tid; i < n_tenants * B; i += nth) {
-                const int u = i / B, b = i - u * B;
-                const int m = bm.model_of_tenant[u];
-                const int tim = bm.tenants_in_model[m], ul = bm.tenant_local[u];
-                bool any = false;
-                for (int e = 0; e < E; ++e) {
-                    if (block_table[m * E + e] != b) continue;
-                    const int bin = bm.bin_base[m] + e * tim + ul;
-                    const int end = bin + 1 < nbins ? s_tot[bin + 1] : R;
-                    any = any || end > s_tot[bin];
-                }
-                if (any) atomicAdd(&s_count[0], 1);
-            }
-        }
-        for (int i = tid; i < M * E; i += nth)
-            if (expert_off[i + 1] > expert_off[i]) atomicAdd(&s_count[1], 1);
-        __syncthreads();
-        if (tid < 2) stats[tid] = s_count[tid];
-        return;
-    }
-    // expert blocks of G experts; invocation statistics
-    const int B = (E + G - 1) / G;
-    for (int i = tid; i <= M * B; i += nth) {
-        int v = R;
-        if (i < M * B) {
-            const int m = i / B, b = i - m * B;
-            const int e0 = b * G, e1 = min(E, e0 + G);
-            v = expert_off[m * E + e0];
-            if (!private_mode && expert_off[m * E + e1] > v) atomicAdd(&s_count[0], 1);
-        }
-        if (group_off) group_off[i] = v;
-    }
-    if (private_mode) {
-        // private orchestrators (Sec. 4.2): every tenant batches its own tokens, so an invocation is a pair
-        // (tenant, block of its model) with at least one row
-        for (int i = tid; i < n_tenants * B; i += nth) {
-            const int u = i / B, b = i - u * B;
-            const int m = bm.model_of_tenant[u];
-            const int tim = bm.tenants_in_model[m], ul = bm.tenant_local[u];
-            bool any = false;
-            for (int e = b * G; e < min(E, (b + 1) * G); ++e) {
-                const int bin = bm.bin_base[m] + e * tim + ul;
-                const int end = bin + 1 < nbins ? s_tot[bin + 1] : R;
-                any = any || end > s_tot[bin];
-            }
-            if (any) atomicAdd(&s_count[0], 1);
-        }
-    }
-    for (int i = tid; i < M * E; i += nth)
-        if (expert_off[i + 1] > expert_off[i]) atomicAdd(&s_count[1], 1);
-    __syncthreads();
-    if (tid < 2) stats[tid] = s_count[tid];
-}
 
 // D1 (large batches): every block ranks the rows of its chunk.  One warp walks the chunk in row order; rows
 // that share a bin inside one step are ranked by lane order (= row order), so the rank of a row inside
@@ -265,68 +139,16 @@ dispatch_place_kernel(int R, int k, int nbins, const int32_t* __restrict__ block
     }
 }
 
-// Small batches: the whole dispatch in one block -- histogram, scan, tables, stable ranks (one warp
-// walks the rows in order), and the gather of the rows.  Same results as the multi-block kernels.
+// Small batches: the whole dispatch in one block (dispatch_small.cuh).
 constexpr int kSmallRows = 2048;   // above this the serial ranking pass of one warp costs more than the extra launches
 
 __global__ void __launch_bounds__(1024, 1)
-dispatch_small_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ tenant_id, int R, int k,
-                      BinMap bm, int nbins, int E, int M, int G, int n_tenants, int32_t* __restrict__ perm,
-                      int32_t* __restrict__ inv_perm, int32_t* __restrict__ tenant_expert_count,
-                      int32_t* __restrict__ expert_off, int32_t* __restrict__ group_off, int32_t* __restrict__ stats,
-                      int32_t* __restrict__ status, const bf16* __restrict__ x, bf16* __restrict__ x_perm, int H,
-                      int do_plan, int plan_ints, PlanArgs pa, int32_t* __restrict__ bin_off, int private_mode,
-                      const int32_t* __restrict__ block_table, int table_blocks)
+dispatch_small_kernel(const __grid_constant__ SmallDispatchArgs a)
 {
     extern __shared__ int32_t s_tot[];       // [nbins], then the plan's scratch, then the bin of every row (u16)
-    __shared__ int32_t s_part[33];
-    __shared__ int32_t s_count[2];
     pdl_wait();
     pdl_launch_dependents();
-    const int tid = threadIdx.x, nth = blockDim.x;
-    unsigned short* s_bin = reinterpret_cast<unsigned short*>(s_tot + nbins + plan_ints);
-    for (int b = tid; b < nbins; b += nth) s_tot[b] = 0;
-    __syncthreads();
-    for (int r = tid; r < R; r += nth) {
-        const int bin = row_bin(bm, tenant_id[r / k], topk_idx[r], status);
-        s_bin[r] = (unsigned short)bin;      // nbins <= 8192: fits; the ranking pass below reads it back
-        atomicAdd(&s_tot[bin], 1);
-    }
-    __syncthreads();
-    scan_and_tables(s_tot, s_part, s_count, nbins, R, E, M, G, n_tenants, bm, bin_off, tenant_expert_count,
-                    expert_off, group_off, stats, private_mode, block_table, table_blocks);
-    __syncthreads();
-    if (tid < 32) {                           // s_tot now holds the next free position of every bin
-        const int lane = tid;
-        for (int rr = 0; rr < R; rr += 32) {
-            const int r = rr + lane;
-            const bool live = r < R;
-            int bin = -1 - lane;
-            if (live) bin = s_bin[r];
-            const unsigned peers = __match_any_sync(0xffffffffu, bin);
-            const int leader = __ffs(peers) - 1;
-            const int rank = __popc(peers & ((1u << lane) - 1u));
-            int start = 0;
-            if (live && lane == leader) { start = s_tot[bin]; s_tot[bin] = start + __popc(peers); }
-            start = __shfl_sync(0xffffffffu, start, leader);
-            if (live) { perm[start + rank] = r; inv_perm[r] = start + rank; }
-            __syncwarp();
-        }
-    }
-    if (do_plan) {
-        __syncthreads();                      // expert_off (written above) is visible to the block
-        plan_body(expert_off, pa, s_tot + nbins, s_part);
-    }
-    if (x_perm) {
-        __syncthreads();                      // perm is complete and visible to the block
-        const int warp = tid >> 5, lane = tid & 31, nw = nth >> 5;
-        for (int pos = warp; pos < R; pos += nw) {
-            const int t = perm[pos] / k;
-            const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t * H);
-            uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)pos * H);
-            for (int v = lane; v < (H >> 3); v += 32) dst[v] = src[v];
-        }
-    }
+    dispatch_small_body(a, s_tot);
 }
 
 // D4: x_perm[pos] = x[perm[pos] / k].  One warp per row, 16-byte vectors.
@@ -424,7 +246,70 @@ BinMap make_binmap(const moe_ctx* c)
     return bm;
 }
 
+// Arguments of the one-block dispatch for a batch of at most kSmallRows rows.
+void small_dispatch_args(moe_ctx* c, const bf16* x, const int32_t* topk_idx, const int32_t* tenant_id, int T, int G,
+                         int32_t* perm, int32_t* inv_perm, int32_t* tenant_expert_count, int32_t* expert_off,
+                         int32_t* group_off, bf16* x_perm, bool with_plan, bool plan_shared, SmallDispatchArgs* out,
+                         size_t* smem_bytes, bool* gather_inside)
+{
+    const moe_config& g = c->cfg;
+    const int k = g.top_k, R = T * k, nbins = c->nbins;
+    SmallDispatchArgs& a = *out;
+    memset(&a, 0, sizeof(a));
+    // the gather rides along while it is small
+    *gather_inside = x_perm && (size_t)R * g.hidden * sizeof(bf16) <= (1u << 20);
+    // the expert work plan rides along when the shared-expert tiles need no token sort (one model)
+    const bool do_plan = with_plan && g.n_models == 1;
+    size_t plan_ints = 0;
+    if (do_plan) { a.pa = make_plan_args(c, T, G, plan_shared); plan_ints = plan_smem_ints(c, G); }
+    a.topk_idx = topk_idx; a.tenant_id = tenant_id; a.R = R; a.k = k; a.bm = make_binmap(c); a.nbins = nbins;
+    a.E = g.n_experts; a.M = g.n_models; a.G = G; a.n_tenants = g.n_tenants;
+    a.perm = perm; a.inv_perm = inv_perm; a.tenant_expert_count = tenant_expert_count; a.expert_off = expert_off;
+    a.group_off = group_off; a.stats = c->ws.stats; a.status = c->ws.status;
+    a.x = x; a.x_perm = *gather_inside ? x_perm : nullptr; a.H = g.hidden;
+    a.do_plan = do_plan ? 1 : 0; a.plan_ints = (int)plan_ints;
+    a.bin_off = c->dispatch_private ? c->ws.bin_off : nullptr; a.private_mode = c->dispatch_private;
+    a.block_table = c->d_block_table; a.table_blocks = c->table_blocks;
+    *smem_bytes = (size_t)nbins * sizeof(int32_t) + plan_ints * sizeof(int32_t) + (((size_t)R * 2 + 15) & ~(size_t)15);
+}
+
 }  // namespace
+
+cudaError_t launch_route_dispatch(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int G,
+                                  int32_t* topk_idx, float* topk_w, float* shared_gate, uint8_t* tie_flag, int32_t* perm,
+                                  int32_t* inv_perm, int32_t* tenant_expert_count, int32_t* expert_off, int32_t* group_off,
+                                  bf16* x_perm, cudaStream_t st, bool plan_shared, bool* fused, bool* plan_done)
+{
+    *fused = false;
+    *plan_done = false;
+    const moe_config& g = c->cfg;
+    const bool tc = c->route_path != MOE_PATH_FMA && route_tc_supported(c);
+    // One CTA routes the batch (at most 128 tokens of one model): it holds every routed row when its top-k step ends
+    // and goes on to the dispatch and the plan -- one launch and one round trip through global memory fewer on the
+    // latency chain of a small batch.
+    if (tc && c->fused_dispatch_enabled && T <= kFusedDispatchTokens && g.n_models == 1 && T * g.top_k <= kSmallRows) {
+        SmallDispatchArgs a;
+        size_t smem_small = 0;
+        bool gather_inside = false;
+        small_dispatch_args(c, x, topk_idx, tenant_id, T, G, perm, inv_perm, tenant_expert_count, expert_off, group_off,
+                            x_perm, true, plan_shared, &a, &smem_small, &gather_inside);
+        if (smem_small <= kFusedDispatchSmem) {
+            const cudaError_t e = launch_route_tc(c, layer, x, tenant_id, T, topk_idx, topk_w, shared_gate, tie_flag, st,
+                                                  &a, smem_small);
+            if (e != cudaSuccess) return e;
+            *fused = true;
+            *plan_done = a.do_plan != 0;
+            if (x_perm && !gather_inside) {
+                // (more rows than one block should copy: the permuted copy is made by a grid of its own)
+                gather_rows_kernel<<<(T * g.top_k * 32 + 255) / 256, 256, 0, st>>>(x, perm, T * g.top_k, g.top_k, g.hidden, x_perm);
+                c->launches += 1;
+                return cudaGetLastError();
+            }
+            return cudaSuccess;
+        }
+    }
+    return launch_route(c, layer, x, tenant_id, T, topk_idx, topk_w, shared_gate, tie_flag, st);
+}
 
 cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, const int32_t* tenant_id, int T, int G,
                             int32_t* perm, int32_t* inv_perm, int32_t* tenant_expert_count, int32_t* expert_off,
@@ -439,24 +324,17 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
     const BinMap bm = make_binmap(c);
     const size_t smem = (size_t)nbins * sizeof(int32_t);
     if (R <= kSmallRows) {
-        // few rows: one block does everything; the gather rides along while it is small
-        const bool gather_inside = x_perm && (size_t)R * g.hidden * sizeof(bf16) <= (1u << 20);
-        // the expert work plan rides along when the shared-expert tiles need no token sort (one model)
-        const bool do_plan = with_plan && g.n_models == 1;
-        PlanArgs pa;
-        memset(&pa, 0, sizeof(pa));
-        size_t plan_ints = 0;
-        if (do_plan) { pa = make_plan_args(c, T, G, plan_shared); plan_ints = plan_smem_ints(c, G); }
+        // few rows: one block does everything
+        SmallDispatchArgs a;
+        size_t smem_small = 0;
+        bool gather_inside = false;
+        small_dispatch_args(c, x, topk_idx, tenant_id, T, G, perm, inv_perm, tenant_expert_count, expert_off, group_off,
+                            x_perm, with_plan, plan_shared, &a, &smem_small, &gather_inside);
         const int threads = (R <= 512 && nbins <= 1024) ? 256 : 1024;
-        const size_t smem_small = smem + plan_ints * sizeof(int32_t) + (((size_t)R * 2 + 15) & ~(size_t)15);
         if (smem_small > 48 * 1024)
             cudaFuncSetAttribute(dispatch_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_small);
-        launch_pdl(dispatch_small_kernel, dim3(1), dim3(threads), smem_small, st,
-            topk_idx, tenant_id, R, k, bm, nbins, g.n_experts, g.n_models, G, g.n_tenants, perm, inv_perm,
-            tenant_expert_count, expert_off, group_off, c->ws.stats, c->ws.status, x, gather_inside ? x_perm : nullptr,
-            g.hidden, do_plan ? 1 : 0, (int)plan_ints, pa, c->dispatch_private ? c->ws.bin_off : nullptr, c->dispatch_private,
-            c->d_block_table, c->table_blocks);
-        if (plan_done) *plan_done = do_plan;
+        launch_pdl(dispatch_small_kernel, dim3(1), dim3(threads), smem_small, st, a);
+        if (plan_done) *plan_done = a.do_plan != 0;
         c->launches += 1;
         if (x_perm && !gather_inside) {
             gather_rows_kernel<<<(R * 32 + 255) / 256, 256, 0, st>>>(x, perm, R, k, g.hidden, x_perm);

@@ -20,6 +20,8 @@ constexpr int kTileRows = 128;       // rows (tokens) of one expert handled by o
 constexpr int kDispatchChunk = 256;  // routed rows ranked by one block of the dispatch kernels
 constexpr int kAccRowsBg = 224;      // pair shape with background lanes: token rows per accumulator of a wide tile (two per tile)
 constexpr int kShortRows = 64;       // pair shape: tiles of at most this many rows may be run by the background lanes
+constexpr int kFusedDispatchTokens = 128;        // tokens one router CTA handles
+constexpr size_t kFusedDispatchSmem = 128 * 1024; // scratch the router's stage ring offers the dispatch behind it
 constexpr int kMaxDevices = 64;      // per-device state of the library (kernel attributes, scratch addresses)
 
 // Per (layer, model) weight pointers, as the kernels see them.
@@ -163,6 +165,7 @@ struct moe_ctx {
     int pair_mode_enabled;        // allow the 2-CTA (cta_group::2) shape of the grouped GEMM for long tiles
     int token_major_enabled;      // one-CTA units take the tokens as the M operand of the MMA (up to 256 weight rows per tile)
     int wide_tiles_enabled;       // allow 512-row tiles (two accumulators per weight tile) in the 2-CTA shape
+    int fused_dispatch_enabled;   // one-tile batches: the router's CTA also runs the dispatch and the work plan
     int background_enabled;       // pair shape: short tiles are run by a second set of lanes beside the long ones
     int dispatch_private;         // 0: shared orchestrator (one request per expert block), 1: private orchestrators
                                   // (one request per tenant and block): invocation statistics and tile formation
@@ -223,8 +226,18 @@ cudaError_t launch_dispatch(moe_ctx* c, const bf16* x, const int32_t* topk_idx, 
 
 cudaError_t launch_route_fma(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,
                              float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st);
+struct SmallDispatchArgs;
+// fused: arguments of the one-block dispatch that the router's CTA runs behind its top-k step (one-tile batch of one
+// model; fused_smem bytes of scratch), or null
 cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,
-                            float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st);
+                            float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st,
+                            const SmallDispatchArgs* fused = nullptr, size_t fused_smem = 0);
+// Router, then -- where one CTA routes the whole batch -- dispatch and work plan in the same launch.  *fused tells the
+// caller whether the dispatch has been done (and *plan_done whether the plan has); if not, launch_dispatch follows.
+cudaError_t launch_route_dispatch(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int G,
+                                  int32_t* topk_idx, float* topk_w, float* shared_gate, uint8_t* tie_flag, int32_t* perm,
+                                  int32_t* inv_perm, int32_t* tenant_expert_count, int32_t* expert_off, int32_t* group_off,
+                                  bf16* x_perm, cudaStream_t st, bool plan_shared, bool* fused, bool* plan_done);
 bool route_tc_supported(const moe_ctx* c);
 void route_tc_destroy(moe_ctx* c);
 

@@ -9,6 +9,7 @@
 #include <cstring>
 
 #include "internal.h"
+#include "dispatch_small.cuh"
 #include "tc_ptx.cuh"
 
 namespace faasmoe {
@@ -23,6 +24,7 @@ constexpr int kRTokens = 128;
 constexpr int kRABytes = kRTokens * kRBK * 2;          // 16 KB of tokens per stage
 constexpr int kRMaxN = 256;                            // router rows of all models, padded
 constexpr int kRTileBudget = 192 * 1024;               // shared memory for the pipeline stages
+static_assert(kFusedDispatchSmem <= (size_t)kRTileBudget, "the dispatch behind the router uses the stage ring as scratch");
 constexpr int kRSmemBytes = kRTileBudget + kRABytes /* a short token tile is read as 128 rows */ + 1024 + 512;
 constexpr int kRThreads = 288;                         // warp 0: TMA (tokens), 1: MMA, 2..5: epilogue, 6 / 7: TMA (routers / gates),
                                                        // 8: second MMA lane
@@ -75,8 +77,14 @@ __device__ __forceinline__ float dot8f(const uint4& a, const uint4& b, float acc
     return acc;
 }
 
+// (a call, not inlined: the registers of the dispatch stay out of the router's own allocation)
+__device__ __noinline__ void dispatch_behind_router(const SmallDispatchArgs& fd, int32_t* scratch)
+{
+    dispatch_small_body(fd, scratch);
+}
+
 __global__ void __launch_bounds__(kRThreads, 1)
-route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
+route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps, const __grid_constant__ SmallDispatchArgs fd)
 {
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -343,6 +351,12 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps)
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
+    // One-tile batch of one model: this block holds every routed row, so it goes on to batch them per expert block
+    // (Sec. 3, Sec. 4.1) and to lay out the experts' work, instead of a kernel of its own doing so after a launch and a
+    // round trip through global memory.  The pipeline stages are free by now (every tile load was consumed by an MMA
+    // that the top-k step waited for) and serve as scratch.  Not after a wait ran out: copies may still be in flight.
+    if (fd.enabled && !s_abort)
+        dispatch_behind_router(fd, reinterpret_cast<int32_t*>(smem_dyn + (smem_base - smem_u32(smem_dyn))));
 }
 
 struct RouterMaps {
@@ -369,7 +383,8 @@ void route_tc_destroy(moe_ctx* c)
 }
 
 cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t* tenant_id, int T, int32_t* topk_idx,
-                            float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st)
+                            float* topk_w, float* shared_gate, uint8_t* tie_flag, cudaStream_t st,
+                            const SmallDispatchArgs* fused, size_t fused_smem)
 {
     const moe_config& g = c->cfg;
     const int M = g.n_models, E = g.n_experts, H = g.hidden;
@@ -438,7 +453,15 @@ cudaError_t launch_route_tc(moe_ctx* c, int layer, const bf16* x, const int32_t*
     if (p.lanes2) p.group = 1;
     p.n_stages -= p.n_stages % p.group;
     p.gate_col = p.gate_merged ? Mc * epad : kRMaxN;
-    launch_pdl(route_tc_kernel, dim3((T + kRTokens - 1) / kRTokens, p.per_model ? M : 1), dim3(kRThreads), kRSmemBytes, st, p, mp);
+    SmallDispatchArgs fd;
+    memset(&fd, 0, sizeof(fd));
+    if (fused) {
+        // (the caller offers the dispatch only for a batch that one CTA routes)
+        if (T > kRTokens || p.per_model || fused_smem > (size_t)kRTileBudget) return cudaErrorInvalidValue;
+        fd = *fused;
+        fd.enabled = 1;
+    }
+    launch_pdl(route_tc_kernel, dim3((T + kRTokens - 1) / kRTokens, p.per_model ? M : 1), dim3(kRThreads), kRSmemBytes, st, p, mp, fd);
     c->launches += 1;
     return cudaGetLastError();
 }

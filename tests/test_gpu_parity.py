@@ -327,6 +327,52 @@ def test_background_lanes_agree_bit_for_bit(qwen_weights, T):
         g.close()
 
 
+@pytest.mark.parametrize("T", [1, 5, 32, 100, 128, 129])
+def test_dispatch_behind_the_router_agrees_bit_for_bit(qwen_weights, T):
+    # a batch that one CTA routes (at most 128 tokens of one model) is dispatched, and its experts' work laid out, by
+    # that CTA in the router's launch; the same code runs as a launch of its own otherwise (129 tokens: always).
+    # Outputs, routing buffers, offsets, statistics and the number of launches are compared, in both orchestrator
+    # modes, with and without a block table, the batch changing from call to call.
+    wl = W.scaled(W.WORKLOADS["decode"], T=T, n_tenants=3, tenant_layout="uniform")
+    x, tenant, mot = W.make_tokens(wl, seed=21)
+    x2, tenant2, _ = W.make_tokens(wl, seed=22)
+    g = GpuLayer(wl, [qwen_weights], wl.T, model_of_tenant=mot)
+    R = T * wl.k
+    try:
+        ws = B.moe_get_workspace(g.ctx)
+        shapes = {"topk_idx": ((R,), torch.int32), "topk_w": ((R,), torch.float32), "shared_gate": ((T,), torch.float32),
+                  "tie_flag": ((T,), torch.uint8), "perm": ((R,), torch.int32), "inv_perm": ((R,), torch.int32),
+                  "expert_off": ((wl.E + 1,), torch.int32)}
+
+        def run(fused, xx, tt, G):
+            B.moe_set_option(g.ctx, B.MOE_OPT_FUSED_DISPATCH, fused)
+            n0 = B.moe_launch_count(g.ctx)
+            out = g.forward(xx, tt, G)
+            n = B.moe_launch_count(g.ctx) - n0
+            bufs = {k: B.wrap_device_pointer(ws[k], sh, dt, g.dev).clone() for k, (sh, dt) in shapes.items()}
+            return out, bufs, B.moe_last_status(g.ctx), B.moe_last_plan(g.ctx, T), n
+
+        for mode in (B.MOE_DISPATCH_SHARED, B.MOE_DISPATCH_PRIVATE):
+            B.moe_set_option(g.ctx, B.MOE_OPT_DISPATCH_MODE, mode)
+            for table in (False, True):
+                if table:
+                    B.moe_set_block_table(g.ctx, torch.tensor([[(7 * e + 3) % 9 for e in range(wl.E)]], dtype=torch.int32), 9)
+                else:
+                    B.moe_set_block_table(g.ctx, None)
+                for G in (1, 4):
+                    for xx, tt in ((x, tenant), (x2, tenant2)):
+                        ref = run(0, xx, tt, G)
+                        got = run(1, xx, tt, G)
+                        assert got[2][0] == 0 and ref[2][0] == 0
+                        assert torch.equal(got[0], ref[0]), (mode, table, G)
+                        for k in shapes:
+                            assert torch.equal(got[1][k], ref[1][k]), (k, mode, table, G)
+                        assert got[2] == ref[2] and got[3] == ref[3]
+                        assert got[4] == ref[4] - (1 if T <= 128 else 0)
+    finally:
+        g.close()
+
+
 @pytest.mark.parametrize("T", [7, 64, 300, 1024, 4096])
 def test_shared_expert_on_second_stream_agrees_bit_for_bit(qwen_weights, T):
     # one model: the shared expert's launches may run on the context's second stream beside the router and the
