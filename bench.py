@@ -195,6 +195,8 @@ NCU_TRAFFIC = {
                "source": "profiles/grouped_gemm_decode_ncu.md (gate/up launch, dram__bytes_read.sum + dram__bytes_write.sum)"},
     "prefill": {"bytes": 935.033600e6 + 84.373760e6, "digest": "5f36453cecdfe1c6",
                 "source": "profiles/grouped_gemm_prefill_ncu.md (merged gate/up launch, dram__bytes_read.sum + dram__bytes_write.sum)"},
+    "pool": {"bytes": 2998.385152e6 + 38.075392e6, "digest": "5f36453cecdfe1c6",
+             "source": "profiles/grouped_gemm_pool_dram.md (merged gate/up launch, dram__bytes_read.sum + dram__bytes_write.sum)"},
 }
 
 
