@@ -107,10 +107,19 @@ enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2,
                                   stages into two accumulators that the epilogue adds; 1: one warp, one accumulator
                                   (another summation order over K: logits differ in the last bits) */,
        MOE_OPT_FUSED_DISPATCH = 11 /* moe_layer_forward and the calls built on it, batches of at most 128 tokens of one
-                                      model with the tensor-core router: 1 (default): the router's one CTA goes on to
-                                      batch the routed rows per expert block (Sec. 3, Sec. 4.1) and to lay out the
-                                      experts' work, in the same launch; 0: the dispatch is a launch of its own, as
-                                      in moe_dispatch.  Results are bit-identical. */ };
+                                      model with the tensor-core router: 1: the router's one CTA goes on to batch the
+                                      routed rows per expert block (Sec. 3, Sec. 4.1) and to lay out the experts' work,
+                                      in the same launch; 0 (default): the dispatch is a launch of its own, as in
+                                      moe_dispatch.  Results are bit-identical.  One launch fewer, but measured about
+                                      1 % slower per step at 32 tokens: the dispatch kernel of its own is already
+                                      resident and waiting when the router ends (programmatic dependent launch), and
+                                      it keeps its tables in L1, which the router's CTA has given up for its stage
+                                      ring. */,
+       MOE_OPT_HEAD_UNITS = 12 /* moe_layer_forward and the calls built on it, batches of at most 64 tokens of one model
+                                  with a shared expert: 1 (default): the gate/up launch works through the shared
+                                  expert's units (tokens and static weights only) before it waits for the router and
+                                  the dispatch of the same pass, so those weights stream in while the routing is being
+                                  worked out; 0: it waits first.  Results are bit-identical. */ };
 
 typedef struct {
     int32_t hidden;        /* H */

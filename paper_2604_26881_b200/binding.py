@@ -31,6 +31,7 @@ MOE_OPT_ROUTE_LANES = 8
 MOE_OPT_DISPATCH_MODE = 9
 MOE_OPT_BACKGROUND_LANES = 10
 MOE_OPT_FUSED_DISPATCH = 11
+MOE_OPT_HEAD_UNITS = 12
 MOE_DISPATCH_SHARED, MOE_DISPATCH_PRIVATE = 0, 1
 MOE_PATH_AUTO, MOE_PATH_FMA, MOE_PATH_TCGEN05 = 0, 1, 2
 

@@ -112,6 +112,11 @@ struct GemmParams {
     int stream_weights;           // 1: every weight tile is read once: mark it evict-first in L2
     int group;                    // stages handed back to the producer per commit (divides the stage count)
     int wide;                     // 1: tiles of up to 512 rows (pair shape only): 4 stages of 48 KB instead of 6 of 32 KB
+    int head_units;               // token-major gate/up launch of a layer pass, one model, one token tile: the shared
+                                  // expert's units at the head of the list (unit i = weight rows 256 i .. of all head_rows
+                                  // tokens).  They depend on nothing the kernels before this one produce, so CTA b runs
+                                  // units b, b + grid, ... of them before it waits for those kernels.  0: none.
+    int head_rows;
     int32_t* status;
 };
 
@@ -273,7 +278,7 @@ __device__ __forceinline__ QEntry read_entry(const QEntry* q)
     const int4 a = *reinterpret_cast<const int4*>(q);
     const int2 b = *reinterpret_cast<const int2*>(&q->colblock);
     QEntry e;
-    e.u = a.x; e.tile_slot = a.y; e.b_row0 = a.z; e.nrows = a.w; e.colblock = b.x; e.shared = b.y; e.pad0 = q->pad0; e.pad1 = 0;
+    e.u = a.x; e.tile_slot = a.y; e.b_row0 = a.z; e.nrows = a.w; e.colblock = b.x; e.shared = b.y; e.pad0 = q->pad0; e.pad1 = q->pad1;
     return e;
 }
 
@@ -570,11 +575,17 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
     // gate/up launch, which had itself waited for the plan before it let this kernel start: the unit lists are
     // complete, and the scheduler and the weight producer (static data) go ahead and fill the ring while the token
     // producer and the epilogue wait for the activations.
-    if (!(MODE == 1 && (warp == 0 || warp == kSchedWarp))) pdl_wait();
-    pdl_launch_dependents();
-    const int n_units = *p.n_units;
-    const int n_shared = *p.n_shared;
-    const int n_short = BG ? *p.n_short : 0;
+    // A gate/up launch with head units (see GemmParams) starts on them at once -- while the router and the dispatch
+    // are still running -- and every role waits when it meets the first unit of the work plan.  Such a launch lets the
+    // down projection start only after the scheduler has waited: that kernel relies on the plan being complete.
+    const bool head = MODE == 0 && SWAP && !PAIR && p.head_units > 0;
+    if (!head) {
+        if (!(MODE == 1 && (warp == 0 || warp == kSchedWarp))) pdl_wait();
+        pdl_launch_dependents();
+    }
+    const int n_units = head ? 0 : *p.n_units;            // (with head units the scheduler reads the counts after its wait)
+    const int n_shared = head ? 0 : *p.n_shared;
+    const int n_short = (BG && !head) ? *p.n_short : 0;
 
     // Units are pulled from a global counter by one scheduler lane per CTA (pair: per CTA pair, the leader's),
     // decoded, and handed to the other roles through a small queue in shared memory; in pair mode the scheduler
@@ -592,7 +603,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
         if (lane == 0) {
             uint32_t stage = 0, phase = 0, q = 0, qphase = 0;
             uint32_t armed = 0, armed_phase = 0;
-            bool ok = true;
+            bool ok = true, planned = false;
             const uint64_t pol_first = l2_evict_first(), pol_last = l2_evict_last();
             const uint64_t pol_x = l2_evict_last();
             while (ok) {
@@ -601,6 +612,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 const QEntry e = read_entry(&s_queue[q]);
                 if (leader) mbar_arrive(bar_qempty + 8 * q); else mbar_arrive_cluster(qempty_leader + 8 * q);
                 if (++q == kQueue) { q = 0; qphase ^= 1; }
+                if (head && !planned && e.pad1) { pdl_wait(); planned = true; }     // the first unit (or the end mark) of the plan
                 if (e.u < 0) break;
                 const UnitInfo ui = unit_info<MODE, PAIR, SWAP, BG>(p, e, rank);
                 const int claim_ks = ui.ksteps > kClaimAhead ? ui.ksteps - kClaimAhead : 0;
@@ -771,7 +783,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const uint32_t stg = bars + kBarBytes + half * kOutGroupBytes;      // this group's staging area
         uint32_t buf = 0, bphase = 0, q = 0, qphase = 0;
-        bool ok = true;
+        bool ok = true, planned = false;
         const uint32_t tempty_leader = PAIR ? map_to_cta(bar_tempty, 0) : bar_tempty;
         while (ok) {
             ok = __all_sync(0xffffffffu, PAIR ? mbar_wait_cluster(bar_qfull + 8 * q, qphase, &s_abort, p.status)
@@ -783,6 +795,7 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                 if (PAIR) mbar_arrive_cluster(qempty_leader + 8 * q); else mbar_arrive(bar_qempty + 8 * q);
             }
             if (++q == kQueue) { q = 0; qphase ^= 1; }
+            if (head && !planned && e.pad1) { pdl_wait(); planned = true; }         // (warp-uniform)
             if (e.u < 0) break;
             const UnitInfo ui = unit_info<MODE, PAIR, SWAP, BG>(p, e, rank);
             const int ld = ui.shared ? p.ld_shared : p.ld_routed;
@@ -1082,7 +1095,9 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
         // ---------------- scheduler (one lane of the leader CTA) ----------------
         if (lane == 0 && leader) {
             uint32_t q = 0, qphase = 0, sphase = 0;
-            bool first = true;
+            bool first = true, planned = !head;
+            int head_next = head ? (int)blockIdx.x : 0;
+            int nu = n_units, nsh = n_shared;         // unit counts of the plan (read after the wait when there are head units)
             const uint32_t peer_queue = PAIR ? map_to_cta(smem_u32(&s_queue[0]), 1) : 0u;
             const uint32_t peer_qfull = PAIR ? map_to_cta(bar_qfull, 1) : 0u;
             for (;;) {
@@ -1096,12 +1111,33 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                            : mbar_wait(bar_qempty + 8 * q, qphase ^ 1, &s_abort, p.status))) break;
                 // one packed counter orders the claims of both ends of the list: a claim is good while fewer than n_units
                 // units have been taken in all
-                const unsigned long long old = atomicAdd(p.counter, 1ull);
-                int u = (int)(uint32_t)old;
-                const bool good = (unsigned long long)(uint32_t)old + (old >> 32) < (unsigned long long)n_units;
                 int4 e0 = make_int4(-1, 0, 0, 0);
                 int2 e1 = make_int2(0, 0);
                 int e0w = 0;                  // token-major shape: weight rows of the unit
+                int from_plan = 1;
+                int u = 0;
+                bool good = false;
+                if (head && head_next < p.head_units) {
+                    // a head unit: the shared expert's weight rows 256 i .. against all tokens (what the plan's list holds
+                    // at index i, written out here because the plan may not exist yet)
+                    u = head_next;
+                    head_next += (int)gridDim.x;
+                    e0 = make_int4(u, 0, 0, p.head_rows);
+                    e1 = make_int2(u * 4, 1);
+                    e0w = 256;
+                    from_plan = 0;
+                } else {
+                    if (!planned) {
+                        pdl_wait();
+                        pdl_launch_dependents();
+                        nu = *p.n_units - p.head_units;          // the list's head has been run
+                        nsh = 0;
+                        planned = true;
+                    }
+                    const unsigned long long old = atomicAdd(p.counter, 1ull);
+                    u = (int)(uint32_t)old;
+                    good = (unsigned long long)(uint32_t)old + (old >> 32) < (unsigned long long)nu;
+                }
                 if (good) {
                     // The list holds the shared expert's units first.  They are fed from L2 (every token tile of the
                     // model reads the same weights) while the routed units stream theirs from HBM, so the two kinds are
@@ -1110,25 +1146,27 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     // long unit handed out at the very end is what the other CTAs then wait for.
                     // (the short units at the tail of the list are taken in list order)
                     int ix = u;
-                    const int n_main = n_units - n_short;
-                    if (n_shared > 0 && u < n_main) {
-                        const int routed = n_main - n_shared;
+                    const int n_main = nu - n_short;
+                    if (nsh > 0 && u < n_main) {
+                        const int routed = n_main - nsh;
                         const int cut = n_main - min(routed, n_main / 6);
                         const int uc = min(u, cut), uc1 = min(u + 1, cut);
-                        const int a = (int)((long long)uc * n_shared / cut), b = (int)((long long)uc1 * n_shared / cut);
-                        ix = b > a ? a : n_shared + (u - a);
+                        const int a = (int)((long long)uc * nsh / cut), b = (int)((long long)uc1 * nsh / cut);
+                        ix = b > a ? a : nsh + (u - a);
                     }
+                    if (head) ix += p.head_units;
                     const Unit un = p.units[ix];
                     const Tile t = un.tile < 0 ? p.stiles[~un.tile] : p.tiles[un.tile];
                     e0 = make_int4(u, t.slot, t.row0, t.nrows);
                     e1 = make_int2(un.colblock & 0xffffff, un.tile < 0 ? 1 : 0);
                     e0w = 256 >> (un.colblock >> 24);
-                } else {
+                } else if (from_plan) {
                     u = -1;
                 }
                 *reinterpret_cast<int4*>(&s_queue[q]) = e0;
                 *reinterpret_cast<int2*>(&s_queue[q].colblock) = e1;
                 s_queue[q].pad0 = e0w;
+                s_queue[q].pad1 = from_plan;
                 mbar_arrive(bar_qfull + 8 * q);
                 if (PAIR) {
                     const uint32_t dst = peer_queue + (uint32_t)sizeof(QEntry) * q;
@@ -1349,7 +1387,7 @@ cudaError_t launch_gemm(moe_ctx* c, const GemmParams& p, const GemmMaps& maps, c
 
 cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, const int32_t* perm, int T,
                               float* y_perm, float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st,
-                              bool shared_only)
+                              bool shared_only, bool tokens_ready)
 {
     const moe_config& g = c->cfg;
     LayerMaps& lm = c->tmaps->layers[layer];
@@ -1406,6 +1444,15 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     p1.wide = tc_wide_mode(c, T) ? 1 : 0;
     p1.group = p1.wide ? 1 : 2;
     if (swap) p1.group = 1;
+    // Token-major shape, one model, all tokens in one tile: the shared expert's gate/up units need the tokens and static
+    // weights only.  When the caller vouches that the tokens are final before the kernels ahead of this launch in the
+    // stream began (a layer pass: router and dispatch only read them), the launch runs those units before it waits for
+    // these kernels -- weight bytes streamed while the routing is still being worked out.
+    if (tokens_ready && c->head_units_enabled && swap && shared && !shared_only && g.n_models == 1 && T <= kTileRows &&
+        shared_dst_rows == nullptr) {
+        p1.head_units = Is / 128;           // units of 256 interleaved gate / up rows
+        p1.head_rows = T;
+    }
     // (the shared expert alone has no short tiles: its launches keep the shape without the background pipeline)
     const bool bg = pair && tc_background_mode(c, T) && !shared_only;
     cudaError_t e = pair ? (bg ? launch_gemm<0, true, false, true>(c, p1, m1, st, cap1)
@@ -1422,6 +1469,7 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     if (shared_only) copy_b(m2.b_routed, m2.b_shared);
     if (!ok) return cudaErrorInvalidValue;
     GemmParams p2 = p1;
+    p2.head_units = 0; p2.head_rows = 0;
     p2.units = shared_only ? c->ws.units2_sh : c->ws.units2;
     p2.n_units = counts + 3; p2.counter = reinterpret_cast<unsigned long long*>(counts + 12); p2.n_shared = counts + 7;
     p2.n_short = counts + 9;

@@ -165,6 +165,7 @@ struct moe_ctx {
     int pair_mode_enabled;        // allow the 2-CTA (cta_group::2) shape of the grouped GEMM for long tiles
     int token_major_enabled;      // one-CTA units take the tokens as the M operand of the MMA (up to 256 weight rows per tile)
     int wide_tiles_enabled;       // allow 512-row tiles (two accumulators per weight tile) in the 2-CTA shape
+    int head_units_enabled;       // token-major gate/up launch of a layer pass: shared-expert units before the wait
     int fused_dispatch_enabled;   // one-tile batches: the router's CTA also runs the dispatch and the work plan
     int background_enabled;       // pair shape: short tiles are run by a second set of lanes beside the long ones
     int dispatch_private;         // 0: shared orchestrator (one request per expert block), 1: private orchestrators
@@ -259,7 +260,7 @@ cudaError_t launch_experts_fma(moe_ctx* c, int layer, const bf16* x_or_xs, const
 
 cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const bf16* x_perm, const int32_t* perm, int T,
                               float* y_perm, float* y_shared, const int32_t* shared_dst_rows, cudaStream_t st,
-                              bool shared_only = false);
+                              bool shared_only = false, bool tokens_ready = false);
 
 cudaError_t launch_combine(moe_ctx* c, const float* y_perm, const int32_t* inv_perm, const float* topk_w,
                            const float* y_shared, const float* shared_gate, const bf16* residual, int T, bf16* out,

@@ -373,6 +373,40 @@ def test_dispatch_behind_the_router_agrees_bit_for_bit(qwen_weights, T):
         g.close()
 
 
+@pytest.mark.parametrize("T", [1, 8, 32, 64])
+def test_shared_units_ahead_of_the_wait_agree_bit_for_bit(qwen_weights, T):
+    # small batches of one model: the gate/up launch may run the shared expert's units (tokens and static weights only)
+    # before it waits for the router and the dispatch of the same pass.  Same units, same arithmetic: the output bits
+    # do not change, with the dispatch inside the router's launch or in its own, call after call without a
+    # synchronisation in between (the launch of one pass starts while kernels of the pass before may still run) and
+    # with the batch changing from call to call.
+    wl = W.scaled(W.WORKLOADS["decode"], T=T, n_tenants=3, tenant_layout="uniform")
+    x, tenant, mot = W.make_tokens(wl, seed=31)
+    x2, tenant2, _ = W.make_tokens(wl, seed=32)
+    g = GpuLayer(wl, [qwen_weights], wl.T, model_of_tenant=mot)
+    try:
+        B.moe_set_option(g.ctx, B.MOE_OPT_HEAD_UNITS, 0)
+        ref, ref2 = g.forward(x, tenant, wl.G), g.forward(x2, tenant2, wl.G)
+        xd, td, xd2, td2 = x.to(g.dev), tenant.to(g.dev), x2.to(g.dev), tenant2.to(g.dev)
+        for fused in (1, 0):
+            B.moe_set_option(g.ctx, B.MOE_OPT_FUSED_DISPATCH, fused)
+            B.moe_set_option(g.ctx, B.MOE_OPT_HEAD_UNITS, 1)
+            outs = [torch.zeros_like(xd) for _ in range(8)]
+            for i, o in enumerate(outs):
+                B.moe_layer_forward(g.ctx, 0, xd if i % 2 == 0 else xd2, td if i % 2 == 0 else td2, T, wl.G, o)
+            torch.cuda.synchronize()
+            assert B.moe_last_status(g.ctx)[0] == 0
+            for i, o in enumerate(outs):
+                assert torch.equal(o, ref if i % 2 == 0 else ref2), (fused, i)
+        # and against the oracle, element by element, through the fused entry point
+        o = g.four_calls(x, tenant, wl.G)
+        want = oracle_layer(wl, qwen_weights, x, tenant, mot, wl.G, o["topk_idx"].cpu().numpy(), o["topk_w"].cpu().numpy())
+        compare_four_calls(o, want, wl, x)
+        assert torch.equal(ref, o["out"])
+    finally:
+        g.close()
+
+
 @pytest.mark.parametrize("T", [7, 64, 300, 1024, 4096])
 def test_shared_expert_on_second_stream_agrees_bit_for_bit(qwen_weights, T):
     # one model: the shared expert's launches may run on the context's second stream beside the router and the
