@@ -191,11 +191,11 @@ def kernel_source_digest() -> str:
 # ncu summaries under profiles/ together with the digest of the kernel sources they were captured on.  bench.py prints
 # the figure only while kernel_source_digest() still equals `digest`; otherwise `traffic` is null.
 NCU_TRAFFIC = {
-    "decode": {"bytes": 657.663232e6 + 4.260608e6, "digest": "5f36453cecdfe1c6",
+    "decode": {"bytes": 657.660416e6 + 3.442176e6, "digest": "9fa52804dc3025e6",
                "source": "profiles/grouped_gemm_decode_ncu.md (gate/up launch, dram__bytes_read.sum + dram__bytes_write.sum)"},
-    "prefill": {"bytes": 935.033600e6 + 84.373760e6, "digest": "5f36453cecdfe1c6",
+    "prefill": {"bytes": 928.787200e6 + 84.617728e6, "digest": "9fa52804dc3025e6",
                 "source": "profiles/grouped_gemm_prefill_ncu.md (merged gate/up launch, dram__bytes_read.sum + dram__bytes_write.sum)"},
-    "pool": {"bytes": 2998.385152e6 + 38.075392e6, "digest": "5f36453cecdfe1c6",
+    "pool": {"bytes": 2997.174528e6 + 38.322176e6, "digest": "9fa52804dc3025e6",
              "source": "profiles/grouped_gemm_pool_dram.md (merged gate/up launch, dram__bytes_read.sum + dram__bytes_write.sum)"},
 }
 
