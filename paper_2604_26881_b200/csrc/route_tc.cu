@@ -119,7 +119,9 @@ route_tc_kernel(const RouteParams p, const __grid_constant__ RouteMaps maps, con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
-    pdl_wait();                     // set-up above overlaps the previous kernel; its results are read from here on
+    // Set-up above overlaps the previous kernel; its results are read from here on.  The producer lanes of the router
+    // and gate rows read static weights only: they fill the first stages while the others still wait.
+    if (!(warp == 6 || warp == 7)) pdl_wait();
     pdl_launch_dependents();
 
     if (warp == 0 || warp == 6 || warp == 7) {
