@@ -117,6 +117,8 @@ struct GemmParams {
                                   // tokens).  They depend on nothing the kernels before this one produce, so CTA b runs
                                   // units b, b + grid, ... of them before it waits for those kernels.  0: none.
     int head_rows;
+    const void* pull_ptr;         // with head units: static bytes that the CTAs without a head unit pull into L2 before they
+    unsigned long long pull_bytes;//   wait (the shared expert's down weights, which the next launch reads); 0: none
     int32_t* status;
 };
 
@@ -1128,6 +1130,17 @@ grouped_gemm_kernel(const GemmParams p, const __grid_constant__ GemmMaps maps)
                     from_plan = 0;
                 } else {
                     if (!planned) {
+                        if (p.pull_bytes && (int)blockIdx.x >= p.head_units) {
+                            // no head unit here: this CTA would only wait.  A hint, in 16 KB pieces dealt out over
+                            // these CTAs; nothing depends on it.
+                            const unsigned nb = gridDim.x - p.head_units, me = blockIdx.x - p.head_units;
+                            const unsigned long long chunk = 16384, nchunks = (p.pull_bytes + chunk - 1) / chunk;
+                            for (unsigned long long ch = me; ch < nchunks; ch += nb) {
+                                const unsigned long long off = ch * chunk;
+                                const unsigned sz = (unsigned)min(chunk, p.pull_bytes - off) & ~15u;
+                                if (sz) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"((const char*)p.pull_ptr + off), "r"(sz) : "memory");
+                            }
+                        }
                         pdl_wait();
                         pdl_launch_dependents();
                         nu = *p.n_units - p.head_units;          // the list's head has been run
@@ -1452,6 +1465,9 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
         shared_dst_rows == nullptr) {
         p1.head_units = Is / 128;           // units of 256 interleaved gate / up rows
         p1.head_rows = T;
+        // the CTAs beyond the head units fetch the shared expert's down weights (fp16 copy, 2 H Is bytes: they fit in L2
+        // beside the head units' own tiles) for the launch that follows
+        p1.pull_ptr = lm.ws_down_f16[0]; p1.pull_bytes = (unsigned long long)H * Is * 2;
     }
     // (the shared expert alone has no short tiles: its launches keep the shape without the background pipeline)
     const bool bg = pair && tc_background_mode(c, T) && !shared_only;
@@ -1469,7 +1485,7 @@ cudaError_t launch_experts_tc(moe_ctx* c, int layer, const bf16* x_or_xs, const 
     if (shared_only) copy_b(m2.b_routed, m2.b_shared);
     if (!ok) return cudaErrorInvalidValue;
     GemmParams p2 = p1;
-    p2.head_units = 0; p2.head_rows = 0;
+    p2.head_units = 0; p2.head_rows = 0; p2.pull_bytes = 0;
     p2.units = shared_only ? c->ws.units2_sh : c->ws.units2;
     p2.n_units = counts + 3; p2.counter = reinterpret_cast<unsigned long long*>(counts + 12); p2.n_shared = counts + 7;
     p2.n_short = counts + 9;
