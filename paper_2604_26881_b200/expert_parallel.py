@@ -9,7 +9,7 @@ steps are passed in as callables, so the same protocol runs on GPUs (the library
 (gloo, with any stand-in for the expert step).
 
 What is NOT here: any overlap of the exchange with the expert GEMMs (one kernel that sends and computes tile by tile
-over peer memory), and any measurement: the protocol has only ever run as CPU ranks over gloo.
+over peer memory), and any measurement: the protocol has run as CPU ranks over gloo and as a single rank over NCCL.
 """
 from __future__ import annotations
 
