@@ -596,11 +596,13 @@ def test_stack_full_size_teacher_forced():
         g.close()
 
 
-@pytest.mark.parametrize("seed", [4, 5])
+@pytest.mark.parametrize("seed", [4, 5, 6])
 def test_random_configurations_agree_across_modes_tables_and_lanes(seed):
     # 25 random layer shapes per seed, four random option settings each -- shared or private orchestrators, blocks by
     # ranges or by a load-aware table, background lanes off or forced on, the shared expert on the second stream or not:
-    # none of them may change a bit of the output or leave a device status bit
+    # none of them may change a bit of the output or leave a device status bit.  Seed 6 draws small batches (at most
+    # 128 tokens) and also switches the shared expert's units ahead of the wait and the dispatch inside the router's
+    # launch on and off (the reference run has both off).
     import random
     rng = random.Random(seed)
     for it in range(25):
@@ -609,18 +611,27 @@ def test_random_configurations_agree_across_modes_tables_and_lanes(seed):
         Is = rng.choice([0, 128, 256, 512]); M = rng.choice([1, 1, 1, 2, 3]); nt = rng.randint(M, M + 5)
         G = rng.randint(1, E)
         T = rng.choice([1, 3, 31, 64, 65, 100, 128, 129, 255, 300, 513, 700, 1025, 1500, 2048, 2600, 4096])
+        if seed >= 6:
+            T = rng.choice([1, 2, 3, 8, 17, 31, 32, 48, 63, 64, 65, 100, 128])
         wl = W.MoEWorkload(f"random{it}", T=T, H=H, E=E, I=I, k=k, Is=Is, M=M, n_tenants=nt, G=G,
                            zipf_bias=rng.random() < 0.6, tenant_layout=rng.choice(["uniform", "contiguous"]))
         wts = W.make_weights(wl, seed=500 + it, shuffle_slots=rng.random() < 0.5)
         x, tenant, mot = W.make_tokens(wl, seed=500 + it)
         g = GpuLayer(wl, [wts], T, model_of_tenant=mot)
         try:
+            if seed >= 6:
+                B.moe_set_option(g.ctx, B.MOE_OPT_HEAD_UNITS, 0)
+                B.moe_set_option(g.ctx, B.MOE_OPT_FUSED_DISPATCH, 0)
             base = g.forward(x, tenant, G)
             ws = B.moe_get_workspace(g.ctx)
             eoff = B.wrap_device_pointer(ws["expert_off"], (M * E + 1,), torch.int32, g.dev).cpu().to(torch.int64)
             table = B.moe_form_blocks((eoff[1:] - eoff[:-1]).view(M, E), G)
             for _ in range(4):
                 opts = dict(mode=rng.choice([0, 1]), bg=rng.choice([0, 2]), early=rng.choice([0, 2]), tab=rng.random() < 0.5)
+                if seed >= 6:
+                    opts.update(head=rng.choice([0, 1]), fused=rng.choice([0, 1]))
+                    B.moe_set_option(g.ctx, B.MOE_OPT_HEAD_UNITS, opts["head"])
+                    B.moe_set_option(g.ctx, B.MOE_OPT_FUSED_DISPATCH, opts["fused"])
                 B.moe_set_option(g.ctx, B.MOE_OPT_DISPATCH_MODE, opts["mode"])
                 B.moe_set_option(g.ctx, B.MOE_OPT_BACKGROUND_LANES, opts["bg"])
                 B.moe_set_option(g.ctx, B.MOE_OPT_EARLY_SHARED, opts["early"])
