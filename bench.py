@@ -191,11 +191,11 @@ def kernel_source_digest() -> str:
 # ncu summaries under profiles/ together with the digest of the kernel sources they were captured on.  bench.py prints
 # the figure only while kernel_source_digest() still equals `digest`; otherwise `traffic` is null.
 NCU_TRAFFIC = {
-    "decode": {"bytes": 678.527744e6 + 6.193408e6, "digest": "4ebfa6a4a9a9b48c",
+    "decode": {"bytes": 678.723072e6 + 3.447552e6, "digest": "767af1952e5f6102",
                "source": "profiles/grouped_gemm_decode_ncu.md (gate/up launch, dram__bytes_read.sum + dram__bytes_write.sum; 23.07 MB of it are the shared expert's down weights pulled into L2 for the next launch)"},
-    "prefill": {"bytes": 931.751424e6 + 84.917248e6, "digest": "4ebfa6a4a9a9b48c",
+    "prefill": {"bytes": 929.690624e6 + 84.762112e6, "digest": "767af1952e5f6102",
                 "source": "profiles/grouped_gemm_prefill_ncu.md (merged gate/up launch, dram__bytes_read.sum + dram__bytes_write.sum)"},
-    "pool": {"bytes": 2998.122496e6 + 38.049536e6, "digest": "4ebfa6a4a9a9b48c",
+    "pool": {"bytes": 2996.817152e6 + 38.470656e6, "digest": "767af1952e5f6102",
              "source": "profiles/grouped_gemm_pool_dram.md (merged gate/up launch, dram__bytes_read.sum + dram__bytes_write.sum)"},
 }
 

@@ -100,7 +100,7 @@ enum { MOE_OPT_EXPERT_PATH = 1, MOE_OPT_ROUTE_PATH = 2,
        MOE_OPT_BACKGROUND_LANES = 10, /* 2-CTA shape: expert tiles of at most 64 rows are run by a second, small pipeline
                                          of every CTA pair (its own stage ring, TMA lane, MMA lane and accumulator)
                                          beside the pair's long tiles, so that the short tiles' weights stream in behind
-                                         tensor-bound work.  1 (default): for batches of at least 2048 tokens of one
+                                         tensor-bound work.  1 (default): for batches of at least 4096 tokens of one
                                          model; 2: every batch of the 2-CTA shape; 0: never (one pipeline runs all tiles
                                          in turn).  Results are bit-identical. */
        MOE_OPT_ROUTE_LANES = 8 /* 2 (default): the tensor-core router issues its MMAs from two warps, even and odd K

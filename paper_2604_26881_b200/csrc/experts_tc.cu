@@ -1284,9 +1284,11 @@ bool tc_background_mode(const moe_ctx* c, int T)
 {
     // measured: it pays where long, tensor-bound tiles dominate and the short tiles can hide behind them (4096-token
     // prefill: step -3 %); where nearly every tile is short the launch is bound by HBM and the background lanes, with
-    // their shallow ring, stream worse than the main ones (240-expert pool +10 %, 1126 tokens +4 %)
+    // their shallow ring, stream worse than the main ones (240-expert pool +8 %, 1126 tokens +6 %).  In between
+    // (Zipf-skewed batches, rounds of 0.6 s alternating in one context): 2048 tokens +3 %, 2560 +1.4 %, 3072 +0.8 %,
+    // 3584 +2 %, 4096 tokens -0.2 % on one part and -6.6 % on another.
     if (!tc_wide_mode(c, T) || c->background_enabled == 0) return false;
-    return c->background_enabled == 2 || (c->cfg.n_models == 1 && T >= 2048);
+    return c->background_enabled == 2 || (c->cfg.n_models == 1 && T >= 4096);
 }
 
 // One-CTA units with the tokens as the M operand: every batch that does not take the pair shape.
