@@ -255,6 +255,40 @@ def test_stack_teacher_forced(path):
         g.close()
 
 
+@pytest.mark.parametrize("T", [5, 40, 64])
+def test_small_stack_agrees_across_wait_options(T):
+    # a stack of four blocks on a decode-sized batch: in every block the gate/up launch may start on the shared
+    # expert's units while the block's RMSNorm output is being routed, and the dispatch may run inside the router's
+    # launch.  The block's input is the previous block's output, so a launch that ran ahead of data it needs would
+    # show in the residual stream; all four settings must give the same bits, twice in a row.
+    wl = W.scaled(W.WORKLOADS["stack"], H=512, I=256, Is=512, E=24, n_layers=4, n_tenants=6, T=T, tenant_layout="uniform")
+    layers = [W.make_weights(wl, seed=11, layer=l) for l in range(wl.n_layers)]
+    x, tenant, mot = W.make_tokens(wl, seed=11)
+    g = GpuLayer(wl, layers, T, model_of_tenant=mot)
+    try:
+        td = tenant.to(g.dev)
+        outs = {}
+        for head in (0, 1):
+            for fused in (0, 1):
+                B.moe_set_option(g.ctx, B.MOE_OPT_HEAD_UNITS, head)
+                B.moe_set_option(g.ctx, B.MOE_OPT_FUSED_DISPATCH, fused)
+                runs = []
+                for _ in range(2):
+                    xd = x.to(g.dev).clone()
+                    B.moe_stack_forward(g.ctx, xd, td, T, wl.G)
+                    runs.append(xd)
+                torch.cuda.synchronize()
+                assert B.moe_last_status(g.ctx)[0] == 0
+                assert torch.equal(runs[0], runs[1])
+                outs[(head, fused)] = runs[0]
+        ref = outs[(0, 0)]
+        assert not torch.equal(ref, x.to(g.dev))
+        for key, o in outs.items():
+            assert torch.equal(o, ref), key
+    finally:
+        g.close()
+
+
 def test_pair_shape_and_single_shape_agree_bit_for_bit(qwen_weights):
     # the 2-CTA (cta_group::2) and the 1-CTA shape of the grouped GEMM tile the work differently but
     # accumulate every output element over K in the same order
